@@ -1,0 +1,361 @@
+#!/usr/bin/env python
+"""Benchmark of the Gossip-PGA iteration (libgpga) on B200.
+
+A "step" is one iteration of Algorithm 1 over the whole n x d state: the fused
+local-update + gossip kernel, or the fused local-update + global-average kernel on
+every H-th iteration.  Prints one JSON line (rank 0).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3_ring_h4] [--impl reference]
+
+Multi-GPU: the state is sharded by columns (columns evolve independently), one
+process per GPU, no data-path collective; every rank holds a full-width shard of a
+problem N times wider (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+METRIC = "Gossip-PGA node-param updates/s and HBM GB/s vs B200 peak (fp32, 1 GPU)"
+UNIT = "node-param updates/s"
+SEED = 20210509
+BYTES_PER_UPDATE = 12          # read X (4) + read b (4) + write X+ (4); the noise never touches HBM
+
+# name: n, d, topology, H, gamma, sigma, K (the configuration's own run length), x0 kind, x0 std, b shift
+WORKLOADS = {
+    "c1_ring_h4": dict(n=8, d=65_536, topo="ring", H=4, gamma=0.1, sigma=0.1, K=32, x0="zero", x0_std=1.0, b_shift=0.0),
+    "c2_exp_h8": dict(n=32, d=1_048_576, topo="exp", H=8, gamma=0.05, sigma=0.1, K=64, x0="zero", x0_std=1.0, b_shift=0.0),
+    "c3_ring_h4": dict(n=64, d=25_557_032, topo="ring", H=4, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),
+    "c3_ring_h16": dict(n=64, d=25_557_032, topo="ring", H=16, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),
+    "c3_ring_hinf": dict(n=64, d=25_557_032, topo="ring", H=0, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),
+    "c3_exp_h4": dict(n=64, d=25_557_032, topo="exp", H=4, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),
+    "c3_exp_h16": dict(n=64, d=25_557_032, topo="exp", H=16, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),
+    "c3_exp_hinf": dict(n=64, d=25_557_032, topo="exp", H=0, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),
+    "c3_global_h1": dict(n=64, d=25_557_032, topo="ring", H=1, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),
+    "c4_exp_h4": dict(n=16, d=335_141_888, topo="exp", H=4, gamma=0.01, sigma=0.01, K=20, x0="zero", x0_std=1.0, b_shift=0.0),
+    "c4_global_h1": dict(n=16, d=335_141_888, topo="exp", H=1, gamma=0.01, sigma=0.01, K=20, x0="zero", x0_std=1.0, b_shift=0.0),
+}
+DEFAULT_WORKLOAD = "c3_ring_h4"
+
+# DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum), as a multiple of the algorithmic bytes of the captured launch, with
+# the digest of the kernel sources at capture time.  A changed source voids it (-> null).
+NCU_TRAFFIC = {
+    # kernel name: (traffic / algorithmic bytes, source digest)
+}
+
+
+def kernel_source_digest() -> str:
+    h = hashlib.sha256()
+    for name in ("gpga_device.cuh", "gpga_kernels.cuh", "gpga_kernels.cu"):
+        h.update((ROOT / "paper_2105_09080_b200" / "csrc" / name).read_bytes())
+    return h.hexdigest()[:16]
+
+
+def measured_peak_gbs():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            return float(json.loads(p.read_text())["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self.active = threading.Event()
+        self.error = None
+
+    def run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            names = {}
+            for attr in dir(nv):
+                if attr.startswith("nvmlClocksEventReason") or attr.startswith("nvmlClocksThrottleReason"):
+                    v = getattr(nv, attr)
+                    if isinstance(v, int) and v and attr not in ("nvmlClocksEventReasonAll", "nvmlClocksThrottleReasonAll"):
+                        names.setdefault(v, attr.replace("nvmlClocksEventReason", "").replace("nvmlClocksThrottleReason", ""))
+            get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                nv.nvmlDeviceGetCurrentClocksThrottleReasons
+            while not self._stop.is_set():
+                if self.active.is_set():
+                    self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                    mask = get_reasons(h)
+                    for bit, nm in names.items():
+                        if mask & bit and bit.bit_count() == 1:
+                            self.reasons.add(nm)
+                time.sleep(self.period)
+            nv.nvmlShutdown()
+        except Exception as exc:          # NVML missing: report it, do not fail the run
+            self.error = repr(exc)
+
+    def finish(self):
+        self._stop.set()
+        self.join(timeout=2)
+        s = sorted(self.samples)
+        return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(r for r in self.reasons if r not in ("GpuIdle", "None")),
+                "samples": len(s), **({"error": self.error} if self.error else {})}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+# ---------------------------------------------------------------------------------
+# CPU baseline: the oracle as it stands, on a bounded column slice of the workload
+# ---------------------------------------------------------------------------------
+def oracle_sample(w, cols, iters, k0=0):
+    """Run `iters` oracle iterations on a `cols`-column slice (all n rows); returns seconds."""
+    import numpy as np
+    from oracle import gpga_oracle as o
+    topo = {"ring": o.TOPO_RING, "exp": o.TOPO_EXP}[w["topo"]]
+    kind = {"zero": o.X0_ZERO, "shared": o.X0_SHARED_NORMAL}[w["x0"]]
+    B = o.init_b(w["n"], cols, SEED, w["b_shift"]).astype(np.float32)
+    X = o.init_x0(w["n"], cols, SEED, kind, w["x0_std"]).astype(np.float32)
+    p = o.Problem(topo, w["H"], w["gamma"], SEED, sigma=w["sigma"], data=B)
+    t0 = time.perf_counter()
+    o.run(p, X, k0, iters)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(w, target_s=12.0):
+    from oracle import gpga_oracle as o
+    iters = max(w["H"], 1) if w["H"] else 4        # one averaging period (or four gossip steps)
+    probe_cols = 4096
+    t = oracle_sample(w, probe_cols, iters)
+    rate = w["n"] * probe_cols * iters / t
+    cols = int(min(w["d"], max(probe_cols, target_s * rate / (w["n"] * iters))))
+    cols -= cols % 4
+    t = oracle_sample(w, cols, iters)
+    return {"value": w["n"] * cols * iters / t, "unit": UNIT, "cores": o.num_threads(), "kind": "oracle",
+            "sample": f"{iters} iterations (k=0..{iters - 1}) on the first {cols} of {w['d']} columns, all "
+                      f"{w['n']} rows, {t:.1f} s; columns are independent so throughput scales linearly in d"}
+
+
+def run_reference(args, w, name):
+    """--impl reference: the oracle on the host cores; each step = one iteration on a bounded slice."""
+    from oracle import gpga_oracle as o
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per_step_s = 1.0
+    t = oracle_sample(w, 4096, 1)
+    cols = int(min(w["d"], max(4096, per_step_s * 4096 / t)))
+    cols -= cols % 4
+    import numpy as np
+    topo = {"ring": o.TOPO_RING, "exp": o.TOPO_EXP}[w["topo"]]
+    kind = {"zero": o.X0_ZERO, "shared": o.X0_SHARED_NORMAL}[w["x0"]]
+    B = o.init_b(w["n"], cols, SEED, w["b_shift"]).astype(np.float32)
+    X = o.init_x0(w["n"], cols, SEED, kind, w["x0_std"]).astype(np.float32)
+    p = o.Problem(topo, w["H"], w["gamma"], SEED, sigma=w["sigma"], data=B)
+    k = 0
+    for _ in range(args.warmup):
+        X = o.step(p, X, k)
+        k += 1
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        X = o.step(p, X, k)
+        k += 1
+    dt = time.perf_counter() - t0
+    value = w["n"] * cols * args.steps / dt
+    sample = (f"each step = one iteration on the first {cols} of {w['d']} columns, all {w['n']} rows "
+              f"(columns are independent)")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": workload_config(name, w, args.gpus),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": o.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def workload_config(name, w, n_gpus):
+    return {"workload": f"{name}: n={w['n']} nodes x d={w['d']} fp32, {w['topo']} topology, H={w['H'] or 'inf'}, "
+                        f"gamma={w['gamma']}, sigma={w['sigma']}, quadratic objective, seed {SEED}",
+            "l2_flush": f"none needed: each step streams {BYTES_PER_UPDATE * w['n'] * w['d'] / 1e9:.2f} GB, larger than the 126 MB L2"
+                        if BYTES_PER_UPDATE * w['n'] * w['d'] > 4 * 126e6 else "state fits in L2; reported as L2-resident",
+            "sharding": f"columns, {n_gpus} shard(s) of d columns each, no collective"}
+
+
+# ---------------------------------------------------------------------------------
+# CUDA arm
+# ---------------------------------------------------------------------------------
+def run_ours(args, w, name):
+    import torch
+    import paper_2105_09080_b200 as pkg
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    n, d = w["n"], w["d"]
+    topo = {"ring": pkg.GPGA_TOPO_RING, "exp": pkg.GPGA_TOPO_EXP}[w["topo"]]
+    kind = {"zero": pkg.GPGA_X0_ZERO, "shared": pkg.GPGA_X0_SHARED_NORMAL}[w["x0"]]
+    g = pkg.Gpga(n, d, topo, w["H"], w["gamma"], SEED)
+    g.set_objective(pkg.GPGA_OBJ_QUADRATIC, sigma=w["sigma"])
+    g.set_column_offset(rank * ((d + 3) // 4 * 4))
+    xa, xb, b = g.allocate()
+    g.init_from_seed(kind, w["x0_std"], w["b_shift"])
+    torch.cuda.synchronize()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        g.step(g.get_k())
+    barrier()
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()
+    launches0 = g.launch_count()
+    k_first = g.get_k()
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    sampler.active.set()
+    events[0].record()
+    for s in range(args.steps):
+        g.step(k_first + s)
+        events[s + 1].record()
+    barrier()
+    sampler.active.clear()
+    clocks = sampler.finish()
+    launches = g.launch_count() - launches0
+    elapsed_ms = events[0].elapsed_time(events[-1])
+    per_step = [events[s].elapsed_time(events[s + 1]) for s in range(args.steps)]
+    if dist is not None:
+        t = torch.tensor([elapsed_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+
+    # per-kernel durations from the per-step events (one kernel per step)
+    glob = [ms for s, ms in enumerate(per_step) if w["H"] and (k_first + s + 1) % w["H"] == 0]
+    goss = [ms for s, ms in enumerate(per_step) if not (w["H"] and (k_first + s + 1) % w["H"] == 0)]
+    peak, peak_kind = measured_peak_gbs()
+    algo_bytes = BYTES_PER_UPDATE * n * d
+    kernels = {}
+    if goss:
+        kernels[f"step_{w['topo']}_kernel"] = sum(goss) / len(goss)
+    if glob:
+        kernels["step_global_kernel"] = sum(glob) / len(glob)
+    dominant = max(kernels, key=lambda nm: kernels[nm] * (len(goss) if nm != "step_global_kernel" else len(glob)))
+    achieved = algo_bytes / (kernels[dominant] * 1e-3) / 1e9
+    traffic = None
+    if dominant in NCU_TRAFFIC and NCU_TRAFFIC[dominant][1] == kernel_source_digest():
+        traffic = NCU_TRAFFIC[dominant][0] * algo_bytes
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
+                "algorithmic_bytes_per_launch": algo_bytes,
+                "per_kernel": {nm: {"ms": ms, "GB/s": algo_bytes / (ms * 1e-3) / 1e9,
+                                    "frac": algo_bytes / (ms * 1e-3) / 1e9 / peak} for nm, ms in kernels.items()},
+                "frac_of_nominal_8TBs": achieved / 8000.0}
+
+    # end to end through the host entry point: pinned host buffers in, K iterations, result out
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(torch, g, w, dist)
+
+    value = n * d * args.steps * world / (elapsed_ms * 1e-3)
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(name, w, world), "hbm_gbs": value * BYTES_PER_UPDATE / 1e9 / world,
+            "roofline": roofline, "clocks": clocks, "e2e": e2e, "gpu_launches": launches}
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(w)
+        print(json.dumps(line))
+    g.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def run_e2e(torch, g, w, dist):
+    n, d, K = w["n"], w["d"], w["K"]
+    x0 = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+    bh = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+    out = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+    # host copies of the seeded inputs (downloaded once, outside the timed region)
+    g.init_from_seed({"zero": 0, "shared": 1}[w["x0"]], w["x0_std"], w["b_shift"])
+    x0.copy_(g.x_bufs[0])
+    bh.copy_(g._keep[2])
+    torch.cuda.synchronize()
+    g.run_host(x0, bh, K, out)                      # warm-up job
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    jobs = 2
+    t0 = time.perf_counter()
+    for _ in range(jobs):
+        g.run_host(x0, bh, K, out)                  # synchronises its stream
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    world = 1
+    if dist is not None:
+        t = torch.tensor([dt], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dt = float(t.item())
+        world = dist.get_world_size()
+    return {"value": n * d * K * jobs * world / dt, "unit": UNIT,
+            "h2d_bytes_per_step": 2 * n * d * 4 / K, "d2h_bytes_per_step": n * d * 4 / K,
+            "job": f"gpga_run_host: pinned host X0 and b copied in ({2 * n * d * 4 / 1e9:.2f} GB), K={K} iterations, "
+                   f"X copied out ({n * d * 4 / 1e9:.2f} GB); bytes per step are the job's bytes / K",
+            "seconds_per_job": dt / jobs}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    w = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w, args.workload)
+    else:
+        run_ours(args, w, args.workload)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,215 @@
+/*
+ * gpga.h -- C ABI of libgpga: one Gossip-PGA iteration over n simulated nodes
+ * held as an n x d fp32 matrix X (row i = node i's parameters) on one GPU.
+ *
+ * Paper: "Accelerating Gossip SGD with Periodic Global Averaging".
+ * Each entry point below names the passage of the paper that defines what it
+ * computes.  Notation follows the paper: n nodes, d parameters, k the 0-based
+ * iteration index of Algorithm 1, gamma the learning rate, H the global
+ * averaging period, W the doubly-stochastic weight matrix (Section 3).
+ *
+ * Conventions
+ *  - Every function returns an int32 status (GPGA_OK = 0).  Nothing throws,
+ *    aborts or traps.  After a non-zero status gpga_last_error() gives text.
+ *  - The handle is owned by the library.  ALL device memory is owned by the
+ *    caller and must outlive the handle; the library never allocates or frees
+ *    device memory.
+ *  - "device pointer" / "host pointer" is stated per argument.  Device
+ *    pointers must be 16-byte aligned.  Matrices are row-major, row stride d,
+ *    fp32.  Element (i, j) of an n x d matrix is at index i * d + j (64-bit).
+ *  - `stream` arguments are a cudaStream_t passed as void* (NULL = default
+ *    stream).  Calls are asynchronous on that stream unless stated otherwise.
+ *  - Random numbers are Philox4x32-10 (Salmon et al., SC'11) keyed by
+ *    key = (seed low word, seed high word), counter = (column >> 2, node i,
+ *    iteration k, stream id); the four output words give four normals for
+ *    columns 4q..4q+3 by Box-Muller with u1 = ((w >> 8) + 1) / 2^24,
+ *    u2 = (w' >> 8) / 2^24.  They are generated in registers and never stored.
+ */
+#ifndef GPGA_H_
+#define GPGA_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gpga_ctx gpga_t;
+
+enum {
+    GPGA_OK = 0,
+    GPGA_ERR_INVALID_ARG = 1,
+    GPGA_ERR_NOT_READY = 2,   /* NULL handle, buffers not bound */
+    GPGA_ERR_CUDA = 3,        /* a CUDA call failed; sticky */
+    GPGA_ERR_UNSUPPORTED = 4
+};
+
+/* Gossip topologies (Section 3; Section 5 for the one-peer exponential graph). */
+enum {
+    GPGA_TOPO_RING = 0,       /* w = 1/3 on i-1, i, i+1 (indices mod n) */
+    GPGA_TOPO_EXP = 1,        /* step k: average with (i + 2^(k mod log2 n)) mod n, w = 1/2; n = 2^m */
+    GPGA_TOPO_GRID = 2,       /* r x c torus, w = 1/5 on the node and its 4 neighbours */
+    GPGA_TOPO_STATIC_EXP = 3, /* w = 1/(log2 n + 1) on i and (i + 2^t) mod n, t < log2 n */
+    GPGA_TOPO_NONE = 4        /* W = I (Local SGD between global averages) */
+};
+
+enum { GPGA_OBJ_QUADRATIC = 0, GPGA_OBJ_LOGISTIC = 1 };
+
+/* Initial state kinds for gpga_init_from_seed. */
+enum { GPGA_X0_ZERO = 0, GPGA_X0_SHARED_NORMAL = 1, GPGA_X0_PER_NODE_NORMAL = 2 };
+
+/* Random stream ids (fourth counter word). */
+enum {
+    GPGA_STREAM_NOISE = 0,
+    GPGA_STREAM_B = 1,
+    GPGA_STREAM_X0 = 2,
+    GPGA_STREAM_NODE_SHIFT = 3,
+    GPGA_STREAM_BATCH = 4
+};
+
+/*
+ * Create a handle for problem (1) of the paper, min_x (1/n) sum_i f_i(x), solved
+ * by Algorithm 1 with learning rate gamma, weight matrix W given by `topology`
+ * and averaging period H.  H = 0 encodes H -> infinity (plain Gossip SGD,
+ * Section 3); H = 1 is parallel SGD.  The default objective is the quadratic
+ * f_i(x) = 1/2 ||x - b_i||^2 with sigma = 0.
+ * Errors: INVALID_ARG for n < 1, d < 1, n >= 2^32, d >= 2^34, H < 0, gamma not
+ * finite or negative, unknown topology, NULL out; UNSUPPORTED for EXP or
+ * STATIC_EXP with n not a power of two.
+ */
+int32_t gpga_create(int64_t n, int64_t d, int32_t topology, int64_t H, float gamma, uint64_t seed,
+                    gpga_t** out);
+
+/*
+ * Choose the stochastic-gradient model (Assumption 2: unbiased, bounded variance).
+ *  QUADRATIC: g_ij = (x_ij - b_ij) + sigma * xi_kij, xi standard normal (stream NOISE).
+ *             l2, m, batch ignored.
+ *  LOGISTIC:  Section 5.1 loss f_i(x) = (1/m) sum_r ln(1 + exp(-y_r a_r^T x)) + (l2/2)||x||^2;
+ *             g_i = mini-batch gradient over `batch` rows drawn with replacement:
+ *             draw t = word (t & 3) of Philox counter (t >> 2, i, k, BATCH), reduced mod m.
+ *             sigma ignored.
+ * Errors: INVALID_ARG for negative / non-finite sigma or l2, m < 1, batch < 1, m >= 2^31.
+ * Must be called before gpga_bind.
+ */
+int32_t gpga_set_objective(gpga_t* ctx, int32_t objective, float sigma, float l2, int64_t m,
+                           int64_t batch);
+
+/* Grid topology only: number of columns c of the r x c torus (n = r * c).
+ * Errors: INVALID_ARG unless c >= 1 and c divides n. */
+int32_t gpga_set_grid_cols(gpga_t* ctx, int64_t cols);
+
+/*
+ * Column sharding: this handle holds global columns col0 .. col0 + d - 1 of a wider
+ * problem.  Only the random-number counters depend on it; W acts on rows, so column
+ * ranges evolve independently (matrix form of the recursion, Appendix A).
+ * Errors: INVALID_ARG unless col0 >= 0, col0 % 4 == 0 and col0 + d < 2^34.
+ */
+int32_t gpga_set_column_offset(gpga_t* ctx, int64_t col0);
+
+/* Bytes of scratch device memory gpga_bind must be given (reduction partials, and
+ * for the logistic objective the per-chunk gradient partials). */
+int64_t gpga_scratch_bytes(const gpga_t* ctx);
+
+/*
+ * Bind caller-owned device buffers.
+ *  x_a, x_b : two n*d fp32 buffers (double buffer for X^(k), X^(k+1)); x_a holds the
+ *             current state.
+ *  data     : QUADRATIC: b, n*d fp32.  LOGISTIC: A, n*m*d fp32 (node-major, then sample).
+ *  labels   : LOGISTIC: y, n*m fp32 in {-1,+1}; otherwise NULL.
+ *  scratch  : at least gpga_scratch_bytes() bytes (scratch_bytes is what was given).
+ * Errors: INVALID_ARG for NULL / misaligned pointers, x_a == x_b, too little scratch.
+ */
+int32_t gpga_bind(gpga_t* ctx, void* x_a, void* x_b, void* data, const void* labels,
+                  void* scratch, int64_t scratch_bytes);
+
+/*
+ * Fill the bound buffers on the device from the seed (quadratic objective only):
+ *  b_ij = z_ij + b_shift * s_i,  z from stream B, s_i the first normal of stream
+ *  NODE_SHIFT for node i;  X^(0) per x0_kind with standard deviation x0_std
+ *  (Algorithm 1 requires equal initial rows: kinds ZERO and SHARED_NORMAL).
+ * Also resets the iteration counter to 0 and makes x_a the current buffer.
+ */
+int32_t gpga_init_from_seed(gpga_t* ctx, int32_t x0_kind, float x0_std, float b_shift,
+                            void* stream);
+
+/*
+ * One iteration of Algorithm 1 for iteration index k: gradient, local update
+ * x^(k+1/2) = x^(k) - gamma g^(k), then the global average if mod(k+1, H) = 0, else one
+ * gossip step with W.  Reads the current buffer, writes the other, flips them, and sets
+ * the internal counter to k + 1.  A pure function of (current X, data, seed, k, params).
+ * Errors: NOT_READY if unbound; INVALID_ARG for k < 0 or k >= 2^32.
+ */
+int32_t gpga_step(gpga_t* ctx, int64_t k, void* stream);
+
+/* K iterations k0 .. k0+K-1 starting at the internal counter k0 (Algorithm 1's loop). */
+int32_t gpga_run(gpga_t* ctx, int64_t K, void* stream);
+
+/*
+ * Same as gpga_run with HOST buffers (quadratic objective): copies x0_host (n*d fp32) and
+ * data_host (n*d fp32) into the bound device buffers, resets the counter to 0, runs K
+ * iterations, copies X^(K) to x_out_host and synchronises the stream.  Host buffers
+ * should be pinned for full copy speed.
+ */
+int32_t gpga_run_host(gpga_t* ctx, const float* x0_host, const float* data_host, int64_t K,
+                      float* x_out_host, void* stream);
+
+/*
+ * Consensus distance sum_i ||x_i - xbar||^2 of the current state (Section 4; Appendix A
+ * notation ||X - Xbar||_F^2), accumulated in fp64.  Synchronises the stream; *out_host is
+ * a host double.
+ */
+int32_t gpga_consensus_distance(gpga_t* ctx, void* stream, double* out_host);
+
+/*
+ * Mean over nodes of the local loss at each node's own iterate, (1/n) sum_i F_i(x_i)
+ * (the quantity Algorithm 2 averages).  QUADRATIC: F_i = 1/2 ||x_i - b_i||^2.
+ * Synchronises the stream.
+ */
+int32_t gpga_mean_loss(gpga_t* ctx, void* stream, double* out_host);
+
+/*
+ * Gossip-AGA (Algorithm 2, period rule with the exponent removed as its appendix states):
+ * K iterations with an adaptive period.  A counter C counts iterations since the last
+ * global average; when C == H the step is a global average, the mean loss F of that
+ * iteration's state is taken, and H is updated: F_init <- (F_init + F)/2 while
+ * k < warmup_iters, afterwards H <- ceil(F_init / F * H_init).  Synchronises at each
+ * global-average iteration.  periods_host (may be NULL) receives up to max_periods period
+ * lengths in order; *num_periods_host their count.
+ */
+int32_t gpga_run_adaptive(gpga_t* ctx, int64_t K, int64_t H_init, int64_t warmup_iters,
+                          void* stream, int64_t* periods_host, int64_t max_periods,
+                          int64_t* num_periods_host);
+
+/* Accessors.  gpga_get_x returns the device pointer of the current state buffer. */
+int32_t gpga_get_x(const gpga_t* ctx, void** x_cur);
+int32_t gpga_get_k(const gpga_t* ctx, int64_t* k);
+int32_t gpga_set_k(gpga_t* ctx, int64_t k);
+int32_t gpga_set_gamma(gpga_t* ctx, float gamma);   /* e.g. the halving schedule of Section 5.1 */
+int32_t gpga_set_period(gpga_t* ctx, int64_t H);
+/* Kernels launched by this handle so far. */
+int64_t gpga_launch_count(const gpga_t* ctx);
+
+/* Text of the last error of this handle (or of gpga_create when ctx is NULL). */
+const char* gpga_last_error(const gpga_t* ctx);
+
+/* Frees the handle only. */
+int32_t gpga_destroy(gpga_t* ctx);
+
+/*
+ * Generator surface (device pointers), used to check the device generator against its
+ * published definition:
+ *  gpga_philox_words:  out[4t..4t+3] = Philox4x32-10(counter = ctr[4t..4t+3], key).
+ *  gpga_box_muller_words: z[2t], z[2t+1] = Box-Muller of the word pair (a[t], b[t]).
+ *  gpga_normal_fill: out[4t..4t+3] = the four normals of counter (q0 + t, i, k, stream_id).
+ */
+int32_t gpga_philox_words(const uint32_t* ctr_dev, uint32_t key0, uint32_t key1, int64_t count,
+                          uint32_t* out_dev, void* stream);
+int32_t gpga_box_muller_words(const uint32_t* a_dev, const uint32_t* b_dev, int64_t count,
+                              float* z_dev, void* stream);
+int32_t gpga_normal_fill(uint64_t seed, uint32_t stream_id, uint32_t k, uint32_t i, uint32_t q0,
+                         int64_t count, float* out_dev, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GPGA_H_ */

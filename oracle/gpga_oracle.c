@@ -356,3 +356,23 @@ void gpga_oracle_aga_update(int64_t k, int64_t warmup_iters, int64_t H_init, dou
         *H = (int64_t)ceil((*F_init / F) * (double)H_init);
     }
 }
+
+/* Box-Muller over arrays of word pairs: z[2t], z[2t+1] from (a[t], b[t]). */
+void gpga_oracle_box_muller_many(const uint32_t* a, const uint32_t* b, int64_t count, double* z)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < count; ++t) gpga_oracle_box_muller(a[t], b[t], z + 2 * t);
+}
+
+/* Mean over nodes of the local quadratic loss at each node's own iterate:
+ * (1/n) sum_i 1/2 ||x_i - b_i||^2  (the loss Algorithm 2 averages, for f_i of the
+ * quadratic objective). */
+double gpga_oracle_quadratic_mean_loss(int64_t n, int64_t d, const double* X, const double* B)
+{
+    double total = 0.0;
+    for (int64_t e = 0; e < n * d; ++e) {
+        double r = X[e] - B[e];
+        total += r * r;
+    }
+    return 0.5 * total / (double)n;
+}

@@ -94,6 +94,10 @@ def lib():
         L.gpga_oracle_init_x0.restype = None
         L.gpga_oracle_aga_update.argtypes = [i64, i64, i64, f64, P, P]
         L.gpga_oracle_aga_update.restype = None
+        L.gpga_oracle_box_muller_many.argtypes = [P, P, i64, P]
+        L.gpga_oracle_box_muller_many.restype = None
+        L.gpga_oracle_quadratic_mean_loss.argtypes = [i64, i64, P, P]
+        L.gpga_oracle_quadratic_mean_loss.restype = f64
         _lib = L
     return _lib
 
@@ -120,6 +124,15 @@ def philox4x32_10(ctr, key) -> np.ndarray:
 def box_muller(a: int, b: int) -> np.ndarray:
     z = np.zeros(2, dtype=np.float64)
     lib().gpga_oracle_box_muller(int(a), int(b), _p(z))
+    return z
+
+
+def box_muller_many(a, b) -> np.ndarray:
+    """Box-Muller of word pairs; returns shape (count, 2) fp64."""
+    a = np.ascontiguousarray(a, dtype=np.uint32)
+    b = np.ascontiguousarray(b, dtype=np.uint32)
+    z = np.empty((a.size, 2), dtype=np.float64)
+    lib().gpga_oracle_box_muller_many(_p(a), _p(b), a.size, _p(z))
     return z
 
 
@@ -368,6 +381,12 @@ def run_f64(p: Problem, X, k0: int, K: int) -> np.ndarray:
     for k in range(k0, k0 + K):
         X = step_f64(p, X, k)
     return X
+
+
+def quadratic_mean_loss(X, B) -> float:
+    X = _f64(X)
+    B = _f64(B)
+    return float(lib().gpga_oracle_quadratic_mean_loss(X.shape[0], X.shape[1], _p(X), _p(B)))
 
 
 def aga_update(k, warmup_iters, H_init, F, F_init, H):

@@ -1,0 +1,495 @@
+// C ABI of libgpga: handle, argument checks, schedule, launches.  See include/gpga.h.
+#include <cmath>
+#include <cstdio>
+#include <new>
+#include <string>
+
+#include "../../include/gpga.h"
+#include "gpga_kernels.cuh"
+#include "gpga_logreg.cuh"
+
+using namespace gpga;
+
+struct gpga_ctx {
+    int64_t n = 0, d = 0, H = 0;
+    int32_t topology = 0;
+    float gamma = 0.f;
+    uint64_t seed = 0;
+    int32_t objective = GPGA_OBJ_QUADRATIC;
+    float sigma = 0.f, l2 = 0.f;
+    int64_t m = 0, batch = 0;
+    int64_t grid_cols = 0;
+    int64_t col0 = 0;
+    float* x[2] = {nullptr, nullptr};
+    float* data = nullptr;
+    const float* labels = nullptr;
+    char* scratch = nullptr;
+    int64_t scratch_bytes = 0;
+    int cur = 0;
+    int64_t k = 0;
+    int64_t launches = 0;
+    bool bound = false;
+    int32_t sticky = GPGA_OK;
+    std::string err;
+    PhiloxKeys keys;
+};
+
+static thread_local std::string g_create_error;
+
+namespace {
+
+constexpr int64_t kMaxTileNodes = 4096;   // shared-memory tile path: n * 16 B <= 64 KB
+
+int32_t fail(gpga_ctx* c, int32_t code, const std::string& msg)
+{
+    if (c) c->err = msg; else g_create_error = msg;
+    return code;
+}
+
+int32_t cuda_fail(gpga_ctx* c, cudaError_t e, const char* where)
+{
+    c->sticky = GPGA_ERR_CUDA;
+    c->err = std::string(where) + ": " + cudaGetErrorString(e);
+    return GPGA_ERR_CUDA;
+}
+
+bool is_pow2(int64_t v) { return v > 0 && (v & (v - 1)) == 0; }
+int log2_floor(int64_t v) { int t = 0; while ((int64_t(1) << (t + 1)) <= v) ++t; return t; }
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+
+// Scratch layout: [reduction partials | result double | G | gradient chunk partials]
+struct ScratchLayout {
+    int64_t partials_off = 0, result_off = 0, G_off = 0, chunk_off = 0, total = 0;
+};
+ScratchLayout scratch_layout(const gpga_ctx* c)
+{
+    ScratchLayout L;
+    int64_t slots = kMaxReduceBlocks;
+    if (c->n > slots) slots = c->n;
+    L.partials_off = 0;
+    L.result_off = round_up(slots * 8, 256);
+    L.total = L.result_off + 256;
+    if (c->objective == GPGA_OBJ_LOGISTIC) {
+        L.G_off = L.total;
+        L.chunk_off = L.G_off + round_up(c->n * c->d * 4, 256);
+        L.total = L.chunk_off + round_up(int64_t(logreg_chunks(c->batch)) * c->n * c->d * 4, 256);
+    }
+    return L;
+}
+
+// Algorithm 1: global average exactly when mod(k + 1, H) = 0 (H = 0: never).
+bool is_global_step(int64_t k, int64_t H) { return H > 0 && ((k + 1) % H) == 0; }
+
+int32_t check_ready(gpga_ctx* c)
+{
+    if (!c) return fail(nullptr, GPGA_ERR_NOT_READY, "NULL handle");
+    if (c->sticky != GPGA_OK) return c->sticky;
+    if (!c->bound) return fail(c, GPGA_ERR_NOT_READY, "buffers not bound (call gpga_bind)");
+    return GPGA_OK;
+}
+
+LogregParams logreg_params(const gpga_ctx* c, int64_t k)
+{
+    const ScratchLayout L = scratch_layout(c);
+    LogregParams lp;
+    lp.A = c->data;
+    lp.y = c->labels;
+    lp.x = c->x[c->cur];
+    lp.G = reinterpret_cast<float*>(c->scratch + L.G_off);
+    lp.partial = reinterpret_cast<float*>(c->scratch + L.chunk_off);
+    lp.n = c->n; lp.d = c->d; lp.m = c->m; lp.batch = c->batch;
+    lp.k = (uint32_t)k;
+    lp.l2 = c->l2;
+    lp.keys = c->keys;
+    return lp;
+}
+
+// One iteration; `global` chosen by the caller (fixed or adaptive period).
+int32_t do_step(gpga_ctx* c, int64_t k, bool global, cudaStream_t s)
+{
+    if (k < 0 || k >= (int64_t(1) << 32)) return fail(c, GPGA_ERR_INVALID_ARG, "k must be in [0, 2^32)");
+    StepParams p;
+    p.x = c->x[c->cur];
+    p.out = c->x[c->cur ^ 1];
+    p.b = c->data;
+    p.n = c->n; p.d = c->d; p.Q = (c->d + 3) / 4;
+    p.q_base = (uint32_t)(c->col0 >> 2);
+    p.k = (uint32_t)k;
+    p.gamma = c->gamma; p.sigma = c->sigma;
+    p.hop_log2 = 0; p.len_log2 = 0;
+    p.grid_cols = (int)c->grid_cols;
+    p.keys = c->keys;
+    const bool vec = (c->d % 4) == 0;
+    int mode = (c->sigma != 0.f) ? GRAD_QUAD_NOISE : GRAD_QUAD;
+    cudaError_t e;
+    if (c->objective == GPGA_OBJ_LOGISTIC) {
+        const LogregParams lp = logreg_params(c, k);
+        e = launch_logreg_grad(lp, s);
+        c->launches += 2;
+        if (e != cudaSuccess) return cuda_fail(c, e, "logistic gradient launch");
+        p.b = lp.G;
+        mode = GRAD_BUFFER;
+    }
+    if (global) {
+        e = launch_step_global(p, mode, vec, s);
+    } else if (c->topology == GPGA_TOPO_RING) {
+        e = launch_step_ring(p, mode, vec, s);
+    } else if (c->topology == GPGA_TOPO_EXP) {
+        const int tau = log2_floor(c->n);
+        if (tau > 0) {
+            p.hop_log2 = (int)(k % tau);
+            p.len_log2 = tau - p.hop_log2;
+        }
+        e = launch_step_exp(p, mode, vec, s);
+    } else {
+        e = launch_step_tile(p, mode, vec, c->topology, s);
+    }
+    c->launches += 1;
+    if (e != cudaSuccess) return cuda_fail(c, e, "step launch");
+    c->cur ^= 1;
+    c->k = k + 1;
+    return GPGA_OK;
+}
+
+int32_t mean_loss_async(gpga_ctx* c, cudaStream_t s, double** result_dev)
+{
+    const ScratchLayout L = scratch_layout(c);
+    double* partials = reinterpret_cast<double*>(c->scratch + L.partials_off);
+    double* result = reinterpret_cast<double*>(c->scratch + L.result_off);
+    cudaError_t e;
+    if (c->objective == GPGA_OBJ_LOGISTIC) {
+        if (c->k >= (int64_t(1) << 32)) return fail(c, GPGA_ERR_INVALID_ARG, "k must be in [0, 2^32)");
+        e = launch_logreg_loss(logreg_params(c, c->k), partials, result, s);
+    } else {
+        e = launch_quadratic_loss(c->x[c->cur], c->data, c->n, c->d, partials, result, s);
+    }
+    c->launches += 2;
+    if (e != cudaSuccess) return cuda_fail(c, e, "loss launch");
+    *result_dev = result;
+    return GPGA_OK;
+}
+
+int32_t read_double(gpga_ctx* c, const double* dev, cudaStream_t s, double* out_host)
+{
+    cudaError_t e = cudaMemcpyAsync(out_host, dev, sizeof(double), cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail(c, e, "result copy");
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(c, e, "stream synchronize");
+    return GPGA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t gpga_create(int64_t n, int64_t d, int32_t topology, int64_t H, float gamma, uint64_t seed,
+                    gpga_t** out)
+{
+    if (!out) return fail(nullptr, GPGA_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    if (n < 1 || n >= (int64_t(1) << 32)) return fail(nullptr, GPGA_ERR_INVALID_ARG, "n must be in [1, 2^32)");
+    if (d < 1 || d >= (int64_t(1) << 34)) return fail(nullptr, GPGA_ERR_INVALID_ARG, "d must be in [1, 2^34)");
+    if (H < 0) return fail(nullptr, GPGA_ERR_INVALID_ARG, "H must be >= 0 (0 = never average globally)");
+    if (!std::isfinite(gamma) || gamma < 0.f) return fail(nullptr, GPGA_ERR_INVALID_ARG, "gamma must be finite and >= 0");
+    if (topology < GPGA_TOPO_RING || topology > GPGA_TOPO_NONE)
+        return fail(nullptr, GPGA_ERR_INVALID_ARG, "unknown topology");
+    if ((topology == GPGA_TOPO_EXP || topology == GPGA_TOPO_STATIC_EXP) && !is_pow2(n))
+        return fail(nullptr, GPGA_ERR_UNSUPPORTED, "exponential graphs need n to be a power of two");
+    if ((topology == GPGA_TOPO_GRID || topology == GPGA_TOPO_STATIC_EXP || topology == GPGA_TOPO_NONE) &&
+        n > kMaxTileNodes)
+        return fail(nullptr, GPGA_ERR_UNSUPPORTED, "this topology supports at most 4096 nodes");
+    gpga_ctx* c = new (std::nothrow) gpga_ctx;
+    if (!c) return fail(nullptr, GPGA_ERR_INVALID_ARG, "out of host memory");
+    c->n = n; c->d = d; c->topology = topology; c->H = H; c->gamma = gamma; c->seed = seed;
+    c->keys = make_philox_keys((uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32));
+    if (topology == GPGA_TOPO_GRID) {   // default: the most square torus
+        int64_t cols = (int64_t)std::floor(std::sqrt((double)n));
+        while (cols > 1 && n % cols != 0) --cols;
+        c->grid_cols = n / cols;
+    }
+    *out = c;
+    return GPGA_OK;
+}
+
+int32_t gpga_set_objective(gpga_t* c, int32_t objective, float sigma, float l2, int64_t m, int64_t batch)
+{
+    if (!c) return fail(nullptr, GPGA_ERR_NOT_READY, "NULL handle");
+    if (c->bound) return fail(c, GPGA_ERR_INVALID_ARG, "set the objective before gpga_bind");
+    if (objective == GPGA_OBJ_QUADRATIC) {
+        if (!std::isfinite(sigma) || sigma < 0.f) return fail(c, GPGA_ERR_INVALID_ARG, "sigma must be finite and >= 0");
+        c->objective = objective; c->sigma = sigma; c->l2 = 0.f; c->m = 0; c->batch = 0;
+        return GPGA_OK;
+    }
+    if (objective == GPGA_OBJ_LOGISTIC) {
+        if (!std::isfinite(l2) || l2 < 0.f) return fail(c, GPGA_ERR_INVALID_ARG, "l2 must be finite and >= 0");
+        if (m < 1 || m >= (int64_t(1) << 31)) return fail(c, GPGA_ERR_INVALID_ARG, "m must be in [1, 2^31)");
+        if (batch < 1 || batch > (int64_t(1) << 20)) return fail(c, GPGA_ERR_INVALID_ARG, "batch must be in [1, 2^20]");
+        if (c->d % 4 != 0) return fail(c, GPGA_ERR_UNSUPPORTED, "logistic objective needs d % 4 == 0");
+        if (c->d > 48 * 1024) return fail(c, GPGA_ERR_UNSUPPORTED, "logistic objective needs d <= 49152");
+        if (c->n > 65535 || c->n * (c->d / 4) >= (int64_t(1) << 31))
+            return fail(c, GPGA_ERR_UNSUPPORTED, "logistic objective: n too large");
+        c->objective = objective; c->sigma = 0.f; c->l2 = l2; c->m = m; c->batch = batch;
+        return GPGA_OK;
+    }
+    return fail(c, GPGA_ERR_INVALID_ARG, "unknown objective");
+}
+
+int32_t gpga_set_grid_cols(gpga_t* c, int64_t cols)
+{
+    if (!c) return fail(nullptr, GPGA_ERR_NOT_READY, "NULL handle");
+    if (cols < 1 || c->n % cols != 0) return fail(c, GPGA_ERR_INVALID_ARG, "cols must divide n");
+    c->grid_cols = cols;
+    return GPGA_OK;
+}
+
+int32_t gpga_set_column_offset(gpga_t* c, int64_t col0)
+{
+    if (!c) return fail(nullptr, GPGA_ERR_NOT_READY, "NULL handle");
+    if (col0 < 0 || (col0 % 4) != 0 || col0 + c->d >= (int64_t(1) << 34))
+        return fail(c, GPGA_ERR_INVALID_ARG, "col0 must be >= 0, a multiple of 4, col0 + d < 2^34");
+    c->col0 = col0;
+    return GPGA_OK;
+}
+
+int64_t gpga_scratch_bytes(const gpga_t* c)
+{
+    if (!c) return 0;
+    return scratch_layout(c).total;
+}
+
+int32_t gpga_bind(gpga_t* c, void* x_a, void* x_b, void* data, const void* labels, void* scratch,
+                  int64_t scratch_bytes)
+{
+    if (!c) return fail(nullptr, GPGA_ERR_NOT_READY, "NULL handle");
+    if (!x_a || !x_b || !data || !scratch) return fail(c, GPGA_ERR_INVALID_ARG, "NULL buffer");
+    if (x_a == x_b) return fail(c, GPGA_ERR_INVALID_ARG, "x_a and x_b must be different buffers");
+    if (!aligned16(x_a) || !aligned16(x_b) || !aligned16(data) || !aligned16(scratch) ||
+        (labels && !aligned16(labels)))
+        return fail(c, GPGA_ERR_INVALID_ARG, "device pointers must be 16-byte aligned");
+    if (c->objective == GPGA_OBJ_LOGISTIC && !labels)
+        return fail(c, GPGA_ERR_INVALID_ARG, "logistic objective needs labels");
+    if (scratch_bytes < scratch_layout(c).total) return fail(c, GPGA_ERR_INVALID_ARG, "scratch too small");
+    c->x[0] = static_cast<float*>(x_a);
+    c->x[1] = static_cast<float*>(x_b);
+    c->data = static_cast<float*>(data);
+    c->labels = static_cast<const float*>(labels);
+    c->scratch = static_cast<char*>(scratch);
+    c->scratch_bytes = scratch_bytes;
+    c->cur = 0;
+    c->k = 0;
+    c->bound = true;
+    return GPGA_OK;
+}
+
+int32_t gpga_init_from_seed(gpga_t* c, int32_t x0_kind, float x0_std, float b_shift, void* stream)
+{
+    int32_t st = check_ready(c);
+    if (st) return st;
+    if (c->objective != GPGA_OBJ_QUADRATIC) return fail(c, GPGA_ERR_UNSUPPORTED, "seeded fill is for the quadratic objective");
+    if (x0_kind < GPGA_X0_ZERO || x0_kind > GPGA_X0_PER_NODE_NORMAL) return fail(c, GPGA_ERR_INVALID_ARG, "unknown x0 kind");
+    if (!std::isfinite(x0_std) || !std::isfinite(b_shift)) return fail(c, GPGA_ERR_INVALID_ARG, "non-finite argument");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool vec = (c->d % 4) == 0;
+    const uint32_t q_base = (uint32_t)(c->col0 >> 2);
+    cudaError_t e = launch_init_b(c->data, c->n, c->d, q_base, b_shift, vec, c->keys, s);
+    if (e != cudaSuccess) return cuda_fail(c, e, "init b launch");
+    e = launch_init_x0(c->x[0], c->n, c->d, q_base, x0_kind, x0_std, vec, c->keys, s);
+    if (e != cudaSuccess) return cuda_fail(c, e, "init x0 launch");
+    c->launches += 2;
+    c->cur = 0;
+    c->k = 0;
+    return GPGA_OK;
+}
+
+int32_t gpga_step(gpga_t* c, int64_t k, void* stream)
+{
+    int32_t st = check_ready(c);
+    if (st) return st;
+    return do_step(c, k, is_global_step(k, c->H), static_cast<cudaStream_t>(stream));
+}
+
+int32_t gpga_run(gpga_t* c, int64_t K, void* stream)
+{
+    int32_t st = check_ready(c);
+    if (st) return st;
+    if (K < 0) return fail(c, GPGA_ERR_INVALID_ARG, "K must be >= 0");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int64_t k0 = c->k;
+    for (int64_t k = k0; k < k0 + K; ++k) {
+        st = do_step(c, k, is_global_step(k, c->H), s);
+        if (st) return st;
+    }
+    return GPGA_OK;
+}
+
+int32_t gpga_run_host(gpga_t* c, const float* x0_host, const float* data_host, int64_t K,
+                      float* x_out_host, void* stream)
+{
+    int32_t st = check_ready(c);
+    if (st) return st;
+    if (c->objective != GPGA_OBJ_QUADRATIC) return fail(c, GPGA_ERR_UNSUPPORTED, "host entry is for the quadratic objective");
+    if (!x0_host || !data_host || !x_out_host) return fail(c, GPGA_ERR_INVALID_ARG, "NULL host buffer");
+    if (K < 0) return fail(c, GPGA_ERR_INVALID_ARG, "K must be >= 0");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t bytes = (size_t)c->n * (size_t)c->d * sizeof(float);
+    cudaError_t e = cudaMemcpyAsync(c->x[0], x0_host, bytes, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(c, e, "x0 upload");
+    e = cudaMemcpyAsync(c->data, data_host, bytes, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(c, e, "data upload");
+    c->cur = 0;
+    c->k = 0;
+    for (int64_t k = 0; k < K; ++k) {
+        st = do_step(c, k, is_global_step(k, c->H), s);
+        if (st) return st;
+    }
+    e = cudaMemcpyAsync(x_out_host, c->x[c->cur], bytes, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail(c, e, "result download");
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(c, e, "stream synchronize");
+    return GPGA_OK;
+}
+
+int32_t gpga_consensus_distance(gpga_t* c, void* stream, double* out_host)
+{
+    int32_t st = check_ready(c);
+    if (st) return st;
+    if (!out_host) return fail(c, GPGA_ERR_INVALID_ARG, "out_host is NULL");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const ScratchLayout L = scratch_layout(c);
+    double* partials = reinterpret_cast<double*>(c->scratch + L.partials_off);
+    double* result = reinterpret_cast<double*>(c->scratch + L.result_off);
+    cudaError_t e = launch_consensus(c->x[c->cur], c->n, c->d, (c->d % 4) == 0, partials, result, s);
+    c->launches += 2;
+    if (e != cudaSuccess) return cuda_fail(c, e, "consensus launch");
+    return read_double(c, result, s, out_host);
+}
+
+int32_t gpga_mean_loss(gpga_t* c, void* stream, double* out_host)
+{
+    int32_t st = check_ready(c);
+    if (st) return st;
+    if (!out_host) return fail(c, GPGA_ERR_INVALID_ARG, "out_host is NULL");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    double* result = nullptr;
+    st = mean_loss_async(c, s, &result);
+    if (st) return st;
+    return read_double(c, result, s, out_host);
+}
+
+int32_t gpga_run_adaptive(gpga_t* c, int64_t K, int64_t H_init, int64_t warmup_iters, void* stream,
+                          int64_t* periods_host, int64_t max_periods, int64_t* num_periods_host)
+{
+    int32_t st = check_ready(c);
+    if (st) return st;
+    if (K < 0 || H_init < 1 || warmup_iters < 0 || max_periods < 0)
+        return fail(c, GPGA_ERR_INVALID_ARG, "need K >= 0, H_init >= 1, warmup_iters >= 0");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int64_t H = H_init, C = 0, periods = 0;
+    double F_init = 0.0;
+    const int64_t k0 = c->k;
+    for (int64_t k = k0; k < k0 + K; ++k) {
+        ++C;
+        const bool global = (C == H);
+        double F = 0.0;
+        if (global) {   // loss of this iteration, taken at x^(k) as Algorithm 2 does
+            double* result = nullptr;
+            st = mean_loss_async(c, s, &result);
+            if (st) return st;
+            st = read_double(c, result, s, &F);
+            if (st) return st;
+        }
+        st = do_step(c, k, global, s);
+        if (st) return st;
+        if (global) {
+            if (periods_host && periods < max_periods) periods_host[periods] = H;
+            ++periods;
+            C = 0;
+            if (k < warmup_iters) {
+                F_init = 0.5 * (F_init + F);
+            } else if (F > 0.0 && std::isfinite(F_init / F)) {
+                const double h = std::ceil(F_init / F * (double)H_init);
+                H = h < 1.0 ? 1 : (h > 9.0e15 ? (int64_t)9.0e15 : (int64_t)h);
+            }
+        }
+    }
+    if (num_periods_host) *num_periods_host = periods;
+    return GPGA_OK;
+}
+
+int32_t gpga_get_x(const gpga_t* c, void** x_cur)
+{
+    if (!c || !x_cur) return GPGA_ERR_NOT_READY;
+    if (!c->bound) return GPGA_ERR_NOT_READY;
+    *x_cur = c->x[c->cur];
+    return GPGA_OK;
+}
+
+int32_t gpga_get_k(const gpga_t* c, int64_t* k)
+{
+    if (!c || !k) return GPGA_ERR_NOT_READY;
+    *k = c->k;
+    return GPGA_OK;
+}
+
+int32_t gpga_set_k(gpga_t* c, int64_t k)
+{
+    if (!c) return fail(nullptr, GPGA_ERR_NOT_READY, "NULL handle");
+    if (k < 0 || k >= (int64_t(1) << 32)) return fail(c, GPGA_ERR_INVALID_ARG, "k must be in [0, 2^32)");
+    c->k = k;
+    return GPGA_OK;
+}
+
+int32_t gpga_set_gamma(gpga_t* c, float gamma)
+{
+    if (!c) return fail(nullptr, GPGA_ERR_NOT_READY, "NULL handle");
+    if (!std::isfinite(gamma) || gamma < 0.f) return fail(c, GPGA_ERR_INVALID_ARG, "gamma must be finite and >= 0");
+    c->gamma = gamma;
+    return GPGA_OK;
+}
+
+int32_t gpga_set_period(gpga_t* c, int64_t H)
+{
+    if (!c) return fail(nullptr, GPGA_ERR_NOT_READY, "NULL handle");
+    if (H < 0) return fail(c, GPGA_ERR_INVALID_ARG, "H must be >= 0");
+    c->H = H;
+    return GPGA_OK;
+}
+
+int64_t gpga_launch_count(const gpga_t* c) { return c ? c->launches : 0; }
+
+const char* gpga_last_error(const gpga_t* c) { return c ? c->err.c_str() : g_create_error.c_str(); }
+
+int32_t gpga_destroy(gpga_t* c)
+{
+    delete c;
+    return GPGA_OK;
+}
+
+int32_t gpga_philox_words(const uint32_t* ctr_dev, uint32_t key0, uint32_t key1, int64_t count,
+                          uint32_t* out_dev, void* stream)
+{
+    if (count < 0 || (count > 0 && (!ctr_dev || !out_dev))) return fail(nullptr, GPGA_ERR_INVALID_ARG, "bad argument");
+    cudaError_t e = launch_philox_words(ctr_dev, make_philox_keys(key0, key1), count, out_dev,
+                                        static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? GPGA_OK : fail(nullptr, GPGA_ERR_CUDA, cudaGetErrorString(e));
+}
+
+int32_t gpga_box_muller_words(const uint32_t* a_dev, const uint32_t* b_dev, int64_t count,
+                              float* z_dev, void* stream)
+{
+    if (count < 0 || (count > 0 && (!a_dev || !b_dev || !z_dev))) return fail(nullptr, GPGA_ERR_INVALID_ARG, "bad argument");
+    cudaError_t e = launch_box_muller_words(a_dev, b_dev, count, z_dev, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? GPGA_OK : fail(nullptr, GPGA_ERR_CUDA, cudaGetErrorString(e));
+}
+
+int32_t gpga_normal_fill(uint64_t seed, uint32_t stream_id, uint32_t k, uint32_t i, uint32_t q0,
+                         int64_t count, float* out_dev, void* stream)
+{
+    if (count < 0 || (count > 0 && !out_dev)) return fail(nullptr, GPGA_ERR_INVALID_ARG, "bad argument");
+    cudaError_t e = launch_normal_fill(make_philox_keys((uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32)),
+                                       stream_id, k, i, q0, count, out_dev, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? GPGA_OK : fail(nullptr, GPGA_ERR_CUDA, cudaGetErrorString(e));
+}
+
+}  // extern "C"

@@ -1,0 +1,390 @@
+// Fused Gossip-PGA kernels for sm_100a.
+//
+// Every step kernel gives one thread a group of four adjacent columns and streams
+// it down the n rows (nodes): each element of X and of b is read once, the
+// half-step Y = X - gamma G (Algorithm 1's local update) lives only in registers,
+// the noise is generated in registers, and each element of X^(k+1) is written once:
+// 12 bytes of HBM traffic per node-parameter update.  The mixing of Algorithm 1
+// (gossip step or global average) acts along the rows of one column group, so no
+// thread ever needs another thread's data.
+#include "gpga_kernels.cuh"
+
+namespace gpga {
+
+constexpr int kBlock = 256;
+
+__device__ __forceinline__ float4 add4(float4 a, float4 b)
+{
+    return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
+}
+__device__ __forceinline__ float4 scale4(float4 a, float s)
+{
+    return make_float4(a.x * s, a.y * s, a.z * s, a.w * s);
+}
+
+// x^(k+1/2) for node i, column group q (Algorithm 1: gradient, then the local update).
+template <int MODE, bool VEC>
+__device__ __forceinline__ float4 half_step(const StepParams& p, long long i, long long q)
+{
+    const long long j0 = q * 4;
+    const float4 x = load4<VEC>(p.x + i * p.d, j0, p.d);
+    const float4 b = load4<VEC>(p.b + i * p.d, j0, p.d);
+    float4 g;
+    if (MODE == GRAD_BUFFER) {
+        g = b;
+    } else {
+        g = make_float4(x.x - b.x, x.y - b.y, x.z - b.z, x.w - b.w);
+        if (MODE == GRAD_QUAD_NOISE) {
+            const float4 z = normal4(p.q_base + (uint32_t)q, (uint32_t)i, p.k, 0u, p.keys);
+            g.x = fmaf(p.sigma, z.x, g.x);
+            g.y = fmaf(p.sigma, z.y, g.y);
+            g.z = fmaf(p.sigma, z.z, g.z);
+            g.w = fmaf(p.sigma, z.w, g.w);
+        }
+    }
+    return make_float4(fmaf(-p.gamma, g.x, x.x), fmaf(-p.gamma, g.y, x.y), fmaf(-p.gamma, g.z, x.z),
+                       fmaf(-p.gamma, g.w, x.w));
+}
+
+// ---------------------------------------------------------------------------
+// Ring: x_i^(k+1) = (y_{i-1} + y_i + y_{i+1}) / 3, indices mod n.  A three-row
+// window slides down the rows; rows 0 and 1 are kept for the wrap-around.
+// ---------------------------------------------------------------------------
+template <int MODE, bool VEC>
+__global__ void __launch_bounds__(kBlock) step_ring_kernel(const StepParams p)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.Q) return;
+    const long long j0 = q * 4;
+    const float third = 0.333333343f;
+    if (p.n <= 2) {
+        const float4 y0 = half_step<MODE, VEC>(p, 0, q);
+        if (p.n == 1) {
+            store4<VEC>(p.out, j0, p.d, scale4(add4(add4(y0, y0), y0), third));
+            return;
+        }
+        const float4 y1 = half_step<MODE, VEC>(p, 1, q);
+        store4<VEC>(p.out, j0, p.d, scale4(add4(add4(y1, y0), y1), third));
+        store4<VEC>(p.out + p.d, j0, p.d, scale4(add4(add4(y0, y1), y0), third));
+        return;
+    }
+    const float4 y0 = half_step<MODE, VEC>(p, 0, q);
+    const float4 y1 = half_step<MODE, VEC>(p, 1, q);
+    float4 a = y0, b = y1;
+#pragma unroll 4
+    for (long long i = 2; i < p.n; ++i) {
+        const float4 c = half_step<MODE, VEC>(p, i, q);
+        store4<VEC>(p.out + (i - 1) * p.d, j0, p.d, scale4(add4(add4(a, b), c), third));
+        a = b;
+        b = c;
+    }
+    store4<VEC>(p.out + (p.n - 1) * p.d, j0, p.d, scale4(add4(add4(a, b), y0), third));
+    store4<VEC>(p.out, j0, p.d, scale4(add4(add4(b, y0), y1), third));
+}
+
+// ---------------------------------------------------------------------------
+// One-peer exponential graph: x_i^(k+1) = (y_i + y_{(i+h) mod n}) / 2, h = 2^t.
+// i -> i + h splits the nodes into h cycles of length n/h; walking a cycle needs
+// only the previous row and the cycle's first row, so each row is read (and its
+// noise generated) once.  Step t of the flattened walk visits row
+// (t / L) + (t mod L) * h with L = n / h.
+// ---------------------------------------------------------------------------
+template <int MODE, bool VEC>
+__global__ void __launch_bounds__(kBlock) step_exp_kernel(const StepParams p)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.Q) return;
+    const long long j0 = q * 4;
+    const long long hop = 1LL << p.hop_log2;
+    const long long lmask = (1LL << p.len_log2) - 1;
+    float4 first = make_float4(0.f, 0.f, 0.f, 0.f), prev = first;
+#pragma unroll 4
+    for (long long t = 0; t < p.n; ++t) {
+        const long long s = t & lmask;
+        const long long row = (t >> p.len_log2) + (s << p.hop_log2);
+        const float4 cur = half_step<MODE, VEC>(p, row, q);
+        if (s == 0)
+            first = cur;
+        else
+            store4<VEC>(p.out + (row - hop) * p.d, j0, p.d, scale4(add4(prev, cur), 0.5f));
+        if (s == lmask) store4<VEC>(p.out + row * p.d, j0, p.d, scale4(add4(cur, first), 0.5f));
+        prev = cur;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Global average: m_j = (1/n) sum_i y_ij, written to every row.  The column sum is
+// accumulated in fp64 (exact for practical n), rounded once.
+// ---------------------------------------------------------------------------
+template <int MODE, bool VEC>
+__global__ void __launch_bounds__(kBlock) step_global_kernel(const StepParams p)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.Q) return;
+    const long long j0 = q * 4;
+    double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+#pragma unroll 4
+    for (long long i = 0; i < p.n; ++i) {
+        const float4 y = half_step<MODE, VEC>(p, i, q);
+        s0 += (double)y.x;
+        s1 += (double)y.y;
+        s2 += (double)y.z;
+        s3 += (double)y.w;
+    }
+    const double inv = (double)p.n;
+    const float4 m = make_float4((float)(s0 / inv), (float)(s1 / inv), (float)(s2 / inv),
+                                 (float)(s3 / inv));
+#pragma unroll 4
+    for (long long i = 0; i < p.n; ++i) store4<VEC>(p.out + i * p.d, j0, p.d, m);
+}
+
+static inline unsigned grid_for(long long Q, int block) { return (unsigned)((Q + block - 1) / block); }
+
+// Small problems: narrower blocks spread the column groups over more SMs.
+static inline int block_for(long long Q) { return (Q >= 148LL * 4 * kBlock) ? kBlock : 64; }
+
+#define GPGA_DISPATCH(kernel, p, mode, vec, s)                                             \
+    do {                                                                                   \
+        const int blk = block_for((p).Q);                                                  \
+        const unsigned grd = grid_for((p).Q, blk);                                         \
+        if (vec) {                                                                         \
+            if (mode == GRAD_QUAD) kernel<GRAD_QUAD, true><<<grd, blk, 0, s>>>(p);         \
+            else if (mode == GRAD_QUAD_NOISE) kernel<GRAD_QUAD_NOISE, true><<<grd, blk, 0, s>>>(p); \
+            else kernel<GRAD_BUFFER, true><<<grd, blk, 0, s>>>(p);                          \
+        } else {                                                                           \
+            if (mode == GRAD_QUAD) kernel<GRAD_QUAD, false><<<grd, blk, 0, s>>>(p);        \
+            else if (mode == GRAD_QUAD_NOISE) kernel<GRAD_QUAD_NOISE, false><<<grd, blk, 0, s>>>(p); \
+            else kernel<GRAD_BUFFER, false><<<grd, blk, 0, s>>>(p);                         \
+        }                                                                                  \
+        return cudaGetLastError();                                                         \
+    } while (0)
+
+cudaError_t launch_step_ring(const StepParams& p, int mode, bool vec, cudaStream_t s)
+{
+    GPGA_DISPATCH(step_ring_kernel, p, mode, vec, s);
+}
+cudaError_t launch_step_exp(const StepParams& p, int mode, bool vec, cudaStream_t s)
+{
+    GPGA_DISPATCH(step_exp_kernel, p, mode, vec, s);
+}
+cudaError_t launch_step_global(const StepParams& p, int mode, bool vec, cudaStream_t s)
+{
+    GPGA_DISPATCH(step_global_kernel, p, mode, vec, s);
+}
+
+// ---------------------------------------------------------------------------
+// Consensus distance sum_j sum_i (x_ij - xbar_j)^2.  One pass over X: with
+// e_i = x_i - x_0 (exact in fp64), sum_i (x_i - xbar)^2 = sum e_i^2 - (sum e_i)^2 / n;
+// shifting by row 0 keeps the subtraction benign when the rows are nearly equal.
+// ---------------------------------------------------------------------------
+constexpr int kReduceBlock = 256;
+
+int consensus_blocks(long long Q)
+{
+    long long b = (Q + kReduceBlock - 1) / kReduceBlock;
+    if (b > kMaxReduceBlocks) b = kMaxReduceBlocks;
+    if (b < 1) b = 1;
+    return (int)b;
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(kReduceBlock) consensus_kernel(const float* __restrict__ x,
+                                                                 long long n, long long d,
+                                                                 long long Q,
+                                                                 double* __restrict__ partials)
+{
+    double acc = 0.0;
+    for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < Q;
+         q += (long long)gridDim.x * blockDim.x) {
+        const long long j0 = q * 4;
+        const float4 r0 = load4<VEC>(x, j0, d);
+        double s1[4] = {0, 0, 0, 0}, s2[4] = {0, 0, 0, 0};
+#pragma unroll 4
+        for (long long i = 1; i < n; ++i) {
+            const float4 v = load4<VEC>(x + i * d, j0, d);
+            const double e0 = (double)v.x - (double)r0.x, e1 = (double)v.y - (double)r0.y;
+            const double e2 = (double)v.z - (double)r0.z, e3 = (double)v.w - (double)r0.w;
+            s1[0] += e0; s2[0] = fma(e0, e0, s2[0]);
+            s1[1] += e1; s2[1] = fma(e1, e1, s2[1]);
+            s1[2] += e2; s2[2] = fma(e2, e2, s2[2]);
+            s1[3] += e3; s2[3] = fma(e3, e3, s2[3]);
+        }
+        const double inv_n = 1.0 / (double)n;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            // columns past d loaded as zeros in every row: they contribute exactly 0
+            const double v = s2[e] - s1[e] * s1[e] * inv_n;
+            acc += v > 0.0 ? v : 0.0;
+        }
+    }
+    acc = block_sum(acc);
+    if (threadIdx.x == 0) partials[blockIdx.x] = acc;
+}
+
+__global__ void final_sum_kernel(const double* __restrict__ partials, int count, double scale,
+                                 double* __restrict__ result)
+{
+    // one warp, fixed order: lane l adds partials l, l+32, ...; then a shuffle tree
+    double v = 0.0;
+    for (int t = threadIdx.x; t < count; t += 32) v += partials[t];
+    v = warp_sum(v);
+    if (threadIdx.x == 0) *result = v * scale;
+}
+
+cudaError_t launch_consensus(const float* x, long long n, long long d, bool vec, double* partials,
+                             double* result, cudaStream_t s)
+{
+    const long long Q = (d + 3) / 4;
+    const int blocks = consensus_blocks(Q);
+    if (vec)
+        consensus_kernel<true><<<blocks, kReduceBlock, 0, s>>>(x, n, d, Q, partials);
+    else
+        consensus_kernel<false><<<blocks, kReduceBlock, 0, s>>>(x, n, d, Q, partials);
+    final_sum_kernel<<<1, 32, 0, s>>>(partials, blocks, 1.0, result);
+    return cudaGetLastError();
+}
+
+// (1/n) sum_i 1/2 ||x_i - b_i||^2 over all elements.
+__global__ void __launch_bounds__(kReduceBlock) quadratic_loss_kernel(const float* __restrict__ x,
+                                                                      const float* __restrict__ b,
+                                                                      long long total,
+                                                                      double* __restrict__ partials)
+{
+    double acc = 0.0;
+    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total;
+         e += (long long)gridDim.x * blockDim.x) {
+        const double r = (double)__ldcs(x + e) - (double)__ldcs(b + e);
+        acc = fma(r, r, acc);
+    }
+    acc = block_sum(acc);
+    if (threadIdx.x == 0) partials[blockIdx.x] = acc;
+}
+
+cudaError_t launch_quadratic_loss(const float* x, const float* b, long long n, long long d,
+                                  double* partials, double* result, cudaStream_t s)
+{
+    const long long total = n * d;
+    const int blocks = consensus_blocks(total);
+    quadratic_loss_kernel<<<blocks, kReduceBlock, 0, s>>>(x, b, total, partials);
+    final_sum_kernel<<<1, 32, 0, s>>>(partials, blocks, 0.5 / (double)n, result);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
+// Seeded fills
+// ---------------------------------------------------------------------------
+template <bool VEC>
+__global__ void __launch_bounds__(kBlock) init_b_kernel(float* __restrict__ b, long long n,
+                                                        long long d, long long Q, uint32_t q_base,
+                                                        float shift, const PhiloxKeys keys)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= Q) return;
+    for (long long i = 0; i < n; ++i) {
+        float4 z = normal4(q_base + (uint32_t)q, (uint32_t)i, 0u, 1u, keys);
+        if (shift != 0.0f) {
+            const float s = normal4(0u, (uint32_t)i, 0u, 3u, keys).x;
+            z.x = fmaf(shift, s, z.x);
+            z.y = fmaf(shift, s, z.y);
+            z.z = fmaf(shift, s, z.z);
+            z.w = fmaf(shift, s, z.w);
+        }
+        store4<VEC>(b + i * d, q * 4, d, z);
+    }
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(kBlock) init_x0_kernel(float* __restrict__ x, long long n,
+                                                         long long d, long long Q, uint32_t q_base,
+                                                         int kind, float std, const PhiloxKeys keys)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= Q) return;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (kind == 1) v = scale4(normal4(q_base + (uint32_t)q, 0u, 0u, 2u, keys), std);
+    for (long long i = 0; i < n; ++i) {
+        if (kind == 2) v = scale4(normal4(q_base + (uint32_t)q, (uint32_t)i, 0u, 2u, keys), std);
+        store4<VEC>(x + i * d, q * 4, d, v);
+    }
+}
+
+cudaError_t launch_init_b(float* b, long long n, long long d, uint32_t q_base, float shift, bool vec,
+                          const PhiloxKeys& keys, cudaStream_t s)
+{
+    const long long Q = (d + 3) / 4;
+    if (vec)
+        init_b_kernel<true><<<grid_for(Q, kBlock), kBlock, 0, s>>>(b, n, d, Q, q_base, shift, keys);
+    else
+        init_b_kernel<false><<<grid_for(Q, kBlock), kBlock, 0, s>>>(b, n, d, Q, q_base, shift, keys);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_init_x0(float* x, long long n, long long d, uint32_t q_base, int kind, float std,
+                           bool vec, const PhiloxKeys& keys, cudaStream_t s)
+{
+    const long long Q = (d + 3) / 4;
+    if (vec)
+        init_x0_kernel<true><<<grid_for(Q, kBlock), kBlock, 0, s>>>(x, n, d, Q, q_base, kind, std, keys);
+    else
+        init_x0_kernel<false><<<grid_for(Q, kBlock), kBlock, 0, s>>>(x, n, d, Q, q_base, kind, std, keys);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
+// Generator surface
+// ---------------------------------------------------------------------------
+__global__ void philox_words_kernel(const uint32_t* __restrict__ ctr, const PhiloxKeys keys,
+                                    long long count, uint32_t* __restrict__ out)
+{
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= count) return;
+    const uint4 w = philox4x32_10(ctr[4 * t], ctr[4 * t + 1], ctr[4 * t + 2], ctr[4 * t + 3], keys);
+    out[4 * t] = w.x;
+    out[4 * t + 1] = w.y;
+    out[4 * t + 2] = w.z;
+    out[4 * t + 3] = w.w;
+}
+
+__global__ void box_muller_words_kernel(const uint32_t* __restrict__ a, const uint32_t* __restrict__ b,
+                                        long long count, float* __restrict__ z)
+{
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= count) return;
+    const float2 v = box_muller(a[t], b[t]);
+    z[2 * t] = v.x;
+    z[2 * t + 1] = v.y;
+}
+
+__global__ void normal_fill_kernel(const PhiloxKeys keys, uint32_t stream_id, uint32_t k, uint32_t i,
+                                   uint32_t q0, long long count, float* __restrict__ out)
+{
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= count) return;
+    const float4 z = normal4(q0 + (uint32_t)t, i, k, stream_id, keys);
+    out[4 * t] = z.x;
+    out[4 * t + 1] = z.y;
+    out[4 * t + 2] = z.z;
+    out[4 * t + 3] = z.w;
+}
+
+cudaError_t launch_philox_words(const uint32_t* ctr, PhiloxKeys keys, long long count, uint32_t* out,
+                                cudaStream_t s)
+{
+    if (count > 0) philox_words_kernel<<<grid_for(count, kBlock), kBlock, 0, s>>>(ctr, keys, count, out);
+    return cudaGetLastError();
+}
+cudaError_t launch_box_muller_words(const uint32_t* a, const uint32_t* b, long long count, float* z,
+                                    cudaStream_t s)
+{
+    if (count > 0) box_muller_words_kernel<<<grid_for(count, kBlock), kBlock, 0, s>>>(a, b, count, z);
+    return cudaGetLastError();
+}
+cudaError_t launch_normal_fill(PhiloxKeys keys, uint32_t stream_id, uint32_t k, uint32_t i,
+                               uint32_t q0, long long count, float* out, cudaStream_t s)
+{
+    if (count > 0)
+        normal_fill_kernel<<<grid_for(count, kBlock), kBlock, 0, s>>>(keys, stream_id, k, i, q0, count, out);
+    return cudaGetLastError();
+}
+
+}  // namespace gpga

@@ -1,0 +1,30 @@
+// Launchers for the per-node logistic-regression gradient and mini-batch loss.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gpga_device.cuh"
+
+namespace gpga {
+
+constexpr int kChunkRows = 32;   // batch rows per block
+
+struct LogregParams {
+    const float* A;   // n x m x d
+    const float* y;   // n x m, +-1
+    const float* x;   // n x d, current state
+    float* partial;   // chunks x n x d
+    float* G;         // n x d
+    long long n, d, m, batch;
+    uint32_t k;
+    float l2;
+    PhiloxKeys keys;
+};
+
+int logreg_chunks(long long batch);
+// Two launches: chunk partials, then the fixed-order sum into G (adds l2 x).
+cudaError_t launch_logreg_grad(const LogregParams& p, cudaStream_t s);
+// Two launches: per-node mini-batch loss (n doubles), then their mean into *result.
+cudaError_t launch_logreg_loss(const LogregParams& p, double* node_loss, double* result, cudaStream_t s);
+
+}  // namespace gpga

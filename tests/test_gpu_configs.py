@@ -1,0 +1,188 @@
+"""Configuration-level parity: the benchmark configurations run through the C ABI and
+compared with the oracle -- fully where the oracle finishes in seconds, on sampled column
+blocks (columns evolve independently under the quadratic objective) at full size."""
+import numpy as np
+import pytest
+
+import paper_2105_09080_b200 as pkg
+from oracle import gpga_oracle as o
+from paper_2105_09080_b200.inputs import logistic_inputs, quadratic_inputs
+from test_gpu_parity import TOL_RUN, TOL_STEP, TOPO, close, make_quadratic
+
+pytestmark = pytest.mark.gpu
+
+SEED = 20210509
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def test_config_1_ring_h4_full_run():
+    # n=8, d=65536, ring, H=4, gamma=0.1, sigma=0.1, K=32, x0 = 0
+    n, d, H, gamma, sigma, K = 8, 65536, 4, 0.1, 0.1, 32
+    X0, B = quadratic_inputs(n, d, SEED)
+    g, p = make_quadratic(n, d, "ring", H, gamma, SEED, sigma, X0, B)
+    want = X0
+    for k in range(K):
+        g.step(k)
+        want = o.step(p, want, k)
+        ok, worst = close(g.get_x().cpu().numpy(), want, TOL_STEP if k == 0 else TOL_RUN)
+        assert ok, (k, worst)
+        if (k + 1) % H == 0:
+            assert g.consensus_distance() == 0.0        # rows identical after a global average
+        elif k % 5 == 0:
+            xi = o.consensus_distance(want)
+            assert abs(g.consensus_distance() - xi) <= 1e-5 * xi + n * d * (2.0**-22 * 8) ** 2
+    # the run ends on a global average: K = 32, H = 4
+    got = g.get_x().cpu().numpy()
+    assert np.all(got == got[0])
+
+
+def test_config_2_exp_h8_full_run():
+    # n=32, d=2^20, one-peer exponential, H=8, gamma=0.05, sigma=0.1, K=64
+    n, d, H, gamma, sigma, K = 32, 1 << 20, 8, 0.05, 0.1, 64
+    X0, B = quadratic_inputs(n, d, SEED + 1)
+    g, p = make_quadratic(n, d, "exp", H, gamma, SEED, sigma, X0, B)
+    g.step(0)
+    want1 = o.step(p, X0, 0)
+    ok, worst = close(g.get_x().cpu().numpy(), want1, TOL_STEP)
+    assert ok, worst
+    g.run(K - 1)
+    want = o.run(p, want1, 1, K - 1)
+    ok, worst = close(g.get_x().cpu().numpy(), want, TOL_RUN)
+    assert ok, worst
+    xi = o.consensus_distance(want)
+    assert abs(g.consensus_distance() - xi) <= 1e-5 * xi + n * d * (2.0**-22 * 8) ** 2
+
+
+def test_config_2_exact_consensus_after_log2n_mixing_steps():
+    # gamma = 0, sigma = 0, random per-node X0: five hops 1,2,4,8,16 give the exact average
+    n, d = 32, 1 << 20
+    X0, B = quadratic_inputs(n, d, SEED + 2, x0="per_node")
+    g, p = make_quadratic(n, d, "exp", 0, 0.0, SEED, 0.0, X0, B)
+    xi0 = g.consensus_distance()
+    assert abs(xi0 - o.consensus_distance(X0)) <= 1e-5 * xi0
+    g.run(4)
+    assert g.consensus_distance() > 1e-3 * xi0            # not yet
+    g.run(1)
+    assert g.consensus_distance() <= 1e-12 * xi0          # float32 storage: exact up to rounding
+    got = g.get_x().cpu().numpy()
+    mean = X0.astype(np.float64).mean(0)
+    assert np.abs(got - mean[None, :]).max() <= 1e-6
+
+
+def test_init_from_seed_matches_oracle_streams():
+    torch = _torch()
+    n, d, c0 = 6, 4104, 8192
+    for kind, okind, std, shift in ((pkg.GPGA_X0_ZERO, o.X0_ZERO, 1.0, 0.0),
+                                    (pkg.GPGA_X0_SHARED_NORMAL, o.X0_SHARED_NORMAL, 0.1, 0.5),
+                                    (pkg.GPGA_X0_PER_NODE_NORMAL, o.X0_PER_NODE_NORMAL, 1.0, 0.0)):
+        g = pkg.Gpga(n, d, pkg.GPGA_TOPO_RING, 0, 0.1, SEED)
+        g.set_column_offset(c0)
+        xa, xb, b = g.allocate()
+        g.init_from_seed(kind, std, shift)
+        # seeded inputs are N(0,1)-scale numbers; the fast device Box-Muller is within 2.5e-5
+        assert np.abs(b.cpu().numpy() - o.init_b(n, d, SEED, shift, c0)).max() <= 3e-5
+        assert np.abs(xa.cpu().numpy() - o.init_x0(n, d, SEED, okind, std, c0)).max() <= 3e-5 * std
+        if kind == pkg.GPGA_X0_SHARED_NORMAL:
+            x = xa.cpu().numpy()
+            assert np.all(x == x[0])
+        g.close()
+    # ragged d (scalar path)
+    g = pkg.Gpga(3, 1031, pkg.GPGA_TOPO_RING, 0, 0.1, SEED)
+    xa, xb, b = g.allocate()
+    g.init_from_seed(pkg.GPGA_X0_PER_NODE_NORMAL, 2.0, 0.25)
+    assert np.abs(b.cpu().numpy() - o.init_b(3, 1031, SEED, 0.25)).max() <= 3e-5
+    assert np.abs(xa.cpu().numpy() - o.init_x0(3, 1031, SEED, o.X0_PER_NODE_NORMAL, 2.0)).max() <= 6e-5
+
+
+def test_run_host_equals_device_run():
+    torch = _torch()
+    n, d, K = 8, 65536, 6
+    X0, B = quadratic_inputs(n, d, SEED + 3)
+    g, _ = make_quadratic(n, d, "ring", 4, 0.1, SEED, 0.1, X0, B)
+    g.run(K)
+    dev = g.get_x().cpu().numpy()
+    g2, _ = make_quadratic(n, d, "ring", 4, 0.1, SEED, 0.1, np.zeros_like(X0), np.zeros_like(B))
+    out = torch.empty((n, d), dtype=torch.float32).pin_memory()
+    g2.run_host(torch.from_numpy(X0).pin_memory(), torch.from_numpy(B).pin_memory(), K, out)
+    assert np.array_equal(out.numpy(), dev)
+
+
+# ------------------------------------------------------------------ logistic objective
+def _make_logistic(n, m, d, batch, topo, H, gamma, l2, seed, A, y, X0):
+    torch = _torch()
+    g = pkg.Gpga(n, d, TOPO[topo][0], H, gamma, seed)
+    g.set_objective(pkg.GPGA_OBJ_LOGISTIC, l2=l2, m=m, batch=batch)
+    xa = torch.from_numpy(X0).cuda()
+    g.bind(xa, torch.empty_like(xa), torch.from_numpy(A).cuda(), torch.from_numpy(y).cuda())
+    p = o.Problem(TOPO[topo][1], H, gamma, seed, objective="logistic", data=A, labels=y, l2=l2,
+                  batch=batch)
+    return g, p
+
+
+@pytest.mark.parametrize("topo", ["ring", "exp"])
+@pytest.mark.parametrize("n,m,d,batch", [(4, 64, 32, 8), (8, 256, 1024, 128), (2, 100, 260, 50)])
+def test_logistic_steps(topo, n, m, d, batch):
+    A, y = logistic_inputs(n, m, d, SEED + n)
+    rng = np.random.default_rng(0)
+    X0 = (0.1 * rng.standard_normal((n, d))).astype(np.float32)
+    g, p = _make_logistic(n, m, d, batch, topo, 4, 0.1, 1e-4, SEED, A, y, X0)
+    g.step(0)
+    want = o.step(p, X0, 0)
+    ok, worst = close(g.get_x().cpu().numpy(), want, TOL_STEP)
+    assert ok, worst
+    g.run(11)
+    want = o.run(p, want, 1, 11)
+    ok, worst = close(g.get_x().cpu().numpy(), want, TOL_RUN)
+    assert ok, worst
+    # mini-batch loss of the next iteration's batch, at each node's own iterate
+    k = g.get_k()
+    f = np.mean([o.logistic_loss(A[i][o.batch_indices(SEED, k, i, batch, m)],
+                                 y[i][o.batch_indices(SEED, k, i, batch, m)], want[i], 1e-4)
+                 for i in range(n)])
+    assert abs(g.mean_loss() - f) <= 1e-4 * abs(f)
+
+
+def test_config_5_logistic_reduced_iterations():
+    # n=64, m=4096, d=1024, batch 128, l2=1e-4, gamma=0.1; the oracle covers the first 40 of
+    # the 2000 iterations in seconds (ring, H=4 and exp, H=16)
+    n, m, d, batch = 64, 4096, 1024, 128
+    A, y = logistic_inputs(n, m, d, SEED)
+    X0 = np.zeros((n, d), dtype=np.float32)
+    for topo, H in (("ring", 4), ("exp", 16)):
+        g, p = _make_logistic(n, m, d, batch, topo, H, 0.1, 1e-4, SEED, A, y, X0)
+        g.run(40)
+        want = o.run(p, X0, 0, 40)
+        ok, worst = close(g.get_x().cpu().numpy(), want, TOL_RUN)
+        assert ok, (topo, worst)
+        xi = o.consensus_distance(want)
+        assert abs(g.consensus_distance() - xi) <= 1e-4 * xi + 1e-12
+        g.close()
+
+
+# ------------------------------------------------------------------ Gossip-AGA
+def test_adaptive_period_sequence_matches_oracle_driven_loop():
+    n, d, K, H_init, warm = 8, 4096, 60, 2, 6
+    X0, B = quadratic_inputs(n, d, SEED + 5, x0="shared", x0_std=3.0)
+    g, p = make_quadratic(n, d, "ring", 0, 0.1, SEED, 0.05, X0, B)
+    periods = g.run_adaptive(K, H_init, warm)
+    # the same loop driven by the oracle (Algorithm 2)
+    X, H, C, F_init, want_periods = X0, H_init, 0, 0.0, []
+    for k in range(K):
+        C += 1
+        glob = C == H
+        F = o.quadratic_mean_loss(X, B) if glob else 0.0
+        p.H = 1 if glob else 0
+        X = o.step(p, X, k)
+        if glob:
+            want_periods.append(H)
+            C = 0
+            F_init, H = o.aga_update(k, warm, H_init, F, F_init, H)
+    assert periods == want_periods
+    assert len(set(periods)) > 1 and periods[-1] > periods[0]      # the period grows as the loss falls
+    ok, worst = close(g.get_x().cpu().numpy(), X, TOL_RUN)
+    assert ok, worst
+    assert abs(g.mean_loss() - o.quadratic_mean_loss(X, B)) <= 1e-5 * o.quadratic_mean_loss(X, B)

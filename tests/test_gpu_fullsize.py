@@ -1,0 +1,119 @@
+"""Full-size configurations (ResNet-50- and BERT-Large-sized parameter counts) in the
+launch configuration the benchmark times, checked on sampled column blocks.
+
+Under the quadratic objective W acts on rows only and the gradient and noise are
+element-wise, so every column evolves independently: the oracle run on a block of columns
+(keyed by the block's global column offset) gives exactly the values a full run would.
+Both sides fill b and X0 from the seed by their own implementation of the same streams;
+nothing computed on the GPU is fed to the oracle."""
+import numpy as np
+import pytest
+
+import paper_2105_09080_b200 as pkg
+from oracle import gpga_oracle as o
+from test_gpu_parity import TOL_RUN, TOL_STEP, TOPO, close
+
+pytestmark = pytest.mark.gpu
+
+SEED = 20210509
+BLOCK = 1024            # columns per sampled block = columns per 256-thread CTA
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def _blocks(d, count, rng):
+    """Column offsets (multiples of 4): first block, last (ragged end), blocks straddling
+    CTA boundaries, and random ones."""
+    offs = {0, (d - BLOCK) // 4 * 4, BLOCK // 2, 148 * BLOCK - 512, (d // 2) // BLOCK * BLOCK + 508}
+    while len(offs) < count:
+        offs.add(int(rng.integers(0, (d - BLOCK) // 4)) * 4)
+    return sorted(offs)
+
+
+def _gpu_block(x, c0, width):
+    return x[:, c0:c0 + width].cpu().numpy()
+
+
+def _free_gib():
+    torch = _torch()
+    free, _ = torch.cuda.mem_get_info()
+    return free / 2**30
+
+
+def _run_case(bufs, n, d, topo, H, gamma, sigma, K, x0_kind, x0_std, b_shift, offs, one_step_ks):
+    xa, xb, b, scratch = bufs
+    okind = {pkg.GPGA_X0_ZERO: o.X0_ZERO, pkg.GPGA_X0_SHARED_NORMAL: o.X0_SHARED_NORMAL}[x0_kind]
+    g = pkg.Gpga(n, d, TOPO[topo][0], H, gamma, SEED)
+    g.set_objective(pkg.GPGA_OBJ_QUADRATIC, sigma=sigma)
+    g.bind(xa, xb, b, scratch=scratch)
+    width = lambda c0: min(BLOCK, d - c0)
+    ora = {}
+    for c0 in offs:
+        w = width(c0)
+        B = o.init_b(n, w, SEED, b_shift, c0).astype(np.float32)
+        X0 = o.init_x0(n, w, SEED, okind, x0_std, c0).astype(np.float32)
+        ora[c0] = (X0, o.Problem(TOPO[topo][1], H, gamma, SEED, sigma=sigma, data=B, col0=c0))
+    # single iterations at chosen k, each from the initial state
+    for k in one_step_ks:
+        g.init_from_seed(x0_kind, x0_std, b_shift)
+        g.step(k)
+        x = g.get_x()
+        for c0 in offs:
+            X0, p = ora[c0]
+            ok, worst = close(_gpu_block(x, c0, width(c0)), o.step(p, X0, k), TOL_STEP)
+            assert ok, (topo, H, "k", k, "col0", c0, worst)
+    # the K-iteration run
+    g.init_from_seed(x0_kind, x0_std, b_shift)
+    g.run(K)
+    x = g.get_x()
+    for c0 in offs:
+        X0, p = ora[c0]
+        ok, worst = close(_gpu_block(x, c0, width(c0)), o.run(p, X0, 0, K), TOL_RUN)
+        assert ok, (topo, H, "run col0", c0, worst)
+    xi = g.consensus_distance()
+    assert np.isfinite(xi) and xi >= 0.0
+    if H and K % H == 0:
+        assert xi == 0.0            # ended on a global average: rows bit-identical
+    g.close()
+
+
+def test_config_3_resnet50_sized():
+    torch = _torch()
+    n, d, gamma, sigma, K = 64, 25_557_032, 0.01, 0.01, 50
+    if _free_gib() < 3 * n * d * 4 / 2**30 + 2:
+        pytest.skip("not enough free device memory")
+    xa = torch.empty((n, d), dtype=torch.float32, device="cuda")
+    xb = torch.empty_like(xa)
+    b = torch.empty_like(xa)
+    scratch = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+    offs = _blocks(d, 12, np.random.default_rng(3))
+    assert d % 128 == 40 and offs[-1] + BLOCK == d
+    for topo in ("ring", "exp"):
+        for H in (4, 16, 0):
+            ks = [0]
+            if H == 4:
+                ks = [0, 3] if topo == "ring" else [0, 1, 2, 3, 4, 5]   # hops 1..32; k=3 is global
+            _run_case((xa, xb, b, scratch), n, d, topo, H, gamma, sigma, K,
+                      pkg.GPGA_X0_SHARED_NORMAL, 0.1, 0.5, offs, ks)
+    del xa, xb, b
+    torch.cuda.empty_cache()
+
+
+def test_config_4_bert_large_sized():
+    torch = _torch()
+    n, d, gamma, sigma, K, H = 16, 335_141_888, 0.01, 0.01, 20, 4
+    if _free_gib() < 3 * n * d * 4 / 2**30 + 2:
+        pytest.skip("not enough free device memory")
+    assert n * d > 2**32            # element indices need 64 bits
+    xa = torch.empty((n, d), dtype=torch.float32, device="cuda")
+    xb = torch.empty_like(xa)
+    b = torch.empty_like(xa)
+    scratch = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+    offs = _blocks(d, 12, np.random.default_rng(4))
+    _run_case((xa, xb, b, scratch), n, d, "exp", H, gamma, sigma, K, pkg.GPGA_X0_ZERO, 1.0, 0.0,
+              offs, [0, 1, 2, 3])
+    del xa, xb, b
+    torch.cuda.empty_cache()

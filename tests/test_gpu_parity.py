@@ -1,0 +1,190 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element,
+on the same seeded inputs.  Tolerances: |gpu - oracle| <= 1e-6 (1 + |oracle|) after one
+iteration, 1e-4 (1 + |oracle|) after a K-iteration run, consensus distance 1e-5 relative."""
+import numpy as np
+import pytest
+
+import paper_2105_09080_b200 as pkg
+from oracle import gpga_oracle as o
+from paper_2105_09080_b200 import binding
+from paper_2105_09080_b200.inputs import logistic_inputs, quadratic_inputs
+
+pytestmark = pytest.mark.gpu
+
+TOL_STEP = 1e-6
+TOL_RUN = 1e-4
+
+TOPO = {"ring": (pkg.GPGA_TOPO_RING, o.TOPO_RING), "exp": (pkg.GPGA_TOPO_EXP, o.TOPO_EXP),
+        "grid": (pkg.GPGA_TOPO_GRID, o.TOPO_GRID),
+        "static_exp": (pkg.GPGA_TOPO_STATIC_EXP, o.TOPO_STATIC_EXP),
+        "none": (pkg.GPGA_TOPO_NONE, o.TOPO_NONE)}
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def close(got, want, tol):
+    err = np.abs(got.astype(np.float64) - want.astype(np.float64))
+    bound = tol * (1 + np.abs(want.astype(np.float64)))
+    worst = float((err / bound).max()) if err.size else 0.0
+    return worst <= 1.0, worst
+
+
+def make_quadratic(n, d, topo, H, gamma, seed, sigma, X0, B, col0=0, grid_cols=0):
+    torch = _torch()
+    g = pkg.Gpga(n, d, TOPO[topo][0], H, gamma, seed)
+    g.set_objective(pkg.GPGA_OBJ_QUADRATIC, sigma=sigma)
+    if col0:
+        g.set_column_offset(col0)
+    if grid_cols:
+        g.set_grid_cols(grid_cols)
+    xa = torch.from_numpy(X0).cuda()
+    g.bind(xa, torch.empty_like(xa), torch.from_numpy(B).cuda())
+    p = o.Problem(TOPO[topo][1], H, gamma, seed, sigma=sigma, data=B, col0=col0, grid_cols=grid_cols)
+    return g, p
+
+
+# ------------------------------------------------------------------ generator
+def test_device_philox_known_answers_and_random_counters():
+    torch = _torch()
+    from pathlib import Path
+    rows = [l.split() for l in (Path(__file__).parent / "golden" / "philox4x32_10_kat.txt")
+            .read_text().splitlines() if l.strip() and not l.startswith("#")]
+    for row in rows:
+        v = [int(t, 16) for t in row]
+        ctr = torch.tensor(np.array([v[0:4]], dtype=np.uint32).view(np.int32), device="cuda")
+        out = binding.philox_words(ctr, v[4], v[5]).cpu().numpy().view(np.uint32)[0]
+        assert [int(x) for x in out] == v[6:10]
+    rng = np.random.default_rng(1)
+    ctr = rng.integers(0, 2**32, (4096, 4), dtype=np.uint64).astype(np.uint32)
+    out = binding.philox_words(torch.tensor(ctr.view(np.int32), device="cuda"), 0xDEADBEEF, 0x1234567)
+    out = out.cpu().numpy().view(np.uint32)
+    for t in range(0, 4096, 37):
+        assert np.array_equal(out[t], o.philox4x32_10(ctr[t], [0xDEADBEEF, 0x1234567]))
+
+
+# The normals enter the state as gamma * sigma * z, so an error dz costs gamma sigma dz.  The
+# largest gamma * sigma of the benchmark configurations is 0.01; keeping that contribution
+# below a quarter of the one-step tolerance needs |dz| <= 2.5e-5.
+DZ_MAX = 2.5e-5
+
+
+def test_device_box_muller_exhaustive_radius_and_angle():
+    torch = _torch()
+    m = np.arange(2**24, dtype=np.uint32)
+    words = torch.tensor((m << 8).view(np.int32), device="cuda")
+    # every value of u1, at angles 0 (z = (r, 0)) and pi/2 + a bit
+    for bword in (0, (2**22 + 12345) << 8):
+        bw = torch.full_like(words, bword)
+        z = binding.box_muller_words(words, bw).cpu().numpy()
+        want = o.box_muller_many(m << 8, np.full(m.shape, bword, dtype=np.uint32))
+        assert np.abs(z - want).max() <= DZ_MAX
+    # every value of u2, at a small, a typical and the largest radius
+    for aword in ((2**24 - 2) << 8, 0x7FFFFF00, 0):
+        aw = torch.full_like(words, np.array([aword], dtype=np.uint32).view(np.int32)[0])
+        z = binding.box_muller_words(aw, words).cpu().numpy()
+        want = o.box_muller_many(np.full(m.shape, aword, dtype=np.uint32), m << 8)
+        assert np.abs(z - want).max() <= DZ_MAX
+
+
+def test_device_normal_fill_matches_oracle_keying():
+    seed = (0xABCDEF12 << 32) | 0x3456789A
+    z = binding.normal_fill(seed, 0, 7, 3, 1000, 257).cpu().numpy()
+    for t in (0, 1, 100, 256):
+        assert np.abs(z[t] - o.normal4(seed, 0, 7, 3, 1000 + t)).max() <= DZ_MAX
+    assert abs(z.mean()) < 0.2 and abs(z.std() - 1) < 0.1
+
+
+# ------------------------------------------------------------------ one step, every kernel
+SHAPES = [(1, 4), (2, 8), (3, 12), (4, 132), (5, 1028), (8, 4100), (16, 1024 + 40), (7, 6), (3, 1),
+          (6, 1031), (64, 520)]
+
+
+@pytest.mark.parametrize("n,d", SHAPES)
+@pytest.mark.parametrize("sigma", [0.0, 0.3])
+def test_ring_and_global_one_step(n, d, sigma):
+    X0, B = quadratic_inputs(n, d, 100 + n, x0="per_node")
+    for H, k in ((0, 5), (3, 2)):           # gossip step; global-average step (mod(k+1,H)=0)
+        g, p = make_quadratic(n, d, "ring", H, 0.25, 77, sigma, X0, B)
+        g.step(k)
+        want = o.step(p, X0, k)
+        ok, worst = close(g.get_x().cpu().numpy(), want, TOL_STEP)
+        assert ok, (H, k, worst)
+        if H:
+            got = g.get_x().cpu().numpy()
+            assert np.all(got == got[0])    # rows bit-identical after a global average
+        g.close()
+
+
+@pytest.mark.parametrize("n", [1, 2, 4, 8, 32, 64])
+@pytest.mark.parametrize("d", [4, 7, 1028, 4096 + 8])
+def test_exp_one_step_every_hop(n, d):
+    X0, B = quadratic_inputs(n, d, 200 + n, x0="per_node")
+    tau = max(1, int(np.log2(n)))
+    for k in range(tau + 1):
+        g, p = make_quadratic(n, d, "exp", 0, 0.1, 5, 0.2, X0, B)
+        g.step(k)
+        ok, worst = close(g.get_x().cpu().numpy(), o.step(p, X0, k), TOL_STEP)
+        assert ok, (k, worst)
+        g.close()
+
+
+@pytest.mark.parametrize("topo,n,gc", [("grid", 12, 4), ("grid", 16, 0), ("grid", 6, 1),
+                                       ("static_exp", 8, 0), ("static_exp", 64, 0), ("none", 5, 0)])
+@pytest.mark.parametrize("d", [8, 1030])
+def test_tile_topologies_one_step(topo, n, gc, d):
+    X0, B = quadratic_inputs(n, d, 300 + n, x0="per_node")
+    g, p = make_quadratic(n, d, topo, 0, 0.2, 9, 0.4, X0, B, grid_cols=gc)
+    if topo == "grid" and gc == 0:
+        p.grid_cols = 4                      # library default: most square torus
+    g.step(3)
+    ok, worst = close(g.get_x().cpu().numpy(), o.step(p, X0, 3), TOL_STEP)
+    assert ok, worst
+    g.close()
+
+
+def test_column_offset_keys_the_noise():
+    n, d, c0 = 4, 64, 4096
+    X0, B = quadratic_inputs(n, d, 1)
+    g, p = make_quadratic(n, d, "ring", 0, 0.1, 3, 1.0, X0, B, col0=c0)
+    g.step(0)
+    ok, worst = close(g.get_x().cpu().numpy(), o.step(p, X0, 0), TOL_STEP)
+    assert ok, worst
+    g0, p0 = make_quadratic(n, d, "ring", 0, 0.1, 3, 1.0, X0, B)
+    g0.step(0)
+    assert not np.array_equal(g0.get_x().cpu().numpy(), g.get_x().cpu().numpy())
+
+
+def test_step_is_a_pure_function_and_resume_is_exact():
+    n, d = 8, 2052
+    X0, B = quadratic_inputs(n, d, 2)
+    g, _ = make_quadratic(n, d, "exp", 4, 0.1, 11, 0.1, X0, B)
+    g.run(10)
+    full = g.get_x().cpu().numpy().copy()
+    g2, _ = make_quadratic(n, d, "exp", 4, 0.1, 11, 0.1, X0, B)
+    g2.run(6)
+    mid = g2.get_x().cpu().numpy().copy()
+    g3, _ = make_quadratic(n, d, "exp", 4, 0.1, 11, 0.1, mid, B)
+    g3.set_k(6)
+    g3.run(4)
+    assert np.array_equal(g3.get_x().cpu().numpy(), full)
+    assert g.get_k() == 10 and g.launch_count() == 10
+
+
+# ------------------------------------------------------------------ consensus distance
+@pytest.mark.parametrize("n,d", [(1, 8), (2, 5), (8, 4100), (64, 777), (16, 100000)])
+def test_consensus_distance(n, d):
+    X0, B = quadratic_inputs(n, d, 400 + n, x0="per_node")
+    g, _ = make_quadratic(n, d, "ring", 0, 0.1, 1, 0.0, X0, B)
+    want = o.consensus_distance(X0)
+    assert abs(g.consensus_distance() - want) <= 1e-5 * want + 1e-300
+    # nearly consensual rows: one row differs in the last bits
+    X1 = np.repeat(X0[:1], n, axis=0).copy()
+    if n > 1:
+        X1[n - 1] = np.nextafter(X1[n - 1], np.float32(10))
+    g, _ = make_quadratic(n, d, "ring", 0, 0.1, 1, 0.0, X1, B)
+    want = o.consensus_distance(X1)
+    assert abs(g.consensus_distance() - want) <= 1e-5 * want
+    g.close()

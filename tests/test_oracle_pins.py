@@ -429,3 +429,15 @@ def test_aga_period_update_worked_example():
     assert (F_init, H) == (2.0, 16)
     F_init, H = o.aga_update(27, 10, 4, 0.6, F_init, H)
     assert (F_init, H) == (2.0, 14)          # ceil(13.33)
+
+
+def test_vector_box_muller_and_mean_loss_helpers():
+    rng = np.random.default_rng(0)
+    a = rng.integers(0, 2**32, 50, dtype=np.uint64).astype(np.uint32)
+    b = rng.integers(0, 2**32, 50, dtype=np.uint64).astype(np.uint32)
+    z = o.box_muller_many(a, b)
+    for t in range(50):
+        assert np.array_equal(z[t], o.box_muller(int(a[t]), int(b[t])))
+    X = rng.standard_normal((3, 4))
+    B = rng.standard_normal((3, 4))
+    assert abs(o.quadratic_mean_loss(X, B) - 0.5 * np.linalg.norm(X - B, "fro") ** 2 / 3) < 1e-13
