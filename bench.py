@@ -42,6 +42,10 @@ WORKLOADS = {
     "c3_exp_h16": dict(n=64, d=25_557_032, topo="exp", H=16, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),
     "c3_exp_hinf": dict(n=64, d=25_557_032, topo="exp", H=0, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),
     "c3_global_h1": dict(n=64, d=25_557_032, topo="ring", H=1, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),
+    # reduced-width copies of c3 / c4 (same n, same ragged d mod 128) for profiler captures
+    "c3s_ring_h4": dict(n=64, d=2_097_192, topo="ring", H=4, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),
+    "c3s_exp_h4": dict(n=64, d=2_097_192, topo="exp", H=4, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),
+    "c4s_exp_h4": dict(n=16, d=8_388_608, topo="exp", H=4, gamma=0.01, sigma=0.01, K=20, x0="zero", x0_std=1.0, b_shift=0.0),
     "c4_exp_h4": dict(n=16, d=335_141_888, topo="exp", H=4, gamma=0.01, sigma=0.01, K=20, x0="zero", x0_std=1.0, b_shift=0.0),
     "c4_global_h1": dict(n=16, d=335_141_888, topo="exp", H=1, gamma=0.01, sigma=0.01, K=20, x0="zero", x0_std=1.0, b_shift=0.0),
 }
@@ -79,7 +83,7 @@ class ClockSampler(threading.Thread):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
-        self._stop = threading.Event()
+        self._halt = threading.Event()
         self.active = threading.Event()
         self.error = None
 
@@ -97,7 +101,7 @@ class ClockSampler(threading.Thread):
                         names.setdefault(v, attr.replace("nvmlClocksEventReason", "").replace("nvmlClocksThrottleReason", ""))
             get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
                 nv.nvmlDeviceGetCurrentClocksThrottleReasons
-            while not self._stop.is_set():
+            while not self._halt.is_set():
                 if self.active.is_set():
                     self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
                     mask = get_reasons(h)
@@ -110,7 +114,7 @@ class ClockSampler(threading.Thread):
             self.error = repr(exc)
 
     def finish(self):
-        self._stop.set()
+        self._halt.set()
         self.join(timeout=2)
         s = sorted(self.samples)
         return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
