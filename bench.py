@@ -201,11 +201,16 @@ def run_reference(args, w, name):
         "gpu_launches": 0}))
 
 
+def padded_stride(d):
+    return (d + 31) // 32 * 32
+
+
 def workload_config(name, w, n_gpus):
     return {"workload": f"{name}: n={w['n']} nodes x d={w['d']} fp32, {w['topo']} topology, H={w['H'] or 'inf'}, "
                         f"gamma={w['gamma']}, sigma={w['sigma']}, quadratic objective, seed {SEED}",
             "l2_flush": f"none needed: each step streams {BYTES_PER_UPDATE * w['n'] * w['d'] / 1e9:.2f} GB, larger than the 126 MB L2"
                         if BYTES_PER_UPDATE * w['n'] * w['d'] > 4 * 126e6 else "state fits in L2; reported as L2-resident",
+            "layout": f"row-major fp32, row stride {padded_stride(w['d'])} floats (rows padded to 128 B)",
             "sharding": f"columns, {n_gpus} shard(s) of d columns each, no collective"}
 
 
@@ -233,6 +238,7 @@ def run_ours(args, w, name):
     g = pkg.Gpga(n, d, topo, w["H"], w["gamma"], SEED)
     g.set_objective(pkg.GPGA_OBJ_QUADRATIC, sigma=w["sigma"])
     g.set_column_offset(rank * ((d + 3) // 4 * 4))
+    g.set_row_stride(padded_stride(d))      # every node's row starts on a 128-byte line
     xa, xb, b = g.allocate()
     g.init_from_seed(kind, w["x0_std"], w["b_shift"])
     torch.cuda.synchronize()
@@ -316,8 +322,8 @@ def run_e2e(torch, g, w, dist):
     out = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
     # host copies of the seeded inputs (downloaded once, outside the timed region)
     g.init_from_seed({"zero": 0, "shared": 1}[w["x0"]], w["x0_std"], w["b_shift"])
-    x0.copy_(g.x_bufs[0])
-    bh.copy_(g._keep[2])
+    x0.copy_(g.x_bufs[0][:, :d])
+    bh.copy_(g._keep[2][:, :d])
     torch.cuda.synchronize()
     g.run_host(x0, bh, K, out)                      # warm-up job
     if dist is not None:

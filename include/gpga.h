@@ -15,8 +15,9 @@
  *    caller and must outlive the handle; the library never allocates or frees
  *    device memory.
  *  - "device pointer" / "host pointer" is stated per argument.  Device
- *    pointers must be 16-byte aligned.  Matrices are row-major, row stride d,
- *    fp32.  Element (i, j) of an n x d matrix is at index i * d + j (64-bit).
+ *    pointers must be 16-byte aligned.  Matrices are row-major fp32 with row
+ *    stride ld >= d (default ld = d, see gpga_set_row_stride): element (i, j) of
+ *    an n x d matrix is at index i * ld + j (64-bit).
  *  - `stream` arguments are a cudaStream_t passed as void* (NULL = default
  *    stream).  Calls are asynchronous on that stream unless stated otherwise.
  *  - Random numbers are Philox4x32-10 (Salmon et al., SC'11) keyed by
@@ -99,6 +100,17 @@ int32_t gpga_set_objective(gpga_t* ctx, int32_t objective, float sigma, float l2
 int32_t gpga_set_grid_cols(gpga_t* ctx, int64_t cols);
 
 /*
+ * Row stride ld (in floats, ld >= d) of the X buffers and, for the quadratic objective, of b:
+ * element (i, j) is at index i * ld + j.  Default ld = d.  Choosing ld a multiple of 32
+ * starts every node's parameter vector on a 128-byte line, which is worth several per cent
+ * of bandwidth when d itself is not a multiple of 32.  Padding columns d .. ld-1 are never
+ * read or written.  The 128-bit access path needs d % 4 == 0 and ld % 4 == 0; other shapes
+ * take a scalar path.  The logistic data A and labels stay dense.  Call before gpga_bind.
+ * Errors: INVALID_ARG for ld < d or after gpga_bind.
+ */
+int32_t gpga_set_row_stride(gpga_t* ctx, int64_t ld);
+
+/*
  * Column sharding: this handle holds global columns col0 .. col0 + d - 1 of a wider
  * problem.  Only the random-number counters depend on it; W acts on rows, so column
  * ranges evolve independently (matrix form of the recursion, Appendix A).
@@ -112,9 +124,9 @@ int64_t gpga_scratch_bytes(const gpga_t* ctx);
 
 /*
  * Bind caller-owned device buffers.
- *  x_a, x_b : two n*d fp32 buffers (double buffer for X^(k), X^(k+1)); x_a holds the
+ *  x_a, x_b : two n*ld fp32 buffers (double buffer for X^(k), X^(k+1)); x_a holds the
  *             current state.
- *  data     : QUADRATIC: b, n*d fp32.  LOGISTIC: A, n*m*d fp32 (node-major, then sample).
+ *  data     : QUADRATIC: b, n*ld fp32.  LOGISTIC: A, n*m*d fp32 (node-major, then sample).
  *  labels   : LOGISTIC: y, n*m fp32 in {-1,+1}; otherwise NULL.
  *  scratch  : at least gpga_scratch_bytes() bytes (scratch_bytes is what was given).
  * Errors: INVALID_ARG for NULL / misaligned pointers, x_a == x_b, too little scratch.
@@ -145,8 +157,8 @@ int32_t gpga_step(gpga_t* ctx, int64_t k, void* stream);
 int32_t gpga_run(gpga_t* ctx, int64_t K, void* stream);
 
 /*
- * Same as gpga_run with HOST buffers (quadratic objective): copies x0_host (n*d fp32) and
- * data_host (n*d fp32) into the bound device buffers, resets the counter to 0, runs K
+ * Same as gpga_run with HOST buffers (quadratic objective): copies x0_host and data_host
+ * (dense n*d fp32 each) into the bound device buffers (row stride ld), resets the counter to 0, runs K
  * iterations, copies X^(K) to x_out_host and synchronises the stream.  Host buffers
  * should be pinned for full copy speed.
  */

@@ -40,6 +40,7 @@ SIGNATURES = {
     "gpga_create": (_i32, [_i64, _i64, _i32, _i64, _f32, _u64, C.POINTER(_P)]),
     "gpga_set_objective": (_i32, [_P, _i32, _f32, _f32, _i64, _i64]),
     "gpga_set_grid_cols": (_i32, [_P, _i64]),
+    "gpga_set_row_stride": (_i32, [_P, _i64]),
     "gpga_set_column_offset": (_i32, [_P, _i64]),
     "gpga_scratch_bytes": (_i64, [_P]),
     "gpga_bind": (_i32, [_P, _P, _P, _P, _P, _P, _i64]),
@@ -108,6 +109,7 @@ class Gpga:
     def __init__(self, n, d, topology, H, gamma, seed):
         self._h = _P()
         self.n, self.d = int(n), int(d)
+        self.ld = int(d)
         st = lib().gpga_create(n, d, topology, H, gamma, seed, C.byref(self._h))
         if st != GPGA_OK:
             raise GpgaError(st, lib().gpga_last_error(None).decode())
@@ -137,6 +139,10 @@ class Gpga:
     def set_grid_cols(self, cols):
         self._check(lib().gpga_set_grid_cols(self._h, cols))
 
+    def set_row_stride(self, ld):
+        self._check(lib().gpga_set_row_stride(self._h, ld))
+        self.ld = int(ld)
+
     def set_column_offset(self, col0):
         self._check(lib().gpga_set_column_offset(self._h, col0))
 
@@ -161,9 +167,9 @@ class Gpga:
         self._check(lib().gpga_bind(self._h, x_a, x_b, data, labels, scratch, scratch_bytes))
 
     def allocate(self, device="cuda"):
-        """Allocate X double buffer, b and scratch for the quadratic objective and bind them."""
+        """Allocate X double buffer, b (n x ld each) and scratch for the quadratic objective and bind."""
         import torch
-        xa = torch.empty((self.n, self.d), dtype=torch.float32, device=device)
+        xa = torch.empty((self.n, self.ld), dtype=torch.float32, device=device)
         xb = torch.empty_like(xa)
         data = torch.empty_like(xa)
         self.bind(xa, xb, data)

@@ -20,6 +20,7 @@ struct gpga_ctx {
     int64_t m = 0, batch = 0;
     int64_t grid_cols = 0;
     int64_t col0 = 0;
+    int64_t ld = 0;   // row stride of X and b in floats
     float* x[2] = {nullptr, nullptr};
     float* data = nullptr;
     const float* labels = nullptr;
@@ -81,6 +82,9 @@ ScratchLayout scratch_layout(const gpga_ctx* c)
 // Algorithm 1: global average exactly when mod(k + 1, H) = 0 (H = 0: never).
 bool is_global_step(int64_t k, int64_t H) { return H > 0 && ((k + 1) % H) == 0; }
 
+// 128-bit path: every row starts 16-byte aligned and ends on a whole group of four.
+bool vec_ok(const gpga_ctx* c) { return (c->d % 4) == 0 && (c->ld % 4) == 0; }
+
 int32_t check_ready(gpga_ctx* c)
 {
     if (!c) return fail(nullptr, GPGA_ERR_NOT_READY, "NULL handle");
@@ -96,6 +100,7 @@ LogregParams logreg_params(const gpga_ctx* c, int64_t k)
     lp.A = c->data;
     lp.y = c->labels;
     lp.x = c->x[c->cur];
+    lp.ldx = c->ld;
     lp.G = reinterpret_cast<float*>(c->scratch + L.G_off);
     lp.partial = reinterpret_cast<float*>(c->scratch + L.chunk_off);
     lp.n = c->n; lp.d = c->d; lp.m = c->m; lp.batch = c->batch;
@@ -113,14 +118,14 @@ int32_t do_step(gpga_ctx* c, int64_t k, bool global, cudaStream_t s)
     p.x = c->x[c->cur];
     p.out = c->x[c->cur ^ 1];
     p.b = c->data;
-    p.n = c->n; p.d = c->d; p.Q = (c->d + 3) / 4;
+    p.n = c->n; p.d = c->d; p.ld = c->ld; p.ldb = c->ld; p.Q = (c->d + 3) / 4;
     p.q_base = (uint32_t)(c->col0 >> 2);
     p.k = (uint32_t)k;
     p.gamma = c->gamma; p.sigma = c->sigma;
     p.hop_log2 = 0; p.len_log2 = 0;
     p.grid_cols = (int)c->grid_cols;
     p.keys = c->keys;
-    const bool vec = (c->d % 4) == 0;
+    const bool vec = vec_ok(c);
     int mode = (c->sigma != 0.f) ? GRAD_QUAD_NOISE : GRAD_QUAD;
     cudaError_t e;
     if (c->objective == GPGA_OBJ_LOGISTIC) {
@@ -129,6 +134,7 @@ int32_t do_step(gpga_ctx* c, int64_t k, bool global, cudaStream_t s)
         c->launches += 2;
         if (e != cudaSuccess) return cuda_fail(c, e, "logistic gradient launch");
         p.b = lp.G;
+        p.ldb = c->d;
         mode = GRAD_BUFFER;
     }
     if (global) {
@@ -162,7 +168,7 @@ int32_t mean_loss_async(gpga_ctx* c, cudaStream_t s, double** result_dev)
         if (c->k >= (int64_t(1) << 32)) return fail(c, GPGA_ERR_INVALID_ARG, "k must be in [0, 2^32)");
         e = launch_logreg_loss(logreg_params(c, c->k), partials, result, s);
     } else {
-        e = launch_quadratic_loss(c->x[c->cur], c->data, c->n, c->d, partials, result, s);
+        e = launch_quadratic_loss(c->x[c->cur], c->data, c->n, c->d, c->ld, vec_ok(c), partials, result, s);
     }
     c->launches += 2;
     if (e != cudaSuccess) return cuda_fail(c, e, "loss launch");
@@ -201,7 +207,7 @@ int32_t gpga_create(int64_t n, int64_t d, int32_t topology, int64_t H, float gam
         return fail(nullptr, GPGA_ERR_UNSUPPORTED, "this topology supports at most 4096 nodes");
     gpga_ctx* c = new (std::nothrow) gpga_ctx;
     if (!c) return fail(nullptr, GPGA_ERR_INVALID_ARG, "out of host memory");
-    c->n = n; c->d = d; c->topology = topology; c->H = H; c->gamma = gamma; c->seed = seed;
+    c->n = n; c->d = d; c->ld = d; c->topology = topology; c->H = H; c->gamma = gamma; c->seed = seed;
     c->keys = make_philox_keys((uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32));
     if (topology == GPGA_TOPO_GRID) {   // default: the most square torus
         int64_t cols = (int64_t)std::floor(std::sqrt((double)n));
@@ -240,6 +246,15 @@ int32_t gpga_set_grid_cols(gpga_t* c, int64_t cols)
     if (!c) return fail(nullptr, GPGA_ERR_NOT_READY, "NULL handle");
     if (cols < 1 || c->n % cols != 0) return fail(c, GPGA_ERR_INVALID_ARG, "cols must divide n");
     c->grid_cols = cols;
+    return GPGA_OK;
+}
+
+int32_t gpga_set_row_stride(gpga_t* c, int64_t ld)
+{
+    if (!c) return fail(nullptr, GPGA_ERR_NOT_READY, "NULL handle");
+    if (c->bound) return fail(c, GPGA_ERR_INVALID_ARG, "set the row stride before gpga_bind");
+    if (ld < c->d || ld >= (int64_t(1) << 35)) return fail(c, GPGA_ERR_INVALID_ARG, "row stride must be >= d");
+    c->ld = ld;
     return GPGA_OK;
 }
 
@@ -290,11 +305,11 @@ int32_t gpga_init_from_seed(gpga_t* c, int32_t x0_kind, float x0_std, float b_sh
     if (x0_kind < GPGA_X0_ZERO || x0_kind > GPGA_X0_PER_NODE_NORMAL) return fail(c, GPGA_ERR_INVALID_ARG, "unknown x0 kind");
     if (!std::isfinite(x0_std) || !std::isfinite(b_shift)) return fail(c, GPGA_ERR_INVALID_ARG, "non-finite argument");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const bool vec = (c->d % 4) == 0;
+    const bool vec = vec_ok(c);
     const uint32_t q_base = (uint32_t)(c->col0 >> 2);
-    cudaError_t e = launch_init_b(c->data, c->n, c->d, q_base, b_shift, vec, c->keys, s);
+    cudaError_t e = launch_init_b(c->data, c->n, c->d, c->ld, q_base, b_shift, vec, c->keys, s);
     if (e != cudaSuccess) return cuda_fail(c, e, "init b launch");
-    e = launch_init_x0(c->x[0], c->n, c->d, q_base, x0_kind, x0_std, vec, c->keys, s);
+    e = launch_init_x0(c->x[0], c->n, c->d, c->ld, q_base, x0_kind, x0_std, vec, c->keys, s);
     if (e != cudaSuccess) return cuda_fail(c, e, "init x0 launch");
     c->launches += 2;
     c->cur = 0;
@@ -332,10 +347,12 @@ int32_t gpga_run_host(gpga_t* c, const float* x0_host, const float* data_host, i
     if (!x0_host || !data_host || !x_out_host) return fail(c, GPGA_ERR_INVALID_ARG, "NULL host buffer");
     if (K < 0) return fail(c, GPGA_ERR_INVALID_ARG, "K must be >= 0");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const size_t bytes = (size_t)c->n * (size_t)c->d * sizeof(float);
-    cudaError_t e = cudaMemcpyAsync(c->x[0], x0_host, bytes, cudaMemcpyHostToDevice, s);
+    const size_t row_bytes = (size_t)c->d * sizeof(float), pitch = (size_t)c->ld * sizeof(float);
+    cudaError_t e = cudaMemcpy2DAsync(c->x[0], pitch, x0_host, row_bytes, row_bytes, (size_t)c->n,
+                                      cudaMemcpyHostToDevice, s);
     if (e != cudaSuccess) return cuda_fail(c, e, "x0 upload");
-    e = cudaMemcpyAsync(c->data, data_host, bytes, cudaMemcpyHostToDevice, s);
+    e = cudaMemcpy2DAsync(c->data, pitch, data_host, row_bytes, row_bytes, (size_t)c->n,
+                          cudaMemcpyHostToDevice, s);
     if (e != cudaSuccess) return cuda_fail(c, e, "data upload");
     c->cur = 0;
     c->k = 0;
@@ -343,7 +360,8 @@ int32_t gpga_run_host(gpga_t* c, const float* x0_host, const float* data_host, i
         st = do_step(c, k, is_global_step(k, c->H), s);
         if (st) return st;
     }
-    e = cudaMemcpyAsync(x_out_host, c->x[c->cur], bytes, cudaMemcpyDeviceToHost, s);
+    e = cudaMemcpy2DAsync(x_out_host, row_bytes, c->x[c->cur], pitch, row_bytes, (size_t)c->n,
+                          cudaMemcpyDeviceToHost, s);
     if (e != cudaSuccess) return cuda_fail(c, e, "result download");
     e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_fail(c, e, "stream synchronize");
@@ -359,7 +377,7 @@ int32_t gpga_consensus_distance(gpga_t* c, void* stream, double* out_host)
     const ScratchLayout L = scratch_layout(c);
     double* partials = reinterpret_cast<double*>(c->scratch + L.partials_off);
     double* result = reinterpret_cast<double*>(c->scratch + L.result_off);
-    cudaError_t e = launch_consensus(c->x[c->cur], c->n, c->d, (c->d % 4) == 0, partials, result, s);
+    cudaError_t e = launch_consensus(c->x[c->cur], c->n, c->d, c->ld, vec_ok(c), partials, result, s);
     c->launches += 2;
     if (e != cudaSuccess) return cuda_fail(c, e, "consensus launch");
     return read_double(c, result, s, out_host);

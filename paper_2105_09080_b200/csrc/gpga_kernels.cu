@@ -22,18 +22,30 @@ __device__ __forceinline__ float4 scale4(float4 a, float s)
     return make_float4(a.x * s, a.y * s, a.z * s, a.w * s);
 }
 
-// x^(k+1/2) for node i, column group q (Algorithm 1: gradient, then the local update).
-template <int MODE, bool VEC>
-__device__ __forceinline__ float4 half_step(const StepParams& p, long long i, long long q)
+// One row's inputs for one column group, and x^(k+1/2) formed from them
+// (Algorithm 1: gradient, then the local update).  Loading and finishing are split
+// so that a thread can have the loads of several rows in flight before it needs any.
+struct RowIn {
+    float4 x, b;
+};
+
+template <bool VEC>
+__device__ __forceinline__ RowIn load_row(const StepParams& p, long long i, long long q)
 {
-    const long long j0 = q * 4;
-    const float4 x = load4<VEC>(p.x + i * p.d, j0, p.d);
-    const float4 b = load4<VEC>(p.b + i * p.d, j0, p.d);
+    RowIn r;
+    r.x = load4<VEC>(p.x + i * p.ld, q * 4, p.d);
+    r.b = load4<VEC>(p.b + i * p.ldb, q * 4, p.d);
+    return r;
+}
+
+template <int MODE>
+__device__ __forceinline__ float4 finish_row(const StepParams& p, const RowIn& r, long long i, long long q)
+{
     float4 g;
     if (MODE == GRAD_BUFFER) {
-        g = b;
+        g = r.b;
     } else {
-        g = make_float4(x.x - b.x, x.y - b.y, x.z - b.z, x.w - b.w);
+        g = make_float4(r.x.x - r.b.x, r.x.y - r.b.y, r.x.z - r.b.z, r.x.w - r.b.w);
         if (MODE == GRAD_QUAD_NOISE) {
             const float4 z = normal4(p.q_base + (uint32_t)q, (uint32_t)i, p.k, 0u, p.keys);
             g.x = fmaf(p.sigma, z.x, g.x);
@@ -42,44 +54,100 @@ __device__ __forceinline__ float4 half_step(const StepParams& p, long long i, lo
             g.w = fmaf(p.sigma, z.w, g.w);
         }
     }
-    return make_float4(fmaf(-p.gamma, g.x, x.x), fmaf(-p.gamma, g.y, x.y), fmaf(-p.gamma, g.z, x.z),
-                       fmaf(-p.gamma, g.w, x.w));
+    return make_float4(fmaf(-p.gamma, g.x, r.x.x), fmaf(-p.gamma, g.y, r.x.y),
+                       fmaf(-p.gamma, g.z, r.x.z), fmaf(-p.gamma, g.w, r.x.w));
+}
+
+template <int MODE, bool VEC>
+__device__ __forceinline__ float4 half_step(const StepParams& p, long long i, long long q)
+{
+    return finish_row<MODE>(p, load_row<VEC>(p, i, q), i, q);
+}
+
+// Visit steps t = t0 .. n-1 of a walk over the rows: row_of(t) is the row read at step
+// t, visit(t, row, y) consumes its half-step value.  Steps are visited in order.
+// A thread issues the loads of U rows before it needs any of them; with PIPE the
+// loads of the next batch are issued before the arithmetic of the current one
+// (software pipeline in registers), so the memory system never waits for the noise
+// arithmetic.  U and PIPE are tuned per kernel.
+template <int MODE, bool VEC, int U, bool PIPE, class RowOf, class Visit>
+__device__ __forceinline__ void stream_rows(const StepParams& p, long long q, long long t0, RowOf row_of,
+                                            Visit visit)
+{
+    const long long n = p.n;
+    long long t = t0;
+    RowIn cur[U], nxt[U];
+    if (t + U <= n) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) cur[u] = load_row<VEC>(p, row_of(t + u), q);
+    }
+    while (t + U <= n) {
+        const bool more = (t + 2 * U <= n);
+        if (PIPE && more) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) nxt[u] = load_row<VEC>(p, row_of(t + U + u), q);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long long row = row_of(t + u);
+            visit(t + u, row, finish_row<MODE>(p, cur[u], row, q));
+        }
+        t += U;
+        if (PIPE) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) cur[u] = nxt[u];
+        } else if (more) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) cur[u] = load_row<VEC>(p, row_of(t + u), q);
+        }
+    }
+    for (; t < n; ++t) {
+        const long long row = row_of(t);
+        visit(t, row, half_step<MODE, VEC>(p, row, q));
+    }
 }
 
 // ---------------------------------------------------------------------------
 // Ring: x_i^(k+1) = (y_{i-1} + y_i + y_{i+1}) / 3, indices mod n.  A three-row
 // window slides down the rows; rows 0 and 1 are kept for the wrap-around.
 // ---------------------------------------------------------------------------
-template <int MODE, bool VEC>
-__global__ void __launch_bounds__(kBlock) step_ring_kernel(const StepParams p)
+__device__ __forceinline__ float4 mix3(float4 a, float4 b, float4 c)
+{
+    const float third = 0.333333343f;
+    return make_float4((a.x + b.x + c.x) * third, (a.y + b.y + c.y) * third, (a.z + b.z + c.z) * third,
+                       (a.w + b.w + c.w) * third);
+}
+
+template <int MODE, bool VEC, int U, bool PIPE, int BLOCK, int MINB>
+__global__ void __launch_bounds__(BLOCK, MINB) step_ring_kernel(const StepParams p)
 {
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (q >= p.Q) return;
     const long long j0 = q * 4;
-    const float third = 0.333333343f;
     if (p.n <= 2) {
         const float4 y0 = half_step<MODE, VEC>(p, 0, q);
         if (p.n == 1) {
-            store4<VEC>(p.out, j0, p.d, scale4(add4(add4(y0, y0), y0), third));
+            store4<VEC>(p.out, j0, p.d, mix3(y0, y0, y0));
             return;
         }
         const float4 y1 = half_step<MODE, VEC>(p, 1, q);
-        store4<VEC>(p.out, j0, p.d, scale4(add4(add4(y1, y0), y1), third));
-        store4<VEC>(p.out + p.d, j0, p.d, scale4(add4(add4(y0, y1), y0), third));
+        store4<VEC>(p.out, j0, p.d, mix3(y1, y0, y1));
+        store4<VEC>(p.out + p.ld, j0, p.d, mix3(y0, y1, y0));
         return;
     }
-    const float4 y0 = half_step<MODE, VEC>(p, 0, q);
-    const float4 y1 = half_step<MODE, VEC>(p, 1, q);
+    const RowIn r0 = load_row<VEC>(p, 0, q), r1 = load_row<VEC>(p, 1, q);
+    const float4 y0 = finish_row<MODE>(p, r0, 0, q);
+    const float4 y1 = finish_row<MODE>(p, r1, 1, q);
     float4 a = y0, b = y1;
-#pragma unroll 4
-    for (long long i = 2; i < p.n; ++i) {
-        const float4 c = half_step<MODE, VEC>(p, i, q);
-        store4<VEC>(p.out + (i - 1) * p.d, j0, p.d, scale4(add4(add4(a, b), c), third));
-        a = b;
-        b = c;
-    }
-    store4<VEC>(p.out + (p.n - 1) * p.d, j0, p.d, scale4(add4(add4(a, b), y0), third));
-    store4<VEC>(p.out, j0, p.d, scale4(add4(add4(b, y0), y1), third));
+    stream_rows<MODE, VEC, U, PIPE>(
+        p, q, 2, [](long long t) { return t; },
+        [&](long long, long long i, float4 c) {
+            store4<VEC>(p.out + (i - 1) * p.ld, j0, p.d, mix3(a, b, c));
+            a = b;
+            b = c;
+        });
+    store4<VEC>(p.out + (p.n - 1) * p.ld, j0, p.d, mix3(a, b, y0));
+    store4<VEC>(p.out, j0, p.d, mix3(b, y0, y1));
 }
 
 // ---------------------------------------------------------------------------
@@ -89,88 +157,96 @@ __global__ void __launch_bounds__(kBlock) step_ring_kernel(const StepParams p)
 // noise generated) once.  Step t of the flattened walk visits row
 // (t / L) + (t mod L) * h with L = n / h.
 // ---------------------------------------------------------------------------
-template <int MODE, bool VEC>
-__global__ void __launch_bounds__(kBlock) step_exp_kernel(const StepParams p)
+template <int MODE, bool VEC, int U, bool PIPE, int BLOCK, int MINB>
+__global__ void __launch_bounds__(BLOCK, MINB) step_exp_kernel(const StepParams p)
 {
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (q >= p.Q) return;
     const long long j0 = q * 4;
     const long long hop = 1LL << p.hop_log2;
     const long long lmask = (1LL << p.len_log2) - 1;
+    const int len_log2 = p.len_log2, hop_log2 = p.hop_log2;
     float4 first = make_float4(0.f, 0.f, 0.f, 0.f), prev = first;
-#pragma unroll 4
-    for (long long t = 0; t < p.n; ++t) {
-        const long long s = t & lmask;
-        const long long row = (t >> p.len_log2) + (s << p.hop_log2);
-        const float4 cur = half_step<MODE, VEC>(p, row, q);
-        if (s == 0)
-            first = cur;
-        else
-            store4<VEC>(p.out + (row - hop) * p.d, j0, p.d, scale4(add4(prev, cur), 0.5f));
-        if (s == lmask) store4<VEC>(p.out + row * p.d, j0, p.d, scale4(add4(cur, first), 0.5f));
-        prev = cur;
-    }
+    stream_rows<MODE, VEC, U, PIPE>(
+        p, q, 0, [=](long long t) { return (t >> len_log2) + ((t & lmask) << hop_log2); },
+        [&](long long t, long long row, float4 cur) {
+            const long long s = t & lmask;
+            if (s == 0)
+                first = cur;
+            else
+                store4<VEC>(p.out + (row - hop) * p.ld, j0, p.d, scale4(add4(prev, cur), 0.5f));
+            if (s == lmask) store4<VEC>(p.out + row * p.ld, j0, p.d, scale4(add4(cur, first), 0.5f));
+            prev = cur;
+        });
 }
 
 // ---------------------------------------------------------------------------
 // Global average: m_j = (1/n) sum_i y_ij, written to every row.  The column sum is
 // accumulated in fp64 (exact for practical n), rounded once.
 // ---------------------------------------------------------------------------
-template <int MODE, bool VEC>
-__global__ void __launch_bounds__(kBlock) step_global_kernel(const StepParams p)
+template <int MODE, bool VEC, int U, bool PIPE, int BLOCK, int MINB>
+__global__ void __launch_bounds__(BLOCK, MINB) step_global_kernel(const StepParams p)
 {
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (q >= p.Q) return;
     const long long j0 = q * 4;
     double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
-#pragma unroll 4
-    for (long long i = 0; i < p.n; ++i) {
-        const float4 y = half_step<MODE, VEC>(p, i, q);
-        s0 += (double)y.x;
-        s1 += (double)y.y;
-        s2 += (double)y.z;
-        s3 += (double)y.w;
-    }
+    stream_rows<MODE, VEC, U, PIPE>(
+        p, q, 0, [](long long t) { return t; },
+        [&](long long, long long, float4 y) {
+            s0 += (double)y.x;
+            s1 += (double)y.y;
+            s2 += (double)y.z;
+            s3 += (double)y.w;
+        });
     const double inv = (double)p.n;
     const float4 m = make_float4((float)(s0 / inv), (float)(s1 / inv), (float)(s2 / inv),
                                  (float)(s3 / inv));
 #pragma unroll 4
-    for (long long i = 0; i < p.n; ++i) store4<VEC>(p.out + i * p.d, j0, p.d, m);
+    for (long long i = 0; i < p.n; ++i) store4<VEC>(p.out + i * p.ld, j0, p.d, m);
 }
 
 static inline unsigned grid_for(long long Q, int block) { return (unsigned)((Q + block - 1) / block); }
 
-// Small problems: narrower blocks spread the column groups over more SMs.
-static inline int block_for(long long Q) { return (Q >= 148LL * 4 * kBlock) ? kBlock : 64; }
+// Launch shape per kernel: rows in flight per thread (U), register pipeline (PIPE),
+// threads per block and minimum resident blocks (the register cap), chosen by timing
+// on B200 at the ResNet-50- and BERT-Large-sized states.
+struct RingTune { static constexpr int U = 2; static constexpr bool PIPE = false; static constexpr int BLOCK = 256; static constexpr int MINB = 4; };
+struct ExpTune { static constexpr int U = 4; static constexpr bool PIPE = false; static constexpr int BLOCK = 128; static constexpr int MINB = 4; };
+struct GlobalTune { static constexpr int U = 4; static constexpr bool PIPE = false; static constexpr int BLOCK = 128; static constexpr int MINB = 4; };
+constexpr int kSmallBlock = 64;   // small problems: narrow blocks spread the column groups over more SMs
 
-#define GPGA_DISPATCH(kernel, p, mode, vec, s)                                             \
-    do {                                                                                   \
-        const int blk = block_for((p).Q);                                                  \
-        const unsigned grd = grid_for((p).Q, blk);                                         \
-        if (vec) {                                                                         \
-            if (mode == GRAD_QUAD) kernel<GRAD_QUAD, true><<<grd, blk, 0, s>>>(p);         \
-            else if (mode == GRAD_QUAD_NOISE) kernel<GRAD_QUAD_NOISE, true><<<grd, blk, 0, s>>>(p); \
-            else kernel<GRAD_BUFFER, true><<<grd, blk, 0, s>>>(p);                          \
-        } else {                                                                           \
-            if (mode == GRAD_QUAD) kernel<GRAD_QUAD, false><<<grd, blk, 0, s>>>(p);        \
-            else if (mode == GRAD_QUAD_NOISE) kernel<GRAD_QUAD_NOISE, false><<<grd, blk, 0, s>>>(p); \
-            else kernel<GRAD_BUFFER, false><<<grd, blk, 0, s>>>(p);                         \
-        }                                                                                  \
-        return cudaGetLastError();                                                         \
+#ifndef GPGA_TUNING_HARNESS
+#define GPGA_DISPATCH(kernel, T, p, mode, vec, s)                                                      \
+    do {                                                                                               \
+        const bool small = (p).Q < 148LL * 4 * T::BLOCK;                                               \
+        const int blk = small ? kSmallBlock : T::BLOCK;                                                \
+        const unsigned grd = grid_for((p).Q, blk);                                                     \
+        if (vec) {                                                                                     \
+            if (mode == GRAD_QUAD) kernel<GRAD_QUAD, true, T::U, T::PIPE, T::BLOCK, T::MINB><<<grd, blk, 0, s>>>(p);             \
+            else if (mode == GRAD_QUAD_NOISE) kernel<GRAD_QUAD_NOISE, true, T::U, T::PIPE, T::BLOCK, T::MINB><<<grd, blk, 0, s>>>(p); \
+            else kernel<GRAD_BUFFER, true, T::U, T::PIPE, T::BLOCK, T::MINB><<<grd, blk, 0, s>>>(p);                             \
+        } else {                                                                                       \
+            if (mode == GRAD_QUAD) kernel<GRAD_QUAD, false, 2, false, T::BLOCK, 1><<<grd, blk, 0, s>>>(p);                       \
+            else if (mode == GRAD_QUAD_NOISE) kernel<GRAD_QUAD_NOISE, false, 2, false, T::BLOCK, 1><<<grd, blk, 0, s>>>(p);      \
+            else kernel<GRAD_BUFFER, false, 2, false, T::BLOCK, 1><<<grd, blk, 0, s>>>(p);                                       \
+        }                                                                                              \
+        return cudaGetLastError();                                                                     \
     } while (0)
 
 cudaError_t launch_step_ring(const StepParams& p, int mode, bool vec, cudaStream_t s)
 {
-    GPGA_DISPATCH(step_ring_kernel, p, mode, vec, s);
+    GPGA_DISPATCH(step_ring_kernel, RingTune, p, mode, vec, s);
 }
 cudaError_t launch_step_exp(const StepParams& p, int mode, bool vec, cudaStream_t s)
 {
-    GPGA_DISPATCH(step_exp_kernel, p, mode, vec, s);
+    GPGA_DISPATCH(step_exp_kernel, ExpTune, p, mode, vec, s);
 }
 cudaError_t launch_step_global(const StepParams& p, int mode, bool vec, cudaStream_t s)
 {
-    GPGA_DISPATCH(step_global_kernel, p, mode, vec, s);
+    GPGA_DISPATCH(step_global_kernel, GlobalTune, p, mode, vec, s);
 }
+#endif  // GPGA_TUNING_HARNESS
 
 // ---------------------------------------------------------------------------
 // Consensus distance sum_j sum_i (x_ij - xbar_j)^2.  One pass over X: with
@@ -190,7 +266,7 @@ int consensus_blocks(long long Q)
 template <bool VEC>
 __global__ void __launch_bounds__(kReduceBlock) consensus_kernel(const float* __restrict__ x,
                                                                  long long n, long long d,
-                                                                 long long Q,
+                                                                 long long ld, long long Q,
                                                                  double* __restrict__ partials)
 {
     double acc = 0.0;
@@ -201,7 +277,7 @@ __global__ void __launch_bounds__(kReduceBlock) consensus_kernel(const float* __
         double s1[4] = {0, 0, 0, 0}, s2[4] = {0, 0, 0, 0};
 #pragma unroll 4
         for (long long i = 1; i < n; ++i) {
-            const float4 v = load4<VEC>(x + i * d, j0, d);
+            const float4 v = load4<VEC>(x + i * ld, j0, d);
             const double e0 = (double)v.x - (double)r0.x, e1 = (double)v.y - (double)r0.y;
             const double e2 = (double)v.z - (double)r0.z, e3 = (double)v.w - (double)r0.w;
             s1[0] += e0; s2[0] = fma(e0, e0, s2[0]);
@@ -231,41 +307,56 @@ __global__ void final_sum_kernel(const double* __restrict__ partials, int count,
     if (threadIdx.x == 0) *result = v * scale;
 }
 
-cudaError_t launch_consensus(const float* x, long long n, long long d, bool vec, double* partials,
+cudaError_t launch_consensus(const float* x, long long n, long long d, long long ld, bool vec, double* partials,
                              double* result, cudaStream_t s)
 {
     const long long Q = (d + 3) / 4;
     const int blocks = consensus_blocks(Q);
     if (vec)
-        consensus_kernel<true><<<blocks, kReduceBlock, 0, s>>>(x, n, d, Q, partials);
+        consensus_kernel<true><<<blocks, kReduceBlock, 0, s>>>(x, n, d, ld, Q, partials);
     else
-        consensus_kernel<false><<<blocks, kReduceBlock, 0, s>>>(x, n, d, Q, partials);
+        consensus_kernel<false><<<blocks, kReduceBlock, 0, s>>>(x, n, d, ld, Q, partials);
     final_sum_kernel<<<1, 32, 0, s>>>(partials, blocks, 1.0, result);
     return cudaGetLastError();
 }
 
 // (1/n) sum_i 1/2 ||x_i - b_i||^2 over all elements.
+template <bool VEC>
 __global__ void __launch_bounds__(kReduceBlock) quadratic_loss_kernel(const float* __restrict__ x,
                                                                       const float* __restrict__ b,
-                                                                      long long total,
+                                                                      long long n, long long d,
+                                                                      long long ld, long long Q,
                                                                       double* __restrict__ partials)
 {
     double acc = 0.0;
-    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total;
-         e += (long long)gridDim.x * blockDim.x) {
-        const double r = (double)__ldcs(x + e) - (double)__ldcs(b + e);
-        acc = fma(r, r, acc);
+    for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < Q;
+         q += (long long)gridDim.x * blockDim.x) {
+        const long long j0 = q * 4;
+#pragma unroll 4
+        for (long long i = 0; i < n; ++i) {
+            const float4 xv = load4<VEC>(x + i * ld, j0, d);   // columns past d load as zeros
+            const float4 bv = load4<VEC>(b + i * ld, j0, d);
+            const double r0 = (double)xv.x - (double)bv.x, r1 = (double)xv.y - (double)bv.y;
+            const double r2 = (double)xv.z - (double)bv.z, r3 = (double)xv.w - (double)bv.w;
+            acc = fma(r0, r0, acc);
+            acc = fma(r1, r1, acc);
+            acc = fma(r2, r2, acc);
+            acc = fma(r3, r3, acc);
+        }
     }
     acc = block_sum(acc);
     if (threadIdx.x == 0) partials[blockIdx.x] = acc;
 }
 
-cudaError_t launch_quadratic_loss(const float* x, const float* b, long long n, long long d,
-                                  double* partials, double* result, cudaStream_t s)
+cudaError_t launch_quadratic_loss(const float* x, const float* b, long long n, long long d, long long ld,
+                                  bool vec, double* partials, double* result, cudaStream_t s)
 {
-    const long long total = n * d;
-    const int blocks = consensus_blocks(total);
-    quadratic_loss_kernel<<<blocks, kReduceBlock, 0, s>>>(x, b, total, partials);
+    const long long Q = (d + 3) / 4;
+    const int blocks = consensus_blocks(Q);
+    if (vec)
+        quadratic_loss_kernel<true><<<blocks, kReduceBlock, 0, s>>>(x, b, n, d, ld, Q, partials);
+    else
+        quadratic_loss_kernel<false><<<blocks, kReduceBlock, 0, s>>>(x, b, n, d, ld, Q, partials);
     final_sum_kernel<<<1, 32, 0, s>>>(partials, blocks, 0.5 / (double)n, result);
     return cudaGetLastError();
 }
@@ -275,7 +366,7 @@ cudaError_t launch_quadratic_loss(const float* x, const float* b, long long n, l
 // ---------------------------------------------------------------------------
 template <bool VEC>
 __global__ void __launch_bounds__(kBlock) init_b_kernel(float* __restrict__ b, long long n,
-                                                        long long d, long long Q, uint32_t q_base,
+                                                        long long d, long long ld, long long Q, uint32_t q_base,
                                                         float shift, const PhiloxKeys keys)
 {
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -289,13 +380,13 @@ __global__ void __launch_bounds__(kBlock) init_b_kernel(float* __restrict__ b, l
             z.z = fmaf(shift, s, z.z);
             z.w = fmaf(shift, s, z.w);
         }
-        store4<VEC>(b + i * d, q * 4, d, z);
+        store4<VEC>(b + i * ld, q * 4, d, z);
     }
 }
 
 template <bool VEC>
 __global__ void __launch_bounds__(kBlock) init_x0_kernel(float* __restrict__ x, long long n,
-                                                         long long d, long long Q, uint32_t q_base,
+                                                         long long d, long long ld, long long Q, uint32_t q_base,
                                                          int kind, float std, const PhiloxKeys keys)
 {
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -304,29 +395,29 @@ __global__ void __launch_bounds__(kBlock) init_x0_kernel(float* __restrict__ x, 
     if (kind == 1) v = scale4(normal4(q_base + (uint32_t)q, 0u, 0u, 2u, keys), std);
     for (long long i = 0; i < n; ++i) {
         if (kind == 2) v = scale4(normal4(q_base + (uint32_t)q, (uint32_t)i, 0u, 2u, keys), std);
-        store4<VEC>(x + i * d, q * 4, d, v);
+        store4<VEC>(x + i * ld, q * 4, d, v);
     }
 }
 
-cudaError_t launch_init_b(float* b, long long n, long long d, uint32_t q_base, float shift, bool vec,
+cudaError_t launch_init_b(float* b, long long n, long long d, long long ld, uint32_t q_base, float shift, bool vec,
                           const PhiloxKeys& keys, cudaStream_t s)
 {
     const long long Q = (d + 3) / 4;
     if (vec)
-        init_b_kernel<true><<<grid_for(Q, kBlock), kBlock, 0, s>>>(b, n, d, Q, q_base, shift, keys);
+        init_b_kernel<true><<<grid_for(Q, kBlock), kBlock, 0, s>>>(b, n, d, ld, Q, q_base, shift, keys);
     else
-        init_b_kernel<false><<<grid_for(Q, kBlock), kBlock, 0, s>>>(b, n, d, Q, q_base, shift, keys);
+        init_b_kernel<false><<<grid_for(Q, kBlock), kBlock, 0, s>>>(b, n, d, ld, Q, q_base, shift, keys);
     return cudaGetLastError();
 }
 
-cudaError_t launch_init_x0(float* x, long long n, long long d, uint32_t q_base, int kind, float std,
+cudaError_t launch_init_x0(float* x, long long n, long long d, long long ld, uint32_t q_base, int kind, float std,
                            bool vec, const PhiloxKeys& keys, cudaStream_t s)
 {
     const long long Q = (d + 3) / 4;
     if (vec)
-        init_x0_kernel<true><<<grid_for(Q, kBlock), kBlock, 0, s>>>(x, n, d, Q, q_base, kind, std, keys);
+        init_x0_kernel<true><<<grid_for(Q, kBlock), kBlock, 0, s>>>(x, n, d, ld, Q, q_base, kind, std, keys);
     else
-        init_x0_kernel<false><<<grid_for(Q, kBlock), kBlock, 0, s>>>(x, n, d, Q, q_base, kind, std, keys);
+        init_x0_kernel<false><<<grid_for(Q, kBlock), kBlock, 0, s>>>(x, n, d, ld, Q, q_base, kind, std, keys);
     return cudaGetLastError();
 }
 

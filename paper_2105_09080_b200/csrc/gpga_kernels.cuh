@@ -19,6 +19,8 @@ struct StepParams {
     const float* b;   // quadratic: targets b; GRAD_BUFFER: gradient matrix G
     float* out;       // X^(k+1), n x d
     long long n, d;
+    long long ld;     // row stride of x and out, in floats (>= d)
+    long long ldb;    // row stride of b, in floats
     long long Q;      // column groups of four: ceil(d / 4)
     uint32_t q_base;  // global index of local group 0 (column offset / 4)
     uint32_t k;       // iteration index (third counter word)
@@ -39,16 +41,16 @@ cudaError_t launch_step_tile(const StepParams& p, int mode, bool vec, int topolo
 // Consensus distance: partials (one double per block) then a fixed-order final sum.
 constexpr int kMaxReduceBlocks = 148 * 8;   // capacity of the partials array, in doubles
 int consensus_blocks(long long Q);
-cudaError_t launch_consensus(const float* x, long long n, long long d, bool vec, double* partials,
+cudaError_t launch_consensus(const float* x, long long n, long long d, long long ld, bool vec, double* partials,
                              double* result, cudaStream_t s);
 // (1/n) sum_i 1/2 ||x_i - b_i||^2, same two-stage reduction.
-cudaError_t launch_quadratic_loss(const float* x, const float* b, long long n, long long d,
-                                  double* partials, double* result, cudaStream_t s);
+cudaError_t launch_quadratic_loss(const float* x, const float* b, long long n, long long d, long long ld,
+                                  bool vec, double* partials, double* result, cudaStream_t s);
 
 // Seeded fills (quadratic objective).
-cudaError_t launch_init_b(float* b, long long n, long long d, uint32_t q_base, float shift, bool vec,
+cudaError_t launch_init_b(float* b, long long n, long long d, long long ld, uint32_t q_base, float shift, bool vec,
                           const PhiloxKeys& keys, cudaStream_t s);
-cudaError_t launch_init_x0(float* x, long long n, long long d, uint32_t q_base, int kind, float std,
+cudaError_t launch_init_x0(float* x, long long n, long long d, long long ld, uint32_t q_base, int kind, float std,
                            bool vec, const PhiloxKeys& keys, cudaStream_t s);
 
 // Generator surface.

@@ -40,7 +40,7 @@ __global__ void __launch_bounds__(kLrBlock) logreg_partial_kernel(const LogregPa
     const int nrows = min(kChunkRows, (int)p.batch - t0);
     const float* A = p.A + (long long)i * p.m * p.d;
     const float* y = p.y + (long long)i * p.m;
-    const float* x = p.x + (long long)i * p.d;
+    const float* x = p.x + (long long)i * p.ldx;
     for (int j = threadIdx.x; j < p.d; j += blockDim.x) xs[j] = x[j];
     if (threadIdx.x < nrows)
         rows[threadIdx.x] = batch_row((uint32_t)(t0 + threadIdx.x), (uint32_t)i, p.k, (uint32_t)p.m, p.keys);
@@ -84,8 +84,10 @@ __global__ void __launch_bounds__(kLrBlock) logreg_partial_kernel(const LogregPa
 __global__ void __launch_bounds__(kLrBlock) logreg_reduce_kernel(const LogregParams p, int chunks)
 {
     const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const long long total4 = p.n * (p.d >> 2);
+    const long long d4 = p.d >> 2;
+    const long long total4 = p.n * d4;
     if (e >= total4) return;
+    const long long row = e / d4, g = e - row * d4;
     const float4* part = reinterpret_cast<const float4*>(p.partial);
     float4 acc = part[e];
     for (int c = 1; c < chunks; ++c) {
@@ -95,7 +97,7 @@ __global__ void __launch_bounds__(kLrBlock) logreg_reduce_kernel(const LogregPar
         acc.z += v.z;
         acc.w += v.w;
     }
-    const float4 xv = reinterpret_cast<const float4*>(p.x)[e];
+    const float4 xv = reinterpret_cast<const float4*>(p.x + row * p.ldx)[g];
     const float inv = 1.0f / (float)p.batch;
     reinterpret_cast<float4*>(p.G)[e] =
         make_float4(fmaf(acc.x, inv, p.l2 * xv.x), fmaf(acc.y, inv, p.l2 * xv.y),
@@ -108,7 +110,7 @@ __global__ void __launch_bounds__(kLrBlock) logreg_loss_kernel(const LogregParam
     const int i = blockIdx.x;
     const float* A = p.A + (long long)i * p.m * p.d;
     const float* y = p.y + (long long)i * p.m;
-    const float* x = p.x + (long long)i * p.d;
+    const float* x = p.x + (long long)i * p.ldx;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     double acc = 0.0;
     for (int t = warp; t < (int)p.batch; t += nwarps) {

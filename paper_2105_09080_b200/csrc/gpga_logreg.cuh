@@ -12,7 +12,8 @@ constexpr int kChunkRows = 32;   // batch rows per block
 struct LogregParams {
     const float* A;   // n x m x d
     const float* y;   // n x m, +-1
-    const float* x;   // n x d, current state
+    const float* x;   // n x d, current state, row stride ldx
+    long long ldx;
     float* partial;   // chunks x n x d
     float* G;         // n x d
     long long n, d, m, batch;

@@ -17,8 +17,8 @@ template <int MODE, bool VEC>
 __device__ __forceinline__ float4 tile_half_step(const StepParams& p, long long i, long long q)
 {
     const long long j0 = q * 4;
-    const float4 x = load4<VEC>(p.x + i * p.d, j0, p.d);
-    const float4 b = load4<VEC>(p.b + i * p.d, j0, p.d);
+    const float4 x = load4<VEC>(p.x + i * p.ld, j0, p.d);
+    const float4 b = load4<VEC>(p.b + i * p.ldb, j0, p.d);
     float4 g;
     if (MODE == GRAD_BUFFER) {
         g = b;
@@ -85,7 +85,7 @@ __global__ void __launch_bounds__(kTileBlock) step_tile_kernel(const StepParams 
         s.y *= w;
         s.z *= w;
         s.w *= w;
-        store4<VEC>(p.out + (long long)i * p.d, q * 4, p.d, s);
+        store4<VEC>(p.out + (long long)i * p.ld, q * 4, p.d, s);
     }
 }
 

@@ -85,6 +85,8 @@ def test_not_ready_and_setter_checks(L):
     assert L.gpga_set_column_offset(h, -4) == pkg.GPGA_ERR_INVALID_ARG
     assert L.gpga_set_column_offset(h, 2**34) == pkg.GPGA_ERR_INVALID_ARG
     assert L.gpga_set_column_offset(h, 1024) == pkg.GPGA_OK
+    assert L.gpga_set_row_stride(h, 63) == pkg.GPGA_ERR_INVALID_ARG
+    assert L.gpga_set_row_stride(h, 96) == pkg.GPGA_OK
     assert L.gpga_set_grid_cols(h, 3) == pkg.GPGA_ERR_INVALID_ARG
     assert L.gpga_set_grid_cols(h, 4) == pkg.GPGA_OK
     assert L.gpga_launch_count(h) == 0
@@ -114,6 +116,7 @@ def test_objective_and_bind_checks(L):
     assert L.gpga_bind(h, a, b, c, None, s, nbytes - 1) == pkg.GPGA_ERR_INVALID_ARG
     assert L.gpga_bind(h, a, b, c, None, s, nbytes) == pkg.GPGA_OK
     assert L.gpga_set_objective(h, 0, 0.2, 0.0, 0, 0) == pkg.GPGA_ERR_INVALID_ARG      # after bind
+    assert L.gpga_set_row_stride(h, 128) == pkg.GPGA_ERR_INVALID_ARG                   # after bind
     assert L.gpga_step(h, -1, None) == pkg.GPGA_ERR_INVALID_ARG
     assert L.gpga_step(h, 2**32, None) == pkg.GPGA_ERR_INVALID_ARG
     assert L.gpga_run(h, -1, None) == pkg.GPGA_ERR_INVALID_ARG

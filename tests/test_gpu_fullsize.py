@@ -43,11 +43,14 @@ def _free_gib():
     return free / 2**30
 
 
-def _run_case(bufs, n, d, topo, H, gamma, sigma, K, x0_kind, x0_std, b_shift, offs, one_step_ks):
+def _run_case(bufs, n, d, topo, H, gamma, sigma, K, x0_kind, x0_std, b_shift, offs, one_step_ks, ld=None):
     xa, xb, b, scratch = bufs
+    ld = ld or d
+    xa, xb, b = (t.view(-1)[:n * ld].view(n, ld) for t in (xa, xb, b))
     okind = {pkg.GPGA_X0_ZERO: o.X0_ZERO, pkg.GPGA_X0_SHARED_NORMAL: o.X0_SHARED_NORMAL}[x0_kind]
     g = pkg.Gpga(n, d, TOPO[topo][0], H, gamma, SEED)
     g.set_objective(pkg.GPGA_OBJ_QUADRATIC, sigma=sigma)
+    g.set_row_stride(ld)
     g.bind(xa, xb, b, scratch=scratch)
     width = lambda c0: min(BLOCK, d - c0)
     ora = {}
@@ -85,7 +88,8 @@ def test_config_3_resnet50_sized():
     n, d, gamma, sigma, K = 64, 25_557_032, 0.01, 0.01, 50
     if _free_gib() < 3 * n * d * 4 / 2**30 + 2:
         pytest.skip("not enough free device memory")
-    xa = torch.empty((n, d), dtype=torch.float32, device="cuda")
+    ld = (d + 31) // 32 * 32          # the benchmark's layout: rows padded to 128 bytes
+    xa = torch.empty((n, ld), dtype=torch.float32, device="cuda")
     xb = torch.empty_like(xa)
     b = torch.empty_like(xa)
     scratch = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
@@ -97,7 +101,10 @@ def test_config_3_resnet50_sized():
             if H == 4:
                 ks = [0, 3] if topo == "ring" else [0, 1, 2, 3, 4, 5]   # hops 1..32; k=3 is global
             _run_case((xa, xb, b, scratch), n, d, topo, H, gamma, sigma, K,
-                      pkg.GPGA_X0_SHARED_NORMAL, 0.1, 0.5, offs, ks)
+                      pkg.GPGA_X0_SHARED_NORMAL, 0.1, 0.5, offs, ks, ld=ld)
+    # the dense layout (row stride d, rows not 128-byte aligned) once as well
+    _run_case((xa, xb, b, scratch), n, d, "ring", 4, gamma, sigma, 8, pkg.GPGA_X0_SHARED_NORMAL, 0.1, 0.5,
+              offs, [0], ld=d)
     del xa, xb, b
     torch.cuda.empty_cache()
 

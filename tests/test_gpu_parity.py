@@ -145,6 +145,54 @@ def test_tile_topologies_one_step(topo, n, gc, d):
     g.close()
 
 
+@pytest.mark.parametrize("topo,H,k", [("ring", 0, 1), ("exp", 0, 2), ("ring", 2, 1), ("grid", 0, 0)])
+@pytest.mark.parametrize("d,ld", [(1000, 1024), (1030, 1056), (7, 9), (1026, 1027)])
+def test_padded_row_stride(topo, H, k, d, ld):
+    """Rows padded to ld floats: same results as the dense layout; padding is never touched."""
+    torch = _torch()
+    n = 8
+    X0, B = quadratic_inputs(n, d, 500 + d, x0="per_node")
+    g = pkg.Gpga(n, d, TOPO[topo][0], H, 0.2, 13)
+    g.set_objective(pkg.GPGA_OBJ_QUADRATIC, sigma=0.3)
+    g.set_row_stride(ld)
+    sentinel = -12345.0
+    bufs = [torch.full((n, ld), sentinel, dtype=torch.float32, device="cuda") for _ in range(3)]
+    bufs[0][:, :d] = torch.from_numpy(X0).cuda()
+    bufs[2][:, :d] = torch.from_numpy(B).cuda()
+    g.bind(*bufs)
+    g.step(k)
+    p = o.Problem(TOPO[topo][1], H, 0.2, 13, sigma=0.3, data=B, grid_cols=4 if topo == "grid" else 0)
+    want = o.step(p, X0, k)
+    out = g.get_x().cpu().numpy()
+    ok, worst = close(out[:, :d], want, TOL_STEP)
+    assert ok, worst
+    assert np.all(out[:, d:] == sentinel)
+    xi = o.consensus_distance(want)
+    assert abs(g.consensus_distance() - xi) <= 1e-5 * xi + n * d * (2.0**-22 * 8) ** 2
+    assert abs(g.mean_loss() - o.quadratic_mean_loss(out[:, :d], B)) <= 1e-6 * o.quadratic_mean_loss(want, B)
+    g.init_from_seed(pkg.GPGA_X0_PER_NODE_NORMAL, 1.0, 0.5)
+    assert np.abs(bufs[2].cpu().numpy()[:, :d] - o.init_b(n, d, 13, 0.5)).max() <= 3e-5
+    assert np.all(bufs[2].cpu().numpy()[:, d:] == sentinel)
+    assert np.all(bufs[0].cpu().numpy()[:, d:] == sentinel)
+    g.close()
+
+
+def test_run_host_with_padded_rows():
+    torch = _torch()
+    n, d, ld, K = 4, 1000, 1024, 5
+    X0, B = quadratic_inputs(n, d, 9)
+    g, _ = make_quadratic(n, d, "ring", 2, 0.1, 3, 0.2, X0, B)
+    g.run(K)
+    want = g.get_x().cpu().numpy()
+    g2 = pkg.Gpga(n, d, pkg.GPGA_TOPO_RING, 2, 0.1, 3)
+    g2.set_objective(pkg.GPGA_OBJ_QUADRATIC, sigma=0.2)
+    g2.set_row_stride(ld)
+    g2.allocate()
+    out = torch.empty((n, d), dtype=torch.float32).pin_memory()
+    g2.run_host(torch.from_numpy(X0).pin_memory(), torch.from_numpy(B).pin_memory(), K, out)
+    assert np.array_equal(out.numpy(), want)
+
+
 def test_column_offset_keys_the_noise():
     n, d, c0 = 4, 64, 4096
     X0, B = quadratic_inputs(n, d, 1)
