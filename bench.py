@@ -55,7 +55,11 @@ DEFAULT_WORKLOAD = "c3_ring_h4"
 # dram__bytes_write.sum), as a multiple of the algorithmic bytes of the captured launch, with
 # the digest of the kernel sources at capture time.  A changed source voids it (-> null).
 NCU_TRAFFIC = {
-    # kernel name: (traffic / algorithmic bytes, source digest)
+    # kernel name: (traffic / algorithmic bytes, source digest); captured at n=64, d=2,097,192 and
+    # n=16, d=8,388,608 -- one pass over three n x d arrays, so traffic scales with n x d
+    "step_ring_kernel": (0.977, "df2c2ab79bfda5b5"),
+    "step_exp_kernel": (0.977, "df2c2ab79bfda5b5"),
+    "step_global_kernel": (0.966, "df2c2ab79bfda5b5"),
 }
 
 
@@ -237,7 +241,8 @@ def run_ours(args, w, name):
     kind = {"zero": pkg.GPGA_X0_ZERO, "shared": pkg.GPGA_X0_SHARED_NORMAL}[w["x0"]]
     g = pkg.Gpga(n, d, topo, w["H"], w["gamma"], SEED)
     g.set_objective(pkg.GPGA_OBJ_QUADRATIC, sigma=w["sigma"])
-    g.set_column_offset(rank * ((d + 3) // 4 * 4))
+    from paper_2105_09080_b200.sharding import weak_shard_offset
+    g.set_column_offset(weak_shard_offset(rank, d))
     g.set_row_stride(padded_stride(d))      # every node's row starts on a 128-byte line
     xa, xb, b = g.allocate()
     g.init_from_seed(kind, w["x0_std"], w["b_shift"])
