@@ -221,6 +221,43 @@ int32_t gpga_box_muller_words(const uint32_t* a_dev, const uint32_t* b_dev, int6
 int32_t gpga_normal_fill(uint64_t seed, uint32_t stream_id, uint32_t k, uint32_t i, uint32_t q0,
                          int64_t count, float* out_dev, void* stream);
 
+/*
+ * (No counterpart in the paper: a packaging variant of the logistic mini-batch gradient
+ * above, for callers that cannot allocate device memory.)
+ *
+ * Some code cannot call cudaMalloc at the point where it needs a gradient: a serving or
+ * training loop that must not synchronise the device, a plug-in that is handed tensors by
+ * a host framework and has no allocator of its own, code running under another runtime's
+ * memory pool.  This entry point computes the same mini-batch gradient matrix as the
+ * logistic objective of gpga_step,
+ *     G[i][:] = -(1/batch) sum_{r in batch(seed,k,i)} y_r a_r / (1 + exp(y_r a_r^T x_i)) + l2 x_i,
+ * without a handle and without any caller-provided scratch: its intermediate partial sums
+ * go to a fixed array of GPGA_NOALLOC_SCRATCH_BYTES built into the library.  Every GPU
+ * that loads the library carries that array until the process exits.
+ *
+ *  A_dev : n*m*d fp32 (device), y_dev : n*m fp32 in {-1,+1} (device),
+ *  x_dev : n rows of d fp32 with row stride ldx (device), G_dev : n*d fp32 OUTPUT (device).
+ *  A_dev, x_dev, G_dev 16-byte aligned; d and ldx multiples of 4.
+ *  needed_bytes_host (host, may be NULL) receives the scratch bytes this problem needs,
+ *  ceil(batch/32) * n * d * 4.
+ *
+ * Behaviour to rely on:
+ *  - It calls no allocating routine.  The first call on a device resolves the array's
+ *    address (a symbol lookup); make that first call before any stream capture begins.
+ *  - Asynchronous on `stream`.  All calls on a device share the one array, which keeps the
+ *    previous call's contents; each call writes every element it later reads, so nothing
+ *    has to be cleared, but calls that overlap on the GPU race.  Issue them on one stream.
+ *  - Errors: INVALID_ARG for NULL or misaligned pointers and out-of-range sizes;
+ *    UNSUPPORTED when the problem needs more than GPGA_NOALLOC_SCRATCH_BYTES (the need is
+ *    reported in *needed_bytes_host; use gpga_step with a bound scratch buffer instead);
+ *    CUDA if a CUDA call fails.
+ */
+#define GPGA_NOALLOC_SCRATCH_BYTES (4 * 1024 * 1024)
+int32_t gpga_logistic_gradient_noalloc(const float* A_dev, const float* y_dev, const float* x_dev,
+                                       int64_t ldx, int64_t n, int64_t d, int64_t m, int64_t batch,
+                                       float l2, uint64_t seed, int64_t k, float* G_dev, void* stream,
+                                       int64_t* needed_bytes_host);
+
 #ifdef __cplusplus
 }
 #endif

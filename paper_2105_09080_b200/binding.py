@@ -62,7 +62,11 @@ SIGNATURES = {
     "gpga_philox_words": (_i32, [_P, _u32, _u32, _i64, _P, _P]),
     "gpga_box_muller_words": (_i32, [_P, _P, _i64, _P, _P]),
     "gpga_normal_fill": (_i32, [_u64, _u32, _u32, _u32, _u32, _i64, _P, _P]),
+    "gpga_logistic_gradient_noalloc": (_i32, [_P, _P, _P, _i64, _i64, _i64, _i64, _i64, _f32, _u64, _i64,
+                                              _P, _P, C.POINTER(_i64)]),
 }
+
+GPGA_NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024
 
 _lib = None
 
@@ -264,3 +268,26 @@ def normal_fill(seed, stream_id, k, i, q0, count, device="cuda", stream=None):
     if st != GPGA_OK:
         raise GpgaError(st, lib().gpga_last_error(None).decode())
     return out
+
+
+def logistic_gradient_noalloc(A, y, x, batch, l2, seed, k, out=None, stream=None):
+    """Mini-batch logistic gradient matrix without any device allocation by the library.
+
+    For callers that cannot allocate device memory themselves at the point of the call
+    (no-sync loops, plug-ins that only receive tensors): the library's built-in scratch
+    array holds the intermediate partial sums.  A (n, m, d), y (n, m), x (n, d or a view
+    with a row stride) and `out` (n, d) are the caller's CUDA tensors; `out` must be given
+    by such callers (it is only created here as a convenience when omitted).  Returns
+    (status, needed_scratch_bytes, out); the status is GPGA_ERR_UNSUPPORTED when the
+    problem needs more than GPGA_NOALLOC_SCRATCH_BYTES.  Calls sharing a device must not
+    overlap on the GPU; make the first call on a device outside stream capture.
+    """
+    import torch
+    n, m, d = A.shape
+    if out is None:
+        out = torch.empty((n, d), dtype=torch.float32, device=A.device)
+    need = _i64()
+    st = lib().gpga_logistic_gradient_noalloc(A.data_ptr(), y.data_ptr(), x.data_ptr(), x.stride(0), n, d, m,
+                                              batch, l2, seed, k, out.data_ptr(), _stream_ptr(stream),
+                                              C.byref(need))
+    return st, int(need.value), out
