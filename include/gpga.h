@@ -74,7 +74,7 @@ enum {
  * and averaging period H.  H = 0 encodes H -> infinity (plain Gossip SGD,
  * Section 3); H = 1 is parallel SGD.  The default objective is the quadratic
  * f_i(x) = 1/2 ||x - b_i||^2 with sigma = 0.
- * Errors: INVALID_ARG for n < 1, d < 1, n >= 2^32, d >= 2^34, H < 0, gamma not
+ * Errors: INVALID_ARG for n < 1, d < 1, n >= 2^31, d >= 2^34, H < 0, gamma not
  * finite or negative, unknown topology, NULL out; UNSUPPORTED for EXP or
  * STATIC_EXP with n not a power of two.
  */

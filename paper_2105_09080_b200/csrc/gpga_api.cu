@@ -40,6 +40,7 @@ static thread_local std::string g_create_error;
 namespace {
 
 constexpr int64_t kMaxTileNodes = 4096;   // shared-memory tile path: n * 16 B <= 64 KB
+constexpr int64_t kNarrowGroups = 148 * 32;   // fewer column groups than this: use the tile kernel
 
 int32_t fail(gpga_ctx* c, int32_t code, const std::string& msg)
 {
@@ -124,32 +125,49 @@ int32_t do_step(gpga_ctx* c, int64_t k, bool global, cudaStream_t s)
     p.gamma = c->gamma; p.sigma = c->sigma;
     p.hop_log2 = 0; p.len_log2 = 0;
     p.grid_cols = (int)c->grid_cols;
+    p.chunks = 0; p.inv_batch = 0.f; p.l2 = 0.f;
     p.keys = c->keys;
     const bool vec = vec_ok(c);
     int mode = (c->sigma != 0.f) ? GRAD_QUAD_NOISE : GRAD_QUAD;
+    // Narrow states (few column groups) go through the tile kernel, which spreads threads over
+    // (row, group) cells; one thread per group would leave most of the GPU idle.
+    const bool narrow = p.Q < kNarrowGroups && tile_supports(c->n);
+    const bool tile_topology = c->topology != GPGA_TOPO_RING && c->topology != GPGA_TOPO_EXP;
     cudaError_t e;
     if (c->objective == GPGA_OBJ_LOGISTIC) {
         const LogregParams lp = logreg_params(c, k);
-        e = launch_logreg_grad(lp, s);
-        c->launches += 2;
+        if (narrow) {   // the step kernel adds the chunk partials itself: one launch fewer
+            e = launch_logreg_partial(lp, s);
+            c->launches += 1;
+            p.b = lp.partial;
+            p.chunks = logreg_chunks(c->batch);
+            p.inv_batch = 1.0f / (float)c->batch;
+            p.l2 = c->l2;
+            mode = GRAD_PARTIALS;
+        } else {
+            e = launch_logreg_grad(lp, s);
+            c->launches += 2;
+            p.b = lp.G;
+            mode = GRAD_BUFFER;
+        }
         if (e != cudaSuccess) return cuda_fail(c, e, "logistic gradient launch");
-        p.b = lp.G;
         p.ldb = c->d;
-        mode = GRAD_BUFFER;
     }
-    if (global) {
-        e = launch_step_global(p, mode, vec, s);
-    } else if (c->topology == GPGA_TOPO_RING) {
-        e = launch_step_ring(p, mode, vec, s);
-    } else if (c->topology == GPGA_TOPO_EXP) {
+    if (c->topology == GPGA_TOPO_EXP) {
         const int tau = log2_floor(c->n);
         if (tau > 0) {
             p.hop_log2 = (int)(k % tau);
             p.len_log2 = tau - p.hop_log2;
         }
-        e = launch_step_exp(p, mode, vec, s);
+    }
+    if (narrow || (tile_topology && !global)) {
+        e = launch_step_tile(p, mode, vec, global ? (int)TILE_MIX_GLOBAL : c->topology, s);
+    } else if (global) {
+        e = launch_step_global(p, mode, vec, s);
+    } else if (c->topology == GPGA_TOPO_RING) {
+        e = launch_step_ring(p, mode, vec, s);
     } else {
-        e = launch_step_tile(p, mode, vec, c->topology, s);
+        e = launch_step_exp(p, mode, vec, s);
     }
     c->launches += 1;
     if (e != cudaSuccess) return cuda_fail(c, e, "step launch");
@@ -194,7 +212,7 @@ int32_t gpga_create(int64_t n, int64_t d, int32_t topology, int64_t H, float gam
 {
     if (!out) return fail(nullptr, GPGA_ERR_INVALID_ARG, "out is NULL");
     *out = nullptr;
-    if (n < 1 || n >= (int64_t(1) << 32)) return fail(nullptr, GPGA_ERR_INVALID_ARG, "n must be in [1, 2^32)");
+    if (n < 1 || n >= (int64_t(1) << 31)) return fail(nullptr, GPGA_ERR_INVALID_ARG, "n must be in [1, 2^31)");
     if (d < 1 || d >= (int64_t(1) << 34)) return fail(nullptr, GPGA_ERR_INVALID_ARG, "d must be in [1, 2^34)");
     if (H < 0) return fail(nullptr, GPGA_ERR_INVALID_ARG, "H must be >= 0 (0 = never average globally)");
     if (!std::isfinite(gamma) || gamma < 0.f) return fail(nullptr, GPGA_ERR_INVALID_ARG, "gamma must be finite and >= 0");
@@ -284,6 +302,8 @@ int32_t gpga_bind(gpga_t* c, void* x_a, void* x_b, void* data, const void* label
         return fail(c, GPGA_ERR_INVALID_ARG, "device pointers must be 16-byte aligned");
     if (c->objective == GPGA_OBJ_LOGISTIC && !labels)
         return fail(c, GPGA_ERR_INVALID_ARG, "logistic objective needs labels");
+    if (c->objective == GPGA_OBJ_LOGISTIC && (c->ld % 4) != 0)
+        return fail(c, GPGA_ERR_INVALID_ARG, "logistic objective needs a row stride that is a multiple of 4");
     if (scratch_bytes < scratch_layout(c).total) return fail(c, GPGA_ERR_INVALID_ARG, "scratch too small");
     c->x[0] = static_cast<float*>(x_a);
     c->x[1] = static_cast<float*>(x_b);

@@ -84,6 +84,7 @@ __device__ __forceinline__ float2 box_muller(uint32_t a, uint32_t b)
         const float t = (float)(0xFFFFFFu - m) * 0x1p-24f;   // 1 - u1, exact
         neg2ln = t * (2.0f + t * (1.0f + t * 0.6666667f));
     } else {
+        // (the exact scaling to (0,1] first: the hardware log2 is most accurate near 1)
         const float u1 = (float)(m + 1u) * 0x1p-24f;
         neg2ln = -1.3862943611198906f * fast_lg2(u1);
     }

@@ -29,17 +29,53 @@ struct RowIn {
     float4 x, b;
 };
 
+// What one thread needs to address its group of four columns in any row.  Row indices
+// are 32-bit (n < 2^31); the element offset row * ld is formed in 64 bits.
+struct ColGroup {
+    const float* x;    // p.x + j0 (128-bit path) or p.x
+    const float* b;
+    float* out;
+    long long j0;      // first local column of the group
+    uint32_t qg;       // global group index = first counter word of the generator
+};
+
 template <bool VEC>
-__device__ __forceinline__ RowIn load_row(const StepParams& p, long long i, long long q)
+__device__ __forceinline__ ColGroup col_group(const StepParams& p, long long q)
+{
+    ColGroup c;
+    c.j0 = q * 4;
+    c.x = VEC ? p.x + c.j0 : p.x;
+    c.b = VEC ? p.b + c.j0 : p.b;
+    c.out = VEC ? p.out + c.j0 : p.out;
+    c.qg = p.q_base + (uint32_t)q;
+    return c;
+}
+
+template <bool VEC>
+__device__ __forceinline__ RowIn load_row(const StepParams& p, const ColGroup& c, int i)
 {
     RowIn r;
-    r.x = load4<VEC>(p.x + i * p.ld, q * 4, p.d);
-    r.b = load4<VEC>(p.b + i * p.ldb, q * 4, p.d);
+    if (VEC) {
+        r.x = ld_stream4(c.x + (long long)i * p.ld);
+        r.b = ld_stream4(c.b + (long long)i * p.ldb);
+    } else {
+        r.x = load4<false>(c.x + (long long)i * p.ld, c.j0, p.d);
+        r.b = load4<false>(c.b + (long long)i * p.ldb, c.j0, p.d);
+    }
     return r;
 }
 
+template <bool VEC>
+__device__ __forceinline__ void store_row(const StepParams& p, const ColGroup& c, int i, float4 v)
+{
+    if (VEC)
+        st_stream4(c.out + (long long)i * p.ld, v);
+    else
+        store4<false>(c.out + (long long)i * p.ld, c.j0, p.d, v);
+}
+
 template <int MODE>
-__device__ __forceinline__ float4 finish_row(const StepParams& p, const RowIn& r, long long i, long long q)
+__device__ __forceinline__ float4 finish_row(const StepParams& p, const ColGroup& c, const RowIn& r, int i)
 {
     float4 g;
     if (MODE == GRAD_BUFFER) {
@@ -47,7 +83,7 @@ __device__ __forceinline__ float4 finish_row(const StepParams& p, const RowIn& r
     } else {
         g = make_float4(r.x.x - r.b.x, r.x.y - r.b.y, r.x.z - r.b.z, r.x.w - r.b.w);
         if (MODE == GRAD_QUAD_NOISE) {
-            const float4 z = normal4(p.q_base + (uint32_t)q, (uint32_t)i, p.k, 0u, p.keys);
+            const float4 z = normal4(c.qg, (uint32_t)i, p.k, 0u, p.keys);
             g.x = fmaf(p.sigma, z.x, g.x);
             g.y = fmaf(p.sigma, z.y, g.y);
             g.z = fmaf(p.sigma, z.z, g.z);
@@ -59,9 +95,9 @@ __device__ __forceinline__ float4 finish_row(const StepParams& p, const RowIn& r
 }
 
 template <int MODE, bool VEC>
-__device__ __forceinline__ float4 half_step(const StepParams& p, long long i, long long q)
+__device__ __forceinline__ float4 half_step(const StepParams& p, const ColGroup& c, int i)
 {
-    return finish_row<MODE>(p, load_row<VEC>(p, i, q), i, q);
+    return finish_row<MODE>(p, c, load_row<VEC>(p, c, i), i);
 }
 
 // Visit steps t = t0 .. n-1 of a walk over the rows: row_of(t) is the row read at step
@@ -71,26 +107,26 @@ __device__ __forceinline__ float4 half_step(const StepParams& p, long long i, lo
 // (software pipeline in registers), so the memory system never waits for the noise
 // arithmetic.  U and PIPE are tuned per kernel.
 template <int MODE, bool VEC, int U, bool PIPE, class RowOf, class Visit>
-__device__ __forceinline__ void stream_rows(const StepParams& p, long long q, long long t0, RowOf row_of,
+__device__ __forceinline__ void stream_rows(const StepParams& p, const ColGroup& c, int t0, RowOf row_of,
                                             Visit visit)
 {
-    const long long n = p.n;
-    long long t = t0;
+    const int n = (int)p.n;
+    int t = t0;
     RowIn cur[U], nxt[U];
     if (t + U <= n) {
 #pragma unroll
-        for (int u = 0; u < U; ++u) cur[u] = load_row<VEC>(p, row_of(t + u), q);
+        for (int u = 0; u < U; ++u) cur[u] = load_row<VEC>(p, c, row_of(t + u));
     }
     while (t + U <= n) {
         const bool more = (t + 2 * U <= n);
         if (PIPE && more) {
 #pragma unroll
-            for (int u = 0; u < U; ++u) nxt[u] = load_row<VEC>(p, row_of(t + U + u), q);
+            for (int u = 0; u < U; ++u) nxt[u] = load_row<VEC>(p, c, row_of(t + U + u));
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const long long row = row_of(t + u);
-            visit(t + u, row, finish_row<MODE>(p, cur[u], row, q));
+            const int row = row_of(t + u);
+            visit(t + u, row, finish_row<MODE>(p, c, cur[u], row));
         }
         t += U;
         if (PIPE) {
@@ -98,12 +134,12 @@ __device__ __forceinline__ void stream_rows(const StepParams& p, long long q, lo
             for (int u = 0; u < U; ++u) cur[u] = nxt[u];
         } else if (more) {
 #pragma unroll
-            for (int u = 0; u < U; ++u) cur[u] = load_row<VEC>(p, row_of(t + u), q);
+            for (int u = 0; u < U; ++u) cur[u] = load_row<VEC>(p, c, row_of(t + u));
         }
     }
     for (; t < n; ++t) {
-        const long long row = row_of(t);
-        visit(t, row, half_step<MODE, VEC>(p, row, q));
+        const int row = row_of(t);
+        visit(t, row, half_step<MODE, VEC>(p, c, row));
     }
 }
 
@@ -123,31 +159,32 @@ __global__ void __launch_bounds__(BLOCK, MINB) step_ring_kernel(const StepParams
 {
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (q >= p.Q) return;
-    const long long j0 = q * 4;
-    if (p.n <= 2) {
-        const float4 y0 = half_step<MODE, VEC>(p, 0, q);
-        if (p.n == 1) {
-            store4<VEC>(p.out, j0, p.d, mix3(y0, y0, y0));
+    const ColGroup c = col_group<VEC>(p, q);
+    const int n = (int)p.n;
+    if (n <= 2) {
+        const float4 y0 = half_step<MODE, VEC>(p, c, 0);
+        if (n == 1) {
+            store_row<VEC>(p, c, 0, mix3(y0, y0, y0));
             return;
         }
-        const float4 y1 = half_step<MODE, VEC>(p, 1, q);
-        store4<VEC>(p.out, j0, p.d, mix3(y1, y0, y1));
-        store4<VEC>(p.out + p.ld, j0, p.d, mix3(y0, y1, y0));
+        const float4 y1 = half_step<MODE, VEC>(p, c, 1);
+        store_row<VEC>(p, c, 0, mix3(y1, y0, y1));
+        store_row<VEC>(p, c, 1, mix3(y0, y1, y0));
         return;
     }
-    const RowIn r0 = load_row<VEC>(p, 0, q), r1 = load_row<VEC>(p, 1, q);
-    const float4 y0 = finish_row<MODE>(p, r0, 0, q);
-    const float4 y1 = finish_row<MODE>(p, r1, 1, q);
+    const RowIn r0 = load_row<VEC>(p, c, 0), r1 = load_row<VEC>(p, c, 1);
+    const float4 y0 = finish_row<MODE>(p, c, r0, 0);
+    const float4 y1 = finish_row<MODE>(p, c, r1, 1);
     float4 a = y0, b = y1;
     stream_rows<MODE, VEC, U, PIPE>(
-        p, q, 2, [](long long t) { return t; },
-        [&](long long, long long i, float4 c) {
-            store4<VEC>(p.out + (i - 1) * p.ld, j0, p.d, mix3(a, b, c));
+        p, c, 2, [](int t) { return t; },
+        [&](int, int i, float4 v) {
+            store_row<VEC>(p, c, i - 1, mix3(a, b, v));
             a = b;
-            b = c;
+            b = v;
         });
-    store4<VEC>(p.out + (p.n - 1) * p.ld, j0, p.d, mix3(a, b, y0));
-    store4<VEC>(p.out, j0, p.d, mix3(b, y0, y1));
+    store_row<VEC>(p, c, n - 1, mix3(a, b, y0));
+    store_row<VEC>(p, c, 0, mix3(b, y0, y1));
 }
 
 // ---------------------------------------------------------------------------
@@ -162,20 +199,20 @@ __global__ void __launch_bounds__(BLOCK, MINB) step_exp_kernel(const StepParams 
 {
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (q >= p.Q) return;
-    const long long j0 = q * 4;
-    const long long hop = 1LL << p.hop_log2;
-    const long long lmask = (1LL << p.len_log2) - 1;
+    const ColGroup c = col_group<VEC>(p, q);
     const int len_log2 = p.len_log2, hop_log2 = p.hop_log2;
+    const int hop = 1 << hop_log2;
+    const int lmask = (1 << len_log2) - 1;
     float4 first = make_float4(0.f, 0.f, 0.f, 0.f), prev = first;
     stream_rows<MODE, VEC, U, PIPE>(
-        p, q, 0, [=](long long t) { return (t >> len_log2) + ((t & lmask) << hop_log2); },
-        [&](long long t, long long row, float4 cur) {
-            const long long s = t & lmask;
+        p, c, 0, [=](int t) { return (t >> len_log2) + ((t & lmask) << hop_log2); },
+        [&](int t, int row, float4 cur) {
+            const int s = t & lmask;
             if (s == 0)
                 first = cur;
             else
-                store4<VEC>(p.out + (row - hop) * p.ld, j0, p.d, scale4(add4(prev, cur), 0.5f));
-            if (s == lmask) store4<VEC>(p.out + row * p.ld, j0, p.d, scale4(add4(cur, first), 0.5f));
+                store_row<VEC>(p, c, row - hop, scale4(add4(prev, cur), 0.5f));
+            if (s == lmask) store_row<VEC>(p, c, row, scale4(add4(cur, first), 0.5f));
             prev = cur;
         });
 }
@@ -189,11 +226,11 @@ __global__ void __launch_bounds__(BLOCK, MINB) step_global_kernel(const StepPara
 {
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (q >= p.Q) return;
-    const long long j0 = q * 4;
+    const ColGroup c = col_group<VEC>(p, q);
     double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
     stream_rows<MODE, VEC, U, PIPE>(
-        p, q, 0, [](long long t) { return t; },
-        [&](long long, long long, float4 y) {
+        p, c, 0, [](int t) { return t; },
+        [&](int, int, float4 y) {
             s0 += (double)y.x;
             s1 += (double)y.y;
             s2 += (double)y.z;
@@ -202,8 +239,9 @@ __global__ void __launch_bounds__(BLOCK, MINB) step_global_kernel(const StepPara
     const double inv = (double)p.n;
     const float4 m = make_float4((float)(s0 / inv), (float)(s1 / inv), (float)(s2 / inv),
                                  (float)(s3 / inv));
+    const int n = (int)p.n;
 #pragma unroll 4
-    for (long long i = 0; i < p.n; ++i) store4<VEC>(p.out + i * p.ld, j0, p.d, m);
+    for (int i = 0; i < n; ++i) store_row<VEC>(p, c, i, m);
 }
 
 static inline unsigned grid_for(long long Q, int block) { return (unsigned)((Q + block - 1) / block); }

@@ -11,8 +11,12 @@ namespace gpga {
 enum GradMode {
     GRAD_QUAD = 0,        // g = x - b
     GRAD_QUAD_NOISE = 1,  // g = (x - b) + sigma * xi, xi generated in registers
-    GRAD_BUFFER = 2       // g read from an n x d buffer (written by the logistic kernel)
+    GRAD_BUFFER = 2,      // g read from an n x d buffer (written by the logistic kernel)
+    GRAD_PARTIALS = 3     // g = (1/B) sum_c partial[c] + l2 x, partials from the logistic kernel (tile kernel only)
 };
+
+// Mixing selector of the tile kernel: a GPGA_TOPO_* value, or the global average.
+enum { TILE_MIX_GLOBAL = 100 };
 
 struct StepParams {
     const float* x;   // X^(k), n x d
@@ -28,6 +32,9 @@ struct StepParams {
     int hop_log2;     // one-peer exponential: hop = 1 << hop_log2
     int len_log2;     // cycle length n / hop = 1 << len_log2
     int grid_cols;    // torus columns (grid topology)
+    int chunks;       // GRAD_PARTIALS: number of chunk partials (b points at them, dense n x d each)
+    float inv_batch;  // GRAD_PARTIALS: 1 / batch
+    float l2;         // GRAD_PARTIALS: l2 coefficient
     PhiloxKeys keys;
 };
 
@@ -36,7 +43,8 @@ cudaError_t launch_step_ring(const StepParams& p, int mode, bool vec, cudaStream
 cudaError_t launch_step_exp(const StepParams& p, int mode, bool vec, cudaStream_t s);
 cudaError_t launch_step_global(const StepParams& p, int mode, bool vec, cudaStream_t s);
 // Generic neighbour-list mix through a shared-memory tile of Y (grid, static exponential, W = I).
-cudaError_t launch_step_tile(const StepParams& p, int mode, bool vec, int topology, cudaStream_t s);
+cudaError_t launch_step_tile(const StepParams& p, int mode, bool vec, int mix, cudaStream_t s);
+bool tile_supports(long long n);   // the n rows of one column group fit the shared-memory tile
 
 // Consensus distance: partials (one double per block) then a fixed-order final sum.
 constexpr int kMaxReduceBlocks = 148 * 8;   // capacity of the partials array, in doubles

@@ -47,27 +47,43 @@ __global__ void __launch_bounds__(kLrBlock) logreg_partial_kernel(const LogregPa
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int d4 = (int)(p.d >> 2);
-    for (int t = warp; t < nrows; t += nwarps) {
+    // margins: a warp takes two rows at a time so that both rows' loads are in flight together
+    for (int t = warp; t < nrows; t += 2 * nwarps) {
+        const int t2 = t + nwarps;
+        const bool two = t2 < nrows;
         const float4* a4 = reinterpret_cast<const float4*>(A + (long long)rows[t] * p.d);
-        float z = 0.f;
+        const float4* b4 = reinterpret_cast<const float4*>(A + (long long)rows[two ? t2 : t] * p.d);
+        float z = 0.f, z2 = 0.f;
+#pragma unroll 4
         for (int g = lane; g < d4; g += 32) {
             const float4 a = __ldg(a4 + g);
+            const float4 b = __ldg(b4 + g);
             const float4 xv = reinterpret_cast<const float4*>(xs)[g];
             z = fmaf(a.x, xv.x, z);
             z = fmaf(a.y, xv.y, z);
             z = fmaf(a.z, xv.z, z);
             z = fmaf(a.w, xv.w, z);
+            z2 = fmaf(b.x, xv.x, z2);
+            z2 = fmaf(b.y, xv.y, z2);
+            z2 = fmaf(b.z, xv.z, z2);
+            z2 = fmaf(b.w, xv.w, z2);
         }
         z = warp_sum_f(z);
+        z2 = warp_sum_f(z2);
         if (lane == 0) {
             const float yr = y[rows[t]];
             coef[t] = -yr / (1.0f + expf(yr * z));
+            if (two) {
+                const float yr2 = y[rows[t2]];
+                coef[t2] = -yr2 / (1.0f + expf(yr2 * z2));
+            }
         }
     }
     __syncthreads();
     float4* out4 = reinterpret_cast<float4*>(p.partial + ((long long)c * p.n + i) * p.d);
     for (int g = threadIdx.x; g < d4; g += blockDim.x) {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
         for (int t = 0; t < nrows; ++t) {
             const float4 a = __ldg(reinterpret_cast<const float4*>(A + (long long)rows[t] * p.d) + g);
             const float s = coef[t];
@@ -139,7 +155,7 @@ __global__ void mean_kernel(const double* v, int count, double* result)
 
 int logreg_chunks(long long batch) { return (int)((batch + kChunkRows - 1) / kChunkRows); }
 
-cudaError_t launch_logreg_grad(const LogregParams& p, cudaStream_t s)
+cudaError_t launch_logreg_partial(const LogregParams& p, cudaStream_t s)
 {
     const int chunks = logreg_chunks(p.batch);
     const size_t smem = (size_t)(p.d + kChunkRows) * sizeof(float);
@@ -147,6 +163,14 @@ cudaError_t launch_logreg_grad(const LogregParams& p, cudaStream_t s)
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
     logreg_partial_kernel<<<dim3((unsigned)p.n, (unsigned)chunks), kLrBlock, smem, s>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_logreg_grad(const LogregParams& p, cudaStream_t s)
+{
+    const int chunks = logreg_chunks(p.batch);
+    cudaError_t e = launch_logreg_partial(p, s);
+    if (e != cudaSuccess) return e;
     const long long total4 = p.n * (p.d >> 2);
     logreg_reduce_kernel<<<(unsigned)((total4 + kLrBlock - 1) / kLrBlock), kLrBlock, 0, s>>>(p, chunks);
     return cudaGetLastError();

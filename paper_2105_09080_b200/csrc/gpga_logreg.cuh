@@ -23,6 +23,8 @@ struct LogregParams {
 };
 
 int logreg_chunks(long long batch);
+// One launch: chunk partials only (the consumer adds them in index order).
+cudaError_t launch_logreg_partial(const LogregParams& p, cudaStream_t s);
 // Two launches: chunk partials, then the fixed-order sum into G (adds l2 x).
 cudaError_t launch_logreg_grad(const LogregParams& p, cudaStream_t s);
 // Two launches: per-node mini-batch loss (n doubles), then their mean into *result.

@@ -51,7 +51,7 @@ def test_create_argument_checks(L):
     assert st == pkg.GPGA_OK and h.value
     assert L.gpga_destroy(h) == pkg.GPGA_OK
     for kw in (dict(n=0), dict(d=0), dict(H=-1), dict(gamma=-0.1), dict(gamma=float("nan")),
-               dict(gamma=float("inf")), dict(topo=9), dict(topo=-1), dict(n=2**32), dict(d=2**34)):
+               dict(gamma=float("inf")), dict(topo=9), dict(topo=-1), dict(n=2**31), dict(d=2**34)):
         st, h = _create(L, **kw)
         assert st == pkg.GPGA_ERR_INVALID_ARG, kw
         assert not h.value

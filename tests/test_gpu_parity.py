@@ -98,8 +98,11 @@ def test_device_normal_fill_matches_oracle_keying():
 
 
 # ------------------------------------------------------------------ one step, every kernel
+# below 148 * 32 column groups (d < 18944) a step goes through the tile kernel, above it through
+# the row-streaming kernels: both ranges, with 128-bit and scalar (d % 4 != 0) shapes
 SHAPES = [(1, 4), (2, 8), (3, 12), (4, 132), (5, 1028), (8, 4100), (16, 1024 + 40), (7, 6), (3, 1),
-          (6, 1031), (64, 520)]
+          (6, 1031), (64, 520),
+          (1, 20004), (2, 20008), (3, 19000), (4, 24580), (5, 20007), (7, 19001), (9, 32772), (64, 19004)]
 
 
 @pytest.mark.parametrize("n,d", SHAPES)
@@ -119,7 +122,7 @@ def test_ring_and_global_one_step(n, d, sigma):
 
 
 @pytest.mark.parametrize("n", [1, 2, 4, 8, 32, 64])
-@pytest.mark.parametrize("d", [4, 7, 1028, 4096 + 8])
+@pytest.mark.parametrize("d", [4, 7, 1028, 4096 + 8, 20004, 19003])
 def test_exp_one_step_every_hop(n, d):
     X0, B = quadratic_inputs(n, d, 200 + n, x0="per_node")
     tau = max(1, int(np.log2(n)))
@@ -146,7 +149,7 @@ def test_tile_topologies_one_step(topo, n, gc, d):
 
 
 @pytest.mark.parametrize("topo,H,k", [("ring", 0, 1), ("exp", 0, 2), ("ring", 2, 1), ("grid", 0, 0)])
-@pytest.mark.parametrize("d,ld", [(1000, 1024), (1030, 1056), (7, 9), (1026, 1027)])
+@pytest.mark.parametrize("d,ld", [(1000, 1024), (1030, 1056), (7, 9), (1026, 1027), (20000, 20032), (19002, 19003)])
 def test_padded_row_stride(topo, H, k, d, ld):
     """Rows padded to ld floats: same results as the dense layout; padding is never touched."""
     torch = _torch()
