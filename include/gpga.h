@@ -42,7 +42,9 @@ enum {
     GPGA_ERR_INVALID_ARG = 1,
     GPGA_ERR_NOT_READY = 2,   /* NULL handle, buffers not bound */
     GPGA_ERR_CUDA = 3,        /* a CUDA call failed; sticky */
-    GPGA_ERR_UNSUPPORTED = 4
+    GPGA_ERR_UNSUPPORTED = 4,
+    GPGA_ERR_TIMEOUT = 5      /* a bounded wait inside a kernel gave up; reported by the next
+                                 synchronising call (consensus distance, mean loss); sticky */
 };
 
 /* Gossip topologies (Section 3; Section 5 for the one-peer exponential graph). */

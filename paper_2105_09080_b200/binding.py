@@ -18,6 +18,7 @@ GPGA_ERR_INVALID_ARG = 1
 GPGA_ERR_NOT_READY = 2
 GPGA_ERR_CUDA = 3
 GPGA_ERR_UNSUPPORTED = 4
+GPGA_ERR_TIMEOUT = 5
 
 GPGA_TOPO_RING = 0
 GPGA_TOPO_EXP = 1

@@ -30,6 +30,7 @@ struct gpga_ctx {
     int64_t k = 0;
     int64_t launches = 0;
     bool bound = false;
+    bool flag_cleared = false;   // the device error word in scratch has been zeroed since bind
     int32_t sticky = GPGA_OK;
     std::string err;
     PhiloxKeys keys;
@@ -103,6 +104,7 @@ LogregParams logreg_params(const gpga_ctx* c, int64_t k)
     lp.x = c->x[c->cur];
     lp.ldx = c->ld;
     lp.G = reinterpret_cast<float*>(c->scratch + L.G_off);
+    lp.error_flag = reinterpret_cast<int*>(c->scratch + L.result_off + 8);
     lp.partial = reinterpret_cast<float*>(c->scratch + L.chunk_off);
     lp.n = c->n; lp.d = c->d; lp.m = c->m; lp.batch = c->batch;
     lp.k = (uint32_t)k;
@@ -136,6 +138,11 @@ int32_t do_step(gpga_ctx* c, int64_t k, bool global, cudaStream_t s)
     cudaError_t e;
     if (c->objective == GPGA_OBJ_LOGISTIC) {
         const LogregParams lp = logreg_params(c, k);
+        if (!c->flag_cleared) {   // kernels with bounded waits report through this word
+            e = cudaMemsetAsync(lp.error_flag, 0, sizeof(int), s);
+            if (e != cudaSuccess) return cuda_fail(c, e, "error word clear");
+            c->flag_cleared = true;
+        }
         if (narrow) {   // the step kernel adds the chunk partials itself: one launch fewer
             e = launch_logreg_partial(lp, s);
             c->launches += 1;
@@ -194,12 +201,20 @@ int32_t mean_loss_async(gpga_ctx* c, cudaStream_t s, double** result_dev)
     return GPGA_OK;
 }
 
+// Reads the result double and, if it has been armed, the device error word beside it.
 int32_t read_double(gpga_ctx* c, const double* dev, cudaStream_t s, double* out_host)
 {
-    cudaError_t e = cudaMemcpyAsync(out_host, dev, sizeof(double), cudaMemcpyDeviceToHost, s);
+    struct { double value; int flag; int pad; } host = {0.0, 0, 0};
+    const size_t bytes = c->flag_cleared ? 12 : sizeof(double);
+    cudaError_t e = cudaMemcpyAsync(&host, dev, bytes, cudaMemcpyDeviceToHost, s);
     if (e != cudaSuccess) return cuda_fail(c, e, "result copy");
     e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_fail(c, e, "stream synchronize");
+    *out_host = host.value;
+    if (host.flag != 0) {
+        c->sticky = GPGA_ERR_TIMEOUT;
+        return fail(c, GPGA_ERR_TIMEOUT, "a bounded wait inside a kernel gave up (asynchronous copy did not complete)");
+    }
     return GPGA_OK;
 }
 
@@ -314,6 +329,7 @@ int32_t gpga_bind(gpga_t* c, void* x_a, void* x_b, void* data, const void* label
     c->cur = 0;
     c->k = 0;
     c->bound = true;
+    c->flag_cleared = false;
     return GPGA_OK;
 }
 

@@ -7,6 +7,7 @@
 // sum over those rows; a second kernel adds the chunks in a fixed order, so the result
 // does not depend on scheduling.
 #include "gpga_logreg.cuh"
+#include "gpga_tma.cuh"
 
 namespace gpga {
 
@@ -35,6 +36,7 @@ __global__ void __launch_bounds__(kLrBlock) logreg_partial_kernel(const LogregPa
     float* xs = smem;                          // d floats: x_i
     float* coef = smem + p.d;                  // kChunkRows floats: s_r
     __shared__ uint32_t rows[kChunkRows];
+    __shared__ float ys[kChunkRows];
     const int i = blockIdx.x, c = blockIdx.y;
     const int t0 = c * kChunkRows;
     const int nrows = min(kChunkRows, (int)p.batch - t0);
@@ -44,6 +46,7 @@ __global__ void __launch_bounds__(kLrBlock) logreg_partial_kernel(const LogregPa
     for (int j = threadIdx.x; j < p.d; j += blockDim.x) xs[j] = x[j];
     if (threadIdx.x < nrows)
         rows[threadIdx.x] = batch_row((uint32_t)(t0 + threadIdx.x), (uint32_t)i, p.k, (uint32_t)p.m, p.keys);
+    if (threadIdx.x < nrows) ys[threadIdx.x] = y[rows[threadIdx.x]];
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int d4 = (int)(p.d >> 2);
@@ -71,10 +74,10 @@ __global__ void __launch_bounds__(kLrBlock) logreg_partial_kernel(const LogregPa
         z = warp_sum_f(z);
         z2 = warp_sum_f(z2);
         if (lane == 0) {
-            const float yr = y[rows[t]];
+            const float yr = ys[t];
             coef[t] = -yr / (1.0f + expf(yr * z));
             if (two) {
-                const float yr2 = y[rows[t2]];
+                const float yr2 = ys[t2];
                 coef[t2] = -yr2 / (1.0f + expf(yr2 * z2));
             }
         }
@@ -93,6 +96,130 @@ __global__ void __launch_bounds__(kLrBlock) logreg_partial_kernel(const LogregPa
             acc.w = fmaf(s, a.w, acc.w);
         }
         out4[g] = acc;
+    }
+}
+
+// The same partial sums with the batch rows staged in shared memory by bulk asynchronous
+// copies (one 16-byte-aligned row of d floats per copy, completion counted on an
+// mbarrier).  Two tiles of rows alternate: while one is consumed the next is in flight,
+// without holding registers, and both passes over a row -- the margin and the weighted
+// sum -- read shared memory, so A is fetched from HBM exactly once.  Used for
+// d <= kTmaMaxD; a thread then owns at most kTmaMaxGroups groups of four columns.
+constexpr int kTmaMaxD = 4096;
+constexpr int kTmaMaxGroups = kTmaMaxD / 4 / kLrBlock;
+constexpr int kTmaTileBytes = 64 * 1024;
+constexpr uint32_t kTmaMaxTries = 1u << 22;
+
+__global__ void __launch_bounds__(kLrBlock) logreg_partial_tma_kernel(const LogregParams p, int tile_rows)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    float* tiles = reinterpret_cast<float*>(smem_raw);         // 2 x tile_rows x d
+    float* xs = tiles + 2 * (size_t)tile_rows * p.d;           // d floats: x_i
+    float* coef = xs + p.d;                                    // kChunkRows floats: s_r
+    __shared__ uint32_t rows[kChunkRows];
+    __shared__ float ys[kChunkRows];
+    __shared__ __align__(8) uint64_t bar[2];
+    const int i = blockIdx.x, c = blockIdx.y;
+    const int t0 = c * kChunkRows;
+    const int nrows = min(kChunkRows, (int)p.batch - t0);
+    const int ntiles = (nrows + tile_rows - 1) / tile_rows;
+    const float* A = p.A + (long long)i * p.m * p.d;
+    const float* y = p.y + (long long)i * p.m;
+    const float* x = p.x + (long long)i * p.ldx;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int d4 = (int)(p.d >> 2);
+    const uint32_t row_bytes = (uint32_t)p.d * 4u;
+    if (threadIdx.x < nrows)
+        rows[threadIdx.x] = batch_row((uint32_t)(t0 + threadIdx.x), (uint32_t)i, p.k, (uint32_t)p.m, p.keys);
+    if (threadIdx.x == 0) {
+        mbar_init(&bar[0], 1);
+        mbar_init(&bar[1], 1);
+        mbar_init_fence();
+    }
+    __syncthreads();
+    // warp 0 starts the copies of tile s into buffer s & 1
+    auto issue = [&](int s) {
+        const int r0 = s * tile_rows;
+        const int rr = min(tile_rows, nrows - r0);
+        float* dst = tiles + (size_t)(s & 1) * tile_rows * p.d;
+        if (lane == 0) mbar_arrive_expect_tx(&bar[s & 1], (uint32_t)rr * row_bytes);
+        __syncwarp();
+        for (int t = lane; t < rr; t += 32)
+            bulk_copy_g2s(dst + (size_t)t * p.d, A + (long long)rows[r0 + t] * p.d, row_bytes, &bar[s & 1]);
+    };
+    if (warp == 0) {
+        issue(0);
+        if (ntiles > 1) issue(1);
+    }
+    // x_i and the labels of the drawn rows arrive while the copies fly
+    if (threadIdx.x < nrows) ys[threadIdx.x] = y[rows[threadIdx.x]];
+    for (int j = threadIdx.x; j < p.d; j += blockDim.x) xs[j] = x[j];
+    __syncthreads();
+    float4 acc[kTmaMaxGroups];
+#pragma unroll
+    for (int u = 0; u < kTmaMaxGroups; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    uint32_t parity0 = 0u, parity1 = 0u;
+    bool failed = false;
+    for (int s = 0; s < ntiles; ++s) {
+        const int buf = s & 1;
+        const int r0 = s * tile_rows;
+        const int rr = min(tile_rows, nrows - r0);
+        const float* tile = tiles + (size_t)buf * tile_rows * p.d;
+        const uint32_t par = buf ? parity1 : parity0;
+        const bool ok = mbar_wait_bounded(&bar[buf], par, kTmaMaxTries);
+        if (__syncthreads_or(!ok)) {
+            // a copy did not report in time: flag it, give the copies in flight (they target
+            // this block's shared memory) one more bounded chance to land, and leave
+            if (!ok) mbar_wait_bounded(&bar[buf], par, kTmaMaxTries);
+            if (s + 1 < ntiles) mbar_wait_bounded(&bar[buf ^ 1], buf ? parity0 : parity1, kTmaMaxTries);
+            if (threadIdx.x == 0 && p.error_flag) atomicExch(p.error_flag, 1);
+            failed = true;
+            break;
+        }
+        if (buf) parity1 ^= 1u; else parity0 ^= 1u;
+        for (int t = warp; t < rr; t += nwarps) {
+            const float4* a4 = reinterpret_cast<const float4*>(tile + (size_t)t * p.d);
+            float z = 0.f;
+#pragma unroll 4
+            for (int g = lane; g < d4; g += 32) {
+                const float4 a = a4[g];
+                const float4 xv = reinterpret_cast<const float4*>(xs)[g];
+                z = fmaf(a.x, xv.x, z);
+                z = fmaf(a.y, xv.y, z);
+                z = fmaf(a.z, xv.z, z);
+                z = fmaf(a.w, xv.w, z);
+            }
+            z = warp_sum_f(z);
+            if (lane == 0) {
+                const float yr = ys[r0 + t];
+                coef[r0 + t] = -yr / (1.0f + expf(yr * z));
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int u = 0; u < kTmaMaxGroups; ++u) {
+            const int g = threadIdx.x + u * kLrBlock;
+            if (g < d4) {
+#pragma unroll 4
+                for (int t = 0; t < rr; ++t) {
+                    const float4 a = reinterpret_cast<const float4*>(tile + (size_t)t * p.d)[g];
+                    const float sc = coef[r0 + t];
+                    acc[u].x = fmaf(sc, a.x, acc[u].x);
+                    acc[u].y = fmaf(sc, a.y, acc[u].y);
+                    acc[u].z = fmaf(sc, a.z, acc[u].z);
+                    acc[u].w = fmaf(sc, a.w, acc[u].w);
+                }
+            }
+        }
+        __syncthreads();   // everyone is done with this buffer before new copies overwrite it
+        if (warp == 0 && s + 2 < ntiles) issue(s + 2);
+    }
+    if (failed) return;
+    float4* out4 = reinterpret_cast<float4*>(p.partial + ((long long)c * p.n + i) * p.d);
+#pragma unroll
+    for (int u = 0; u < kTmaMaxGroups; ++u) {
+        const int g = threadIdx.x + u * kLrBlock;
+        if (g < d4) out4[g] = acc[u];
     }
 }
 
@@ -158,6 +285,16 @@ int logreg_chunks(long long batch) { return (int)((batch + kChunkRows - 1) / kCh
 cudaError_t launch_logreg_partial(const LogregParams& p, cudaStream_t s)
 {
     const int chunks = logreg_chunks(p.batch);
+    if (p.d <= kTmaMaxD) {
+        int tile_rows = kTmaTileBytes / 2 / (int)(p.d * 4);   // two tiles share the budget
+        if (tile_rows > kChunkRows) tile_rows = kChunkRows;
+        const size_t smem_tma = (2 * (size_t)tile_rows * p.d + p.d + kChunkRows) * sizeof(float);
+        cudaError_t e = cudaFuncSetAttribute(logreg_partial_tma_kernel,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+        if (e != cudaSuccess) return e;
+        logreg_partial_tma_kernel<<<dim3((unsigned)p.n, (unsigned)chunks), kLrBlock, smem_tma, s>>>(p, tile_rows);
+        return cudaGetLastError();
+    }
     const size_t smem = (size_t)(p.d + kChunkRows) * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(logreg_partial_kernel,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);

@@ -16,6 +16,7 @@ struct LogregParams {
     long long ldx;
     float* partial;   // chunks x n x d
     float* G;         // n x d
+    int* error_flag;  // set to 1 if a bounded wait inside a kernel gave up (may be NULL)
     long long n, d, m, batch;
     uint32_t k;
     float l2;

@@ -87,6 +87,7 @@ int32_t gpga_logistic_gradient_noalloc(const float* A_dev, const float* y_dev, c
     p.ldx = ldx;
     p.partial = scratch;
     p.G = G_dev;
+    p.error_flag = nullptr;
     p.n = n; p.d = d; p.m = m; p.batch = batch;
     p.k = (uint32_t)k;
     p.l2 = l2;
