@@ -7,6 +7,7 @@
 // sum over those rows; a second kernel adds the chunks in a fixed order, so the result
 // does not depend on scheduling.
 #include "gpga_logreg.cuh"
+#include "gpga_launch.cuh"
 #include "gpga_tma.cuh"
 
 namespace gpga {
@@ -289,15 +290,15 @@ cudaError_t launch_logreg_partial(const LogregParams& p, cudaStream_t s)
         int tile_rows = kTmaTileBytes / 2 / (int)(p.d * 4);   // two tiles share the budget
         if (tile_rows > kChunkRows) tile_rows = kChunkRows;
         const size_t smem_tma = (2 * (size_t)tile_rows * p.d + p.d + kChunkRows) * sizeof(float);
-        cudaError_t e = cudaFuncSetAttribute(logreg_partial_tma_kernel,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+        static unsigned long long tma_limit_set = 0;
+        cudaError_t e = ensure_smem_limit(logreg_partial_tma_kernel, 100 * 1024, tma_limit_set);
         if (e != cudaSuccess) return e;
         logreg_partial_tma_kernel<<<dim3((unsigned)p.n, (unsigned)chunks), kLrBlock, smem_tma, s>>>(p, tile_rows);
         return cudaGetLastError();
     }
     const size_t smem = (size_t)(p.d + kChunkRows) * sizeof(float);
-    cudaError_t e = cudaFuncSetAttribute(logreg_partial_kernel,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    static unsigned long long plain_limit_set = 0;
+    cudaError_t e = ensure_smem_limit(logreg_partial_kernel, 200 * 1024, plain_limit_set);
     if (e != cudaSuccess) return e;
     logreg_partial_kernel<<<dim3((unsigned)p.n, (unsigned)chunks), kLrBlock, smem, s>>>(p);
     return cudaGetLastError();

@@ -12,6 +12,7 @@
 //    the GPU idle (the logistic workload: d = 1024).
 #include "../../include/gpga.h"
 #include "gpga_kernels.cuh"
+#include "gpga_launch.cuh"
 
 namespace gpga {
 
@@ -147,9 +148,8 @@ cudaError_t launch_step_tile(const StepParams& p, int mode, bool vec, int mix, c
     const int blk = cells >= kTileBlock ? kTileBlock : (int)((cells + 31) / 32 * 32);
 #define GPGA_TILE(M, V)                                                                          \
     do {                                                                                         \
-        cudaError_t e = cudaFuncSetAttribute(step_tile_kernel<M, V>,                             \
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize,        \
-                                             kTileSmemBytes);                                    \
+        static unsigned long long limit_set = 0;                                                 \
+        cudaError_t e = ensure_smem_limit(step_tile_kernel<M, V>, kTileSmemBytes, limit_set);    \
         if (e != cudaSuccess) return e;                                                          \
         step_tile_kernel<M, V><<<grd, blk, smem, s>>>(p, mix, tile_groups, log2n);               \
     } while (0)
