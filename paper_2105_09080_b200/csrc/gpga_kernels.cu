@@ -218,8 +218,11 @@ __global__ void __launch_bounds__(BLOCK, MINB) step_exp_kernel(const StepParams 
 }
 
 // ---------------------------------------------------------------------------
-// Global average: m_j = (1/n) sum_i y_ij, written to every row.  The column sum is
-// accumulated in fp64 (exact for practical n), rounded once.
+// Global average: m_j = (1/n) sum_i y_ij, written to every row.  Rows are added
+// pairwise in fp32 in groups of four, (y0 + y1) + (y2 + y3), and the group sums are
+// accumulated in fp64 and rounded once.  A group sum carries at most three fp32
+// roundings, so the mean is within a few 1e-8 (1 + |y|) of the exact one; and when all
+// rows are equal every group sum (v, 2v or 4v) is exact, so the mean is exactly v.
 // ---------------------------------------------------------------------------
 template <int MODE, bool VEC, int U, bool PIPE, int BLOCK, int MINB>
 __global__ void __launch_bounds__(BLOCK, MINB) step_global_kernel(const StepParams p)
@@ -228,18 +231,42 @@ __global__ void __launch_bounds__(BLOCK, MINB) step_global_kernel(const StepPara
     if (q >= p.Q) return;
     const ColGroup c = col_group<VEC>(p, q);
     double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
     stream_rows<MODE, VEC, U, PIPE>(
         p, c, 0, [](int t) { return t; },
-        [&](int, int, float4 y) {
-            s0 += (double)y.x;
-            s1 += (double)y.y;
-            s2 += (double)y.z;
-            s3 += (double)y.w;
+        [&](int t, int, float4 y) {
+            const int phase = t & 3;
+            if (phase == 0) {
+                a = y;
+            } else if (phase == 1) {
+                a = add4(a, y);
+            } else if (phase == 2) {
+                b = y;
+            } else {
+                b = add4(b, y);
+                const float4 g = add4(a, b);
+                s0 += (double)g.x;
+                s1 += (double)g.y;
+                s2 += (double)g.z;
+                s3 += (double)g.w;
+            }
         });
+    const int n = (int)p.n, rest = n & 3;   // rows of an unfinished last group
+    if (rest >= 1) {
+        s0 += (double)a.x;
+        s1 += (double)a.y;
+        s2 += (double)a.z;
+        s3 += (double)a.w;
+    }
+    if (rest == 3) {
+        s0 += (double)b.x;
+        s1 += (double)b.y;
+        s2 += (double)b.z;
+        s3 += (double)b.w;
+    }
     const double inv = (double)p.n;
     const float4 m = make_float4((float)(s0 / inv), (float)(s1 / inv), (float)(s2 / inv),
                                  (float)(s3 / inv));
-    const int n = (int)p.n;
 #pragma unroll 4
     for (int i = 0; i < n; ++i) store_row<VEC>(p, c, i, m);
 }
@@ -250,8 +277,8 @@ static inline unsigned grid_for(long long Q, int block) { return (unsigned)((Q +
 // threads per block and minimum resident blocks (the register cap), chosen by timing
 // on B200 at the ResNet-50- and BERT-Large-sized states.
 struct RingTune { static constexpr int U = 2; static constexpr bool PIPE = false; static constexpr int BLOCK = 256; static constexpr int MINB = 4; };
-struct ExpTune { static constexpr int U = 4; static constexpr bool PIPE = false; static constexpr int BLOCK = 128; static constexpr int MINB = 4; };
-struct GlobalTune { static constexpr int U = 4; static constexpr bool PIPE = false; static constexpr int BLOCK = 128; static constexpr int MINB = 4; };
+struct ExpTune { static constexpr int U = 4; static constexpr bool PIPE = false; static constexpr int BLOCK = 256; static constexpr int MINB = 4; };
+struct GlobalTune { static constexpr int U = 4; static constexpr bool PIPE = false; static constexpr int BLOCK = 256; static constexpr int MINB = 4; };
 constexpr int kSmallBlock = 64;   // small problems: narrow blocks spread the column groups over more SMs
 
 #ifndef GPGA_TUNING_HARNESS
