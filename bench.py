@@ -353,12 +353,8 @@ def run_logistic(args, w, name):
         raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
     n, d, m, batch = w["n"], w["d"], w["m"], w["batch"]
-    gen = torch.Generator(device="cuda").manual_seed(SEED)
-    A = torch.randn((n, m, d), device="cuda", generator=gen) / d ** 0.5
-    x_star = torch.randn(d, device="cuda", generator=gen)
-    xi = x_star[None, :] + 0.5 * torch.randn((n, d), device="cuda", generator=gen)
-    margin = torch.einsum("nmd,nd->nm", A, xi) + 0.1 * torch.randn((n, m), device="cuda", generator=gen)
-    y = torch.where(margin >= 0, 1.0, -1.0).to(torch.float32).contiguous()
+    from paper_2105_09080_b200.inputs import logistic_inputs_device
+    A, y = logistic_inputs_device(n, m, d, SEED)
     topo = {"ring": pkg.GPGA_TOPO_RING, "exp": pkg.GPGA_TOPO_EXP}[w["topo"]]
     g = pkg.Gpga(n, d, topo, w["H"], w["gamma"], SEED)
     g.set_objective(pkg.GPGA_OBJ_LOGISTIC, l2=w["l2"], m=m, batch=batch)
@@ -400,7 +396,7 @@ def run_logistic(args, w, name):
     hout.copy_(g2.get_x(), non_blocking=True)
     torch.cuda.synchronize()
     dt = time.perf_counter() - t0
-    loss, xi_dist = g2.mean_loss(), g2.consensus_distance()
+    loss, xi_dist, gloss = g2.mean_loss(), g2.consensus_distance(), g2.global_loss()
     line = {"metric": METRIC, "value": n * d * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
@@ -416,7 +412,7 @@ def run_logistic(args, w, name):
             "e2e": {"value": n * d * w["K"] / dt, "unit": UNIT, "h2d_bytes_per_step": (A.numel() + y.numel() + n * d) * 4 / w["K"],
                     "d2h_bytes_per_step": n * d * 4 / w["K"],
                     "job": f"pinned host A, y, X0 copied in, K={w['K']} iterations, X copied out", "seconds_per_job": dt},
-            "after_K": {"mean_minibatch_loss": loss, "consensus_distance": xi_dist},
+            "after_K": {"mean_minibatch_loss": loss, "consensus_distance": xi_dist, "global_loss": gloss},
             "gpu_launches": launches}
     print(json.dumps(line))
 

@@ -182,6 +182,14 @@ int32_t gpga_consensus_distance(gpga_t* ctx, void* stream, double* out_host);
 int32_t gpga_mean_loss(gpga_t* ctx, void* stream, double* out_host);
 
 /*
+ * Global loss of problem (1) at the node average: f(xbar) = (1/n) sum_i f_i(xbar),
+ * xbar = (1/n) sum_i x_i (the quantity the paper's convergence figures plot).
+ * QUADRATIC: f_i = 1/2 ||x - b_i||^2.  LOGISTIC: the Section 5.1 loss over all m local samples
+ * of every node plus (l2/2)||x||^2.  fp64 accumulation.  Synchronises the stream.
+ */
+int32_t gpga_global_loss(gpga_t* ctx, void* stream, double* out_host);
+
+/*
  * Gossip-AGA (Algorithm 2, period rule with the exponent removed as its appendix states):
  * K iterations with an adaptive period.  A counter C counts iterations since the last
  * global average; when C == H the step is a global average, the mean loss F of that

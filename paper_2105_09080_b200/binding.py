@@ -51,6 +51,7 @@ SIGNATURES = {
     "gpga_run_host": (_i32, [_P, _P, _P, _i64, _P, _P]),
     "gpga_consensus_distance": (_i32, [_P, _P, C.POINTER(C.c_double)]),
     "gpga_mean_loss": (_i32, [_P, _P, C.POINTER(C.c_double)]),
+    "gpga_global_loss": (_i32, [_P, _P, C.POINTER(C.c_double)]),
     "gpga_run_adaptive": (_i32, [_P, _i64, _i64, _i64, _P, C.POINTER(_i64), _i64, C.POINTER(_i64)]),
     "gpga_get_x": (_i32, [_P, C.POINTER(_P)]),
     "gpga_get_k": (_i32, [_P, C.POINTER(_i64)]),
@@ -203,6 +204,11 @@ class Gpga:
     def mean_loss(self, stream=None) -> float:
         out = C.c_double()
         self._check(lib().gpga_mean_loss(self._h, _stream_ptr(stream), C.byref(out)))
+        return out.value
+
+    def global_loss(self, stream=None) -> float:
+        out = C.c_double()
+        self._check(lib().gpga_global_loss(self._h, _stream_ptr(stream), C.byref(out)))
         return out.value
 
     def run_adaptive(self, K, H_init, warmup_iters, stream=None, max_periods=4096):

@@ -7,6 +7,7 @@
 #include "../../include/gpga.h"
 #include "gpga_kernels.cuh"
 #include "gpga_logreg.cuh"
+#include "gpga_loss.cuh"
 
 using namespace gpga;
 
@@ -428,6 +429,33 @@ int32_t gpga_mean_loss(gpga_t* c, void* stream, double* out_host)
     double* result = nullptr;
     st = mean_loss_async(c, s, &result);
     if (st) return st;
+    return read_double(c, result, s, out_host);
+}
+
+int32_t gpga_global_loss(gpga_t* c, void* stream, double* out_host)
+{
+    int32_t st = check_ready(c);
+    if (st) return st;
+    if (!out_host) return fail(c, GPGA_ERR_INVALID_ARG, "out_host is NULL");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const ScratchLayout L = scratch_layout(c);
+    double* partials = reinterpret_cast<double*>(c->scratch + L.partials_off);
+    double* result = reinterpret_cast<double*>(c->scratch + L.result_off);
+    cudaError_t e;
+    if (c->objective == GPGA_OBJ_LOGISTIC) {
+        if (c->d > 12288) return fail(c, GPGA_ERR_UNSUPPORTED, "logistic global loss needs d <= 12288");
+        // xbar borrows the gradient buffer, which is dead between iterations
+        float* xbar = reinterpret_cast<float*>(c->scratch + L.G_off);
+        int64_t slots = kMaxReduceBlocks;
+        if (c->n > slots) slots = c->n;
+        e = launch_logistic_global_loss(c->data, c->labels, c->x[c->cur], c->ld, c->n, c->d, c->m, c->l2, xbar,
+                                        partials, slots, result, s);
+        c->launches += 3;
+    } else {
+        e = launch_quadratic_global_loss(c->x[c->cur], c->data, c->n, c->d, c->ld, vec_ok(c), partials, result, s);
+        c->launches += 2;
+    }
+    if (e != cudaSuccess) return cuda_fail(c, e, "global loss launch");
     return read_double(c, result, s, out_host);
 }
 

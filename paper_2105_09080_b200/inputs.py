@@ -55,3 +55,18 @@ def logistic_inputs(n: int, m: int, d: int, seed: int, hetero: float = 0.5,
         margin = A[i].astype(np.float64) @ xi + label_noise * rng.standard_normal(m)
         y[i] = np.where(margin >= 0.0, 1.0, -1.0)
     return np.ascontiguousarray(A), np.ascontiguousarray(y)
+
+
+def logistic_inputs_device(n: int, m: int, d: int, seed: int, device="cuda", hetero: float = 0.5,
+                           label_noise: float = 0.1):
+    """Same recipe as ``logistic_inputs`` drawn on the device with torch's seeded generator
+    (a different random stream, hence different numbers): (A, y) as float32 CUDA tensors.
+    For workloads too large to ship from the host on every run."""
+    import torch
+    gen = torch.Generator(device=device).manual_seed(seed)
+    A = torch.randn((n, m, d), device=device, generator=gen) / d ** 0.5
+    x_star = torch.randn(d, device=device, generator=gen)
+    xi = x_star[None, :] + hetero * torch.randn((n, d), device=device, generator=gen)
+    margin = torch.einsum("nmd,nd->nm", A, xi) + label_noise * torch.randn((n, m), device=device, generator=gen)
+    y = torch.where(margin >= 0, 1.0, -1.0).to(torch.float32).contiguous()
+    return A.contiguous(), y

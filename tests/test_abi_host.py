@@ -123,6 +123,7 @@ def test_objective_and_bind_checks(L):
     assert L.gpga_run(h, 0, None) == pkg.GPGA_OK                                      # no launch
     assert L.gpga_run_host(h, None, None, 1, None, None) == pkg.GPGA_ERR_INVALID_ARG
     assert L.gpga_consensus_distance(h, None, None) == pkg.GPGA_ERR_INVALID_ARG
+    assert L.gpga_global_loss(h, None, None) == pkg.GPGA_ERR_INVALID_ARG
     assert L.gpga_run_adaptive(h, 4, 0, 0, None, None, 0, None) == pkg.GPGA_ERR_INVALID_ARG
     L.gpga_destroy(h)
     # logistic objective needs labels at bind, and d % 4 == 0

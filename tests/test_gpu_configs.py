@@ -144,6 +144,9 @@ def test_logistic_steps(topo, n, m, d, batch):
                                  y[i][o.batch_indices(SEED, k, i, batch, m)], want[i], 1e-4)
                  for i in range(n)])
     assert abs(g.mean_loss() - f) <= 1e-4 * abs(f)
+    # global loss of problem (1) at the node average, over every local sample
+    f_glob = o.global_logistic_loss(A, y, want.astype(np.float64).mean(0), 1e-4)
+    assert abs(g.global_loss() - f_glob) <= 1e-4 * abs(f_glob)
 
 
 def test_config_5_logistic_reduced_iterations():
@@ -186,3 +189,6 @@ def test_adaptive_period_sequence_matches_oracle_driven_loop():
     ok, worst = close(g.get_x().cpu().numpy(), X, TOL_RUN)
     assert ok, worst
     assert abs(g.mean_loss() - o.quadratic_mean_loss(X, B)) <= 1e-5 * o.quadratic_mean_loss(X, B)
+    xbar = np.repeat(X.astype(np.float64).mean(0, keepdims=True), n, axis=0)
+    f_glob = o.quadratic_mean_loss(xbar, B)         # (1/n) sum_i 1/2 ||xbar - b_i||^2
+    assert abs(g.global_loss() - f_glob) <= 1e-5 * f_glob

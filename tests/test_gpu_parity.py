@@ -173,6 +173,8 @@ def test_padded_row_stride(topo, H, k, d, ld):
     xi = o.consensus_distance(want)
     assert abs(g.consensus_distance() - xi) <= 1e-5 * xi + n * d * (2.0**-22 * 8) ** 2
     assert abs(g.mean_loss() - o.quadratic_mean_loss(out[:, :d], B)) <= 1e-6 * o.quadratic_mean_loss(want, B)
+    xbar = np.repeat(want.astype(np.float64).mean(0, keepdims=True), n, axis=0)
+    assert abs(g.global_loss() - o.quadratic_mean_loss(xbar, B)) <= 1e-5 * o.quadratic_mean_loss(xbar, B)
     g.init_from_seed(pkg.GPGA_X0_PER_NODE_NORMAL, 1.0, 0.5)
     assert np.abs(bufs[2].cpu().numpy()[:, :d] - o.init_b(n, d, 13, 0.5)).max() <= 3e-5
     assert np.all(bufs[2].cpu().numpy()[:, d:] == sentinel)
