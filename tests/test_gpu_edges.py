@@ -1,0 +1,168 @@
+"""Edge cases and invariants of the CUDA path: extreme node counts, counters at the end of their
+range, structural properties the paper's setting fixes (checked on the GPU results themselves)."""
+import numpy as np
+import pytest
+
+import paper_2105_09080_b200 as pkg
+from oracle import gpga_oracle as o
+from paper_2105_09080_b200.inputs import logistic_inputs, quadratic_inputs
+from test_gpu_parity import TOL_RUN, TOL_STEP, TOPO, close, make_quadratic
+
+pytestmark = pytest.mark.gpu
+
+
+def _torch():
+    import torch
+    return torch
+
+
+@pytest.mark.parametrize("topo,n,d", [("ring", 4096, 8), ("exp", 4096, 12), ("ring", 4097, 8), ("ring", 5000, 5),
+                                      ("exp", 8192, 4), ("static_exp", 1024, 8), ("grid", 4096, 4)])
+def test_many_nodes_few_columns(topo, n, d):
+    """n at and beyond what the shared-memory tile holds (4096 rows): both kernel families."""
+    X0, B = quadratic_inputs(n, d, n + d, x0="per_node")
+    for H, k in ((0, 3), (2, 1)):
+        g, p = make_quadratic(n, d, topo, H, 0.3, 5, 0.2, X0, B)
+        if topo == "grid":
+            p.grid_cols = 64
+        g.step(k)
+        ok, worst = close(g.get_x().cpu().numpy(), o.step(p, X0, k), TOL_STEP)
+        assert ok, (H, k, worst)
+        xi = o.consensus_distance(o.step(p, X0, k))
+        assert abs(g.consensus_distance() - xi) <= 1e-5 * xi + 1e-9
+        g.close()
+
+
+def test_counters_at_the_end_of_their_range():
+    """Largest iteration index, a seed using all 64 bits, the largest column offset."""
+    n, d = 4, 64
+    X0, B = quadratic_inputs(n, d, 3, x0="per_node")
+    seed = 0xFEDCBA9876543210
+    k = 2**32 - 1
+    col0 = 2**34 - 64 - 4
+    g, p = make_quadratic(n, d, "exp", 0, 0.1, seed, 1.0, X0, B, col0=col0)
+    g.step(k)
+    ok, worst = close(g.get_x().cpu().numpy(), o.step(p, X0, k), TOL_STEP)
+    assert ok, worst
+    # a wide state keyed far into the column range goes through the streaming kernels
+    d2 = 19_004
+    X0, B = quadratic_inputs(n, d2, 4, x0="per_node")
+    col0 = 2**34 - d2 - 4
+    g, p = make_quadratic(n, d2, "ring", 0, 0.1, seed, 1.0, X0, B, col0=col0)
+    g.step(k)
+    ok, worst = close(g.get_x().cpu().numpy(), o.step(p, X0, k), TOL_STEP)
+    assert ok, worst
+
+
+@pytest.mark.parametrize("topo,d", [("ring", 1 << 18), ("exp", 1 << 18), ("grid", 20_000), ("ring", 1024)])
+def test_mixing_preserves_the_node_mean_on_the_gpu(topo, d):
+    """W is doubly stochastic: with no gradient step the column means do not move (Section 3)."""
+    n = 16
+    X0, B = quadratic_inputs(n, d, 11, x0="per_node")
+    g, _ = make_quadratic(n, d, topo, 0, 0.0, 1, 0.0, X0, B)
+    before = X0.astype(np.float64).mean(0)
+    g.run(5)
+    after = g.get_x().cpu().numpy().astype(np.float64).mean(0)
+    assert np.abs(after - before).max() <= 5e-7
+    assert g.consensus_distance() < o.consensus_distance(X0)
+
+
+def test_ring_contracts_by_lambda2_on_the_gpu():
+    """No gradient, no noise, state on the second eigenvector: each ring step multiplies it by
+    lambda_2 = (1 + 2 cos(2 pi / n)) / 3 (Appendix A: ||(W - J)^k|| <= beta^k with equality here)."""
+    n, d = 32, 1 << 16
+    lam = (1 + 2 * np.cos(2 * np.pi / n)) / 3
+    rng = np.random.default_rng(0)
+    X0 = (np.cos(2 * np.pi * np.arange(n) / n)[:, None] * rng.standard_normal((1, d))).astype(np.float32)
+    g, _ = make_quadratic(n, d, "ring", 0, 0.0, 1, 0.0, X0, np.zeros_like(X0))
+    xi_prev = g.consensus_distance()
+    for _ in range(6):
+        g.run(1)
+        xi = g.consensus_distance()
+        assert abs(np.sqrt(xi / xi_prev) - lam) < 1e-5
+        xi_prev = xi
+
+
+def test_period_one_is_parallel_sgd():
+    """H = 1: W = (1/n) 1 1^T every step, all rows identical after every iteration (Section 3)."""
+    n, d = 8, 32_768
+    X0, B = quadratic_inputs(n, d, 12)
+    g, p = make_quadratic(n, d, "exp", 1, 0.1, 9, 0.3, X0, B)
+    want = X0
+    for k in range(5):
+        g.step(k)
+        want = o.step(p, want, k)
+        got = g.get_x().cpu().numpy()
+        assert np.all(got == got[0])
+        assert g.consensus_distance() == 0.0
+    ok, worst = close(got, want, TOL_RUN)
+    assert ok, worst
+
+
+def test_step_size_schedule_and_period_change_between_steps():
+    """gamma halved mid-run (the convex experiment's schedule) and H changed on the fly."""
+    n, d = 8, 20_004
+    X0, B = quadratic_inputs(n, d, 13)
+    g, p = make_quadratic(n, d, "ring", 4, 0.2, 9, 0.1, X0, B)
+    g.run(6)
+    want = o.run(p, X0, 0, 6)
+    g.set_gamma(0.1)
+    g.set_period(2)
+    p.gamma, p.H = 0.1, 2
+    g.run(6)
+    want = o.run(p, want, 6, 6)
+    ok, worst = close(g.get_x().cpu().numpy(), want, TOL_RUN)
+    assert ok, worst
+    assert g.get_k() == 12
+
+
+def test_adaptive_period_with_the_logistic_objective():
+    torch = _torch()
+    n, m, d, batch, K, H_init, warm = 8, 256, 64, 32, 40, 2, 6
+    A, y = logistic_inputs(n, m, d, 21)
+    X0 = np.zeros((n, d), dtype=np.float32)
+    g = pkg.Gpga(n, d, pkg.GPGA_TOPO_RING, 0, 0.5, 7)
+    g.set_objective(pkg.GPGA_OBJ_LOGISTIC, l2=1e-3, m=m, batch=batch)
+    xa = torch.from_numpy(X0).cuda()
+    g.bind(xa, torch.empty_like(xa), torch.from_numpy(A).cuda(), torch.from_numpy(y).cuda())
+    periods = g.run_adaptive(K, H_init, warm)
+    p = o.Problem(o.TOPO_RING, 0, 0.5, 7, objective="logistic", data=A, labels=y, l2=1e-3, batch=batch)
+    X, H, C, F_init, want_periods = X0, H_init, 0, 0.0, []
+    for k in range(K):
+        C += 1
+        glob = C == H
+        if glob:   # Algorithm 2: mean over nodes of the mini-batch loss of this iteration at x^(k)
+            F = np.mean([o.logistic_loss(A[i][o.batch_indices(7, k, i, batch, m)],
+                                         y[i][o.batch_indices(7, k, i, batch, m)], X[i], 1e-3) for i in range(n)])
+        p.H = 1 if glob else 0
+        X = o.step(p, X, k)
+        if glob:
+            want_periods.append(H)
+            C = 0
+            F_init, H = o.aga_update(k, warm, H_init, F, F_init, H)
+    assert periods == want_periods
+    ok, worst = close(g.get_x().cpu().numpy(), X, TOL_RUN)
+    assert ok, worst
+
+
+def test_logistic_with_padded_state_rows():
+    torch = _torch()
+    n, m, d, ld, batch = 4, 64, 32, 48, 16
+    A, y = logistic_inputs(n, m, d, 22)
+    rng = np.random.default_rng(2)
+    X0 = (0.2 * rng.standard_normal((n, d))).astype(np.float32)
+    g = pkg.Gpga(n, d, pkg.GPGA_TOPO_EXP, 3, 0.3, 7)
+    g.set_objective(pkg.GPGA_OBJ_LOGISTIC, l2=1e-3, m=m, batch=batch)
+    g.set_row_stride(ld)
+    bufs = [torch.full((n, ld), -7.0, dtype=torch.float32, device="cuda") for _ in range(2)]
+    bufs[0][:, :d] = torch.from_numpy(X0).cuda()
+    g.bind(bufs[0], bufs[1], torch.from_numpy(A).cuda(), torch.from_numpy(y).cuda())
+    g.run(7)
+    p = o.Problem(o.TOPO_EXP, 3, 0.3, 7, objective="logistic", data=A, labels=y, l2=1e-3, batch=batch)
+    want = o.run(p, X0, 0, 7)
+    out = g.get_x().cpu().numpy()
+    ok, worst = close(out[:, :d], want, TOL_RUN)
+    assert ok, worst
+    assert np.all(out[:, d:] == -7.0)
+    f = o.global_logistic_loss(A, y, want.astype(np.float64).mean(0), 1e-3)
+    assert abs(g.global_loss() - f) <= 1e-4 * f
