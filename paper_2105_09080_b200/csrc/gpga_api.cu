@@ -443,7 +443,6 @@ int32_t gpga_global_loss(gpga_t* c, void* stream, double* out_host)
     double* result = reinterpret_cast<double*>(c->scratch + L.result_off);
     cudaError_t e;
     if (c->objective == GPGA_OBJ_LOGISTIC) {
-        if (c->d > 12288) return fail(c, GPGA_ERR_UNSUPPORTED, "logistic global loss needs d <= 12288");
         // xbar borrows the gradient buffer, which is dead between iterations
         float* xbar = reinterpret_cast<float*>(c->scratch + L.G_off);
         int64_t slots = kMaxReduceBlocks;

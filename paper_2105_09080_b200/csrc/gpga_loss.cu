@@ -5,6 +5,7 @@
 #include "gpga_loss.cuh"
 
 #include "gpga_kernels.cuh"
+#include "gpga_launch.cuh"
 
 namespace gpga {
 
@@ -140,6 +141,11 @@ cudaError_t launch_logistic_global_loss(const float* A, const float* y, const fl
     if (chunks > 65535) chunks = 65535;
     const int rows_per_block = (int)((m + chunks - 1) / chunks);
     chunks = (m + rows_per_block - 1) / rows_per_block;
+    if ((size_t)d * sizeof(float) > 48 * 1024) {   // xbar in shared memory beyond the default limit
+        static unsigned long long limit_set = 0;
+        cudaError_t e = ensure_smem_limit(logistic_full_loss_kernel, 200 * 1024, limit_set);
+        if (e != cudaSuccess) return e;
+    }
     logistic_full_loss_kernel<<<dim3((unsigned)n, (unsigned)chunks), kLossBlock, (size_t)d * sizeof(float), s>>>(
         A, y, xbar, d, m, rows_per_block, partials);
     loss_final_kernel<<<1, 32, 0, s>>>(partials, (int)(n * chunks), 1.0 / ((double)n * (double)m), xbar, (int)d,
