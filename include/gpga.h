@@ -155,7 +155,10 @@ int32_t gpga_init_from_seed(gpga_t* ctx, int32_t x0_kind, float x0_std, float b_
  */
 int32_t gpga_step(gpga_t* ctx, int64_t k, void* stream);
 
-/* K iterations k0 .. k0+K-1 starting at the internal counter k0 (Algorithm 1's loop). */
+/* K iterations k0 .. k0+K-1 starting at the internal counter k0 (Algorithm 1's loop).  A quadratic-
+ * objective state of at most 64 MB (X, X+ and b together) is advanced many iterations per launch with
+ * its column strips resident in shared memory -- columns evolve independently -- with results
+ * bit-identical to K calls of gpga_step; larger states take one launch per iteration. */
 int32_t gpga_run(gpga_t* ctx, int64_t K, void* stream);
 
 /*

@@ -8,6 +8,7 @@
 #include "gpga_kernels.cuh"
 #include "gpga_logreg.cuh"
 #include "gpga_loss.cuh"
+#include "gpga_tile.cuh"
 
 using namespace gpga;
 
@@ -181,6 +182,49 @@ int32_t do_step(gpga_ctx* c, int64_t k, bool global, cudaStream_t s)
     if (e != cudaSuccess) return cuda_fail(c, e, "step launch");
     c->cur ^= 1;
     c->k = k + 1;
+    return GPGA_OK;
+}
+
+// K iterations starting at c->k.  A quadratic-objective state small enough to sit in L2 is
+// bound by launch latency when stepped one launch per iteration; it runs instead in launches
+// of up to kFusedSteps iterations with its strips resident in shared memory.
+constexpr int64_t kFusedStateBytes = 64ll << 20;
+constexpr int64_t kFusedSteps = 1024;
+
+int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)
+{
+    const int64_t k_end = c->k + K;
+    if (k_end > (int64_t(1) << 32)) return fail(c, GPGA_ERR_INVALID_ARG, "iteration index must stay below 2^32");
+    const bool fused = c->objective == GPGA_OBJ_QUADRATIC && K >= 2 && run_tile_supports(c->n) &&
+                       12 * c->n * c->ld <= kFusedStateBytes;
+    if (!fused) {
+        for (int64_t k = c->k; k < k_end; ++k) {
+            const int32_t st = do_step(c, k, is_global_step(k, c->H), s);
+            if (st) return st;
+        }
+        return GPGA_OK;
+    }
+    while (c->k < k_end) {
+        const int64_t steps = (k_end - c->k < kFusedSteps) ? k_end - c->k : kFusedSteps;
+        StepParams p;
+        p.x = c->x[c->cur];
+        p.out = c->x[c->cur ^ 1];
+        p.b = c->data;
+        p.n = c->n; p.d = c->d; p.ld = c->ld; p.ldb = c->ld; p.Q = (c->d + 3) / 4;
+        p.q_base = (uint32_t)(c->col0 >> 2);
+        p.k = (uint32_t)c->k;
+        p.gamma = c->gamma; p.sigma = c->sigma;
+        p.hop_log2 = 0; p.len_log2 = 0;
+        p.grid_cols = (int)c->grid_cols;
+        p.chunks = 0; p.inv_batch = 0.f; p.l2 = 0.f;
+        p.keys = c->keys;
+        const cudaError_t e = launch_run_tile(p, (c->sigma != 0.f) ? GRAD_QUAD_NOISE : GRAD_QUAD, vec_ok(c),
+                                              c->topology, c->H, (int)steps, s);
+        c->launches += 1;
+        if (e != cudaSuccess) return cuda_fail(c, e, "fused run launch");
+        c->cur ^= 1;
+        c->k += steps;
+    }
     return GPGA_OK;
 }
 
@@ -366,13 +410,7 @@ int32_t gpga_run(gpga_t* c, int64_t K, void* stream)
     int32_t st = check_ready(c);
     if (st) return st;
     if (K < 0) return fail(c, GPGA_ERR_INVALID_ARG, "K must be >= 0");
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const int64_t k0 = c->k;
-    for (int64_t k = k0; k < k0 + K; ++k) {
-        st = do_step(c, k, is_global_step(k, c->H), s);
-        if (st) return st;
-    }
-    return GPGA_OK;
+    return run_steps(c, K, static_cast<cudaStream_t>(stream));
 }
 
 int32_t gpga_run_host(gpga_t* c, const float* x0_host, const float* data_host, int64_t K,
@@ -393,10 +431,8 @@ int32_t gpga_run_host(gpga_t* c, const float* x0_host, const float* data_host, i
     if (e != cudaSuccess) return cuda_fail(c, e, "data upload");
     c->cur = 0;
     c->k = 0;
-    for (int64_t k = 0; k < K; ++k) {
-        st = do_step(c, k, is_global_step(k, c->H), s);
-        if (st) return st;
-    }
+    st = run_steps(c, K, s);
+    if (st) return st;
     e = cudaMemcpy2DAsync(x_out_host, row_bytes, c->x[c->cur], pitch, row_bytes, (size_t)c->n,
                           cudaMemcpyDeviceToHost, s);
     if (e != cudaSuccess) return cuda_fail(c, e, "result download");

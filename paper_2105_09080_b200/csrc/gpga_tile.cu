@@ -10,26 +10,50 @@
 //    exponential graph) and W = I, at any width;
 //  - every topology when d is so small that one thread per column group would leave
 //    the GPU idle (the logistic workload: d = 1024).
+// A second kernel keeps the strip of X and b in shared memory across several
+// iterations (columns evolve independently under the quadratic objective), for states
+// so small that an iteration per launch is bound by launch latency, not by memory.
 #include "../../include/gpga.h"
 #include "gpga_kernels.cuh"
 #include "gpga_launch.cuh"
+#include "gpga_tile.cuh"
 
 namespace gpga {
 
 constexpr int kTileBlock = 256;
 constexpr int kTileSmemBytes = 64 * 1024;
 
+// y = x - gamma g for the quadratic objective (with or without noise) or a given gradient.
+template <int MODE>
+__device__ __forceinline__ float4 tile_finish(const StepParams& p, float4 x, float4 b, int i, long long q, uint32_t k)
+{
+    float4 g;
+    if (MODE == GRAD_BUFFER) {
+        g = b;
+    } else {
+        g = make_float4(x.x - b.x, x.y - b.y, x.z - b.z, x.w - b.w);
+        if (MODE == GRAD_QUAD_NOISE) {
+            const float4 z = normal4(p.q_base + (uint32_t)q, (uint32_t)i, k, 0u, p.keys);
+            g.x = fmaf(p.sigma, z.x, g.x);
+            g.y = fmaf(p.sigma, z.y, g.y);
+            g.z = fmaf(p.sigma, z.z, g.z);
+            g.w = fmaf(p.sigma, z.w, g.w);
+        }
+    }
+    return make_float4(fmaf(-p.gamma, g.x, x.x), fmaf(-p.gamma, g.y, x.y), fmaf(-p.gamma, g.z, x.z),
+                       fmaf(-p.gamma, g.w, x.w));
+}
+
 template <int MODE, bool VEC>
 __device__ __forceinline__ float4 tile_half_step(const StepParams& p, int i, long long q)
 {
     const long long j0 = q * 4;
     const float4 x = load4<VEC>(p.x + (long long)i * p.ld, j0, p.d);
-    float4 g;
     if (MODE == GRAD_PARTIALS) {
         // g = (1/B) sum_c partial[c][i][:] + l2 x, chunks added in index order
         const long long stride = p.n * p.d;
         const float* part = p.b + (long long)i * p.d + j0;
-        g = *reinterpret_cast<const float4*>(part);
+        float4 g = *reinterpret_cast<const float4*>(part);
         for (int c = 1; c < p.chunks; ++c) {
             const float4 v = *reinterpret_cast<const float4*>(part + c * stride);
             g.x += v.x;
@@ -39,23 +63,10 @@ __device__ __forceinline__ float4 tile_half_step(const StepParams& p, int i, lon
         }
         g = make_float4(fmaf(g.x, p.inv_batch, p.l2 * x.x), fmaf(g.y, p.inv_batch, p.l2 * x.y),
                         fmaf(g.z, p.inv_batch, p.l2 * x.z), fmaf(g.w, p.inv_batch, p.l2 * x.w));
-    } else {
-        const float4 b = load4<VEC>(p.b + (long long)i * p.ldb, j0, p.d);
-        if (MODE == GRAD_BUFFER) {
-            g = b;
-        } else {
-            g = make_float4(x.x - b.x, x.y - b.y, x.z - b.z, x.w - b.w);
-            if (MODE == GRAD_QUAD_NOISE) {
-                const float4 z = normal4(p.q_base + (uint32_t)q, (uint32_t)i, p.k, 0u, p.keys);
-                g.x = fmaf(p.sigma, z.x, g.x);
-                g.y = fmaf(p.sigma, z.y, g.y);
-                g.z = fmaf(p.sigma, z.z, g.z);
-                g.w = fmaf(p.sigma, z.w, g.w);
-            }
-        }
+        return tile_finish<GRAD_BUFFER>(p, x, g, i, q, p.k);
     }
-    return make_float4(fmaf(-p.gamma, g.x, x.x), fmaf(-p.gamma, g.y, x.y), fmaf(-p.gamma, g.z, x.z),
-                       fmaf(-p.gamma, g.w, x.w));
+    const float4 b = load4<VEC>(p.b + (long long)i * p.ldb, j0, p.d);
+    return tile_finish<MODE>(p, x, b, i, q, p.k);
 }
 
 __device__ __forceinline__ void acc4(float4& s, const float4 v)
@@ -64,6 +75,81 @@ __device__ __forceinline__ void acc4(float4& s, const float4 v)
     s.y += v.y;
     s.z += v.z;
     s.w += v.w;
+}
+
+// x_i^(k+1) for cell (row i, group g) from the tile of Y.  `mix` is a GPGA_TOPO_* value or
+// TILE_MIX_GLOBAL.
+__device__ __forceinline__ float4 tile_mix(const float4* ytile, int i, int g, int n, int tile_groups, int mix,
+                                           int hop_log2, int grid_cols, int log2n)
+{
+    float4 s = ytile[i * tile_groups + g];
+    if (mix == TILE_MIX_GLOBAL) {
+        // the column mean exactly as the row-streaming kernel forms it: rows added pairwise in
+        // fp32 in groups of four, group sums accumulated in fp64; the same sum in the same
+        // order for every row, so the rows come out bit-identical
+        double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+        int r = 0;
+        for (; r + 4 <= n; r += 4) {
+            float4 a = ytile[r * tile_groups + g], b = ytile[(r + 2) * tile_groups + g];
+            acc4(a, ytile[(r + 1) * tile_groups + g]);
+            acc4(b, ytile[(r + 3) * tile_groups + g]);
+            acc4(a, b);
+            s0 += (double)a.x;
+            s1 += (double)a.y;
+            s2 += (double)a.z;
+            s3 += (double)a.w;
+        }
+        const int rest = n - r;
+        if (rest >= 1) {
+            float4 a = ytile[r * tile_groups + g];
+            if (rest >= 2) acc4(a, ytile[(r + 1) * tile_groups + g]);
+            s0 += (double)a.x;
+            s1 += (double)a.y;
+            s2 += (double)a.z;
+            s3 += (double)a.w;
+        }
+        if (rest == 3) {
+            const float4 b = ytile[(r + 2) * tile_groups + g];
+            s0 += (double)b.x;
+            s1 += (double)b.y;
+            s2 += (double)b.z;
+            s3 += (double)b.w;
+        }
+        if ((n & (n - 1)) == 0) {   // 1/n is exact: the product equals the quotient
+            const double inv = 1.0 / (double)n;
+            s = make_float4((float)(s0 * inv), (float)(s1 * inv), (float)(s2 * inv), (float)(s3 * inv));
+        } else {
+            const double dn = (double)n;
+            s = make_float4((float)(s0 / dn), (float)(s1 / dn), (float)(s2 / dn), (float)(s3 / dn));
+        }
+    } else if (mix == GPGA_TOPO_RING) {
+        const float4 up = ytile[(i == 0 ? n - 1 : i - 1) * tile_groups + g];
+        const float4 dn = ytile[(i == n - 1 ? 0 : i + 1) * tile_groups + g];
+        const float third = 0.333333343f;
+        s = make_float4((up.x + s.x + dn.x) * third, (up.y + s.y + dn.y) * third, (up.z + s.z + dn.z) * third,
+                        (up.w + s.w + dn.w) * third);
+    } else if (mix == GPGA_TOPO_EXP) {
+        const float4 peer = ytile[((i + (1 << hop_log2)) & (n - 1)) * tile_groups + g];
+        s = make_float4((s.x + peer.x) * 0.5f, (s.y + peer.y) * 0.5f, (s.z + peer.z) * 0.5f,
+                        (s.w + peer.w) * 0.5f);
+    } else if (mix == GPGA_TOPO_GRID) {
+        const int cols = grid_cols, rows = n / cols;
+        const int a = i / cols, b = i - a * cols;
+        const int up = (a == 0 ? rows - 1 : a - 1) * cols + b;
+        const int dn = (a == rows - 1 ? 0 : a + 1) * cols + b;
+        const int lf = a * cols + (b == 0 ? cols - 1 : b - 1);
+        const int rt = a * cols + (b == cols - 1 ? 0 : b + 1);
+        acc4(s, ytile[up * tile_groups + g]);
+        acc4(s, ytile[lf * tile_groups + g]);
+        acc4(s, ytile[rt * tile_groups + g]);
+        acc4(s, ytile[dn * tile_groups + g]);
+        s = make_float4(s.x * 0.2f, s.y * 0.2f, s.z * 0.2f, s.w * 0.2f);
+    } else if (mix == GPGA_TOPO_STATIC_EXP) {
+        for (int t = 0; t < log2n; ++t) acc4(s, ytile[((i + (1 << t)) & (n - 1)) * tile_groups + g]);
+        const float w = 1.0f / (float)(log2n + 1);
+        s = make_float4(s.x * w, s.y * w, s.z * w, s.w * w);
+    }   // GPGA_TOPO_NONE: W = I
+    return s;
 }
 
 template <int MODE, bool VEC>
@@ -84,67 +170,105 @@ __global__ void __launch_bounds__(kTileBlock) step_tile_kernel(const StepParams 
         const int i = c / tile_groups, g = c - i * tile_groups;
         const long long q = q_first + g;
         if (q >= p.Q) continue;
-        float4 s = ytile[c];
-        if (mix == TILE_MIX_GLOBAL) {
-            // the same fp64 sum in the same order for every row: rows come out bit-identical
-            double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
-            for (int r = 0; r < n; ++r) {
-                const float4 v = ytile[r * tile_groups + g];
-                s0 += (double)v.x;
-                s1 += (double)v.y;
-                s2 += (double)v.z;
-                s3 += (double)v.w;
-            }
-            const double dn = (double)n;
-            s = make_float4((float)(s0 / dn), (float)(s1 / dn), (float)(s2 / dn), (float)(s3 / dn));
-        } else if (mix == GPGA_TOPO_RING) {
-            const float4 up = ytile[(i == 0 ? n - 1 : i - 1) * tile_groups + g];
-            const float4 dn = ytile[(i == n - 1 ? 0 : i + 1) * tile_groups + g];
-            const float third = 0.333333343f;
-            s = make_float4((up.x + s.x + dn.x) * third, (up.y + s.y + dn.y) * third,
-                            (up.z + s.z + dn.z) * third, (up.w + s.w + dn.w) * third);
-        } else if (mix == GPGA_TOPO_EXP) {
-            const float4 peer = ytile[((i + (1 << p.hop_log2)) & (n - 1)) * tile_groups + g];
-            s = make_float4((s.x + peer.x) * 0.5f, (s.y + peer.y) * 0.5f, (s.z + peer.z) * 0.5f,
-                            (s.w + peer.w) * 0.5f);
-        } else if (mix == GPGA_TOPO_GRID) {
-            const int cols = p.grid_cols, rows = n / cols;
-            const int a = i / cols, b = i - a * cols;
-            const int up = (a == 0 ? rows - 1 : a - 1) * cols + b;
-            const int dn = (a == rows - 1 ? 0 : a + 1) * cols + b;
-            const int lf = a * cols + (b == 0 ? cols - 1 : b - 1);
-            const int rt = a * cols + (b == cols - 1 ? 0 : b + 1);
-            acc4(s, ytile[up * tile_groups + g]);
-            acc4(s, ytile[lf * tile_groups + g]);
-            acc4(s, ytile[rt * tile_groups + g]);
-            acc4(s, ytile[dn * tile_groups + g]);
-            s = make_float4(s.x * 0.2f, s.y * 0.2f, s.z * 0.2f, s.w * 0.2f);
-        } else if (mix == GPGA_TOPO_STATIC_EXP) {
-            for (int t = 0; t < log2n; ++t) acc4(s, ytile[((i + (1 << t)) & (n - 1)) * tile_groups + g]);
-            const float w = 1.0f / (float)(log2n + 1);
-            s = make_float4(s.x * w, s.y * w, s.z * w, s.w * w);
-        }   // GPGA_TOPO_NONE: W = I
+        const float4 s = tile_mix(ytile, i, g, n, tile_groups, mix, p.hop_log2, p.grid_cols, log2n);
         store4<VEC>(p.out + (long long)i * p.ld, q * 4, p.d, s);
     }
 }
 
+// K iterations k0 .. k0+K-1 of Algorithm 1 on one strip of column groups, with the strip of
+// X, b and Y resident in shared memory: X and b are read from global memory once and X written
+// once for all K iterations.  Quadratic objective only (its columns are independent).  Each
+// iteration does exactly what step_tile_kernel does, so the result is bit-identical to K
+// single-iteration launches.
+template <int MODE, bool VEC>
+__global__ void __launch_bounds__(kTileBlock) run_tile_kernel(const StepParams p, int topology, long long H,
+                                                              long long phase0, int hop0, int steps,
+                                                              int tile_groups, int log2n)
+{
+    extern __shared__ float4 tile_smem[];   // X, b, Y: [n][tile_groups] each
+    const int n = (int)p.n;
+    const int cells = n * tile_groups;
+    float4* xtile = tile_smem;
+    float4* btile = tile_smem + cells;
+    float4* ytile = tile_smem + 2 * cells;
+    const long long q_first = (long long)blockIdx.x * tile_groups;
+    for (int c = threadIdx.x; c < cells; c += blockDim.x) {
+        const int i = c / tile_groups, g = c - i * tile_groups;
+        const long long q = q_first + g;
+        if (q < p.Q) {
+            xtile[c] = load4<VEC>(p.x + (long long)i * p.ld, q * 4, p.d);
+            btile[c] = load4<VEC>(p.b + (long long)i * p.ldb, q * 4, p.d);
+        }
+    }
+    __syncthreads();
+    // schedule counters kept incrementally (no division in the loop):
+    // phase = (k + 1) mod H, global average when it is 0; hop_log2 = k mod log2(n)
+    long long phase = phase0;
+    int hop_log2 = hop0;
+    // a thread's first cell, with its coordinates worked out once; further cells (strips with
+    // more cells than threads) go through the generic loops
+    const int c0 = threadIdx.x;
+    const int i0 = c0 / tile_groups, g0 = c0 - i0 * tile_groups;
+    const bool own0 = c0 < cells && q_first + g0 < p.Q;
+    for (int t = 0; t < steps; ++t) {
+        const uint32_t k = p.k + (uint32_t)t;
+        const bool global = H > 0 && phase == 0;            // Algorithm 1's test mod(k + 1, H) = 0
+        const int mix = global ? (int)TILE_MIX_GLOBAL : topology;
+        if (own0) ytile[c0] = tile_finish<MODE>(p, xtile[c0], btile[c0], i0, q_first + g0, k);
+        for (int c = c0 + blockDim.x; c < cells; c += blockDim.x) {
+            const int i = c / tile_groups, g = c - i * tile_groups;
+            const long long q = q_first + g;
+            if (q < p.Q) ytile[c] = tile_finish<MODE>(p, xtile[c], btile[c], i, q, k);
+        }
+        __syncthreads();
+        if (own0) xtile[c0] = tile_mix(ytile, i0, g0, n, tile_groups, mix, hop_log2, p.grid_cols, log2n);
+        for (int c = c0 + blockDim.x; c < cells; c += blockDim.x) {
+            const int i = c / tile_groups, g = c - i * tile_groups;
+            if (q_first + g < p.Q) xtile[c] = tile_mix(ytile, i, g, n, tile_groups, mix, hop_log2, p.grid_cols, log2n);
+        }
+        __syncthreads();
+        if (++phase >= H) phase = 0;
+        if (++hop_log2 >= log2n) hop_log2 = 0;
+    }
+    for (int c = threadIdx.x; c < cells; c += blockDim.x) {
+        const int i = c / tile_groups, g = c - i * tile_groups;
+        const long long q = q_first + g;
+        if (q < p.Q) store4<VEC>(p.out + (long long)i * p.ld, q * 4, p.d, xtile[c]);
+    }
+}
+
 bool tile_supports(long long n) { return n * 16 <= kTileSmemBytes; }
+bool run_tile_supports(long long n) { return n * 2 * 48 <= kTileSmemBytes; }   // X, b, Y strips of >= 2 groups
+
+static int log2_floor(long long n)
+{
+    int t = 0;
+    while ((1LL << (t + 1)) <= n) ++t;
+    return t;
+}
+
+// Strip width: enough blocks to cover the SMs, at most 64 groups, within the shared-memory budget.
+static int strip_groups(long long Q, long long n, int bytes_per_cell, int blocks_per_sm = 2)
+{
+    long long tg = (Q + blocks_per_sm * 148 - 1) / (blocks_per_sm * 148);
+    if (tg < 2) tg = 2;
+    if (tg > 64) tg = 64;
+    if (tg > kTileSmemBytes / bytes_per_cell / n) tg = kTileSmemBytes / bytes_per_cell / n;
+    if (tg > Q) tg = Q;
+    // whole warps of cells where the strip can be narrowed to get them
+    for (long long t = tg; t >= 2 && t * 2 > tg; --t)
+        if ((n * t) % 32 == 0) { tg = t; break; }
+    return (int)tg;
+}
 
 cudaError_t launch_step_tile(const StepParams& p, int mode, bool vec, int mix, cudaStream_t s)
 {
     if (!tile_supports(p.n)) return cudaErrorInvalidConfiguration;   // callers bound n
-    // strip width: enough blocks to cover the SMs, at most 64 groups, at most 64 KB of tile
-    long long tg = (p.Q + 2 * 148 - 1) / (2 * 148);
-    if (tg < 2) tg = 2;
-    if (tg > 64) tg = 64;
-    if (tg > kTileSmemBytes / 16 / p.n) tg = kTileSmemBytes / 16 / p.n;
-    if (tg > p.Q) tg = p.Q;
-    const int tile_groups = (int)tg;
-    int log2n = 0;
-    while ((1LL << (log2n + 1)) <= p.n) ++log2n;
+    const int tile_groups = strip_groups(p.Q, p.n, 16);
+    const int log2n = log2_floor(p.n);
     const unsigned grd = (unsigned)((p.Q + tile_groups - 1) / tile_groups);
     const size_t smem = (size_t)p.n * tile_groups * 16;
-    long long cells = p.n * tile_groups;
+    const long long cells = p.n * tile_groups;
     const int blk = cells >= kTileBlock ? kTileBlock : (int)((cells + 31) / 32 * 32);
 #define GPGA_TILE(M, V)                                                                          \
     do {                                                                                         \
@@ -165,6 +289,37 @@ cudaError_t launch_step_tile(const StepParams& p, int mode, bool vec, int mix, c
         else GPGA_TILE(GRAD_BUFFER, false);
     }
 #undef GPGA_TILE
+    return cudaGetLastError();
+}
+
+cudaError_t launch_run_tile(const StepParams& p, int mode, bool vec, int topology, long long H, int steps,
+                            cudaStream_t s)
+{
+    if (!run_tile_supports(p.n) || (mode != GRAD_QUAD && mode != GRAD_QUAD_NOISE))
+        return cudaErrorInvalidConfiguration;   // callers check
+    const int tile_groups = strip_groups(p.Q, p.n, 48, 8);   // compute-bound: fill every SM with warps
+    const int log2n = log2_floor(p.n);
+    const unsigned grd = (unsigned)((p.Q + tile_groups - 1) / tile_groups);
+    const size_t smem = (size_t)p.n * tile_groups * 48;
+    const long long cells = p.n * tile_groups;
+    const int blk = cells >= kTileBlock ? kTileBlock : (int)((cells + 31) / 32 * 32);
+    const long long phase0 = H > 0 ? ((long long)p.k + 1) % H : 1;
+    const int hop0 = log2n > 0 ? (int)(p.k % (uint32_t)log2n) : 0;
+#define GPGA_RUN_TILE(M, V)                                                                      \
+    do {                                                                                         \
+        static unsigned long long limit_set = 0;                                                 \
+        cudaError_t e = ensure_smem_limit(run_tile_kernel<M, V>, kTileSmemBytes, limit_set);     \
+        if (e != cudaSuccess) return e;                                                          \
+        run_tile_kernel<M, V><<<grd, blk, smem, s>>>(p, topology, H, phase0, hop0, steps, tile_groups, log2n); \
+    } while (0)
+    if (vec) {
+        if (mode == GRAD_QUAD) GPGA_RUN_TILE(GRAD_QUAD, true);
+        else GPGA_RUN_TILE(GRAD_QUAD_NOISE, true);
+    } else {
+        if (mode == GRAD_QUAD) GPGA_RUN_TILE(GRAD_QUAD, false);
+        else GPGA_RUN_TILE(GRAD_QUAD_NOISE, false);
+    }
+#undef GPGA_RUN_TILE
     return cudaGetLastError();
 }
 

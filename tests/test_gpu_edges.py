@@ -166,3 +166,41 @@ def test_logistic_with_padded_state_rows():
     assert np.all(out[:, d:] == -7.0)
     f = o.global_logistic_loss(A, y, want.astype(np.float64).mean(0), 1e-3)
     assert abs(g.global_loss() - f) <= 1e-4 * f
+
+
+@pytest.mark.parametrize("topo,n,d,H", [("ring", 8, 65_536, 4), ("exp", 32, 4096, 8), ("ring", 7, 1031, 3),
+                                        ("grid", 12, 520, 5), ("static_exp", 16, 64, 0), ("none", 5, 36, 2),
+                                        ("ring", 1, 8, 2), ("exp", 2, 20_004, 1), ("ring", 600, 24, 4)])
+def test_multi_iteration_launch_equals_single_iterations(topo, n, d, H):
+    """gpga_run keeps a small state in shared memory across iterations (one launch for many
+    iterations); the result is bit-identical to stepping one launch per iteration."""
+    X0, B = quadratic_inputs(n, d, 31 + n, x0="shared", x0_std=0.5)
+    K = 13
+    g, p = make_quadratic(n, d, topo, H, 0.1, 17, 0.2, X0, B)
+    if topo == "grid":
+        p.grid_cols = 4
+    g.run(K)
+    assert g.launch_count() == 1 and g.get_k() == K
+    fused = g.get_x().cpu().numpy().copy()
+    g2, _ = make_quadratic(n, d, topo, H, 0.1, 17, 0.2, X0, B)
+    for k in range(K):
+        g2.step(k)
+    assert g2.launch_count() == K
+    assert np.array_equal(fused, g2.get_x().cpu().numpy())
+    ok, worst = close(fused, o.run(p, X0, 0, K), TOL_RUN)
+    assert ok, worst
+    # continuing from the middle of a period gives the same as one long run
+    g3, _ = make_quadratic(n, d, topo, H, 0.1, 17, 0.2, X0, B)
+    g3.run(5)
+    g3.run(K - 5)
+    assert np.array_equal(fused, g3.get_x().cpu().numpy())
+
+
+def test_multi_iteration_launch_is_chunked_for_long_runs():
+    n, d, K = 4, 256, 2500            # more than one launch worth of iterations
+    X0, B = quadratic_inputs(n, d, 5)
+    g, p = make_quadratic(n, d, "ring", 16, 0.05, 3, 0.1, X0, B)
+    g.run(K)
+    assert g.launch_count() == 3 and g.get_k() == K
+    ok, worst = close(g.get_x().cpu().numpy(), o.run(p, X0, 0, K), TOL_RUN)
+    assert ok, worst
