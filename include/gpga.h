@@ -179,8 +179,9 @@ int32_t gpga_consensus_distance(gpga_t* ctx, void* stream, double* out_host);
 
 /*
  * Mean over nodes of the local loss at each node's own iterate, (1/n) sum_i F_i(x_i)
- * (the quantity Algorithm 2 averages).  QUADRATIC: F_i = 1/2 ||x_i - b_i||^2.
- * Synchronises the stream.
+ * (the quantity Algorithm 2 averages).  QUADRATIC: F_i = 1/2 ||x_i - b_i||^2 (the additive
+ * noise model has no per-sample loss).  LOGISTIC: the loss over the mini-batch that node i
+ * draws for the current iteration counter k, plus (l2/2)||x_i||^2.  Synchronises the stream.
  */
 int32_t gpga_mean_loss(gpga_t* ctx, void* stream, double* out_host);
 

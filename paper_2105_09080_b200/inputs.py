@@ -70,3 +70,22 @@ def logistic_inputs_device(n: int, m: int, d: int, seed: int, device="cuda", het
     margin = torch.einsum("nmd,nd->nm", A, xi) + label_noise * torch.randn((n, m), device=device, generator=gen)
     y = torch.where(margin >= 0, 1.0, -1.0).to(torch.float32).contiguous()
     return A.contiguous(), y
+
+
+def convex_experiment_inputs(n: int, m: int = 8000, d: int = 10, seed: int = 0, iid: bool = False):
+    """Synthetic data of the paper's logistic-regression experiment (Section 5.1): features
+    h ~ N(0, 10 I_d); a unit-norm x*_i per node (one shared x* when iid); label +1 with
+    probability 1 / (1 + exp(-h^T x*_i)), else -1.  Returns (A, y) float32 with the feature
+    dimension zero-padded to a multiple of 4 (padded weights receive zero gradient and stay 0)."""
+    rng = np.random.default_rng(seed)
+    dp = (d + 3) // 4 * 4
+    A = np.zeros((n, m, dp), dtype=np.float32)
+    A[:, :, :d] = rng.normal(0.0, np.sqrt(10.0), size=(n, m, d)).astype(np.float32)
+    shared = rng.standard_normal(d)
+    y = np.empty((n, m), dtype=np.float32)
+    for i in range(n):
+        xs = shared if iid else rng.standard_normal(d)
+        xs = xs / np.linalg.norm(xs)
+        prob = 1.0 / (1.0 + np.exp(-(A[i, :, :d].astype(np.float64) @ xs)))
+        y[i] = np.where(rng.uniform(size=m) <= prob, 1.0, -1.0)
+    return np.ascontiguousarray(A), np.ascontiguousarray(y)
