@@ -35,10 +35,12 @@ def run_one(A_dev, y_dev, topology, H, iters, every, batch, seed, gamma0=0.2, ha
     done = 0
     while done < iters:
         g.set_gamma(gamma0 * 0.5 ** (done // halve_every))
-        step = min(every, iters - done, halve_every - done % halve_every)
+        next_record = min((done // every + 1) * every, iters)
+        next_halving = (done // halve_every + 1) * halve_every
+        step = min(next_record, next_halving) - done
         g.run(step)
         done += step
-        if done % every == 0 or done == iters:
+        if done == next_record:
             loss.append(g.global_loss())
             cons.append(g.consensus_distance())
     g.close()

@@ -64,3 +64,13 @@ def test_sharded_run_equals_unsharded_run(tmp_path):
     assert np.array_equal(got, want)
     xi = float(np.load(tmp_path / "xi.npy")[0])
     assert abs(xi - o.consensus_distance(want)) <= 1e-12 * xi
+
+
+def test_convex_experiment_inputs_follow_the_recipe():
+    from paper_2105_09080_b200.inputs import convex_experiment_inputs
+    A, y = convex_experiment_inputs(6, 2000, 10, seed=1)
+    assert A.shape == (6, 2000, 12) and not A[:, :, 10:].any()           # zero padding to a multiple of 4
+    assert abs(A[:, :, :10].std() - np.sqrt(10)) < 0.05
+    assert set(np.unique(y)) == {-1.0, 1.0}
+    A2, y2 = convex_experiment_inputs(6, 2000, 10, seed=1, iid=True)
+    assert A2.shape == A.shape and abs(y2.mean()) < 0.1
