@@ -53,7 +53,8 @@ enum {
     GPGA_TOPO_EXP = 1,        /* step k: average with (i + 2^(k mod log2 n)) mod n, w = 1/2; n = 2^m */
     GPGA_TOPO_GRID = 2,       /* r x c torus, w = 1/5 on the node and its 4 neighbours */
     GPGA_TOPO_STATIC_EXP = 3, /* w = 1/(log2 n + 1) on i and (i + 2^t) mod n, t < log2 n */
-    GPGA_TOPO_NONE = 4        /* W = I (Local SGD between global averages) */
+    GPGA_TOPO_NONE = 4,       /* W = I (Local SGD between global averages) */
+    GPGA_TOPO_SPARSE = 5      /* any doubly-stochastic W given in CSR form (gpga_set_weight_matrix) */
 };
 
 enum { GPGA_OBJ_QUADRATIC = 0, GPGA_OBJ_LOGISTIC = 1 };
@@ -100,6 +101,16 @@ int32_t gpga_set_objective(gpga_t* ctx, int32_t objective, float sigma, float l2
 /* Grid topology only: number of columns c of the r x c torus (n = r * c).
  * Errors: INVALID_ARG unless c >= 1 and c divides n. */
 int32_t gpga_set_grid_cols(gpga_t* ctx, int64_t cols);
+
+/*
+ * Topology SPARSE: the weight matrix W of Section 3 (doubly stochastic, w_ij > 0 only between
+ * neighbours or for i = j) in CSR form, DEVICE pointers owned by the caller: row_ptr (n + 1
+ * int32), col_idx and weights (nnz entries; row i holds x_i^(k+1) = sum_e w[e] y_{col_idx[e]}).
+ * The library does not check stochasticity (the arrays live on the device).  n <= 4096.
+ * Errors: INVALID_ARG for NULL pointers, nnz < n or a handle with another topology.
+ */
+int32_t gpga_set_weight_matrix(gpga_t* ctx, const int32_t* row_ptr_dev, const int32_t* col_idx_dev,
+                               const float* weights_dev, int64_t nnz);
 
 /*
  * Row stride ld (in floats, ld >= d) of the X buffers and, for the quadratic objective, of b:

@@ -28,6 +28,7 @@ TOPO_EXP = 1
 TOPO_GRID = 2
 TOPO_STATIC_EXP = 3
 TOPO_NONE = 4
+TOPO_SPARSE = 5   # any doubly-stochastic W given explicitly
 
 X0_ZERO = 0
 X0_SHARED_NORMAL = 1
@@ -197,7 +198,24 @@ def dense_w_static_exp(n: int) -> np.ndarray:
     return W
 
 
-def dense_w(topology: int, n: int, k: int, grid_cols: int = 0) -> np.ndarray:
+def metropolis_w(adjacency: np.ndarray) -> np.ndarray:
+    """Metropolis-Hastings weights of an undirected graph: w_ij = 1 / (1 + max(deg_i, deg_j)) on
+    edges, the rest of each row on the diagonal; symmetric, hence doubly stochastic (Section 3)."""
+    adj = np.asarray(adjacency, dtype=bool)
+    n = adj.shape[0]
+    deg = adj.sum(1)
+    W = np.zeros((n, n))
+    for i in range(n):
+        for j in range(n):
+            if i != j and adj[i, j]:
+                W[i, j] = 1.0 / (1.0 + max(deg[i], deg[j]))
+        W[i, i] = 1.0 - W[i].sum()
+    return W
+
+
+def dense_w(topology: int, n: int, k: int, grid_cols: int = 0, W=None) -> np.ndarray:
+    if topology == TOPO_SPARSE:
+        return np.asarray(W, dtype=np.float64)
     if topology == TOPO_RING:
         return dense_w_ring(n)
     if topology == TOPO_EXP:
@@ -232,12 +250,19 @@ def gradient_half_step(X, G, gamma) -> np.ndarray:
     return Y
 
 
-def mix(Y, topology: int, k: int, global_step: bool, grid_cols: int = 0) -> np.ndarray:
+def mix(Y, topology: int, k: int, global_step: bool, grid_cols: int = 0, W=None) -> np.ndarray:
     """Sparse-path mixing of the half-step matrix Y (fp64 in, fp64 out)."""
     Y = _f64(Y)
     n, d = Y.shape
     Z = np.empty_like(Y)
     L = lib()
+    if topology == TOPO_SPARSE and not global_step:
+        # x_i = sum_{j in N_i} w_ij y_j, row by row over the stored neighbours (Algorithm 1)
+        Wd = np.asarray(W, dtype=np.float64)
+        for i in range(n):
+            nb = np.nonzero(Wd[i])[0]
+            Z[i] = sum(Wd[i, j] * Y[j] for j in nb)
+        return Z
     if global_step:
         L.gpga_oracle_mix_global(n, d, _p(Y), _p(Z))
     elif topology == TOPO_RING:
@@ -255,12 +280,12 @@ def mix(Y, topology: int, k: int, global_step: bool, grid_cols: int = 0) -> np.n
     return Z
 
 
-def mix_dense(Y, topology: int, k: int, global_step: bool, grid_cols: int = 0) -> np.ndarray:
+def mix_dense(Y, topology: int, k: int, global_step: bool, grid_cols: int = 0, W=None) -> np.ndarray:
     """Dense-W mixing, X+ = W Y (tiny n only)."""
     Y = _f64(Y)
     n = Y.shape[0]
-    W = dense_w_global(n) if global_step else dense_w(topology, n, k, grid_cols)
-    return W @ Y
+    Wd = dense_w_global(n) if global_step else dense_w(topology, n, k, grid_cols, W)
+    return Wd @ Y
 
 
 def consensus_distance(X) -> float:
@@ -336,7 +361,7 @@ class Problem:
     (data = A of shape n x m x d, labels = y of shape n x m)."""
 
     def __init__(self, topology, H, gamma, seed, sigma=0.0, objective="quadratic", data=None,
-                 labels=None, l2=0.0, batch=0, col0=0, grid_cols=0):
+                 labels=None, l2=0.0, batch=0, col0=0, grid_cols=0, W=None):
         self.topology = topology
         self.H = H
         self.gamma = gamma
@@ -349,6 +374,7 @@ class Problem:
         self.batch = batch
         self.col0 = col0
         self.grid_cols = grid_cols
+        self.W = W
 
 
 def step_f64(p: Problem, X, k: int, dense: bool = False) -> np.ndarray:
@@ -360,7 +386,7 @@ def step_f64(p: Problem, X, k: int, dense: bool = False) -> np.ndarray:
         Y = gradient_half_step(X, G, p.gamma)
     g = is_global(k, p.H)
     mixer = mix_dense if dense else mix
-    return mixer(Y, p.topology, k, g, p.grid_cols)
+    return mixer(Y, p.topology, k, g, p.grid_cols, p.W)
 
 
 def step(p: Problem, X32, k: int, dense: bool = False) -> np.ndarray:

@@ -25,6 +25,7 @@ GPGA_TOPO_EXP = 1
 GPGA_TOPO_GRID = 2
 GPGA_TOPO_STATIC_EXP = 3
 GPGA_TOPO_NONE = 4
+GPGA_TOPO_SPARSE = 5
 
 GPGA_OBJ_QUADRATIC = 0
 GPGA_OBJ_LOGISTIC = 1
@@ -41,6 +42,7 @@ SIGNATURES = {
     "gpga_create": (_i32, [_i64, _i64, _i32, _i64, _f32, _u64, C.POINTER(_P)]),
     "gpga_set_objective": (_i32, [_P, _i32, _f32, _f32, _i64, _i64]),
     "gpga_set_grid_cols": (_i32, [_P, _i64]),
+    "gpga_set_weight_matrix": (_i32, [_P, _P, _P, _P, _i64]),
     "gpga_set_row_stride": (_i32, [_P, _i64]),
     "gpga_set_column_offset": (_i32, [_P, _i64]),
     "gpga_scratch_bytes": (_i64, [_P]),
@@ -144,6 +146,12 @@ class Gpga:
 
     def set_grid_cols(self, cols):
         self._check(lib().gpga_set_grid_cols(self._h, cols))
+
+    def set_weight_matrix(self, row_ptr, col_idx, weights):
+        """CSR weight matrix as torch CUDA tensors (int32, int32, float32); kept alive by this object."""
+        self._w = (row_ptr, col_idx, weights)
+        self._check(lib().gpga_set_weight_matrix(self._h, row_ptr.data_ptr(), col_idx.data_ptr(),
+                                                 weights.data_ptr(), weights.numel()))
 
     def set_row_stride(self, ld):
         self._check(lib().gpga_set_row_stride(self._h, ld))

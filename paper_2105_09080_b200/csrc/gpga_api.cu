@@ -36,6 +36,7 @@ struct gpga_ctx {
     int32_t sticky = GPGA_OK;
     std::string err;
     PhiloxKeys keys;
+    SparseW sparse;   // topology SPARSE: caller-owned CSR arrays on the device
 };
 
 static thread_local std::string g_create_error;
@@ -169,8 +170,10 @@ int32_t do_step(gpga_ctx* c, int64_t k, bool global, cudaStream_t s)
             p.len_log2 = tau - p.hop_log2;
         }
     }
+    if (c->topology == GPGA_TOPO_SPARSE && !c->sparse.row_ptr)
+        return fail(c, GPGA_ERR_NOT_READY, "topology SPARSE needs gpga_set_weight_matrix");
     if (narrow || (tile_topology && !global)) {
-        e = launch_step_tile(p, mode, vec, global ? (int)TILE_MIX_GLOBAL : c->topology, s);
+        e = launch_step_tile_w(p, mode, vec, global ? (int)TILE_MIX_GLOBAL : c->topology, c->sparse, s);
     } else if (global) {
         e = launch_step_global(p, mode, vec, s);
     } else if (c->topology == GPGA_TOPO_RING) {
@@ -195,6 +198,8 @@ int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)
 {
     const int64_t k_end = c->k + K;
     if (k_end > (int64_t(1) << 32)) return fail(c, GPGA_ERR_INVALID_ARG, "iteration index must stay below 2^32");
+    if (c->topology == GPGA_TOPO_SPARSE && !c->sparse.row_ptr)
+        return fail(c, GPGA_ERR_NOT_READY, "topology SPARSE needs gpga_set_weight_matrix");
     const bool fused = c->objective == GPGA_OBJ_QUADRATIC && K >= 2 && run_tile_supports(c->n) &&
                        12 * c->n * c->ld <= kFusedStateBytes;
     if (!fused) {
@@ -219,7 +224,7 @@ int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)
         p.chunks = 0; p.inv_batch = 0.f; p.l2 = 0.f;
         p.keys = c->keys;
         const cudaError_t e = launch_run_tile(p, (c->sigma != 0.f) ? GRAD_QUAD_NOISE : GRAD_QUAD, vec_ok(c),
-                                              c->topology, c->H, (int)steps, s);
+                                              c->topology, c->H, (int)steps, c->sparse, s);
         c->launches += 1;
         if (e != cudaSuccess) return cuda_fail(c, e, "fused run launch");
         c->cur ^= 1;
@@ -276,11 +281,12 @@ int32_t gpga_create(int64_t n, int64_t d, int32_t topology, int64_t H, float gam
     if (d < 1 || d >= (int64_t(1) << 34)) return fail(nullptr, GPGA_ERR_INVALID_ARG, "d must be in [1, 2^34)");
     if (H < 0) return fail(nullptr, GPGA_ERR_INVALID_ARG, "H must be >= 0 (0 = never average globally)");
     if (!std::isfinite(gamma) || gamma < 0.f) return fail(nullptr, GPGA_ERR_INVALID_ARG, "gamma must be finite and >= 0");
-    if (topology < GPGA_TOPO_RING || topology > GPGA_TOPO_NONE)
+    if (topology < GPGA_TOPO_RING || topology > GPGA_TOPO_SPARSE)
         return fail(nullptr, GPGA_ERR_INVALID_ARG, "unknown topology");
     if ((topology == GPGA_TOPO_EXP || topology == GPGA_TOPO_STATIC_EXP) && !is_pow2(n))
         return fail(nullptr, GPGA_ERR_UNSUPPORTED, "exponential graphs need n to be a power of two");
-    if ((topology == GPGA_TOPO_GRID || topology == GPGA_TOPO_STATIC_EXP || topology == GPGA_TOPO_NONE) &&
+    if ((topology == GPGA_TOPO_GRID || topology == GPGA_TOPO_STATIC_EXP || topology == GPGA_TOPO_NONE ||
+         topology == GPGA_TOPO_SPARSE) &&
         n > kMaxTileNodes)
         return fail(nullptr, GPGA_ERR_UNSUPPORTED, "this topology supports at most 4096 nodes");
     gpga_ctx* c = new (std::nothrow) gpga_ctx;
@@ -324,6 +330,19 @@ int32_t gpga_set_grid_cols(gpga_t* c, int64_t cols)
     if (!c) return fail(nullptr, GPGA_ERR_NOT_READY, "NULL handle");
     if (cols < 1 || c->n % cols != 0) return fail(c, GPGA_ERR_INVALID_ARG, "cols must divide n");
     c->grid_cols = cols;
+    return GPGA_OK;
+}
+
+int32_t gpga_set_weight_matrix(gpga_t* c, const int32_t* row_ptr_dev, const int32_t* col_idx_dev,
+                               const float* weights_dev, int64_t nnz)
+{
+    if (!c) return fail(nullptr, GPGA_ERR_NOT_READY, "NULL handle");
+    if (c->topology != GPGA_TOPO_SPARSE) return fail(c, GPGA_ERR_INVALID_ARG, "handle was not created with topology SPARSE");
+    if (!row_ptr_dev || !col_idx_dev || !weights_dev || nnz < c->n)
+        return fail(c, GPGA_ERR_INVALID_ARG, "need non-NULL CSR arrays with at least one entry per row");
+    c->sparse.row_ptr = row_ptr_dev;
+    c->sparse.col = col_idx_dev;
+    c->sparse.w = weights_dev;
     return GPGA_OK;
 }
 

@@ -80,7 +80,7 @@ __device__ __forceinline__ void acc4(float4& s, const float4 v)
 // x_i^(k+1) for cell (row i, group g) from the tile of Y.  `mix` is a GPGA_TOPO_* value or
 // TILE_MIX_GLOBAL.
 __device__ __forceinline__ float4 tile_mix(const float4* ytile, int i, int g, int n, int tile_groups, int mix,
-                                           int hop_log2, int grid_cols, int log2n)
+                                           int hop_log2, int grid_cols, int log2n, const SparseW& sw)
 {
     float4 s = ytile[i * tile_groups + g];
     if (mix == TILE_MIX_GLOBAL) {
@@ -148,13 +148,24 @@ __device__ __forceinline__ float4 tile_mix(const float4* ytile, int i, int g, in
         for (int t = 0; t < log2n; ++t) acc4(s, ytile[((i + (1 << t)) & (n - 1)) * tile_groups + g]);
         const float w = 1.0f / (float)(log2n + 1);
         s = make_float4(s.x * w, s.y * w, s.z * w, s.w * w);
+    } else if (mix == GPGA_TOPO_SPARSE) {
+        // x_i = sum_j w_ij y_j over the stored entries of row i, in storage order
+        s = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int e = sw.row_ptr[i]; e < sw.row_ptr[i + 1]; ++e) {
+            const float w = sw.w[e];
+            const float4 v = ytile[sw.col[e] * tile_groups + g];
+            s.x = fmaf(w, v.x, s.x);
+            s.y = fmaf(w, v.y, s.y);
+            s.z = fmaf(w, v.z, s.z);
+            s.w = fmaf(w, v.w, s.w);
+        }
     }   // GPGA_TOPO_NONE: W = I
     return s;
 }
 
 template <int MODE, bool VEC>
 __global__ void __launch_bounds__(kTileBlock) step_tile_kernel(const StepParams p, int mix, int tile_groups,
-                                                               int log2n)
+                                                               int log2n, const SparseW sw)
 {
     extern __shared__ float4 ytile[];   // [n][tile_groups]
     const long long q_first = (long long)blockIdx.x * tile_groups;
@@ -170,7 +181,7 @@ __global__ void __launch_bounds__(kTileBlock) step_tile_kernel(const StepParams 
         const int i = c / tile_groups, g = c - i * tile_groups;
         const long long q = q_first + g;
         if (q >= p.Q) continue;
-        const float4 s = tile_mix(ytile, i, g, n, tile_groups, mix, p.hop_log2, p.grid_cols, log2n);
+        const float4 s = tile_mix(ytile, i, g, n, tile_groups, mix, p.hop_log2, p.grid_cols, log2n, sw);
         store4<VEC>(p.out + (long long)i * p.ld, q * 4, p.d, s);
     }
 }
@@ -183,7 +194,7 @@ __global__ void __launch_bounds__(kTileBlock) step_tile_kernel(const StepParams 
 template <int MODE, bool VEC>
 __global__ void __launch_bounds__(kTileBlock) run_tile_kernel(const StepParams p, int topology, long long H,
                                                               long long phase0, int hop0, int steps,
-                                                              int tile_groups, int log2n)
+                                                              int tile_groups, int log2n, const SparseW sw)
 {
     extern __shared__ float4 tile_smem[];   // X, b, Y: [n][tile_groups] each
     const int n = (int)p.n;
@@ -221,10 +232,10 @@ __global__ void __launch_bounds__(kTileBlock) run_tile_kernel(const StepParams p
             if (q < p.Q) ytile[c] = tile_finish<MODE>(p, xtile[c], btile[c], i, q, k);
         }
         __syncthreads();
-        if (own0) xtile[c0] = tile_mix(ytile, i0, g0, n, tile_groups, mix, hop_log2, p.grid_cols, log2n);
+        if (own0) xtile[c0] = tile_mix(ytile, i0, g0, n, tile_groups, mix, hop_log2, p.grid_cols, log2n, sw);
         for (int c = c0 + blockDim.x; c < cells; c += blockDim.x) {
             const int i = c / tile_groups, g = c - i * tile_groups;
-            if (q_first + g < p.Q) xtile[c] = tile_mix(ytile, i, g, n, tile_groups, mix, hop_log2, p.grid_cols, log2n);
+            if (q_first + g < p.Q) xtile[c] = tile_mix(ytile, i, g, n, tile_groups, mix, hop_log2, p.grid_cols, log2n, sw);
         }
         __syncthreads();
         if (++phase >= H) phase = 0;
@@ -263,6 +274,11 @@ static int strip_groups(long long Q, long long n, int bytes_per_cell, int blocks
 
 cudaError_t launch_step_tile(const StepParams& p, int mode, bool vec, int mix, cudaStream_t s)
 {
+    return launch_step_tile_w(p, mode, vec, mix, SparseW(), s);
+}
+
+cudaError_t launch_step_tile_w(const StepParams& p, int mode, bool vec, int mix, const SparseW& sw, cudaStream_t s)
+{
     if (!tile_supports(p.n)) return cudaErrorInvalidConfiguration;   // callers bound n
     const int tile_groups = strip_groups(p.Q, p.n, 16);
     const int log2n = log2_floor(p.n);
@@ -275,7 +291,7 @@ cudaError_t launch_step_tile(const StepParams& p, int mode, bool vec, int mix, c
         static unsigned long long limit_set = 0;                                                 \
         cudaError_t e = ensure_smem_limit(step_tile_kernel<M, V>, kTileSmemBytes, limit_set);    \
         if (e != cudaSuccess) return e;                                                          \
-        step_tile_kernel<M, V><<<grd, blk, smem, s>>>(p, mix, tile_groups, log2n);               \
+        step_tile_kernel<M, V><<<grd, blk, smem, s>>>(p, mix, tile_groups, log2n, sw);           \
     } while (0)
     if (mode == GRAD_PARTIALS) {
         GPGA_TILE(GRAD_PARTIALS, true);   // logistic objective: d % 4 == 0 is required upstream
@@ -293,7 +309,7 @@ cudaError_t launch_step_tile(const StepParams& p, int mode, bool vec, int mix, c
 }
 
 cudaError_t launch_run_tile(const StepParams& p, int mode, bool vec, int topology, long long H, int steps,
-                            cudaStream_t s)
+                            const SparseW& sw, cudaStream_t s)
 {
     if (!run_tile_supports(p.n) || (mode != GRAD_QUAD && mode != GRAD_QUAD_NOISE))
         return cudaErrorInvalidConfiguration;   // callers check
@@ -310,7 +326,7 @@ cudaError_t launch_run_tile(const StepParams& p, int mode, bool vec, int topolog
         static unsigned long long limit_set = 0;                                                 \
         cudaError_t e = ensure_smem_limit(run_tile_kernel<M, V>, kTileSmemBytes, limit_set);     \
         if (e != cudaSuccess) return e;                                                          \
-        run_tile_kernel<M, V><<<grd, blk, smem, s>>>(p, topology, H, phase0, hop0, steps, tile_groups, log2n); \
+        run_tile_kernel<M, V><<<grd, blk, smem, s>>>(p, topology, H, phase0, hop0, steps, tile_groups, log2n, sw); \
     } while (0)
     if (vec) {
         if (mode == GRAD_QUAD) GPGA_RUN_TILE(GRAD_QUAD, true);

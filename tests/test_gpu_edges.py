@@ -220,3 +220,39 @@ def test_convex_experiment_driver_small():
         assert len(loss) == 7 and loss[-1] < loss[0]
     assert np.all(out["parallel_sgd"][1] == 0.0)
     assert out["gossip_pga"][1][1:].mean() < out["gossip_sgd"][1][1:].mean()
+
+
+@pytest.mark.parametrize("n,d", [(9, 40), (30, 1030), (16, 20_004)])
+def test_general_sparse_weight_matrix(n, d):
+    """Topology SPARSE: Metropolis weights of a random connected graph, given in CSR form."""
+    torch = _torch()
+    rng = np.random.default_rng(n)
+    adj = np.triu(rng.uniform(size=(n, n)) < 0.3, 1)
+    adj[np.arange(n - 1), np.arange(1, n)] = True
+    adj = adj | adj.T
+    W = o.metropolis_w(adj)
+    row_ptr, col, val = [0], [], []
+    for i in range(n):
+        nz = np.nonzero(W[i])[0]
+        col += list(nz)
+        val += list(W[i, nz])
+        row_ptr.append(len(col))
+    X0, B = quadratic_inputs(n, d, 77, x0="per_node")
+    for H, K in ((0, 1), (3, 7)):
+        g = pkg.Gpga(n, d, pkg.GPGA_TOPO_SPARSE, H, 0.2, 5)
+        g.set_objective(pkg.GPGA_OBJ_QUADRATIC, sigma=0.3)
+        xa = torch.from_numpy(X0).cuda()
+        g.bind(xa, torch.empty_like(xa), torch.from_numpy(B).cuda())
+        with pytest.raises(pkg.GpgaError):
+            g.step(0)                                   # no weight matrix yet
+        g.set_weight_matrix(torch.tensor(row_ptr, dtype=torch.int32, device="cuda"),
+                            torch.tensor(col, dtype=torch.int32, device="cuda"),
+                            torch.tensor(val, dtype=torch.float32, device="cuda"))
+        p = o.Problem(o.TOPO_SPARSE, H, 0.2, 5, sigma=0.3, data=B, W=W)
+        if K == 1:
+            g.step(0)
+        else:
+            g.run(K)
+        ok, worst = close(g.get_x().cpu().numpy(), o.run(p, X0, 0, K), TOL_STEP if K == 1 else TOL_RUN)
+        assert ok, (H, K, worst)
+        g.close()

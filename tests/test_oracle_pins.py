@@ -441,3 +441,26 @@ def test_vector_box_muller_and_mean_loss_helpers():
     X = rng.standard_normal((3, 4))
     B = rng.standard_normal((3, 4))
     assert abs(o.quadratic_mean_loss(X, B) - 0.5 * np.linalg.norm(X - B, "fro") ** 2 / 3) < 1e-13
+
+
+def test_metropolis_weights_are_doubly_stochastic_and_mix_like_dense_w():
+    rng = np.random.default_rng(12)
+    n = 9
+    adj = rng.uniform(size=(n, n)) < 0.35
+    adj = np.triu(adj, 1)
+    adj = adj | adj.T
+    adj[np.arange(n), (np.arange(n) + 1) % n] = True          # keep it connected: add a ring
+    adj = adj | adj.T
+    W = o.metropolis_w(adj)
+    assert (W >= 0).all() and np.allclose(W, W.T)
+    assert np.allclose(W.sum(0), 1, atol=1e-15) and np.allclose(W.sum(1), 1, atol=1e-15)
+    assert np.array_equal(W > 0, adj | np.eye(n, dtype=bool))   # w_ij > 0 exactly on neighbours and i = j
+    assert np.linalg.norm(W - np.full((n, n), 1.0 / n), 2) < 1.0  # beta < 1: connected graph (Assumption 3)
+    B = rng.standard_normal((n, 6))
+    X = rng.standard_normal((n, 6))
+    p = o.Problem(o.TOPO_SPARSE, 3, 0.2, 4, sigma=0.3, data=B, W=W)
+    for k in range(5):
+        a, b = o.step_f64(p, X, k, dense=False), o.step_f64(p, X, k, dense=True)
+        assert np.allclose(a, b, rtol=1e-12, atol=1e-13)
+        assert np.allclose(a.mean(0), o.quadratic_half_step(X, B, 0.2, 0.3, 4, k).mean(0), atol=1e-13)
+        X = a
