@@ -25,3 +25,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_libraries():
+    """Make sure the in-tree CUDA library and the C oracle exist and are current before any test
+    loads them (both builds are no-ops when nothing changed)."""
+    from paper_2105_09080_b200 import build
+    from oracle import gpga_oracle
+    build.build_library()
+    gpga_oracle.build()
