@@ -438,9 +438,20 @@ def run_logistic(args, w, name):
 
 def run_e2e(torch, g, w, dist):
     n, d, K = w["n"], w["d"], w["K"]
-    x0 = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
-    bh = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
-    out = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+    problem = None
+    try:
+        x0 = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+        bh = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+        out = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+    except Exception as exc:        # not enough pinnable host memory on this rank
+        problem = repr(exc)[:200]
+    if dist is not None:            # every rank must take the same branch before the next collective
+        ok = torch.tensor([0 if problem else 1], device="cuda")
+        dist.all_reduce(ok, op=dist.ReduceOp.MIN)
+        if int(ok.item()) == 0 and not problem:
+            problem = "another rank could not pin its host buffers"
+    if problem:
+        return {"value": None, "unit": UNIT, "error": problem}
     # host copies of the seeded inputs (downloaded once, outside the timed region)
     g.init_from_seed({"zero": 0, "shared": 1}[w["x0"]], w["x0_std"], w["b_shift"])
     x0.copy_(g.x_bufs[0][:, :d])
