@@ -217,6 +217,15 @@ int32_t gpga_run_adaptive(gpga_t* ctx, int64_t K, int64_t H_init, int64_t warmup
                           void* stream, int64_t* periods_host, int64_t max_periods,
                           int64_t* num_periods_host);
 
+/*
+ * Self-test of the in-kernel wait limit (no counterpart in the paper): launches one block that
+ * waits, a bounded number of polls, on a barrier that nothing will ever complete.  The wait must
+ * give up and raise the handle's device error word, so that the NEXT synchronising call
+ * (gpga_consensus_distance, gpga_mean_loss, gpga_global_loss) returns GPGA_ERR_TIMEOUT, after
+ * which the handle stays in that state.  Nothing faults, traps or hangs.  For tests only.
+ */
+int32_t gpga_selftest_bounded_wait(gpga_t* ctx, void* stream);
+
 /* Accessors.  gpga_get_x returns the device pointer of the current state buffer. */
 int32_t gpga_get_x(const gpga_t* ctx, void** x_cur);
 int32_t gpga_get_k(const gpga_t* ctx, int64_t* k);

@@ -54,6 +54,7 @@ SIGNATURES = {
     "gpga_consensus_distance": (_i32, [_P, _P, C.POINTER(C.c_double)]),
     "gpga_mean_loss": (_i32, [_P, _P, C.POINTER(C.c_double)]),
     "gpga_global_loss": (_i32, [_P, _P, C.POINTER(C.c_double)]),
+    "gpga_selftest_bounded_wait": (_i32, [_P, _P]),
     "gpga_run_adaptive": (_i32, [_P, _i64, _i64, _i64, _P, C.POINTER(_i64), _i64, C.POINTER(_i64)]),
     "gpga_get_x": (_i32, [_P, C.POINTER(_P)]),
     "gpga_get_k": (_i32, [_P, C.POINTER(_i64)]),
@@ -218,6 +219,9 @@ class Gpga:
         out = C.c_double()
         self._check(lib().gpga_global_loss(self._h, _stream_ptr(stream), C.byref(out)))
         return out.value
+
+    def selftest_bounded_wait(self, stream=None):
+        self._check(lib().gpga_selftest_bounded_wait(self._h, _stream_ptr(stream)))
 
     def run_adaptive(self, K, H_init, warmup_iters, stream=None, max_periods=4096):
         periods = (_i64 * max_periods)()

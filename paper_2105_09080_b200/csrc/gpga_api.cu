@@ -513,6 +513,21 @@ int32_t gpga_global_loss(gpga_t* c, void* stream, double* out_host)
     return read_double(c, result, s, out_host);
 }
 
+int32_t gpga_selftest_bounded_wait(gpga_t* c, void* stream)
+{
+    int32_t st = check_ready(c);
+    if (st) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int* flag = reinterpret_cast<int*>(c->scratch + scratch_layout(c).result_off + 8);
+    cudaError_t e = cudaMemsetAsync(flag, 0, sizeof(int), s);
+    if (e != cudaSuccess) return cuda_fail(c, e, "error word clear");
+    c->flag_cleared = true;
+    e = launch_bounded_wait_selftest(flag, s);
+    c->launches += 1;
+    if (e != cudaSuccess) return cuda_fail(c, e, "self-test launch");
+    return GPGA_OK;
+}
+
 int32_t gpga_run_adaptive(gpga_t* c, int64_t K, int64_t H_init, int64_t warmup_iters, void* stream,
                           int64_t* periods_host, int64_t max_periods, int64_t* num_periods_host)
 {

@@ -281,6 +281,26 @@ __global__ void mean_kernel(const double* v, int count, double* result)
     if (threadIdx.x == 0) *result = s / (double)count;
 }
 
+// A wait that cannot succeed: the barrier expects one arrival that never comes.  Exercises the
+// give-up path of mbar_wait_bounded and the error word without any copy in flight.
+__global__ void bounded_wait_selftest_kernel(int* error_flag, uint32_t tries)
+{
+    __shared__ __align__(8) uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mbar_init_fence();
+    }
+    __syncthreads();
+    const bool ok = mbar_wait_bounded(&bar, 0u, tries);
+    if (!ok && threadIdx.x == 0) atomicExch(error_flag, 1);
+}
+
+cudaError_t launch_bounded_wait_selftest(int* error_flag, cudaStream_t s)
+{
+    bounded_wait_selftest_kernel<<<1, 32, 0, s>>>(error_flag, 2000u);
+    return cudaGetLastError();
+}
+
 int logreg_chunks(long long batch) { return (int)((batch + kChunkRows - 1) / kChunkRows); }
 
 cudaError_t launch_logreg_partial(const LogregParams& p, cudaStream_t s)

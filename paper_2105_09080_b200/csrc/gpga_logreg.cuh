@@ -24,6 +24,8 @@ struct LogregParams {
 };
 
 int logreg_chunks(long long batch);
+// One block waits (bounded) on a barrier nobody completes and must set *error_flag.
+cudaError_t launch_bounded_wait_selftest(int* error_flag, cudaStream_t s);
 // One launch: chunk partials only (the consumer adds them in index order).
 cudaError_t launch_logreg_partial(const LogregParams& p, cudaStream_t s);
 // Two launches: chunk partials, then the fixed-order sum into G (adds l2 x).

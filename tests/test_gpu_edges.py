@@ -256,3 +256,25 @@ def test_general_sparse_weight_matrix(n, d):
         ok, worst = close(g.get_x().cpu().numpy(), o.run(p, X0, 0, K), TOL_STEP if K == 1 else TOL_RUN)
         assert ok, (H, K, worst)
         g.close()
+
+
+def test_bounded_wait_gives_up_and_reports_timeout():
+    """A wait inside a kernel that can never be satisfied ends by itself and surfaces as
+    GPGA_ERR_TIMEOUT at the next synchronising call; the GPU context stays usable."""
+    n, d = 4, 64
+    X0, B = quadratic_inputs(n, d, 1)
+    g, _ = make_quadratic(n, d, "ring", 0, 0.1, 1, 0.0, X0, B)
+    assert g.consensus_distance() == 0.0
+    g.selftest_bounded_wait()
+    with pytest.raises(pkg.GpgaError) as err:
+        g.consensus_distance()
+    assert err.value.status == pkg.GPGA_ERR_TIMEOUT
+    with pytest.raises(pkg.GpgaError) as err:       # sticky
+        g.step(0)
+    assert err.value.status == pkg.GPGA_ERR_TIMEOUT
+    g.close()
+    # another handle on the same device works as before
+    g2, p = make_quadratic(n, d, "ring", 0, 0.1, 1, 0.2, X0, B)
+    g2.step(0)
+    ok, worst = close(g2.get_x().cpu().numpy(), o.step(p, X0, 0), TOL_STEP)
+    assert ok, worst
