@@ -47,11 +47,11 @@ def build(force: bool = False) -> Path:
 _lib = None
 
 
-def lib():
-    global _lib
-    if _lib is None:
-        build()
-        L = C.CDLL(str(_LIB))
+def load(path):
+    """Load an oracle shared library (the built one, or a deliberately broken copy that a test
+    compiled to see whether the pins notice) and declare its signatures."""
+    if True:
+        L = C.CDLL(str(path))
         i64, i32, u32, u64, f64 = C.c_int64, C.c_int32, C.c_uint32, C.c_uint64, C.c_double
         P = C.c_void_p
         L.gpga_oracle_philox4x32_10.argtypes = [P, P, P]
@@ -99,7 +99,14 @@ def lib():
         L.gpga_oracle_box_muller_many.restype = None
         L.gpga_oracle_quadratic_mean_loss.argtypes = [i64, i64, P, P]
         L.gpga_oracle_quadratic_mean_loss.restype = f64
-        _lib = L
+    return L
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = load(_LIB)
     return _lib
 
 

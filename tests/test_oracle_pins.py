@@ -464,3 +464,12 @@ def test_metropolis_weights_are_doubly_stochastic_and_mix_like_dense_w():
         assert np.allclose(a, b, rtol=1e-12, atol=1e-13)
         assert np.allclose(a.mean(0), o.quadratic_half_step(X, B, 0.2, 0.3, 4, k).mean(0), atol=1e-13)
         X = a
+
+
+def test_counter_layout_of_the_noise_generator():
+    # the documented keying: counter = (column group q, node i, iteration k, stream id),
+    # key = (seed low word, seed high word); (z0,z1) from words 0,1 and (z2,z3) from words 2,3
+    seed, stream, k, i, q = (0x89ABCDEF << 32) | 0x01234567, 3, 1000, 17, 123456
+    w = o.philox4x32_10([q, i, k, stream], [0x01234567, 0x89ABCDEF])
+    want = np.concatenate([o.box_muller(int(w[0]), int(w[1])), o.box_muller(int(w[2]), int(w[3]))])
+    assert np.array_equal(o.normal4(seed, stream, k, i, q), want)
