@@ -178,7 +178,8 @@ def run_reference(args, w, name):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    per_step_s = 1.0
+    # each step is a bounded sample sized so that warm-up + timed steps take about a minute in all
+    per_step_s = min(1.0, 60.0 / max(1, args.steps + args.warmup))
     t = oracle_sample(w, 4096, 1)
     cols = int(min(w["d"], max(4096, per_step_s * 4096 / t)))
     cols -= cols % 4
