@@ -329,7 +329,7 @@ int consensus_blocks(long long Q)
 }
 
 template <bool VEC>
-__global__ void __launch_bounds__(kReduceBlock) consensus_kernel(const float* __restrict__ x,
+__global__ void __launch_bounds__(kReduceBlock, 3) consensus_kernel(const float* __restrict__ x,
                                                                  long long n, long long d,
                                                                  long long ld, long long Q,
                                                                  double* __restrict__ partials)
@@ -387,7 +387,7 @@ cudaError_t launch_consensus(const float* x, long long n, long long d, long long
 
 // (1/n) sum_i 1/2 ||x_i - b_i||^2 over all elements.
 template <bool VEC>
-__global__ void __launch_bounds__(kReduceBlock) quadratic_loss_kernel(const float* __restrict__ x,
+__global__ void __launch_bounds__(kReduceBlock, 3) quadratic_loss_kernel(const float* __restrict__ x,
                                                                       const float* __restrict__ b,
                                                                       long long n, long long d,
                                                                       long long ld, long long Q,
