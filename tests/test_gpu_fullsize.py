@@ -93,7 +93,7 @@ def test_config_3_resnet50_sized():
     xb = torch.empty_like(xa)
     b = torch.empty_like(xa)
     scratch = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
-    offs = _blocks(d, 12, np.random.default_rng(3))
+    offs = _blocks(d, 64, np.random.default_rng(3))
     assert d % 128 == 40 and offs[-1] + BLOCK == d
     for topo in ("ring", "exp"):
         for H in (4, 16, 0):
@@ -119,7 +119,7 @@ def test_config_4_bert_large_sized():
     xb = torch.empty_like(xa)
     b = torch.empty_like(xa)
     scratch = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
-    offs = _blocks(d, 12, np.random.default_rng(4))
+    offs = _blocks(d, 48, np.random.default_rng(4))
     _run_case((xa, xb, b, scratch), n, d, "exp", H, gamma, sigma, K, pkg.GPGA_X0_ZERO, 1.0, 0.0,
               offs, [0, 1, 2, 3])
     del xa, xb, b
