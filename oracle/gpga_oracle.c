@@ -40,7 +40,12 @@
  * gap against the beta values the paper prints in Section 5.1; closed forms
  * of the mean recursion; eigenvector contraction; finite-time consensus of
  * the one-peer exponential graph; dense-W agreement; finite differences for
- * the logistic gradient; brute force on tiny inputs.
+ * the logistic gradient; brute force on tiny inputs.  tests/test_oracle_mutations.py
+ * plants single mistakes in a copy of this file and requires a pin to fail for each.
+ *
+ * Parity unpinned: whole-run trajectories of the benchmark configurations (the paper
+ * prints no loss or consensus-distance values for them); they are covered only by
+ * the invariants above and by the comparison of the two implementations.
  */
 #include <math.h>
 #include <stdint.h>
