@@ -224,6 +224,128 @@ __global__ void __launch_bounds__(kLrBlock) logreg_partial_tma_kernel(const Logr
     }
 }
 
+// Narrow rows (d <= kRegMaxD): the same staging by bulk asynchronous copies, but each warp
+// takes one staged row through registers once -- the margin a^T x against x held in
+// registers, then s * a added to per-lane accumulators -- so a row is read from shared
+// memory once instead of twice and x not at all.  The per-warp accumulators are added in
+// warp order at the end (fixed order: the result does not depend on scheduling).
+constexpr int kRegMaxD = 1024;
+constexpr int kRegGroups = kRegMaxD / 4 / 32;   // float4 per lane
+
+__global__ void __launch_bounds__(kLrBlock, 2) logreg_partial_tma_reg_kernel(const LogregParams p, int tile_rows)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    float* tiles = reinterpret_cast<float*>(smem_raw);         // 2 x tile_rows x d, later nwarps x d
+    __shared__ uint32_t rows[kChunkRows];
+    __shared__ float ys[kChunkRows];
+    __shared__ __align__(8) uint64_t bar[2];
+    const int i = blockIdx.x, c = blockIdx.y;
+    const int t0 = c * kChunkRows;
+    const int nrows = min(kChunkRows, (int)p.batch - t0);
+    const int ntiles = (nrows + tile_rows - 1) / tile_rows;
+    const float* A = p.A + (long long)i * p.m * p.d;
+    const float* y = p.y + (long long)i * p.m;
+    const float4* x4 = reinterpret_cast<const float4*>(p.x + (long long)i * p.ldx);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int d4 = (int)(p.d >> 2);
+    const uint32_t row_bytes = (uint32_t)p.d * 4u;
+    if (threadIdx.x < nrows)
+        rows[threadIdx.x] = batch_row((uint32_t)(t0 + threadIdx.x), (uint32_t)i, p.k, (uint32_t)p.m, p.keys);
+    if (threadIdx.x == 0) {
+        mbar_init(&bar[0], 1);
+        mbar_init(&bar[1], 1);
+        mbar_init_fence();
+    }
+    __syncthreads();
+    auto issue = [&](int s) {
+        const int r0 = s * tile_rows;
+        const int rr = min(tile_rows, nrows - r0);
+        float* dst = tiles + (size_t)(s & 1) * tile_rows * p.d;
+        if (lane == 0) mbar_arrive_expect_tx(&bar[s & 1], (uint32_t)rr * row_bytes);
+        __syncwarp();
+        for (int t = lane; t < rr; t += 32)
+            bulk_copy_g2s(dst + (size_t)t * p.d, A + (long long)rows[r0 + t] * p.d, row_bytes, &bar[s & 1]);
+    };
+    if (warp == 0) {
+        issue(0);
+        if (ntiles > 1) issue(1);
+    }
+    if (threadIdx.x < nrows) ys[threadIdx.x] = y[rows[threadIdx.x]];
+    float4 xr[kRegGroups], acc[kRegGroups];
+#pragma unroll
+    for (int j = 0; j < kRegGroups; ++j) {
+        const int g = lane + 32 * j;
+        xr[j] = g < d4 ? x4[g] : make_float4(0.f, 0.f, 0.f, 0.f);
+        acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    __syncthreads();
+    uint32_t parity0 = 0u, parity1 = 0u;
+    bool failed = false;
+    for (int s = 0; s < ntiles; ++s) {
+        const int buf = s & 1;
+        const int r0 = s * tile_rows;
+        const int rr = min(tile_rows, nrows - r0);
+        const float* tile = tiles + (size_t)buf * tile_rows * p.d;
+        const uint32_t par = buf ? parity1 : parity0;
+        const bool ok = mbar_wait_bounded(&bar[buf], par, kTmaMaxTries);
+        if (__syncthreads_or(!ok)) {
+            if (!ok) mbar_wait_bounded(&bar[buf], par, kTmaMaxTries);
+            if (s + 1 < ntiles) mbar_wait_bounded(&bar[buf ^ 1], buf ? parity0 : parity1, kTmaMaxTries);
+            if (threadIdx.x == 0 && p.error_flag) atomicExch(p.error_flag, 1);
+            failed = true;
+            break;
+        }
+        if (buf) parity1 ^= 1u; else parity0 ^= 1u;
+        for (int t = warp; t < rr; t += nwarps) {
+            const float4* a4 = reinterpret_cast<const float4*>(tile + (size_t)t * p.d);
+            float4 a[kRegGroups];
+            float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
+#pragma unroll
+            for (int j = 0; j < kRegGroups; ++j) {
+                const int g = lane + 32 * j;
+                a[j] = g < d4 ? a4[g] : make_float4(0.f, 0.f, 0.f, 0.f);
+                z0 = fmaf(a[j].x, xr[j].x, z0);
+                z1 = fmaf(a[j].y, xr[j].y, z1);
+                z2 = fmaf(a[j].z, xr[j].z, z2);
+                z3 = fmaf(a[j].w, xr[j].w, z3);
+            }
+            const float z = warp_sum_f((z0 + z1) + (z2 + z3));   // every lane holds the sum
+            const float yr = ys[r0 + t];
+            const float sc = -yr / (1.0f + expf(yr * z));
+#pragma unroll
+            for (int j = 0; j < kRegGroups; ++j) {
+                acc[j].x = fmaf(sc, a[j].x, acc[j].x);
+                acc[j].y = fmaf(sc, a[j].y, acc[j].y);
+                acc[j].z = fmaf(sc, a[j].z, acc[j].z);
+                acc[j].w = fmaf(sc, a[j].w, acc[j].w);
+            }
+        }
+        __syncthreads();   // everyone is done with this buffer before new copies overwrite it
+        if (warp == 0 && s + 2 < ntiles) issue(s + 2);
+    }
+    if (failed) return;
+    // the tiles are free now: park the per-warp sums there and add them in warp order
+    float4* red = reinterpret_cast<float4*>(tiles);            // [nwarps][d4]
+#pragma unroll
+    for (int j = 0; j < kRegGroups; ++j) {
+        const int g = lane + 32 * j;
+        if (g < d4) red[warp * d4 + g] = acc[j];
+    }
+    __syncthreads();
+    float4* out4 = reinterpret_cast<float4*>(p.partial + ((long long)c * p.n + i) * p.d);
+    for (int g = threadIdx.x; g < d4; g += blockDim.x) {
+        float4 sum = red[g];
+        for (int w = 1; w < nwarps; ++w) {
+            const float4 v = red[w * d4 + g];
+            sum.x += v.x;
+            sum.y += v.y;
+            sum.z += v.z;
+            sum.w += v.w;
+        }
+        out4[g] = sum;
+    }
+}
+
 // G[i][:] = (1/B) sum_c partial[c][i][:] + l2 x_i, chunks added in index order.
 __global__ void __launch_bounds__(kLrBlock) logreg_reduce_kernel(const LogregParams p, int chunks)
 {
@@ -306,6 +428,18 @@ int logreg_chunks(long long batch) { return (int)((batch + kChunkRows - 1) / kCh
 cudaError_t launch_logreg_partial(const LogregParams& p, cudaStream_t s)
 {
     const int chunks = logreg_chunks(p.batch);
+    if (p.d <= kRegMaxD) {
+        int tile_rows = kTmaTileBytes / 2 / (int)(p.d * 4);   // two tiles share the budget
+        if (tile_rows > kChunkRows) tile_rows = kChunkRows;
+        size_t smem_reg = 2 * (size_t)tile_rows * p.d * sizeof(float);
+        const size_t red_bytes = (size_t)(kLrBlock / 32) * p.d * sizeof(float);   // the final per-warp sums
+        if (smem_reg < red_bytes) smem_reg = red_bytes;
+        static unsigned long long reg_limit_set = 0;
+        cudaError_t e = ensure_smem_limit(logreg_partial_tma_reg_kernel, 100 * 1024, reg_limit_set);
+        if (e != cudaSuccess) return e;
+        logreg_partial_tma_reg_kernel<<<dim3((unsigned)p.n, (unsigned)chunks), kLrBlock, smem_reg, s>>>(p, tile_rows);
+        return cudaGetLastError();
+    }
     if (p.d <= kTmaMaxD) {
         int tile_rows = kTmaTileBytes / 2 / (int)(p.d * 4);   // two tiles share the budget
         if (tile_rows > kChunkRows) tile_rows = kChunkRows;
