@@ -169,7 +169,11 @@ int32_t gpga_step(gpga_t* ctx, int64_t k, void* stream);
 /* K iterations k0 .. k0+K-1 starting at the internal counter k0 (Algorithm 1's loop).  A quadratic-
  * objective state of at most 64 MB (X, X+ and b together) is advanced many iterations per launch with
  * its column strips resident in shared memory -- columns evolve independently -- with results
- * bit-identical to K calls of gpga_step; larger states take one launch per iteration. */
+ * bit-identical to K calls of gpga_step; larger states take one launch per iteration.
+ * Logistic objective: within one call the launches of consecutive iterations overlap (the rows of A and
+ * the labels of iteration k+1 are fetched while iteration k finishes); A and the labels are inputs that
+ * no kernel of the library writes, and the caller must not write them while the call's work is in
+ * flight on the stream.  Results are the same as K calls of gpga_step. */
 int32_t gpga_run(gpga_t* ctx, int64_t K, void* stream);
 
 /*

@@ -117,7 +117,7 @@ LogregParams logreg_params(const gpga_ctx* c, int64_t k)
 }
 
 // One iteration; `global` chosen by the caller (fixed or adaptive period).
-int32_t do_step(gpga_ctx* c, int64_t k, bool global, cudaStream_t s)
+int32_t do_step(gpga_ctx* c, int64_t k, bool global, cudaStream_t s, bool after_own_step = false)
 {
     if (k < 0 || k >= (int64_t(1) << 32)) return fail(c, GPGA_ERR_INVALID_ARG, "k must be in [0, 2^32)");
     StepParams p;
@@ -140,7 +140,8 @@ int32_t do_step(gpga_ctx* c, int64_t k, bool global, cudaStream_t s)
     const bool tile_topology = c->topology != GPGA_TOPO_RING && c->topology != GPGA_TOPO_EXP;
     cudaError_t e;
     if (c->objective == GPGA_OBJ_LOGISTIC) {
-        const LogregParams lp = logreg_params(c, k);
+        LogregParams lp = logreg_params(c, k);
+        lp.after_own_step = after_own_step && narrow;   // the narrow path's step kernel releases its successor early
         if (!c->flag_cleared) {   // kernels with bounded waits report through this word
             e = cudaMemsetAsync(lp.error_flag, 0, sizeof(int), s);
             if (e != cudaSuccess) return cuda_fail(c, e, "error word clear");
@@ -204,7 +205,8 @@ int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)
                        12 * c->n * c->ld <= kFusedStateBytes;
     if (!fused) {
         for (int64_t k = c->k; k < k_end; ++k) {
-            const int32_t st = do_step(c, k, is_global_step(k, c->H), s);
+            // from the second iteration on, the launch before the gradient kernel is our own step kernel
+            const int32_t st = do_step(c, k, is_global_step(k, c->H), s, k > k_end - K);
             if (st) return st;
         }
         return GPGA_OK;

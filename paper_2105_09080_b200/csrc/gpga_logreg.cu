@@ -224,53 +224,61 @@ __global__ void __launch_bounds__(kLrBlock) logreg_partial_tma_kernel(const Logr
     }
 }
 
-// Narrow rows (d <= kRegMaxD): the same staging by bulk asynchronous copies, but each warp
-// takes one staged row through registers once -- the margin a^T x against x held in
-// registers, then s * a added to per-lane accumulators -- so a row is read from shared
-// memory once instead of twice and x not at all.  The per-warp accumulators are added in
-// warp order at the end (fixed order: the result does not depend on scheduling).
+// Narrow rows (d <= kRegMaxD): the same staging by bulk asynchronous copies, but every warp
+// runs its own pipeline -- it draws the indices of its rows (rows warp, warp + 8, ... of the
+// chunk), copies each into one of its `slots` row buffers, and takes a staged row through
+// registers once: the margin a^T x against x held in registers, then s * a added to per-lane
+// accumulators.  A row is read from shared memory once instead of twice, x not at all, and
+// no block-wide barrier stands between rows.  The per-warp accumulators are added in warp
+// order at the end (fixed order: the result does not depend on scheduling).
 constexpr int kRegMaxD = 1024;
 constexpr int kRegGroups = kRegMaxD / 4 / 32;   // float4 per lane
+constexpr int kRegWarps = kLrBlock / 32;
+constexpr int kRegMaxSlots = 4;                 // kChunkRows / kRegWarps rows per warp at most
+constexpr int kRegSmemBytes = 96 * 1024;
+static_assert(kRegWarps * kRegMaxSlots >= kChunkRows, "a warp must be able to hold all its rows");
 
-__global__ void __launch_bounds__(kLrBlock, 2) logreg_partial_tma_reg_kernel(const LogregParams p, int tile_rows)
+__global__ void __launch_bounds__(kLrBlock, 2) logreg_partial_tma_reg_kernel(const LogregParams p, int slots)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    float* tiles = reinterpret_cast<float*>(smem_raw);         // 2 x tile_rows x d, later nwarps x d
-    __shared__ uint32_t rows[kChunkRows];
-    __shared__ float ys[kChunkRows];
-    __shared__ __align__(8) uint64_t bar[2];
+    __shared__ __align__(8) uint64_t bars[kRegWarps * kRegMaxSlots];
     const int i = blockIdx.x, c = blockIdx.y;
     const int t0 = c * kChunkRows;
     const int nrows = min(kChunkRows, (int)p.batch - t0);
-    const int ntiles = (nrows + tile_rows - 1) / tile_rows;
     const float* A = p.A + (long long)i * p.m * p.d;
     const float* y = p.y + (long long)i * p.m;
     const float4* x4 = reinterpret_cast<const float4*>(p.x + (long long)i * p.ldx);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int d4 = (int)(p.d >> 2);
     const uint32_t row_bytes = (uint32_t)p.d * 4u;
-    if (threadIdx.x < nrows)
-        rows[threadIdx.x] = batch_row((uint32_t)(t0 + threadIdx.x), (uint32_t)i, p.k, (uint32_t)p.m, p.keys);
-    if (threadIdx.x == 0) {
-        mbar_init(&bar[0], 1);
-        mbar_init(&bar[1], 1);
+    float* mine = reinterpret_cast<float*>(smem_raw) + (size_t)warp * slots * p.d;   // this warp's row buffers
+    uint64_t* bar = bars + warp * kRegMaxSlots;
+    const int my_rows = warp < nrows ? (nrows - warp + kRegWarps - 1) / kRegWarps : 0;
+    // lane r holds the index and the label of this warp's r-th row
+    uint32_t my_idx = 0u;
+    float my_y = 0.f;
+    if (lane < my_rows) {
+        my_idx = batch_row((uint32_t)(t0 + warp + lane * kRegWarps), (uint32_t)i, p.k, (uint32_t)p.m, p.keys);
+        my_y = y[my_idx];
+    }
+    if (lane == 0) {
+        for (int s = 0; s < slots; ++s) mbar_init(&bar[s], 1);
         mbar_init_fence();
     }
-    __syncthreads();
-    auto issue = [&](int s) {
-        const int r0 = s * tile_rows;
-        const int rr = min(tile_rows, nrows - r0);
-        float* dst = tiles + (size_t)(s & 1) * tile_rows * p.d;
-        if (lane == 0) mbar_arrive_expect_tx(&bar[s & 1], (uint32_t)rr * row_bytes);
-        __syncwarp();
-        for (int t = lane; t < rr; t += 32)
-            bulk_copy_g2s(dst + (size_t)t * p.d, A + (long long)rows[r0 + t] * p.d, row_bytes, &bar[s & 1]);
+    __syncwarp();
+    auto issue = [&](int r) {   // whole warp calls; lane 0 starts the copy of row r into slot r % slots
+        const uint32_t idx = __shfl_sync(0xFFFFFFFFu, my_idx, r);
+        if (lane == 0) {
+            const int s = r % slots;
+            mbar_arrive_expect_tx(&bar[s], row_bytes);
+            bulk_copy_g2s(mine + (size_t)s * p.d, A + (long long)idx * p.d, row_bytes, &bar[s]);
+        }
     };
-    if (warp == 0) {
-        issue(0);
-        if (ntiles > 1) issue(1);
-    }
-    if (threadIdx.x < nrows) ys[threadIdx.x] = y[rows[threadIdx.x]];
+    const int first = min(slots, my_rows);
+    for (int r = 0; r < first; ++r) issue(r);
+    // everything above reads only A, y and the iteration index; x is the previous step's output and
+    // the partial sums may still be read by it
+    grid_dependency_wait();
     float4 xr[kRegGroups], acc[kRegGroups];
 #pragma unroll
     for (int j = 0; j < kRegGroups; ++j) {
@@ -278,65 +286,61 @@ __global__ void __launch_bounds__(kLrBlock, 2) logreg_partial_tma_reg_kernel(con
         xr[j] = g < d4 ? x4[g] : make_float4(0.f, 0.f, 0.f, 0.f);
         acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    __syncthreads();
-    uint32_t parity0 = 0u, parity1 = 0u;
     bool failed = false;
-    for (int s = 0; s < ntiles; ++s) {
-        const int buf = s & 1;
-        const int r0 = s * tile_rows;
-        const int rr = min(tile_rows, nrows - r0);
-        const float* tile = tiles + (size_t)buf * tile_rows * p.d;
-        const uint32_t par = buf ? parity1 : parity0;
-        const bool ok = mbar_wait_bounded(&bar[buf], par, kTmaMaxTries);
-        if (__syncthreads_or(!ok)) {
-            if (!ok) mbar_wait_bounded(&bar[buf], par, kTmaMaxTries);
-            if (s + 1 < ntiles) mbar_wait_bounded(&bar[buf ^ 1], buf ? parity0 : parity1, kTmaMaxTries);
-            if (threadIdx.x == 0 && p.error_flag) atomicExch(p.error_flag, 1);
+    for (int r = 0; r < my_rows; ++r) {
+        const int s = r % slots;
+        const uint32_t parity = (uint32_t)(r / slots) & 1u;
+        if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&bar[s], parity, kTmaMaxTries))) {   // warp-uniform
+            // give the copies still in flight (this one and the later slots') one more bounded chance to land
+            for (int q = r; q < min(my_rows, r + slots); ++q)
+                mbar_wait_bounded(&bar[q % slots], (uint32_t)(q / slots) & 1u, kTmaMaxTries);
             failed = true;
             break;
         }
-        if (buf) parity1 ^= 1u; else parity0 ^= 1u;
-        for (int t = warp; t < rr; t += nwarps) {
-            const float4* a4 = reinterpret_cast<const float4*>(tile + (size_t)t * p.d);
-            float4 a[kRegGroups];
-            float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
+        const float4* a4 = reinterpret_cast<const float4*>(mine + (size_t)s * p.d);
+        float4 a[kRegGroups];
+        float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
 #pragma unroll
-            for (int j = 0; j < kRegGroups; ++j) {
-                const int g = lane + 32 * j;
-                a[j] = g < d4 ? a4[g] : make_float4(0.f, 0.f, 0.f, 0.f);
-                z0 = fmaf(a[j].x, xr[j].x, z0);
-                z1 = fmaf(a[j].y, xr[j].y, z1);
-                z2 = fmaf(a[j].z, xr[j].z, z2);
-                z3 = fmaf(a[j].w, xr[j].w, z3);
-            }
-            const float z = warp_sum_f((z0 + z1) + (z2 + z3));   // every lane holds the sum
-            const float yr = ys[r0 + t];
-            const float sc = -yr / (1.0f + expf(yr * z));
-#pragma unroll
-            for (int j = 0; j < kRegGroups; ++j) {
-                acc[j].x = fmaf(sc, a[j].x, acc[j].x);
-                acc[j].y = fmaf(sc, a[j].y, acc[j].y);
-                acc[j].z = fmaf(sc, a[j].z, acc[j].z);
-                acc[j].w = fmaf(sc, a[j].w, acc[j].w);
-            }
+        for (int j = 0; j < kRegGroups; ++j) {
+            const int g = lane + 32 * j;
+            a[j] = g < d4 ? a4[g] : make_float4(0.f, 0.f, 0.f, 0.f);
+            z0 = fmaf(a[j].x, xr[j].x, z0);
+            z1 = fmaf(a[j].y, xr[j].y, z1);
+            z2 = fmaf(a[j].z, xr[j].z, z2);
+            z3 = fmaf(a[j].w, xr[j].w, z3);
         }
-        __syncthreads();   // everyone is done with this buffer before new copies overwrite it
-        if (warp == 0 && s + 2 < ntiles) issue(s + 2);
+        const float z = warp_sum_f((z0 + z1) + (z2 + z3));   // every lane holds the sum
+        // the sum needed every lane's loads, so the slot is free: refill it before the arithmetic
+        if (r + slots < my_rows) issue(r + slots);
+        const float yr = __shfl_sync(0xFFFFFFFFu, my_y, r);
+        const float sc = -yr / (1.0f + expf(yr * z));
+#pragma unroll
+        for (int j = 0; j < kRegGroups; ++j) {
+            acc[j].x = fmaf(sc, a[j].x, acc[j].x);
+            acc[j].y = fmaf(sc, a[j].y, acc[j].y);
+            acc[j].z = fmaf(sc, a[j].z, acc[j].z);
+            acc[j].w = fmaf(sc, a[j].w, acc[j].w);
+        }
     }
-    if (failed) return;
-    // the tiles are free now: park the per-warp sums there and add them in warp order
-    float4* red = reinterpret_cast<float4*>(tiles);            // [nwarps][d4]
+    grid_launch_dependents();   // the step kernel may take its place; it waits for this grid before reading
+    if (__syncthreads_or(failed)) {
+        if (threadIdx.x == 0 && p.error_flag) atomicExch(p.error_flag, 1);
+        return;
+    }
+    // every copy has landed and been read: park the per-warp sums in each warp's first slot
+    float4* red = reinterpret_cast<float4*>(smem_raw);
+    const int wstride = slots * d4;
 #pragma unroll
     for (int j = 0; j < kRegGroups; ++j) {
         const int g = lane + 32 * j;
-        if (g < d4) red[warp * d4 + g] = acc[j];
+        if (g < d4) red[warp * wstride + g] = acc[j];
     }
     __syncthreads();
     float4* out4 = reinterpret_cast<float4*>(p.partial + ((long long)c * p.n + i) * p.d);
     for (int g = threadIdx.x; g < d4; g += blockDim.x) {
         float4 sum = red[g];
-        for (int w = 1; w < nwarps; ++w) {
-            const float4 v = red[w * d4 + g];
+        for (int w = 1; w < kRegWarps; ++w) {
+            const float4 v = red[w * wstride + g];
             sum.x += v.x;
             sum.y += v.y;
             sum.z += v.z;
@@ -429,16 +433,14 @@ cudaError_t launch_logreg_partial(const LogregParams& p, cudaStream_t s)
 {
     const int chunks = logreg_chunks(p.batch);
     if (p.d <= kRegMaxD) {
-        int tile_rows = kTmaTileBytes / 2 / (int)(p.d * 4);   // two tiles share the budget
-        if (tile_rows > kChunkRows) tile_rows = kChunkRows;
-        size_t smem_reg = 2 * (size_t)tile_rows * p.d * sizeof(float);
-        const size_t red_bytes = (size_t)(kLrBlock / 32) * p.d * sizeof(float);   // the final per-warp sums
-        if (smem_reg < red_bytes) smem_reg = red_bytes;
+        int slots = kRegSmemBytes / (kRegWarps * (int)p.d * 4);   // row buffers per warp
+        if (slots > kRegMaxSlots) slots = kRegMaxSlots;
+        const size_t smem_reg = (size_t)kRegWarps * slots * p.d * sizeof(float);
         static unsigned long long reg_limit_set = 0;
-        cudaError_t e = ensure_smem_limit(logreg_partial_tma_reg_kernel, 100 * 1024, reg_limit_set);
+        cudaError_t e = ensure_smem_limit(logreg_partial_tma_reg_kernel, kRegSmemBytes, reg_limit_set);
         if (e != cudaSuccess) return e;
-        logreg_partial_tma_reg_kernel<<<dim3((unsigned)p.n, (unsigned)chunks), kLrBlock, smem_reg, s>>>(p, tile_rows);
-        return cudaGetLastError();
+        return launch_after_trigger(logreg_partial_tma_reg_kernel, dim3((unsigned)p.n, (unsigned)chunks),
+                                    dim3(kLrBlock), smem_reg, s, p.after_own_step, p, slots);
     }
     if (p.d <= kTmaMaxD) {
         int tile_rows = kTmaTileBytes / 2 / (int)(p.d * 4);   // two tiles share the budget

@@ -21,6 +21,10 @@ struct LogregParams {
     uint32_t k;
     float l2;
     PhiloxKeys keys;
+    // true only when the launch before this one on the stream is this library's own step kernel of
+    // the previous iteration: the gradient kernel may then start drawing and copying rows of A
+    // (which no kernel writes) while that step kernel is still running
+    bool after_own_step = false;
 };
 
 int logreg_chunks(long long batch);

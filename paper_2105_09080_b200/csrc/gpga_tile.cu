@@ -168,6 +168,12 @@ __global__ void __launch_bounds__(kTileBlock) step_tile_kernel(const StepParams 
                                                                int log2n, const SparseW sw)
 {
     extern __shared__ float4 ytile[];   // [n][tile_groups]
+    if (MODE == GRAD_PARTIALS) {
+        // the next iteration's gradient kernel may start staging its rows of A beside this kernel;
+        // this kernel itself may have been started before the gradient kernel it follows was done
+        grid_launch_dependents();
+        grid_dependency_wait();
+    }
     const long long q_first = (long long)blockIdx.x * tile_groups;
     const int n = (int)p.n;
     const int cells = n * tile_groups;
@@ -293,8 +299,14 @@ cudaError_t launch_step_tile_w(const StepParams& p, int mode, bool vec, int mix,
         if (e != cudaSuccess) return e;                                                          \
         step_tile_kernel<M, V><<<grd, blk, smem, s>>>(p, mix, tile_groups, log2n, sw);           \
     } while (0)
-    if (mode == GRAD_PARTIALS) {
-        GPGA_TILE(GRAD_PARTIALS, true);   // logistic objective: d % 4 == 0 is required upstream
+    if (mode == GRAD_PARTIALS) {   // logistic objective: d % 4 == 0 is required upstream
+        // always follows the gradient kernel on the stream and waits for it first thing, so it may
+        // be made resident while that kernel drains
+        static unsigned long long limit_set = 0;
+        cudaError_t e = ensure_smem_limit(step_tile_kernel<GRAD_PARTIALS, true>, kTileSmemBytes, limit_set);
+        if (e != cudaSuccess) return e;
+        return launch_after_trigger(step_tile_kernel<GRAD_PARTIALS, true>, dim3(grd), dim3(blk), smem, s, true, p,
+                                    mix, tile_groups, log2n, sw);
     } else if (vec) {
         if (mode == GRAD_QUAD) GPGA_TILE(GRAD_QUAD, true);
         else if (mode == GRAD_QUAD_NOISE) GPGA_TILE(GRAD_QUAD_NOISE, true);

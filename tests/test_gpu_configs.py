@@ -128,7 +128,7 @@ def _make_logistic(n, m, d, batch, topo, H, gamma, l2, seed, A, y, X0):
 # lane busy; d = 260: ragged over the lanes); d <= 4096: staged, two passes over shared memory
 # (d = 4096: two-row tiles); wider: plain loads; d >= 18944: gradient buffer + row-streaming step
 # kernels instead of the tile kernel
-@pytest.mark.parametrize("n,m,d,batch", [(4, 64, 32, 8), (8, 256, 1024, 128), (2, 100, 260, 50), (3, 20, 4, 33),
+@pytest.mark.parametrize("n,m,d,batch", [(4, 64, 32, 8), (8, 256, 1024, 128), (2, 100, 260, 50), (4, 20, 4, 33),
                                          (2, 64, 1028, 40), (4, 24, 4096, 40), (2, 16, 8192, 8),
                                          (2, 16, 20000, 33)])
 def test_logistic_steps(topo, n, m, d, batch):
