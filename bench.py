@@ -466,7 +466,7 @@ def run_e2e(torch, g, w, dist):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(jobs):
-        g.run_host(x0, bh, K, out)                  # copies and kernels are ordered on the launching stream
+        g.run_host(x0, bh, K, out)                  # returns when its copies and kernels are done
     e1.record()
     torch.cuda.synchronize()
     dt = e0.elapsed_time(e1) * 1e-3                 # device time, copies included

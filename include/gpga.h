@@ -179,8 +179,16 @@ int32_t gpga_run(gpga_t* ctx, int64_t K, void* stream);
 /*
  * Same as gpga_run with HOST buffers (quadratic objective): copies x0_host and data_host
  * (dense n*d fp32 each) into the bound device buffers (row stride ld), resets the counter to 0, runs K
- * iterations, copies X^(K) to x_out_host and synchronises the stream.  Host buffers
+ * iterations, copies X^(K) to x_out_host and returns when all of that is done.  Host buffers
  * should be pinned for full copy speed.
+ * Columns of X evolve independently (W mixes rows; gradient and noise are element-wise and keyed by
+ * the absolute column), so a state above 64 MB with d % 4 == 0 moves through the call as column
+ * chunks of about 128 MB per buffer: the upload of one chunk, the K iterations of the one before
+ * and the download of the one before that run at the same time on two internal copy streams and on
+ * `stream`.  Every element goes through the same arithmetic as in the unchunked run (results
+ * bit-identical to bind + gpga_run), and on return the bound device buffers hold the whole X^(K).
+ * Work already queued on `stream` is waited for; the internal streams and events are created on
+ * the first call and released by gpga_destroy.
  */
 int32_t gpga_run_host(gpga_t* ctx, const float* x0_host, const float* data_host, int64_t K,
                       float* x_out_host, void* stream);

@@ -3,6 +3,7 @@
 #include <cstdio>
 #include <new>
 #include <string>
+#include <vector>
 
 #include "../../include/gpga.h"
 #include "gpga_kernels.cuh"
@@ -37,6 +38,16 @@ struct gpga_ctx {
     std::string err;
     PhiloxKeys keys;
     SparseW sparse;   // topology SPARSE: caller-owned CSR arrays on the device
+    // gpga_run_host only: copy streams and per-chunk events, created on first use
+    cudaStream_t up = nullptr, down = nullptr;
+    std::vector<cudaEvent_t> events;
+
+    ~gpga_ctx()
+    {
+        for (cudaEvent_t ev : events) cudaEventDestroy(ev);
+        if (up) cudaStreamDestroy(up);
+        if (down) cudaStreamDestroy(down);
+    }
 };
 
 static thread_local std::string g_create_error;
@@ -434,6 +445,34 @@ int32_t gpga_run(gpga_t* c, int64_t K, void* stream)
     return run_steps(c, K, static_cast<cudaStream_t>(stream));
 }
 
+namespace {
+
+// Column chunks of the host entry: about this many bytes of one n x chunk buffer, whole 128-byte
+// lines per row.  Small enough that the first upload and the last download, which nothing
+// overlaps, are a small part of the job; large enough that a chunk's step kernels fill the GPU.
+constexpr int64_t kHostChunkBytes = 128ll << 20;
+
+int32_t host_streams(gpga_ctx* c, size_t events)
+{
+    cudaError_t e;
+    if (!c->up && (e = cudaStreamCreateWithFlags(&c->up, cudaStreamNonBlocking)) != cudaSuccess)
+        return cuda_fail(c, e, "copy stream");
+    if (!c->down && (e = cudaStreamCreateWithFlags(&c->down, cudaStreamNonBlocking)) != cudaSuccess)
+        return cuda_fail(c, e, "copy stream");
+    while (c->events.size() < events) {
+        cudaEvent_t ev;
+        if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(c, e, "event");
+        c->events.push_back(ev);
+    }
+    return GPGA_OK;
+}
+
+}  // namespace
+
+// Columns evolve independently of one another (W acts on rows; gradient and noise are element-wise
+// and keyed by the absolute column), so the job is cut into column chunks that move through three
+// streams: upload of chunk c+1, the K iterations of chunk c and the download of chunk c-1 run at
+// the same time, and every element goes through exactly the arithmetic of the unchunked run.
 int32_t gpga_run_host(gpga_t* c, const float* x0_host, const float* data_host, int64_t K,
                       float* x_out_host, void* stream)
 {
@@ -443,22 +482,61 @@ int32_t gpga_run_host(gpga_t* c, const float* x0_host, const float* data_host, i
     if (!x0_host || !data_host || !x_out_host) return fail(c, GPGA_ERR_INVALID_ARG, "NULL host buffer");
     if (K < 0) return fail(c, GPGA_ERR_INVALID_ARG, "K must be >= 0");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const size_t row_bytes = (size_t)c->d * sizeof(float), pitch = (size_t)c->ld * sizeof(float);
-    cudaError_t e = cudaMemcpy2DAsync(c->x[0], pitch, x0_host, row_bytes, row_bytes, (size_t)c->n,
-                                      cudaMemcpyHostToDevice, s);
-    if (e != cudaSuccess) return cuda_fail(c, e, "x0 upload");
-    e = cudaMemcpy2DAsync(c->data, pitch, data_host, row_bytes, row_bytes, (size_t)c->n,
-                          cudaMemcpyHostToDevice, s);
-    if (e != cudaSuccess) return cuda_fail(c, e, "data upload");
-    c->cur = 0;
-    c->k = 0;
-    st = run_steps(c, K, s);
+    const size_t host_pitch = (size_t)c->d * sizeof(float), pitch = (size_t)c->ld * sizeof(float);
+    // whole column groups only (d % 4 == 0), so that every chunk takes the 128-bit path of the full run
+    int64_t chunks = 1;
+    if (vec_ok(c) && 12 * c->n * c->ld > kFusedStateBytes) chunks = (c->n * c->d * 4 + kHostChunkBytes - 1) / kHostChunkBytes;
+    const int64_t width = chunks > 1 ? round_up((c->d + chunks - 1) / chunks, 32) : c->d;
+    chunks = (c->d + width - 1) / width;
+    st = host_streams(c, (size_t)(2 * chunks + 2));
     if (st) return st;
-    e = cudaMemcpy2DAsync(x_out_host, row_bytes, c->x[c->cur], pitch, row_bytes, (size_t)c->n,
-                          cudaMemcpyDeviceToHost, s);
-    if (e != cudaSuccess) return cuda_fail(c, e, "result download");
-    e = cudaStreamSynchronize(s);
-    if (e != cudaSuccess) return cuda_fail(c, e, "stream synchronize");
+    cudaEvent_t* ev = c->events.data();   // [0]: work already on s; [1 + 2c]: chunk c uploaded; [2 + 2c]: chunk c done
+    cudaError_t e = cudaEventRecord(ev[0], s);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(c->up, ev[0], 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(c->down, ev[0], 0);
+    if (e != cudaSuccess) return cuda_fail(c, e, "stream order");
+    // the full-width view, put back whatever happens
+    float* const x0_full = c->x[0];
+    float* const x1_full = c->x[1];
+    float* const data_full = c->data;
+    const int64_t d_full = c->d, col0_full = c->col0;
+    auto restore = [&]() {
+        c->x[0] = x0_full; c->x[1] = x1_full; c->data = data_full; c->d = d_full; c->col0 = col0_full;
+    };
+    const char* where = nullptr;
+    for (int64_t ch = 0; ch < chunks && !st && !where; ++ch) {
+        const int64_t j0 = ch * width;
+        const int64_t w = (d_full - j0 < width) ? d_full - j0 : width;
+        const size_t wb = (size_t)w * sizeof(float);
+        e = cudaMemcpy2DAsync(x0_full + j0, pitch, x0_host + j0, host_pitch, wb, (size_t)c->n, cudaMemcpyHostToDevice, c->up);
+        if (e == cudaSuccess)
+            e = cudaMemcpy2DAsync(data_full + j0, pitch, data_host + j0, host_pitch, wb, (size_t)c->n, cudaMemcpyHostToDevice, c->up);
+        if (e == cudaSuccess) e = cudaEventRecord(ev[1 + 2 * ch], c->up);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s, ev[1 + 2 * ch], 0);
+        if (e != cudaSuccess) { where = "upload"; break; }
+        c->x[0] = x0_full + j0; c->x[1] = x1_full + j0; c->data = data_full + j0;
+        c->d = w; c->col0 = col0_full + j0;
+        c->cur = 0;
+        c->k = 0;
+        st = run_steps(c, K, s);
+        restore();
+        if (st) break;
+        e = cudaEventRecord(ev[2 + 2 * ch], s);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(c->down, ev[2 + 2 * ch], 0);
+        if (e == cudaSuccess)
+            e = cudaMemcpy2DAsync(x_out_host + j0, host_pitch, c->x[c->cur] + j0, pitch, wb, (size_t)c->n,
+                                  cudaMemcpyDeviceToHost, c->down);
+        if (e != cudaSuccess) where = "download";
+    }
+    // nothing of this call stays in flight when it returns, whatever happened
+    const cudaError_t e_up = cudaStreamSynchronize(c->up);
+    const cudaError_t e_s = cudaStreamSynchronize(s);
+    const cudaError_t e_down = cudaStreamSynchronize(c->down);
+    if (st) return st;
+    if (where) return cuda_fail(c, e, where);
+    if (e_up != cudaSuccess) return cuda_fail(c, e_up, "upload stream");
+    if (e_s != cudaSuccess) return cuda_fail(c, e_s, "stream synchronize");
+    if (e_down != cudaSuccess) return cuda_fail(c, e_down, "download stream");
     return GPGA_OK;
 }
 

@@ -198,6 +198,40 @@ def test_run_host_with_padded_rows():
     assert np.array_equal(out.numpy(), want)
 
 
+@pytest.mark.parametrize("topo,H", [("ring", 3), ("exp", 2)])
+def test_run_host_in_column_chunks_equals_the_device_run(topo, H):
+    """A state too large for one chunk goes through the host entry as a pipeline of column chunks
+    (upload, K iterations, download on three streams); every element must come out exactly as from
+    the unchunked run on resident buffers.  384 MB per buffer = 3 chunks, the last one ragged."""
+    torch = _torch()
+    n, d, K = 8, 12_000_040, 5
+    rng = np.random.default_rng(17)
+    X0 = rng.standard_normal((n, d), dtype=np.float32)
+    B = rng.standard_normal((n, d), dtype=np.float32)
+    ld = (d + 31) // 32 * 32
+    outs = []
+    for host in (False, True):
+        g = pkg.Gpga(n, d, TOPO[topo][0], H, 0.1, 5)
+        g.set_objective(pkg.GPGA_OBJ_QUADRATIC, sigma=0.3)
+        g.set_row_stride(ld)
+        xa, _, data = g.allocate()
+        if host:
+            out = torch.empty((n, d), dtype=torch.float32).pin_memory()
+            out.fill_(float("nan"))
+            g.run_host(torch.from_numpy(X0).pin_memory(), torch.from_numpy(B).pin_memory(), K, out)
+            assert g.get_k() == K
+            assert np.array_equal(g.get_x()[:, :d].cpu().numpy(), out.numpy())   # the device state is whole too
+            outs.append(out.numpy())
+        else:
+            xa[:, :d] = torch.from_numpy(X0).cuda()
+            data[:, :d] = torch.from_numpy(B).cuda()
+            g.run(K)
+            outs.append(g.get_x()[:, :d].cpu().numpy())
+        g.close()
+        del xa, data
+    assert np.array_equal(outs[0], outs[1])
+
+
 def test_column_offset_keys_the_noise():
     n, d, c0 = 4, 64, 4096
     X0, B = quadratic_inputs(n, d, 1)
