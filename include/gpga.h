@@ -138,11 +138,15 @@ int64_t gpga_scratch_bytes(const gpga_t* ctx);
 /*
  * Bind caller-owned device buffers.
  *  x_a, x_b : two n*ld fp32 buffers (double buffer for X^(k), X^(k+1)); x_a holds the
- *             current state.
+ *             current state.  x_b == x_a selects the in-place update: every kernel gives all n
+ *             rows of a column group to one thread (or one block's shared-memory tile), which
+ *             has read a row before it overwrites it, so X^(k+1) may replace X^(k) and the
+ *             footprint drops from three n*ld buffers to two.  Results are bit-identical.
  *  data     : QUADRATIC: b, n*ld fp32.  LOGISTIC: A, n*m*d fp32 (node-major, then sample).
  *  labels   : LOGISTIC: y, n*m fp32 in {-1,+1}; otherwise NULL.
  *  scratch  : at least gpga_scratch_bytes() bytes (scratch_bytes is what was given).
- * Errors: INVALID_ARG for NULL / misaligned pointers, x_a == x_b, too little scratch.
+ * Errors: INVALID_ARG for NULL / misaligned pointers, x_a and x_b overlapping without being
+ * equal, too little scratch.
  */
 int32_t gpga_bind(gpga_t* ctx, void* x_a, void* x_b, void* data, const void* labels,
                   void* scratch, int64_t scratch_bytes);

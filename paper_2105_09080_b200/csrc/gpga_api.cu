@@ -388,7 +388,11 @@ int32_t gpga_bind(gpga_t* c, void* x_a, void* x_b, void* data, const void* label
 {
     if (!c) return fail(nullptr, GPGA_ERR_NOT_READY, "NULL handle");
     if (!x_a || !x_b || !data || !scratch) return fail(c, GPGA_ERR_INVALID_ARG, "NULL buffer");
-    if (x_a == x_b) return fail(c, GPGA_ERR_INVALID_ARG, "x_a and x_b must be different buffers");
+    if (x_a != x_b) {   // the same buffer twice means "update in place"; anything between is a mistake
+        const uintptr_t a = reinterpret_cast<uintptr_t>(x_a), b = reinterpret_cast<uintptr_t>(x_b);
+        const uintptr_t bytes = (uintptr_t)c->n * (uintptr_t)c->ld * sizeof(float);
+        if ((a < b ? b - a : a - b) < bytes) return fail(c, GPGA_ERR_INVALID_ARG, "x_a and x_b overlap partly");
+    }
     if (!aligned16(x_a) || !aligned16(x_b) || !aligned16(data) || !aligned16(scratch) ||
         (labels && !aligned16(labels)))
         return fail(c, GPGA_ERR_INVALID_ARG, "device pointers must be 16-byte aligned");

@@ -111,7 +111,8 @@ def test_objective_and_bind_checks(L):
     nbytes = L.gpga_scratch_bytes(h)
     a, b, c, s = 0x10000, 0x20000, 0x30000, 0x40000       # fake aligned addresses, never dereferenced
     assert L.gpga_bind(h, None, b, c, None, s, nbytes) == pkg.GPGA_ERR_INVALID_ARG
-    assert L.gpga_bind(h, a, a, c, None, s, nbytes) == pkg.GPGA_ERR_INVALID_ARG
+    assert L.gpga_bind(h, a, a + 16, c, None, s, nbytes) == pkg.GPGA_ERR_INVALID_ARG   # partial overlap
+    assert L.gpga_bind(h, a, a, c, None, s, nbytes) == pkg.GPGA_OK                     # in-place update
     assert L.gpga_bind(h, a + 4, b, c, None, s, nbytes) == pkg.GPGA_ERR_INVALID_ARG
     assert L.gpga_bind(h, a, b, c, None, s, nbytes - 1) == pkg.GPGA_ERR_INVALID_ARG
     assert L.gpga_bind(h, a, b, c, None, s, nbytes) == pkg.GPGA_OK

@@ -196,6 +196,74 @@ def test_multi_iteration_launch_equals_single_iterations(topo, n, d, H):
     assert np.array_equal(fused, g3.get_x().cpu().numpy())
 
 
+# row-streaming kernels (wide d, scalar tail included), the shared-memory tile kernel (narrow d and
+# the grid / static exponential / W = I mixes) and the multi-iteration launch
+@pytest.mark.parametrize("topo,n,d,H", [("ring", 8, 40_000, 3), ("exp", 16, 24_004, 2), ("ring", 2, 30_001, 2),
+                                        ("exp", 8, 20_003, 0), ("ring", 7, 1031, 3), ("grid", 12, 520, 5),
+                                        ("static_exp", 16, 64, 0), ("none", 5, 36, 2), ("exp", 32, 4096, 8)])
+def test_in_place_update_equals_the_double_buffered_one(topo, n, d, H):
+    """Binding the same buffer as x_a and x_b overwrites X^(k) with X^(k+1); every element must come
+    out exactly as with two buffers, stepping one launch per iteration and through gpga_run."""
+    torch = _torch()
+    X0, B = quadratic_inputs(n, d, 77 + n, x0="shared", x0_std=0.5)
+    K = 6
+    g, p = make_quadratic(n, d, topo, H, 0.1, 23, 0.2, X0, B)
+    if topo == "grid":
+        p.grid_cols = 4               # the library's default for n = 12
+    for k in range(K):
+        g.step(k)
+    want = g.get_x().cpu().numpy().copy()
+    for stepwise in (True, False):
+        h = pkg.Gpga(n, d, TOPO[topo][0], H, 0.1, 23)
+        h.set_objective(pkg.GPGA_OBJ_QUADRATIC, sigma=0.2)
+        x = torch.from_numpy(X0).cuda()
+        h.bind(x, x, torch.from_numpy(B).cuda())
+        if stepwise:
+            for k in range(K):
+                h.step(k)
+        else:
+            h.run(K)
+        assert h.get_k() == K
+        assert np.array_equal(x.cpu().numpy(), want), (topo, stepwise)
+        h.close()
+    ok, worst = close(want, o.run(p, X0, 0, K), TOL_RUN)
+    assert ok, worst
+
+
+def test_in_place_update_with_the_logistic_objective():
+    torch = _torch()
+    n, m, d, batch, K = 8, 128, 256, 48, 7
+    A, y = logistic_inputs(n, m, d, 5)
+    rng = np.random.default_rng(4)
+    X0 = (0.2 * rng.standard_normal((n, d))).astype(np.float32)
+    outs = []
+    for in_place in (False, True):
+        g = pkg.Gpga(n, d, pkg.GPGA_TOPO_RING, 3, 0.3, 9)
+        g.set_objective(pkg.GPGA_OBJ_LOGISTIC, l2=1e-3, m=m, batch=batch)
+        xa = torch.from_numpy(X0).cuda()
+        g.bind(xa, xa if in_place else torch.empty_like(xa), torch.from_numpy(A).cuda(), torch.from_numpy(y).cuda())
+        g.run(K)
+        outs.append(g.get_x().cpu().numpy().copy())
+        g.close()
+    assert np.array_equal(outs[0], outs[1])
+    p = o.Problem(o.TOPO_RING, 3, 0.3, 9, objective="logistic", data=A, labels=y, l2=1e-3, batch=batch)
+    ok, worst = close(outs[1], o.run(p, X0, 0, K), TOL_RUN)
+    assert ok, worst
+
+
+def test_partly_overlapping_state_buffers_are_rejected():
+    torch = _torch()
+    n, d = 4, 64
+    g = pkg.Gpga(n, d, pkg.GPGA_TOPO_RING, 2, 0.1, 1)
+    big = torch.zeros(2 * n * d, dtype=torch.float32, device="cuda")
+    data = torch.zeros(n * d, dtype=torch.float32, device="cuda")
+    scratch = torch.empty(g.scratch_bytes(), dtype=torch.uint8, device="cuda")
+    with pytest.raises(pkg.GpgaError) as err:
+        g.bind_raw(big.data_ptr(), big.data_ptr() + 64, data.data_ptr(), None, scratch.data_ptr(), scratch.numel())
+    assert err.value.status == pkg.GPGA_ERR_INVALID_ARG
+    g.bind_raw(big.data_ptr(), big.data_ptr() + n * d * 4, data.data_ptr(), None, scratch.data_ptr(), scratch.numel())
+
+
 def test_multi_iteration_launch_is_chunked_for_long_runs():
     n, d, K = 4, 256, 2500            # more than one launch worth of iterations
     X0, B = quadratic_inputs(n, d, 5)
