@@ -254,6 +254,49 @@ __global__ void __launch_bounds__(kTileBlock) run_tile_kernel(const StepParams p
     }
 }
 
+// The same K iterations for strips with at most one cell per thread (n * tile_groups <= block
+// size): a thread keeps its cell's x and b in registers for the whole run, and only Y goes
+// through shared memory, in two tiles used alternately so that one barrier per iteration is
+// enough (a tile is rewritten two iterations later, and every thread passes the barrier in
+// between only after its reads of it).  Same arithmetic per element as run_tile_kernel.
+template <int MODE, bool VEC>
+__global__ void __launch_bounds__(kTileBlock) run_cell_kernel(const StepParams p, int topology, long long H,
+                                                              long long phase0, int hop0, int steps,
+                                                              int tile_groups, int log2n, const SparseW sw)
+{
+    extern __shared__ float4 tile_smem[];   // Y twice: [2][n][tile_groups]
+    const int n = (int)p.n;
+    const int cells = n * tile_groups;
+    const long long q_first = (long long)blockIdx.x * tile_groups;
+    const int c = threadIdx.x;
+    const int i = c / tile_groups, g = c - i * tile_groups;
+    const long long q = q_first + g;
+    const bool own = c < cells && q < p.Q;
+    float4 x = make_float4(0.f, 0.f, 0.f, 0.f), b = x;
+    if (own) {
+        x = load4<VEC>(p.x + (long long)i * p.ld, q * 4, p.d);
+        b = load4<VEC>(p.b + (long long)i * p.ldb, q * 4, p.d);
+    }
+    long long phase = phase0;   // (k + 1) mod H, global average when it is 0
+    int hop_log2 = hop0;        // k mod log2(n)
+    float4* ycur = tile_smem;
+    float4* ynext = tile_smem + cells;
+    for (int t = 0; t < steps; ++t) {
+        const uint32_t k = p.k + (uint32_t)t;
+        const bool global = H > 0 && phase == 0;            // Algorithm 1's test mod(k + 1, H) = 0
+        const int mix = global ? (int)TILE_MIX_GLOBAL : topology;
+        if (own) ycur[c] = tile_finish<MODE>(p, x, b, i, q, k);
+        __syncthreads();
+        if (own) x = tile_mix(ycur, i, g, n, tile_groups, mix, hop_log2, p.grid_cols, log2n, sw);
+        float4* const swap = ycur;
+        ycur = ynext;
+        ynext = swap;
+        if (++phase >= H) phase = 0;
+        if (++hop_log2 >= log2n) hop_log2 = 0;
+    }
+    if (own) store4<VEC>(p.out + (long long)i * p.ld, q * 4, p.d, x);
+}
+
 bool tile_supports(long long n) { return n * 16 <= kTileSmemBytes; }
 bool run_tile_supports(long long n) { return n * 2 * 48 <= kTileSmemBytes; }   // X, b, Y strips of >= 2 groups
 
@@ -325,14 +368,40 @@ cudaError_t launch_run_tile(const StepParams& p, int mode, bool vec, int topolog
 {
     if (!run_tile_supports(p.n) || (mode != GRAD_QUAD && mode != GRAD_QUAD_NOISE))
         return cudaErrorInvalidConfiguration;   // callers check
-    const int tile_groups = strip_groups(p.Q, p.n, 48, 8);   // compute-bound: fill every SM with warps
     const int log2n = log2_floor(p.n);
+    const long long phase0 = H > 0 ? ((long long)p.k + 1) % H : 1;
+    const int hop0 = log2n > 0 ? (int)(p.k % (uint32_t)log2n) : 0;
+    if (p.n <= kTileBlock) {
+        // one cell per thread: the narrowest strip that fills whole warps (small blocks balance
+        // best over the SMs and wait least at their barrier), two warps' worth when there are more
+        // blocks than fit on the GPU at once
+        long long tg = kTileBlock / p.n;
+        for (long long t = 1; t * p.n <= kTileBlock; ++t)
+            if ((t * p.n) % 32 == 0) { tg = t; break; }
+        if ((p.Q + tg - 1) / tg > 148 * 32 && 2 * tg * p.n <= kTileBlock / 2) tg *= 2;
+        if (tg > p.Q) tg = p.Q;
+        const int tile_groups = (int)tg;
+        const unsigned grd = (unsigned)((p.Q + tile_groups - 1) / tile_groups);
+        const long long cells = p.n * tile_groups;
+        const int blk = (int)((cells + 31) / 32 * 32);
+        const size_t smem = (size_t)cells * 32;
+#define GPGA_RUN_CELL(M, V) \
+    run_cell_kernel<M, V><<<grd, blk, smem, s>>>(p, topology, H, phase0, hop0, steps, tile_groups, log2n, sw)
+        if (vec) {
+            if (mode == GRAD_QUAD) GPGA_RUN_CELL(GRAD_QUAD, true);
+            else GPGA_RUN_CELL(GRAD_QUAD_NOISE, true);
+        } else {
+            if (mode == GRAD_QUAD) GPGA_RUN_CELL(GRAD_QUAD, false);
+            else GPGA_RUN_CELL(GRAD_QUAD_NOISE, false);
+        }
+#undef GPGA_RUN_CELL
+        return cudaGetLastError();
+    }
+    const int tile_groups = strip_groups(p.Q, p.n, 48, 8);   // compute-bound: fill every SM with warps
     const unsigned grd = (unsigned)((p.Q + tile_groups - 1) / tile_groups);
     const size_t smem = (size_t)p.n * tile_groups * 48;
     const long long cells = p.n * tile_groups;
     const int blk = cells >= kTileBlock ? kTileBlock : (int)((cells + 31) / 32 * 32);
-    const long long phase0 = H > 0 ? ((long long)p.k + 1) % H : 1;
-    const int hop0 = log2n > 0 ? (int)(p.k % (uint32_t)log2n) : 0;
 #define GPGA_RUN_TILE(M, V)                                                                      \
     do {                                                                                         \
         static unsigned long long limit_set = 0;                                                 \
