@@ -109,6 +109,57 @@ def test_config_3_resnet50_sized():
     torch.cuda.empty_cache()
 
 
+def test_config_3_through_the_host_pipeline():
+    """The ResNet-50-sized job through the host entry (pinned X0 and b in, X^(K) out, moved as
+    column chunks on three streams): bit-identical to the resident run on sampled blocks, and
+    within tolerance of the oracle on blocks that straddle chunk boundaries."""
+    torch = _torch()
+    n, d, gamma, sigma, K, H = 64, 25_557_032, 0.01, 0.01, 8, 4
+    if _free_gib() < 3 * n * d * 4 / 2**30 + 2:
+        pytest.skip("not enough free device memory")
+    ld = (d + 31) // 32 * 32
+    try:
+        host = [torch.empty((n, d), dtype=torch.float32, pin_memory=True) for _ in range(3)]
+    except RuntimeError:
+        pytest.skip("cannot pin 3 x 6.5 GB of host memory")
+    x0_h, b_h, out_h = host
+    g = pkg.Gpga(n, d, pkg.GPGA_TOPO_RING, H, gamma, SEED)
+    g.set_objective(pkg.GPGA_OBJ_QUADRATIC, sigma=sigma)
+    g.set_row_stride(ld)
+    xa, xb, b = g.allocate()
+    g.init_from_seed(pkg.GPGA_X0_SHARED_NORMAL, 0.1, 0.5)
+    x0_h.copy_(xa[:, :d])
+    b_h.copy_(b[:, :d])
+    torch.cuda.synchronize()
+    chunks = -(-n * d * 4 // (128 << 20))                 # the library's rule: ~128 MB of one buffer per chunk
+    width = -(-(-(-d // chunks)) // 32) * 32
+    assert chunks == 49 and width == 521_600
+    rng = np.random.default_rng(8)
+    offs = sorted({0, (d - BLOCK) // 4 * 4, width - 512, 2 * width - 4, 48 * width - 1020} |
+                  {int(rng.integers(0, (d - BLOCK) // 4)) * 4 for _ in range(27)})
+    g.run(K)
+    resident = {c0: _gpu_block(g.get_x(), c0, min(BLOCK, d - c0)) for c0 in offs}
+    out_h.fill_(float("nan"))
+    g.run_host(x0_h, b_h, K, out_h)
+    assert g.get_k() == K
+    out = out_h.numpy()
+    assert not np.isnan(out[:, ::4099]).any()
+    for c0 in offs:
+        w = min(BLOCK, d - c0)
+        assert np.array_equal(out[:, c0:c0 + w], resident[c0]), c0
+        assert np.array_equal(_gpu_block(g.get_x(), c0, w), resident[c0]), c0
+    for c0 in (width - 512, 2 * width - 4, 48 * width - 1020):      # across chunk boundaries
+        w = min(BLOCK, d - c0)
+        B = o.init_b(n, w, SEED, 0.5, c0).astype(np.float32)
+        X0 = o.init_x0(n, w, SEED, o.X0_SHARED_NORMAL, 0.1, c0).astype(np.float32)
+        p = o.Problem(o.TOPO_RING, H, gamma, SEED, sigma=sigma, data=B, col0=c0)
+        ok, worst = close(out[:, c0:c0 + w], o.run(p, X0, 0, K), TOL_RUN)
+        assert ok, (c0, worst)
+    g.close()
+    del xa, xb, b, host, x0_h, b_h, out_h
+    torch.cuda.empty_cache()
+
+
 def test_config_4_bert_large_sized():
     torch = _torch()
     n, d, gamma, sigma, K, H = 16, 335_141_888, 0.01, 0.01, 20, 4
