@@ -152,8 +152,10 @@ __global__ void __launch_bounds__(kLrBlock) logreg_partial_tma_kernel(const Logr
         issue(0);
         if (ntiles > 1) issue(1);
     }
-    // x_i and the labels of the drawn rows arrive while the copies fly
+    // x_i and the labels of the drawn rows arrive while the copies fly; x is the previous step's
+    // output (and the partial sums may still be read by it), everything before reads A and y only
     if (threadIdx.x < nrows) ys[threadIdx.x] = y[rows[threadIdx.x]];
+    grid_dependency_wait();
     for (int j = threadIdx.x; j < p.d; j += blockDim.x) xs[j] = x[j];
     __syncthreads();
     float4 acc[kTmaMaxGroups];
@@ -215,6 +217,7 @@ __global__ void __launch_bounds__(kLrBlock) logreg_partial_tma_kernel(const Logr
         __syncthreads();   // everyone is done with this buffer before new copies overwrite it
         if (warp == 0 && s + 2 < ntiles) issue(s + 2);
     }
+    grid_launch_dependents();   // the step kernel may take its place; it waits for this grid before reading
     if (failed) return;
     float4* out4 = reinterpret_cast<float4*>(p.partial + ((long long)c * p.n + i) * p.d);
 #pragma unroll
@@ -449,8 +452,8 @@ cudaError_t launch_logreg_partial(const LogregParams& p, cudaStream_t s)
         static unsigned long long tma_limit_set = 0;
         cudaError_t e = ensure_smem_limit(logreg_partial_tma_kernel, 100 * 1024, tma_limit_set);
         if (e != cudaSuccess) return e;
-        logreg_partial_tma_kernel<<<dim3((unsigned)p.n, (unsigned)chunks), kLrBlock, smem_tma, s>>>(p, tile_rows);
-        return cudaGetLastError();
+        return launch_after_trigger(logreg_partial_tma_kernel, dim3((unsigned)p.n, (unsigned)chunks), dim3(kLrBlock),
+                                    smem_tma, s, p.after_own_step, p, tile_rows);
     }
     const size_t smem = (size_t)(p.d + kChunkRows) * sizeof(float);
     static unsigned long long plain_limit_set = 0;
