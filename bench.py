@@ -369,7 +369,7 @@ def run_ours(args, w, name):
 
 
 def run_logistic(args, w, name):
-    """Convex workload: per-node mini-batch logistic gradient + fused step/mix, 3 launches per step."""
+    """Convex workload: per-node mini-batch logistic gradient + fused step/mix, 2 launches per step."""
     import torch
     import paper_2105_09080_b200 as pkg
     if not torch.cuda.is_available():
