@@ -187,7 +187,7 @@ int32_t gpga_run(gpga_t* ctx, int64_t K, void* stream);
  * should be pinned for full copy speed.
  * Columns of X evolve independently (W mixes rows; gradient and noise are element-wise and keyed by
  * the absolute column), so a state above 64 MB with d % 4 == 0 moves through the call as column
- * chunks of about 128 MB per buffer: the upload of one chunk, the K iterations of the one before
+ * chunks (a sixteenth of a buffer, between 16 and 128 MB): the upload of one chunk, the K iterations of the one before
  * and the download of the one before that run at the same time on two internal copy streams and on
  * `stream`.  Every element goes through the same arithmetic as in the unchunked run (results
  * bit-identical to bind + gpga_run), and on return the bound device buffers hold the whole X^(K).

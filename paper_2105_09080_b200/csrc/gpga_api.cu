@@ -451,10 +451,11 @@ int32_t gpga_run(gpga_t* c, int64_t K, void* stream)
 
 namespace {
 
-// Column chunks of the host entry: about this many bytes of one n x chunk buffer, whole 128-byte
-// lines per row.  Small enough that the first upload and the last download, which nothing
-// overlaps, are a small part of the job; large enough that a chunk's step kernels fill the GPU.
-constexpr int64_t kHostChunkBytes = 128ll << 20;
+// Column chunks of the host entry: a sixteenth of one n x d buffer, between 16 MB and 128 MB, in
+// whole 128-byte lines per row.  Small enough that the first upload and the last chunk's
+// iterations and download, which nothing overlaps, are a small part of the job; large enough that
+// a chunk's step kernels fill the GPU.
+constexpr int64_t kHostChunkMinBytes = 16ll << 20, kHostChunkMaxBytes = 128ll << 20;
 
 int32_t host_streams(gpga_ctx* c, size_t events)
 {
@@ -489,7 +490,13 @@ int32_t gpga_run_host(gpga_t* c, const float* x0_host, const float* data_host, i
     const size_t host_pitch = (size_t)c->d * sizeof(float), pitch = (size_t)c->ld * sizeof(float);
     // whole column groups only (d % 4 == 0), so that every chunk takes the 128-bit path of the full run
     int64_t chunks = 1;
-    if (vec_ok(c) && 12 * c->n * c->ld > kFusedStateBytes) chunks = (c->n * c->d * 4 + kHostChunkBytes - 1) / kHostChunkBytes;
+    if (vec_ok(c) && 12 * c->n * c->ld > kFusedStateBytes) {
+        const int64_t buffer_bytes = c->n * c->d * 4;
+        int64_t chunk_bytes = buffer_bytes / 16;
+        if (chunk_bytes < kHostChunkMinBytes) chunk_bytes = kHostChunkMinBytes;
+        if (chunk_bytes > kHostChunkMaxBytes) chunk_bytes = kHostChunkMaxBytes;
+        chunks = (buffer_bytes + chunk_bytes - 1) / chunk_bytes;
+    }
     const int64_t width = chunks > 1 ? round_up((c->d + chunks - 1) / chunks, 32) : c->d;
     chunks = (c->d + width - 1) / width;
     st = host_streams(c, (size_t)(2 * chunks + 2));

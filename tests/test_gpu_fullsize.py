@@ -131,7 +131,7 @@ def test_config_3_through_the_host_pipeline():
     x0_h.copy_(xa[:, :d])
     b_h.copy_(b[:, :d])
     torch.cuda.synchronize()
-    chunks = -(-n * d * 4 // (128 << 20))                 # the library's rule: ~128 MB of one buffer per chunk
+    chunks = -(-n * d * 4 // (128 << 20))                 # the library's rule at this size: 128 MB of one buffer per chunk
     width = -(-(-(-d // chunks)) // 32) * 32
     assert chunks == 49 and width == 521_600
     rng = np.random.default_rng(8)

@@ -202,7 +202,7 @@ def test_run_host_with_padded_rows():
 def test_run_host_in_column_chunks_equals_the_device_run(topo, H):
     """A state too large for one chunk goes through the host entry as a pipeline of column chunks
     (upload, K iterations, download on three streams); every element must come out exactly as from
-    the unchunked run on resident buffers.  384 MB per buffer = 3 chunks, the last one ragged."""
+    the unchunked run on resident buffers.  384 MB per buffer = 16 chunks, the last one ragged."""
     torch = _torch()
     n, d, K = 8, 12_000_040, 5
     rng = np.random.default_rng(17)
