@@ -100,132 +100,9 @@ __global__ void __launch_bounds__(kLrBlock) logreg_partial_kernel(const LogregPa
     }
 }
 
-// The same partial sums with the batch rows staged in shared memory by bulk asynchronous
-// copies (one 16-byte-aligned row of d floats per copy, completion counted on an
-// mbarrier).  Two tiles of rows alternate: while one is consumed the next is in flight,
-// without holding registers, and both passes over a row -- the margin and the weighted
-// sum -- read shared memory, so A is fetched from HBM exactly once.  Used for
-// d <= kTmaMaxD; a thread then owns at most kTmaMaxGroups groups of four columns.
-constexpr int kTmaMaxD = 4096;
-constexpr int kTmaMaxGroups = kTmaMaxD / 4 / kLrBlock;
-constexpr int kTmaTileBytes = 64 * 1024;
+// Polls of an mbarrier before a kernel gives up on a bulk copy (each poll may block for a short,
+// hardware-defined time): far beyond any copy's latency, and finite.
 constexpr uint32_t kTmaMaxTries = 1u << 22;
-
-__global__ void __launch_bounds__(kLrBlock) logreg_partial_tma_kernel(const LogregParams p, int tile_rows)
-{
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    float* tiles = reinterpret_cast<float*>(smem_raw);         // 2 x tile_rows x d
-    float* xs = tiles + 2 * (size_t)tile_rows * p.d;           // d floats: x_i
-    float* coef = xs + p.d;                                    // kChunkRows floats: s_r
-    __shared__ uint32_t rows[kChunkRows];
-    __shared__ float ys[kChunkRows];
-    __shared__ __align__(8) uint64_t bar[2];
-    const int i = blockIdx.x, c = blockIdx.y;
-    const int t0 = c * kChunkRows;
-    const int nrows = min(kChunkRows, (int)p.batch - t0);
-    const int ntiles = (nrows + tile_rows - 1) / tile_rows;
-    const float* A = p.A + (long long)i * p.m * p.d;
-    const float* y = p.y + (long long)i * p.m;
-    const float* x = p.x + (long long)i * p.ldx;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    const int d4 = (int)(p.d >> 2);
-    const uint32_t row_bytes = (uint32_t)p.d * 4u;
-    if (threadIdx.x < nrows)
-        rows[threadIdx.x] = batch_row((uint32_t)(t0 + threadIdx.x), (uint32_t)i, p.k, (uint32_t)p.m, p.keys);
-    if (threadIdx.x == 0) {
-        mbar_init(&bar[0], 1);
-        mbar_init(&bar[1], 1);
-        mbar_init_fence();
-    }
-    __syncthreads();
-    // warp 0 starts the copies of tile s into buffer s & 1
-    auto issue = [&](int s) {
-        const int r0 = s * tile_rows;
-        const int rr = min(tile_rows, nrows - r0);
-        float* dst = tiles + (size_t)(s & 1) * tile_rows * p.d;
-        if (lane == 0) mbar_arrive_expect_tx(&bar[s & 1], (uint32_t)rr * row_bytes);
-        __syncwarp();
-        for (int t = lane; t < rr; t += 32)
-            bulk_copy_g2s(dst + (size_t)t * p.d, A + (long long)rows[r0 + t] * p.d, row_bytes, &bar[s & 1]);
-    };
-    if (warp == 0) {
-        issue(0);
-        if (ntiles > 1) issue(1);
-    }
-    // x_i and the labels of the drawn rows arrive while the copies fly; x is the previous step's
-    // output (and the partial sums may still be read by it), everything before reads A and y only
-    if (threadIdx.x < nrows) ys[threadIdx.x] = y[rows[threadIdx.x]];
-    grid_dependency_wait();
-    for (int j = threadIdx.x; j < p.d; j += blockDim.x) xs[j] = x[j];
-    __syncthreads();
-    float4 acc[kTmaMaxGroups];
-#pragma unroll
-    for (int u = 0; u < kTmaMaxGroups; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-    uint32_t parity0 = 0u, parity1 = 0u;
-    bool failed = false;
-    for (int s = 0; s < ntiles; ++s) {
-        const int buf = s & 1;
-        const int r0 = s * tile_rows;
-        const int rr = min(tile_rows, nrows - r0);
-        const float* tile = tiles + (size_t)buf * tile_rows * p.d;
-        const uint32_t par = buf ? parity1 : parity0;
-        const bool ok = mbar_wait_bounded(&bar[buf], par, kTmaMaxTries);
-        if (__syncthreads_or(!ok)) {
-            // a copy did not report in time: flag it, give the copies in flight (they target
-            // this block's shared memory) one more bounded chance to land, and leave
-            if (!ok) mbar_wait_bounded(&bar[buf], par, kTmaMaxTries);
-            if (s + 1 < ntiles) mbar_wait_bounded(&bar[buf ^ 1], buf ? parity0 : parity1, kTmaMaxTries);
-            if (threadIdx.x == 0 && p.error_flag) atomicExch(p.error_flag, 1);
-            failed = true;
-            break;
-        }
-        if (buf) parity1 ^= 1u; else parity0 ^= 1u;
-        for (int t = warp; t < rr; t += nwarps) {
-            const float4* a4 = reinterpret_cast<const float4*>(tile + (size_t)t * p.d);
-            float z = 0.f;
-#pragma unroll 4
-            for (int g = lane; g < d4; g += 32) {
-                const float4 a = a4[g];
-                const float4 xv = reinterpret_cast<const float4*>(xs)[g];
-                z = fmaf(a.x, xv.x, z);
-                z = fmaf(a.y, xv.y, z);
-                z = fmaf(a.z, xv.z, z);
-                z = fmaf(a.w, xv.w, z);
-            }
-            z = warp_sum_f(z);
-            if (lane == 0) {
-                const float yr = ys[r0 + t];
-                coef[r0 + t] = -yr / (1.0f + expf(yr * z));
-            }
-        }
-        __syncthreads();
-#pragma unroll
-        for (int u = 0; u < kTmaMaxGroups; ++u) {
-            const int g = threadIdx.x + u * kLrBlock;
-            if (g < d4) {
-#pragma unroll 4
-                for (int t = 0; t < rr; ++t) {
-                    const float4 a = reinterpret_cast<const float4*>(tile + (size_t)t * p.d)[g];
-                    const float sc = coef[r0 + t];
-                    acc[u].x = fmaf(sc, a.x, acc[u].x);
-                    acc[u].y = fmaf(sc, a.y, acc[u].y);
-                    acc[u].z = fmaf(sc, a.z, acc[u].z);
-                    acc[u].w = fmaf(sc, a.w, acc[u].w);
-                }
-            }
-        }
-        __syncthreads();   // everyone is done with this buffer before new copies overwrite it
-        if (warp == 0 && s + 2 < ntiles) issue(s + 2);
-    }
-    grid_launch_dependents();   // the step kernel may take its place; it waits for this grid before reading
-    if (failed) return;
-    float4* out4 = reinterpret_cast<float4*>(p.partial + ((long long)c * p.n + i) * p.d);
-#pragma unroll
-    for (int u = 0; u < kTmaMaxGroups; ++u) {
-        const int g = threadIdx.x + u * kLrBlock;
-        if (g < d4) out4[g] = acc[u];
-    }
-}
 
 // Narrow rows (d <= kRegMaxD): the same staging by bulk asynchronous copies, but every warp
 // runs its own pipeline -- it draws the indices of its rows (rows warp, warp + 8, ... of the
@@ -353,6 +230,138 @@ __global__ void __launch_bounds__(kLrBlock, 2) logreg_partial_tma_reg_kernel(con
     }
 }
 
+// Wider rows (kRegMaxD < d <= kTmaMaxD): the batch rows are staged in shared memory by bulk
+// asynchronous copies (one 16-byte-aligned row of d floats per copy, completion counted on an
+// mbarrier), two tiles of rows alternating: while one is consumed the next is in flight.  A
+// thread owns J groups of four columns (group t + 256 u): x_i of those columns and its slice of
+// the tile's rows sit in registers, so a staged row is read from shared memory once; the
+// margins of the tile's rows are reduced over the block (lanes by shuffle, warps in index
+// order through shared memory), and s * a is added to the thread's accumulators from the
+// registers.  One block barrier per tile; A is fetched from HBM exactly once.
+constexpr int kTmaMaxD = 8192;
+constexpr int kColsCells = 8;            // (rows per tile) x (groups per thread), in registers
+
+template <int J>
+__global__ void __launch_bounds__(kLrBlock, 2) logreg_partial_tma_cols_kernel(const LogregParams p)
+{
+    constexpr int T = kColsCells / J;   // rows per tile
+    constexpr int kWarps = kLrBlock / 32;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    float* tiles = reinterpret_cast<float*>(smem_raw);         // 2 x T x d
+    __shared__ uint32_t rows[kChunkRows];
+    __shared__ float ys[kChunkRows];
+    __shared__ float wsum[2][T][kWarps];                       // per-warp margin sums, by tile parity
+    __shared__ __align__(8) uint64_t bar[2];
+    const int i = blockIdx.x, c = blockIdx.y;
+    const int t0 = c * kChunkRows;
+    const int nrows = min(kChunkRows, (int)p.batch - t0);
+    const int ntiles = (nrows + T - 1) / T;
+    const float* A = p.A + (long long)i * p.m * p.d;
+    const float* y = p.y + (long long)i * p.m;
+    const float4* x4 = reinterpret_cast<const float4*>(p.x + (long long)i * p.ldx);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int d4 = (int)(p.d >> 2);
+    const uint32_t row_bytes = (uint32_t)p.d * 4u;
+    if (threadIdx.x < nrows)
+        rows[threadIdx.x] = batch_row((uint32_t)(t0 + threadIdx.x), (uint32_t)i, p.k, (uint32_t)p.m, p.keys);
+    if (threadIdx.x == 0) {
+        mbar_init(&bar[0], 1);
+        mbar_init(&bar[1], 1);
+        mbar_init_fence();
+    }
+    __syncthreads();
+    // warp 0 starts the copies of tile s into buffer s & 1
+    auto issue = [&](int s) {
+        const int r0 = s * T;
+        const int rr = min(T, nrows - r0);
+        float* dst = tiles + (size_t)(s & 1) * T * p.d;
+        if (lane == 0) mbar_arrive_expect_tx(&bar[s & 1], (uint32_t)rr * row_bytes);
+        __syncwarp();
+        if (lane < rr) bulk_copy_g2s(dst + (size_t)lane * p.d, A + (long long)rows[r0 + lane] * p.d, row_bytes, &bar[s & 1]);
+    };
+    if (warp == 0) {
+        issue(0);
+        if (ntiles > 1) issue(1);
+    }
+    if (threadIdx.x < nrows) ys[threadIdx.x] = y[rows[threadIdx.x]];
+    // everything above reads only A, y and the iteration index; x is the previous step's output and
+    // the partial sums may still be read by it
+    grid_dependency_wait();
+    float4 xr[J], acc[J];
+#pragma unroll
+    for (int u = 0; u < J; ++u) {
+        const int g = threadIdx.x + u * kLrBlock;
+        xr[u] = g < d4 ? x4[g] : make_float4(0.f, 0.f, 0.f, 0.f);
+        acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    __syncthreads();   // ys
+    uint32_t parity0 = 0u, parity1 = 0u;
+    bool failed = false;
+    for (int s = 0; s < ntiles; ++s) {
+        const int buf = s & 1;
+        const int r0 = s * T;
+        const int rr = min(T, nrows - r0);
+        const float* tile = tiles + (size_t)buf * T * p.d;
+        const uint32_t par = buf ? parity1 : parity0;
+        const bool ok = mbar_wait_bounded(&bar[buf], par, kTmaMaxTries);
+        if (__syncthreads_or(!ok)) {
+            // a copy did not report in time: flag it, give the copies in flight (they target
+            // this block's shared memory) one more bounded chance to land, and leave
+            if (!ok) mbar_wait_bounded(&bar[buf], par, kTmaMaxTries);
+            if (s + 1 < ntiles) mbar_wait_bounded(&bar[buf ^ 1], buf ? parity0 : parity1, kTmaMaxTries);
+            if (threadIdx.x == 0 && p.error_flag) atomicExch(p.error_flag, 1);
+            failed = true;
+            break;
+        }
+        if (buf) parity1 ^= 1u; else parity0 ^= 1u;
+        // this thread's slice of the tile, and its part of every row's margin
+        float4 a[T][J];
+#pragma unroll
+        for (int t = 0; t < T; ++t) {
+            float z = 0.f;
+#pragma unroll
+            for (int u = 0; u < J; ++u) {
+                const int g = threadIdx.x + u * kLrBlock;
+                a[t][u] = (t < rr && g < d4) ? reinterpret_cast<const float4*>(tile + (size_t)t * p.d)[g]
+                                             : make_float4(0.f, 0.f, 0.f, 0.f);
+                z = fmaf(a[t][u].x, xr[u].x, z);
+                z = fmaf(a[t][u].y, xr[u].y, z);
+                z = fmaf(a[t][u].z, xr[u].z, z);
+                z = fmaf(a[t][u].w, xr[u].w, z);
+            }
+            z = warp_sum_f(z);
+            if (lane == 0) wsum[buf][t][warp] = z;
+        }
+        __syncthreads();   // margins complete; every thread holds its slice, so the buffer is free
+        if (warp == 0 && s + 2 < ntiles) issue(s + 2);
+#pragma unroll
+        for (int t = 0; t < T; ++t) {
+            if (t < rr) {
+                float z = wsum[buf][t][0];
+#pragma unroll
+                for (int w = 1; w < kWarps; ++w) z += wsum[buf][t][w];
+                const float yr = ys[r0 + t];
+                const float sc = -yr / (1.0f + expf(yr * z));
+#pragma unroll
+                for (int u = 0; u < J; ++u) {
+                    acc[u].x = fmaf(sc, a[t][u].x, acc[u].x);
+                    acc[u].y = fmaf(sc, a[t][u].y, acc[u].y);
+                    acc[u].z = fmaf(sc, a[t][u].z, acc[u].z);
+                    acc[u].w = fmaf(sc, a[t][u].w, acc[u].w);
+                }
+            }
+        }
+    }
+    grid_launch_dependents();   // the step kernel may take its place; it waits for this grid before reading
+    if (failed) return;
+    float4* out4 = reinterpret_cast<float4*>(p.partial + ((long long)c * p.n + i) * p.d);
+#pragma unroll
+    for (int u = 0; u < J; ++u) {
+        const int g = threadIdx.x + u * kLrBlock;
+        if (g < d4) out4[g] = acc[u];
+    }
+}
+
 // G[i][:] = (1/B) sum_c partial[c][i][:] + l2 x_i, chunks added in index order.
 __global__ void __launch_bounds__(kLrBlock) logreg_reduce_kernel(const LogregParams p, int chunks)
 {
@@ -446,14 +455,21 @@ cudaError_t launch_logreg_partial(const LogregParams& p, cudaStream_t s)
                                     dim3(kLrBlock), smem_reg, s, p.after_own_step, p, slots);
     }
     if (p.d <= kTmaMaxD) {
-        int tile_rows = kTmaTileBytes / 2 / (int)(p.d * 4);   // two tiles share the budget
-        if (tile_rows > kChunkRows) tile_rows = kChunkRows;
-        const size_t smem_tma = (2 * (size_t)tile_rows * p.d + p.d + kChunkRows) * sizeof(float);
-        static unsigned long long tma_limit_set = 0;
-        cudaError_t e = ensure_smem_limit(logreg_partial_tma_kernel, 100 * 1024, tma_limit_set);
-        if (e != cudaSuccess) return e;
-        return launch_after_trigger(logreg_partial_tma_kernel, dim3((unsigned)p.n, (unsigned)chunks), dim3(kLrBlock),
-                                    smem_tma, s, p.after_own_step, p, tile_rows);
+        const int groups = (int)((p.d / 4 + kLrBlock - 1) / kLrBlock);   // groups of four columns per thread
+        const dim3 grid((unsigned)p.n, (unsigned)chunks);
+        const size_t smem_cols = 2 * (size_t)kColsCells * p.d * sizeof(float);   // before / J below
+#define GPGA_COLS(J)                                                                                   \
+    do {                                                                                               \
+        static unsigned long long limit_set = 0;                                                       \
+        cudaError_t e = ensure_smem_limit(logreg_partial_tma_cols_kernel<J>, 64 * 1024, limit_set);    \
+        if (e != cudaSuccess) return e;                                                                \
+        return launch_after_trigger(logreg_partial_tma_cols_kernel<J>, grid, dim3(kLrBlock), smem_cols / J, s, \
+                                    p.after_own_step, p);                                              \
+    } while (0)
+        if (groups <= 2) GPGA_COLS(2);
+        else if (groups <= 4) GPGA_COLS(4);
+        else GPGA_COLS(8);
+#undef GPGA_COLS
     }
     const size_t smem = (size_t)(p.d + kChunkRows) * sizeof(float);
     static unsigned long long plain_limit_set = 0;

@@ -124,13 +124,14 @@ def _make_logistic(n, m, d, batch, topo, H, gamma, l2, seed, A, y, X0):
 
 
 @pytest.mark.parametrize("topo", ["ring", "exp"])
-# d <= 1024: rows staged by bulk asynchronous copies and taken through registers once (d = 4: one
-# lane busy; d = 260: ragged over the lanes); d <= 4096: staged, two passes over shared memory
-# (d = 4096: two-row tiles); wider: plain loads; d >= 18944: gradient buffer + row-streaming step
-# kernels instead of the tile kernel
+# d <= 1024: rows staged by bulk asynchronous copies, one pipeline per warp, rows through registers
+# once (d = 4: one lane busy; d = 260: ragged over the lanes); d <= 8192: staged in two alternating
+# tiles, a thread owns 2 / 4 / 8 groups of four columns (d = 1028, 2052: ragged over the threads;
+# 4096 and 8192: full); wider: plain loads; d >= 18944: gradient buffer + row-streaming step kernels
+# instead of the tile kernel
 @pytest.mark.parametrize("n,m,d,batch", [(4, 64, 32, 8), (8, 256, 1024, 128), (2, 100, 260, 50), (4, 20, 4, 33),
-                                         (2, 64, 1028, 40), (4, 24, 4096, 40), (2, 16, 8192, 8),
-                                         (2, 16, 20000, 33)])
+                                         (2, 64, 1028, 40), (4, 40, 2052, 70), (4, 24, 4096, 40),
+                                         (2, 16, 8192, 8), (2, 16, 8196, 8), (2, 16, 20000, 33)])
 def test_logistic_steps(topo, n, m, d, batch):
     A, y = logistic_inputs(n, m, d, SEED + n)
     rng = np.random.default_rng(0)
