@@ -104,12 +104,13 @@ __global__ void __launch_bounds__(kLrBlock) logreg_partial_kernel(const LogregPa
 // hardware-defined time): far beyond any copy's latency, and finite.
 constexpr uint32_t kTmaMaxTries = 1u << 22;
 
-// Narrow rows (d <= kRegMaxD): the same staging by bulk asynchronous copies, but every warp
-// runs its own pipeline -- it draws the indices of its rows (rows warp, warp + 8, ... of the
-// chunk), copies each into one of its `slots` row buffers, and takes a staged row through
+// Narrow rows (d <= kRegMaxD): the batch rows are staged in shared memory by bulk asynchronous
+// copies (one 16-byte-aligned row of d floats per copy, completion counted on an mbarrier) and
+// every warp runs its own pipeline -- it draws the indices of its rows (rows warp, warp + 8, ...
+// of the chunk), copies each into one of its `slots` row buffers, and takes a staged row through
 // registers once: the margin a^T x against x held in registers, then s * a added to per-lane
-// accumulators.  A row is read from shared memory once instead of twice, x not at all, and
-// no block-wide barrier stands between rows.  The per-warp accumulators are added in warp
+// accumulators.  A row is read from shared memory once, x not at all, and no block-wide
+// barrier stands between rows; A is fetched from HBM exactly once.  The per-warp accumulators are added in warp
 // order at the end (fixed order: the result does not depend on scheduling).
 constexpr int kRegMaxD = 1024;
 constexpr int kRegGroups = kRegMaxD / 4 / 32;   // float4 per lane
