@@ -170,10 +170,13 @@ int32_t gpga_init_from_seed(gpga_t* ctx, int32_t x0_kind, float x0_std, float b_
  */
 int32_t gpga_step(gpga_t* ctx, int64_t k, void* stream);
 
-/* K iterations k0 .. k0+K-1 starting at the internal counter k0 (Algorithm 1's loop).  A quadratic-
- * objective state of at most 64 MB (X, X+ and b together) is advanced many iterations per launch with
- * its column strips resident in shared memory -- columns evolve independently -- with results
- * bit-identical to K calls of gpga_step; larger states take one launch per iteration.
+/* K iterations k0 .. k0+K-1 starting at the internal counter k0 (Algorithm 1's loop).  Columns of X
+ * evolve independently, so under the quadratic objective a strip of columns can be advanced many
+ * iterations per launch with its cells held on chip (HBM touched once per launch, the time per
+ * iteration set by the noise arithmetic).  gpga_run does so for a state of at most 64 MB (X, X+ and b
+ * together), and at any size for n <= 32 and K >= 32, where that is faster than streaming the state
+ * from HBM every iteration; otherwise it takes one launch per iteration.  Results are bit-identical
+ * to K calls of gpga_step either way.
  * Logistic objective: within one call the launches of consecutive iterations overlap (the rows of A and
  * the labels of iteration k+1 are fetched while iteration k finishes); A and the labels are inputs that
  * no kernel of the library writes, and the caller must not write them while the call's work is in

@@ -200,11 +200,20 @@ int32_t do_step(gpga_ctx* c, int64_t k, bool global, cudaStream_t s, bool after_
     return GPGA_OK;
 }
 
-// K iterations starting at c->k.  A quadratic-objective state small enough to sit in L2 is
-// bound by launch latency when stepped one launch per iteration; it runs instead in launches
-// of up to kFusedSteps iterations with its strips resident in shared memory.
+// K iterations starting at c->k.  Columns evolve independently, so a strip of columns can be taken
+// through many iterations on chip (launch_run_tile) with HBM touched once per launch; the time per
+// iteration is then set by the noise arithmetic, not by memory.  That path is taken
+//  - for a state small enough to sit in L2 (one launch per iteration would be launch-bound), and
+//  - for n <= 32 and runs of at least kFusedMinSteps iterations at any size: there the arithmetic
+//    bound (6.0-6.2e11 updates/s measured at n = 16, 32) is above what the row-streaming kernels
+//    reach from HBM (at most 5.5e11), and the one extra pass over the state is amortised.  At
+//    n = 64 the multi-iteration kernel runs at 4.8e11 (two-warp blocks, longer column sums) and
+//    the row-streaming kernels stay in use.
+// A launch is kept to about half a second of work.
 constexpr int64_t kFusedStateBytes = 64ll << 20;
 constexpr int64_t kFusedSteps = 1024;
+constexpr int64_t kFusedWideNodes = 32, kFusedMinSteps = 32;
+constexpr double kFusedUpdatesPerLaunch = 2.75e11;
 
 int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)
 {
@@ -213,7 +222,10 @@ int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)
     if (c->topology == GPGA_TOPO_SPARSE && !c->sparse.row_ptr)
         return fail(c, GPGA_ERR_NOT_READY, "topology SPARSE needs gpga_set_weight_matrix");
     const bool fused = c->objective == GPGA_OBJ_QUADRATIC && K >= 2 && run_tile_supports(c->n) &&
-                       12 * c->n * c->ld <= kFusedStateBytes;
+                       (12 * c->n * c->ld <= kFusedStateBytes || (c->n <= kFusedWideNodes && K >= kFusedMinSteps));
+    int64_t per_launch = (int64_t)(kFusedUpdatesPerLaunch / ((double)c->n * (double)c->d));
+    if (per_launch > kFusedSteps) per_launch = kFusedSteps;
+    if (per_launch < 16) per_launch = 16;
     if (!fused) {
         for (int64_t k = c->k; k < k_end; ++k) {
             // from the second iteration on, the launch before the gradient kernel is our own step kernel
@@ -223,7 +235,7 @@ int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)
         return GPGA_OK;
     }
     while (c->k < k_end) {
-        const int64_t steps = (k_end - c->k < kFusedSteps) ? k_end - c->k : kFusedSteps;
+        const int64_t steps = (k_end - c->k < per_launch) ? k_end - c->k : per_launch;
         StepParams p;
         p.x = c->x[c->cur];
         p.out = c->x[c->cur ^ 1];

@@ -264,7 +264,7 @@ __global__ void __launch_bounds__(kTileBlock) run_cell_kernel(const StepParams p
                                                               long long phase0, int hop0, int steps,
                                                               int tile_groups, int log2n, const SparseW sw)
 {
-    extern __shared__ float4 tile_smem[];   // Y twice: [2][n][tile_groups]
+    extern __shared__ float4 tile_smem[];   // Y twice: [2][n][tile_groups], then the column-mean addends
     const int n = (int)p.n;
     const int cells = n * tile_groups;
     const long long q_first = (long long)blockIdx.x * tile_groups;
@@ -281,13 +281,55 @@ __global__ void __launch_bounds__(kTileBlock) run_cell_kernel(const StepParams p
     int hop_log2 = hop0;        // k mod log2(n)
     float4* ycur = tile_smem;
     float4* ynext = tile_smem + cells;
+    float4* gsum = tile_smem + 2 * cells;   // [n / 4 + 2][tile_groups]: the fp32 addends of the column mean
     for (int t = 0; t < steps; ++t) {
         const uint32_t k = p.k + (uint32_t)t;
         const bool global = H > 0 && phase == 0;            // Algorithm 1's test mod(k + 1, H) = 0
-        const int mix = global ? (int)TILE_MIX_GLOBAL : topology;
+        const int mix = topology;
         if (own) ycur[c] = tile_finish<MODE>(p, x, b, i, q, k);
         __syncthreads();
-        if (own) x = tile_mix(ycur, i, g, n, tile_groups, mix, hop_log2, p.grid_cols, log2n, sw);
+        if (global) {
+            // The column mean, formed once per column group instead of once per cell: the first
+            // row of every group of four adds its group in fp32, (y0 + y1) + (y2 + y3), as
+            // tile_mix and the row-streaming kernel do; after a barrier every cell adds the
+            // group sums in fp64 in row order.  Same addends, same order, same result.
+            const int full = n >> 2, rest = n & 3;
+            if (own) {
+                if ((i & 3) == 0 && i + 4 <= n) {
+                    float4 a = ycur[c], b2 = ycur[(i + 2) * tile_groups + g];
+                    acc4(a, ycur[(i + 1) * tile_groups + g]);
+                    acc4(b2, ycur[(i + 3) * tile_groups + g]);
+                    acc4(a, b2);
+                    gsum[(i >> 2) * tile_groups + g] = a;
+                } else if (i == 4 * full) {            // the unfinished last group: one or two addends
+                    float4 a = ycur[c];
+                    if (rest >= 2) acc4(a, ycur[(i + 1) * tile_groups + g]);
+                    gsum[full * tile_groups + g] = a;
+                    if (rest == 3) gsum[(full + 1) * tile_groups + g] = ycur[(i + 2) * tile_groups + g];
+                }
+            }
+            __syncthreads();
+            if (own) {
+                const int addends = full + (rest >= 1 ? 1 : 0) + (rest == 3 ? 1 : 0);
+                double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+                for (int j = 0; j < addends; ++j) {
+                    const float4 v = gsum[j * tile_groups + g];
+                    s0 += (double)v.x;
+                    s1 += (double)v.y;
+                    s2 += (double)v.z;
+                    s3 += (double)v.w;
+                }
+                if ((n & (n - 1)) == 0) {   // 1/n is exact: the product equals the quotient
+                    const double inv = 1.0 / (double)n;
+                    x = make_float4((float)(s0 * inv), (float)(s1 * inv), (float)(s2 * inv), (float)(s3 * inv));
+                } else {
+                    const double dn = (double)n;
+                    x = make_float4((float)(s0 / dn), (float)(s1 / dn), (float)(s2 / dn), (float)(s3 / dn));
+                }
+            }
+        } else if (own) {
+            x = tile_mix(ycur, i, g, n, tile_groups, mix, hop_log2, p.grid_cols, log2n, sw);
+        }
         float4* const swap = ycur;
         ycur = ynext;
         ynext = swap;
@@ -384,7 +426,7 @@ cudaError_t launch_run_tile(const StepParams& p, int mode, bool vec, int topolog
         const unsigned grd = (unsigned)((p.Q + tile_groups - 1) / tile_groups);
         const long long cells = p.n * tile_groups;
         const int blk = (int)((cells + 31) / 32 * 32);
-        const size_t smem = (size_t)cells * 32;
+        const size_t smem = (size_t)cells * 32 + (size_t)(p.n / 4 + 2) * tile_groups * 16;
 #define GPGA_RUN_CELL(M, V) \
     run_cell_kernel<M, V><<<grd, blk, smem, s>>>(p, topology, H, phase0, hop0, steps, tile_groups, log2n, sw)
         if (vec) {

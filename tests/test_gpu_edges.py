@@ -264,6 +264,34 @@ def test_partly_overlapping_state_buffers_are_rejected():
     g.bind_raw(big.data_ptr(), big.data_ptr() + n * d * 4, data.data_ptr(), None, scratch.data_ptr(), scratch.numel())
 
 
+@pytest.mark.parametrize("topo,n,d,H,fused", [("exp", 16, 1_500_004, 8, True), ("ring", 32, 600_000, 5, True),
+                                              ("ring", 64, 300_000, 4, False)])
+def test_long_runs_with_few_nodes_take_the_multi_iteration_launch_at_any_size(topo, n, d, H, fused):
+    """Above 64 MB of state gpga_run still advances many iterations per launch when n <= 32 and the
+    run has at least 32 iterations (the on-chip arithmetic is then faster than streaming the state
+    from HBM every iteration); n = 64 keeps one launch per iteration.  Either way the result is
+    bit-identical to stepping, and within tolerance of the oracle on a slice of columns."""
+    X0, B = quadratic_inputs(n, d, 5 + n, x0="shared", x0_std=0.5)
+    assert 12 * n * d > 64 << 20
+    K = 40
+    g, _ = make_quadratic(n, d, topo, H, 0.05, 29, 0.1, X0, B)
+    g.run(K)
+    assert g.launch_count() == (1 if fused else K)
+    got = g.get_x().cpu().numpy().copy()
+    g2, _ = make_quadratic(n, d, topo, H, 0.05, 29, 0.1, X0, B)
+    for k in range(K):
+        g2.step(k)
+    assert np.array_equal(got, g2.get_x().cpu().numpy())
+    g3, _ = make_quadratic(n, d, topo, H, 0.05, 29, 0.1, X0, B)
+    g3.run(K - 1)                      # fewer than 32 left after the first call: falls back to stepping
+    g3.run(1)
+    assert np.array_equal(got, g3.get_x().cpu().numpy())
+    c0, w = (d // 2) // 4 * 4, 2048
+    p = o.Problem(TOPO[topo][1], H, 0.05, 29, sigma=0.1, data=np.ascontiguousarray(B[:, c0:c0 + w]), col0=c0)
+    ok, worst = close(got[:, c0:c0 + w], o.run(p, np.ascontiguousarray(X0[:, c0:c0 + w]), 0, K), TOL_RUN)
+    assert ok, worst
+
+
 def test_multi_iteration_launch_is_chunked_for_long_runs():
     n, d, K = 4, 256, 2500            # more than one launch worth of iterations
     X0, B = quadratic_inputs(n, d, 5)
