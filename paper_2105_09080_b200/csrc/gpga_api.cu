@@ -204,15 +204,15 @@ int32_t do_step(gpga_ctx* c, int64_t k, bool global, cudaStream_t s, bool after_
 // through many iterations on chip (launch_run_tile) with HBM touched once per launch; the time per
 // iteration is then set by the noise arithmetic, not by memory.  That path is taken
 //  - for a state small enough to sit in L2 (one launch per iteration would be launch-bound), and
-//  - for n <= 32 and runs of at least kFusedMinSteps iterations at any size: there the arithmetic
-//    bound (6.0-6.2e11 updates/s measured at n = 16, 32) is above what the row-streaming kernels
-//    reach from HBM (at most 5.5e11), and the one extra pass over the state is amortised.  At
-//    n = 64 the multi-iteration kernel runs at 4.8e11 (two-warp blocks, longer column sums) and
-//    the row-streaming kernels stay in use.
+//  - for n <= kFusedWideNodes and runs of at least kFusedMinSteps iterations at any size: there the
+//    arithmetic bound (6.0-6.9e11 updates/s measured for n = 8 ... 64, 5.3e11 at n = 128) is above
+//    what the row-streaming kernels reach from HBM (at most 5.5e11, 4.9-5.3e11 at 0.8 GB of
+//    state), and the one extra pass over the state is amortised.  At n = 256 the two are equal,
+//    and wider n would go through the several-cells-per-thread kernel, which is far slower.
 // A launch is kept to about half a second of work.
 constexpr int64_t kFusedStateBytes = 64ll << 20;
 constexpr int64_t kFusedSteps = 1024;
-constexpr int64_t kFusedWideNodes = 32, kFusedMinSteps = 32;
+constexpr int64_t kFusedWideNodes = 128, kFusedMinSteps = 32;
 constexpr double kFusedUpdatesPerLaunch = 2.75e11;
 
 int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)

@@ -282,6 +282,7 @@ __global__ void __launch_bounds__(kTileBlock) run_cell_kernel(const StepParams p
     float4* ycur = tile_smem;
     float4* ynext = tile_smem + cells;
     float4* gsum = tile_smem + 2 * cells;   // [n / 4 + 2][tile_groups]: the fp32 addends of the column mean
+    float4* gmean = gsum + (n / 4 + 2) * tile_groups;   // [tile_groups]: the column means
     for (int t = 0; t < steps; ++t) {
         const uint32_t k = p.k + (uint32_t)t;
         const bool global = H > 0 && phase == 0;            // Algorithm 1's test mod(k + 1, H) = 0
@@ -291,8 +292,9 @@ __global__ void __launch_bounds__(kTileBlock) run_cell_kernel(const StepParams p
         if (global) {
             // The column mean, formed once per column group instead of once per cell: the first
             // row of every group of four adds its group in fp32, (y0 + y1) + (y2 + y3), as
-            // tile_mix and the row-streaming kernel do; after a barrier every cell adds the
-            // group sums in fp64 in row order.  Same addends, same order, same result.
+            // tile_mix and the row-streaming kernel do; after a barrier one thread per column group
+            // adds the group sums in fp64 in row order and hands the mean to the column's cells.
+            // Same addends, same order, same result.
             const int full = n >> 2, rest = n & 3;
             if (own) {
                 if ((i & 3) == 0 && i + 4 <= n) {
@@ -309,24 +311,28 @@ __global__ void __launch_bounds__(kTileBlock) run_cell_kernel(const StepParams p
                 }
             }
             __syncthreads();
-            if (own) {
+            if (c < tile_groups && q_first + c < p.Q) {      // thread c: the mean of column group c
                 const int addends = full + (rest >= 1 ? 1 : 0) + (rest == 3 ? 1 : 0);
                 double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
                 for (int j = 0; j < addends; ++j) {
-                    const float4 v = gsum[j * tile_groups + g];
+                    const float4 v = gsum[j * tile_groups + c];
                     s0 += (double)v.x;
                     s1 += (double)v.y;
                     s2 += (double)v.z;
                     s3 += (double)v.w;
                 }
+                float4 m;
                 if ((n & (n - 1)) == 0) {   // 1/n is exact: the product equals the quotient
                     const double inv = 1.0 / (double)n;
-                    x = make_float4((float)(s0 * inv), (float)(s1 * inv), (float)(s2 * inv), (float)(s3 * inv));
+                    m = make_float4((float)(s0 * inv), (float)(s1 * inv), (float)(s2 * inv), (float)(s3 * inv));
                 } else {
                     const double dn = (double)n;
-                    x = make_float4((float)(s0 / dn), (float)(s1 / dn), (float)(s2 / dn), (float)(s3 / dn));
+                    m = make_float4((float)(s0 / dn), (float)(s1 / dn), (float)(s2 / dn), (float)(s3 / dn));
                 }
+                gmean[c] = m;
             }
+            __syncthreads();
+            if (own) x = gmean[g];
         } else if (own) {
             x = tile_mix(ycur, i, g, n, tile_groups, mix, hop_log2, p.grid_cols, log2n, sw);
         }
@@ -415,18 +421,19 @@ cudaError_t launch_run_tile(const StepParams& p, int mode, bool vec, int topolog
     const int hop0 = log2n > 0 ? (int)(p.k % (uint32_t)log2n) : 0;
     if (p.n <= kTileBlock) {
         // one cell per thread: the narrowest strip that fills whole warps (small blocks balance
-        // best over the SMs and wait least at their barrier), two warps' worth when there are more
-        // blocks than fit on the GPU at once
+        // best over the SMs and wait least at their barrier); up to four warps' worth when there
+        // are more blocks than fit on the GPU at once (the column means of a global-average
+        // iteration are formed by one thread per column group: wider strips fill that warp)
         long long tg = kTileBlock / p.n;
         for (long long t = 1; t * p.n <= kTileBlock; ++t)
             if ((t * p.n) % 32 == 0) { tg = t; break; }
-        if ((p.Q + tg - 1) / tg > 148 * 32 && 2 * tg * p.n <= kTileBlock / 2) tg *= 2;
+        while ((p.Q + tg - 1) / tg > 148 * 32 && 2 * tg * p.n <= kTileBlock / 2) tg *= 2;
         if (tg > p.Q) tg = p.Q;
         const int tile_groups = (int)tg;
         const unsigned grd = (unsigned)((p.Q + tile_groups - 1) / tile_groups);
         const long long cells = p.n * tile_groups;
         const int blk = (int)((cells + 31) / 32 * 32);
-        const size_t smem = (size_t)cells * 32 + (size_t)(p.n / 4 + 2) * tile_groups * 16;
+        const size_t smem = (size_t)cells * 32 + (size_t)(p.n / 4 + 3) * tile_groups * 16;
 #define GPGA_RUN_CELL(M, V) \
     run_cell_kernel<M, V><<<grd, blk, smem, s>>>(p, topology, H, phase0, hop0, steps, tile_groups, log2n, sw)
         if (vec) {

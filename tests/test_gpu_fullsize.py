@@ -173,7 +173,7 @@ def test_config_4_bert_large_sized():
     offs = _blocks(d, 48, np.random.default_rng(4))
     _run_case((xa, xb, b, scratch), n, d, "exp", H, gamma, sigma, K, pkg.GPGA_X0_ZERO, 1.0, 0.0,
               offs, [0, 1, 2, 3])
-    # a run of 32 iterations goes through the multi-iteration launch (n <= 32): 41.9 M one-warp strips
+    # a run of 32 iterations goes through the multi-iteration launch: 10.5 M strips of 8 column groups
     _run_case((xa, xb, b, scratch), n, d, "exp", H, gamma, sigma, 32, pkg.GPGA_X0_ZERO, 1.0, 0.0,
               offs[::2], [])
     del xa, xb, b
