@@ -8,6 +8,7 @@
 #include "../../include/gpga.h"
 #include "gpga_kernels.cuh"
 #include "gpga_logreg.cuh"
+#include "gpga_logrun.cuh"
 #include "gpga_loss.cuh"
 #include "gpga_tile.cuh"
 
@@ -75,9 +76,9 @@ int log2_floor(int64_t v) { int t = 0; while ((int64_t(1) << (t + 1)) <= v) ++t;
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
 
-// Scratch layout: [reduction partials | result double | G | gradient chunk partials]
+// Scratch layout: [reduction partials | result double | G | gradient chunk partials | published rows]
 struct ScratchLayout {
-    int64_t partials_off = 0, result_off = 0, G_off = 0, chunk_off = 0, total = 0;
+    int64_t partials_off = 0, result_off = 0, G_off = 0, chunk_off = 0, ytag_off = 0, ytag_bytes = 0, total = 0;
 };
 ScratchLayout scratch_layout(const gpga_ctx* c)
 {
@@ -91,6 +92,13 @@ ScratchLayout scratch_layout(const gpga_ctx* c)
         L.G_off = L.total;
         L.chunk_off = L.G_off + round_up(c->n * c->d * 4, 256);
         L.total = L.chunk_off + round_up(int64_t(logreg_chunks(c->batch)) * c->n * c->d * 4, 256);
+        // rows published by the many-iterations-per-launch kernel (narrow states only)
+        if (c->d <= 1024 && c->n <= 88 && (c->topology == GPGA_TOPO_RING || c->topology == GPGA_TOPO_EXP)) {
+            const int nbuf = 2 + logreg_run_buffers(c->topology == GPGA_TOPO_EXP, log2_floor(c->n));
+            L.ytag_off = L.total;
+            L.ytag_bytes = (int64_t)logreg_run_ytag_bytes((int)c->n, (int)c->d, nbuf);
+            L.total = L.ytag_off + round_up(L.ytag_bytes, 256);
+        }
     }
     return L;
 }
@@ -215,6 +223,55 @@ constexpr int64_t kFusedSteps = 1024;
 constexpr int64_t kFusedWideNodes = 128, kFusedMinSteps = 32;
 constexpr double kFusedUpdatesPerLaunch = 2.75e11;
 
+// Logistic objective, narrow state: many iterations per launch with x_i resident on chip (a pair of
+// blocks per node, see gpga_logrun.cu); bit-identical to single steps.  The rows the blocks publish
+// to one another have their own part of the scratch area; the stop word is the first word of its
+// reduction area (not in use between iterations).
+constexpr int64_t kLogRunMinSteps = 2;
+constexpr int64_t kLogRunSteps = 1 << 14;   // per launch: about a tenth of a second
+
+int32_t run_logistic_resident(gpga_ctx* c, int64_t K, cudaStream_t s)
+{
+    const ScratchLayout L = scratch_layout(c);
+    const int64_t k_end = c->k + K;
+    cudaError_t e;
+    if (!c->flag_cleared) {
+        e = cudaMemsetAsync(c->scratch + L.result_off + 8, 0, sizeof(int), s);
+        if (e != cudaSuccess) return cuda_fail(c, e, "error word clear");
+        c->flag_cleared = true;
+    }
+    while (c->k < k_end) {
+        const int64_t steps = (k_end - c->k < kLogRunSteps) ? k_end - c->k : kLogRunSteps;
+        LogRunParams p;
+        p.A = c->data;
+        p.y = c->labels;
+        p.x_in = c->x[c->cur];
+        p.x_out = c->x[c->cur ^ (int)(steps & 1)];
+        p.ldx = c->ld;
+        p.ytag = reinterpret_cast<unsigned long long*>(c->scratch + L.ytag_off);
+        p.nbuf = 2 + logreg_run_buffers(c->topology == GPGA_TOPO_EXP, log2_floor(c->n));
+        p.stop = reinterpret_cast<int*>(c->scratch + L.partials_off);
+        p.error_flag = reinterpret_cast<int*>(c->scratch + L.result_off + 8);
+        p.n = (int)c->n; p.d = (int)c->d; p.m = (int)c->m; p.batch = (int)c->batch;
+        p.k0 = (uint32_t)c->k;
+        p.steps = (int)steps;
+        p.topology = c->topology;
+        p.H = (int)c->H;
+        p.log2n = log2_floor(c->n);
+        p.gamma = c->gamma; p.l2 = c->l2;
+        p.keys = c->keys;
+        e = cudaMemsetAsync(p.stop, 0, sizeof(int), s);
+        if (e == cudaSuccess) e = cudaMemsetAsync(p.ytag, 0, (size_t)L.ytag_bytes, s);   // no tag of an earlier launch survives
+        if (e != cudaSuccess) return cuda_fail(c, e, "published-row buffers clear");
+        e = launch_logreg_run(p, s);
+        c->launches += 1;
+        if (e != cudaSuccess) return cuda_fail(c, e, "resident logistic launch");
+        c->cur ^= (int)(steps & 1);
+        c->k += steps;
+    }
+    return GPGA_OK;
+}
+
 int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)
 {
     const int64_t k_end = c->k + K;
@@ -226,6 +283,12 @@ int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)
     int64_t per_launch = (int64_t)(kFusedUpdatesPerLaunch / ((double)c->n * (double)c->d));
     if (per_launch > kFusedSteps) per_launch = kFusedSteps;
     if (per_launch < 16) per_launch = 16;
+    if (c->objective == GPGA_OBJ_LOGISTIC && K >= kLogRunMinSteps) {
+        bool ok = false;
+        const cudaError_t e = logreg_run_supported((int)c->n, (int)c->d, (int)c->batch, c->topology, c->H, &ok);
+        if (e != cudaSuccess) return cuda_fail(c, e, "occupancy query");
+        if (ok && scratch_layout(c).ytag_bytes > 0) return run_logistic_resident(c, K, s);
+    }
     if (!fused) {
         for (int64_t k = c->k; k < k_end; ++k) {
             // from the second iteration on, the launch before the gradient kernel is our own step kernel

@@ -103,6 +103,46 @@ __device__ __forceinline__ float4 normal4(uint32_t q, uint32_t i, uint32_t k, ui
     return make_float4(za.x, za.y, zb.x, zb.y);
 }
 
+// Row index of the t-th mini-batch draw of node i at iteration k (drawn with replacement):
+// word t & 3 of the generator call with counter (t >> 2, i, k, stream 4), reduced mod m.
+__device__ __forceinline__ uint32_t batch_row(uint32_t t, uint32_t i, uint32_t k, uint32_t m,
+                                              const PhiloxKeys& ks)
+{
+    const uint4 w = philox4x32_10(t >> 2, i, k, 4u, ks);
+    const uint32_t sel = t & 3u;
+    const uint32_t word = sel == 0 ? w.x : sel == 1 ? w.y : sel == 2 ? w.z : w.w;
+    return word % m;
+}
+
+__device__ __forceinline__ float warp_sum_f(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// ---- packed pairs of fp32 (two IEEE fused multiply-adds per instruction on sm_100) ----------
+// Each half is rounded exactly as a scalar fmaf of the same operands.
+typedef unsigned long long f32x2_t;
+__device__ __forceinline__ f32x2_t pack2(float lo, float hi)
+{
+    f32x2_t v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+    return v;
+}
+__device__ __forceinline__ float2 unpack2(f32x2_t v)
+{
+    float2 r;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(r.x), "=f"(r.y) : "l"(v));
+    return r;
+}
+__device__ __forceinline__ f32x2_t fma2(f32x2_t a, f32x2_t b, f32x2_t c)
+{
+    f32x2_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
 // ---- streaming (read-once / write-once) 128-bit accesses -------------------
 __device__ __forceinline__ float4 ld_stream4(const float* p)
 {

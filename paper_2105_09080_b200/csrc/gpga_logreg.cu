@@ -14,22 +14,6 @@ namespace gpga {
 
 constexpr int kLrBlock = 256;
 
-__device__ __forceinline__ uint32_t batch_row(uint32_t t, uint32_t i, uint32_t k, uint32_t m,
-                                              const PhiloxKeys& ks)
-{
-    const uint4 w = philox4x32_10(t >> 2, i, k, 4u, ks);
-    const uint32_t sel = t & 3u;
-    const uint32_t word = sel == 0 ? w.x : sel == 1 ? w.y : sel == 2 ? w.z : w.w;
-    return word % m;
-}
-
-__device__ __forceinline__ float warp_sum_f(float v)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-    return v;
-}
-
 // partial[c][i][:] = sum over the chunk's rows of s_r a_r,  s_r = -y_r / (1 + exp(y_r z_r)).
 __global__ void __launch_bounds__(kLrBlock) logreg_partial_kernel(const LogregParams p)
 {

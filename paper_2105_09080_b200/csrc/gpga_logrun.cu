@@ -1,0 +1,607 @@
+// Many Gossip-PGA iterations of the logistic objective in ONE launch (Algorithm 1 with the
+// Section 5.1 loss), for states narrow enough that an iteration per launch is bound by the
+// launch-to-launch dependency chain rather than by memory.
+//
+// A pair of blocks (one thread-block cluster of two) owns node i for the whole run:
+//  - x_i stays on chip (every warp holds it in registers);
+//  - the batch rows of A stream into per-warp shared-memory buffers by bulk asynchronous
+//    copies, the copies of the next iteration's rows (their indices depend only on the seed,
+//    the node and the iteration) already in flight while this iteration is reduced and mixed,
+//    and every row asked into L2 more than an iteration before it is copied;
+//  - the per-warp gradient sums are added in shared memory; the chunk sums go to the block that
+//    finishes the column group by asynchronous stores into its shared memory, which count
+//    themselves off on an mbarrier there (no cluster-wide barrier in the loop); each block
+//    finishes one half of the columns: gradient, local update y_i = x_i - gamma g_i;
+//  - y_i is published to global memory as 64-bit words (value, iteration tag), each written and
+//    read whole, so a reader needs no flag and no fence: it reads the rows of its neighbours (ring,
+//    one-peer exponential graph) or of all nodes (global average) until the tags are this
+//    iteration's, forms its half of x_i^(k+1) and sends it to both blocks of the pair, again by
+//    counted asynchronous stores.
+// Every sum is formed in the order the one-iteration kernels use (rows of a warp in order,
+// eight warps of a chunk in order, chunks in order; ring (up + self) + down; global mean by
+// groups of four rows in fp32, groups in fp64), so a run is bit-identical to the same number of
+// single steps.
+//
+// Buffers of published rows.  Gossip iteration `it` of the launch uses buffer it % G, global-average
+// iterations alternate between two buffers of their own.  A block overwrites what it published G
+// gossip iterations (two global averages) earlier; every reader is done with that by then:
+// on the ring a node publishes iteration it only after its neighbours' rows of it - 1, which they
+// publish after reading its row of it - 2 (G = 2); on the one-peer exponential graph a node at
+// iteration it has, through log2 n hops, waited for every node's row of it - log2 n
+// (G = log2 n + 2); a global average waits for every node, and the one before it was read
+// before those rows were published.
+//
+// Waiting: a block only waits for data of the SAME iteration, which its owner publishes before it
+// waits for anything of that iteration, so the waits cannot form a cycle as long as all blocks
+// are resident (checked before the launch; the launch is cooperative where the driver allows).
+// Every wait is bounded; one that gives up raises the error word and a stop word that ends the
+// other blocks' waits.  Both blocks of a pair meet at a cluster barrier before they exit, so no
+// asynchronous store is ever aimed at a block that has left.
+#include <cooperative_groups.h>
+
+#include "../../include/gpga.h"
+#include "gpga_launch.cuh"
+#include "gpga_logrun.cuh"
+#include "gpga_tma.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace gpga {
+
+constexpr int kRunThreads = 512;
+constexpr int kRunWarps = kRunThreads / 32;   // 16 = two chunks of eight row-warps per block
+constexpr int kRunMaxD = 1024;
+constexpr int kRunGroups = kRunMaxD / 4 / 32;   // float4 per lane
+constexpr int kRunMaxSlots = 4;                 // row buffers per warp
+constexpr int kRunChunkRows = 32, kRunChunkWarps = 8;   // the batch is cut as by the one-iteration kernel
+constexpr int kRunMaxChunks = 2 * kRunWarps / kRunChunkWarps;   // 4: batch <= 128
+constexpr int kRunMaxNodes = 88;
+constexpr int kRunSmemLimit = 226 * 1024;       // dynamic; the static arrays take under 1 KB
+constexpr uint32_t kRunCopyTries = 1u << 22;    // polls of an mbarrier before a copy is given up
+constexpr uint32_t kRunPollTries = 1u << 21;    // reads of a published group (about a microsecond each)
+
+__device__ __forceinline__ int ld_relaxed_gpu(const int* p)
+{
+    int v;
+    asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_gpu(int* p, int v)
+{
+    asm volatile("st.relaxed.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// ---- published rows: (value, tag) words -------------------------------------------------------
+// A group of four columns is four 64-bit words, low half the fp32 value, high half the tag.  Each
+// word is written and read by one 64-bit access, so a word whose tag matches carries its value.
+__device__ __forceinline__ void publish4(unsigned long long* dst, float4 v, uint32_t tag)
+{
+    const unsigned long long t = (unsigned long long)tag << 32;
+    const unsigned long long w0 = t | __float_as_uint(v.x), w1 = t | __float_as_uint(v.y);
+    const unsigned long long w2 = t | __float_as_uint(v.z), w3 = t | __float_as_uint(v.w);
+    asm volatile("st.relaxed.gpu.global.v2.b64 [%0], {%1, %2};" ::"l"(dst), "l"(w0), "l"(w1) : "memory");
+    asm volatile("st.relaxed.gpu.global.v2.b64 [%0], {%1, %2};" ::"l"(dst + 2), "l"(w2), "l"(w3) : "memory");
+}
+// Reads the group until all four tags equal `tag`.  Gives up after kRunPollTries reads, or as soon
+// as *stop is set; returns false then (v is not meaningful).
+__device__ __forceinline__ bool read4(const unsigned long long* src, uint32_t tag, const int* stop, float4* v)
+{
+    for (uint32_t t = 0; t < kRunPollTries; ++t) {
+        unsigned long long w0, w1, w2, w3;
+        asm volatile("ld.relaxed.gpu.global.v2.b64 {%0, %1}, [%2];" : "=l"(w0), "=l"(w1) : "l"(src) : "memory");
+        asm volatile("ld.relaxed.gpu.global.v2.b64 {%0, %1}, [%2];" : "=l"(w2), "=l"(w3) : "l"(src + 2) : "memory");
+        const uint32_t t0 = (uint32_t)(w0 >> 32), t1 = (uint32_t)(w1 >> 32), t2 = (uint32_t)(w2 >> 32),
+                       t3 = (uint32_t)(w3 >> 32);
+        if (t0 == tag && t1 == tag && t2 == tag && t3 == tag) {
+            *v = make_float4(__uint_as_float((uint32_t)w0), __uint_as_float((uint32_t)w1),
+                             __uint_as_float((uint32_t)w2), __uint_as_float((uint32_t)w3));
+            return true;
+        }
+        if ((t & 63u) == 63u && ld_relaxed_gpu(stop) != 0) return false;
+    }
+    return false;
+}
+
+// One read of the group, no retry: true if all four tags equal `tag`.
+__device__ __forceinline__ bool try4(const unsigned long long* src, uint32_t tag, float4* v)
+{
+    unsigned long long w0, w1, w2, w3;
+    asm volatile("ld.relaxed.gpu.global.v2.b64 {%0, %1}, [%2];" : "=l"(w0), "=l"(w1) : "l"(src) : "memory");
+    asm volatile("ld.relaxed.gpu.global.v2.b64 {%0, %1}, [%2];" : "=l"(w2), "=l"(w3) : "l"(src + 2) : "memory");
+    *v = make_float4(__uint_as_float((uint32_t)w0), __uint_as_float((uint32_t)w1), __uint_as_float((uint32_t)w2),
+                     __uint_as_float((uint32_t)w3));
+    return (uint32_t)(w0 >> 32) == tag && (uint32_t)(w1 >> 32) == tag && (uint32_t)(w2 >> 32) == tag &&
+           (uint32_t)(w3 >> 32) == tag;
+}
+// Polls one word until its tag equals `tag` (bounded, ends on the stop word).
+__device__ __forceinline__ bool wait_tag(const unsigned long long* word, uint32_t tag, const int* stop)
+{
+    for (uint32_t t = 0; t < kRunPollTries; ++t) {
+        unsigned long long w;
+        asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];" : "=l"(w) : "l"(word) : "memory");
+        if ((uint32_t)(w >> 32) == tag) return true;
+        if ((t & 63u) == 63u && ld_relaxed_gpu(stop) != 0) return false;
+    }
+    return false;
+}
+// The same for a whole warp reading 32 adjacent groups of one row, all written by one warp of the
+// publisher with the same two store instructions: lane 0 alone polls the last word of the segment
+// (`gate`), then every active lane reads and checks its own group (and keeps reading in the rare
+// case that its words are not there yet).  One poller per warp keeps the polling traffic small.
+// The whole warp must call.
+__device__ __forceinline__ bool read4_warp(bool active, const unsigned long long* src, const unsigned long long* gate,
+                                           uint32_t tag, const int* stop, float4* v)
+{
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) {
+        ok = 0;
+        for (uint32_t t = 0; t < kRunPollTries; ++t) {
+            unsigned long long w;
+            asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];" : "=l"(w) : "l"(gate) : "memory");
+            if ((uint32_t)(w >> 32) == tag) {
+                ok = 1;
+                break;
+            }
+            if ((t & 63u) == 63u && ld_relaxed_gpu(stop) != 0) break;
+        }
+    }
+    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+    if (!ok) return false;
+    return active ? read4(src, tag, stop, v) : true;
+}
+
+// ---- counted asynchronous stores into a block of the pair (distributed shared memory) ----------
+// Address of a shared-memory location of this block as seen in block `rank` of the cluster.
+__device__ __forceinline__ uint32_t cluster_addr(const void* smem_ptr, uint32_t rank)
+{
+    uint32_t a;
+    asm("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(smem_u32(smem_ptr)), "r"(rank));
+    return a;
+}
+// 16 bytes to `dst`; on arrival they count as 16 bytes of the current phase of the barrier at `bar`
+// (both cluster addresses of the same block).
+__device__ __forceinline__ void send4(uint32_t dst, uint32_t bar, float4 v)
+{
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::
+                     "r"(dst),
+                 "r"(__float_as_uint(v.x)), "r"(__float_as_uint(v.y)), "r"(__float_as_uint(v.z)),
+                 "r"(__float_as_uint(v.w)), "r"(bar)
+                 : "memory");
+}
+// Waits for the phase of `bar` with the given parity; gives up after kRunCopyTries polls, or as soon
+// as *stop is set.
+__device__ __forceinline__ bool wait_phase(uint64_t* bar, uint32_t parity, const int* stop)
+{
+    for (uint32_t t = 0; t < kRunCopyTries; ++t) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((t & 255u) == 255u && ld_relaxed_gpu(stop) != 0) return false;
+    }
+    return false;
+}
+
+__device__ __forceinline__ void add4_to(float4& s, const float4 v)
+{
+    s.x += v.x;
+    s.y += v.y;
+    s.z += v.z;
+    s.w += v.w;
+}
+
+// Shared-memory plan for row width d: row buffers [16 warps][slots][d], the reduction area, the
+// chunk sums of this block's half [4][h0] and x_i [d].
+struct RunSmem {
+    int slots;
+    int red_f4;      // float4 entries of the reduction area
+    size_t bytes;
+};
+__host__ __device__ inline RunSmem run_smem_plan(int d)
+{
+    const int d4 = d >> 2, h0 = (d4 + 1) >> 1;
+    RunSmem s;
+    s.red_f4 = kRunWarps * d4 > kRunThreads ? kRunWarps * d4 : kRunThreads;   // row sums; (group, row) items of a column mean
+    const size_t fixed = ((size_t)s.red_f4 + (size_t)kRunMaxChunks * h0 + (size_t)d4) * sizeof(float4);
+    const size_t per_slot = (size_t)kRunWarps * d * sizeof(float);
+    long long slots = ((long long)kRunSmemLimit - (long long)fixed) / (long long)per_slot;
+    if (slots > kRunMaxSlots) slots = kRunMaxSlots;
+    s.slots = (int)slots;
+    s.bytes = fixed + (size_t)(slots > 0 ? slots : 0) * per_slot;
+    return s;
+}
+
+// FULL: d == kRunMaxD, every lane holds kRunGroups whole groups (no guards in the row loop).
+template <bool FULL>
+__global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRunParams p, int slots, int red_f4)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t bars[kRunWarps * kRunMaxSlots];
+    __shared__ __align__(8) uint64_t sums_bar, x_bar;   // chunk sums of this block's half; x_i^(k+1)
+    cg::cluster_group cluster = cg::this_cluster();
+    const int r = (int)cluster.block_rank();   // which half of the columns this block finishes
+    const int i = (int)(blockIdx.x >> 1);      // node
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n = p.n, d = p.d, d4 = d >> 2;
+    const int h0 = (d4 + 1) >> 1;              // block 0 finishes groups [0, h0), block 1 [h0, d4)
+    const int g_lo = r ? h0 : 0;
+    const int owned = r ? d4 - h0 : h0;
+    const int chunks = (p.batch + kRunChunkRows - 1) / kRunChunkRows;
+    const float inv_batch = 1.0f / (float)p.batch;
+    const int gossip_bufs = p.nbuf - 2;        // then two buffers for global-average iterations
+    const size_t buf_words = (size_t)n * d;
+
+    float* slot_base = reinterpret_cast<float*>(smem_raw);
+    float4* red = reinterpret_cast<float4*>(slot_base + (size_t)kRunWarps * slots * d);
+    float4* pbuf = red + red_f4;                    // [chunk][h0]: chunk sums of this block's groups
+    float4* xnew = pbuf + kRunMaxChunks * h0;       // [d4]: x_i^(k+1), both halves
+    // the same locations in both blocks of the pair, as cluster addresses
+    const uint32_t pbuf_at[2] = {cluster_addr(pbuf, 0), cluster_addr(pbuf, 1)};
+    const uint32_t xnew_at[2] = {cluster_addr(xnew, 0), cluster_addr(xnew, 1)};
+    const uint32_t sums_bar_at[2] = {cluster_addr(&sums_bar, 0), cluster_addr(&sums_bar, 1)};
+    const uint32_t x_bar_at[2] = {cluster_addr(&x_bar, 0), cluster_addr(&x_bar, 1)};
+    const int* stop = p.stop;
+
+    // ---- this warp's rows: warp (chunk c, w) of the one-iteration kernel ----------------------
+    const int pair = r * kRunWarps + warp;
+    const int c = pair / kRunChunkWarps, w = pair % kRunChunkWarps;
+    const int nrows_c = c < chunks ? min(kRunChunkRows, p.batch - c * kRunChunkRows) : 0;
+    const int my_rows = w < nrows_c ? (nrows_c - w + kRunChunkWarps - 1) / kRunChunkWarps : 0;
+    const int depth = min(slots, my_rows);   // copies this warp keeps in flight
+    const uint32_t t_mine = (uint32_t)(c * kRunChunkRows + w + lane * kRunChunkWarps);   // lane rho <-> row rho
+    const float* A = p.A + (long long)i * p.m * d;
+    const float* labels = p.y + (long long)i * p.m;
+    float* mine = slot_base + (size_t)warp * slots * d;
+    uint64_t* bar = bars + warp * kRunMaxSlots;
+    const uint32_t row_bytes = (uint32_t)d * 4u;
+
+    uint32_t idx_cur = 0u, idx_nxt = 0u;   // lane rho: row rho of this / the next iteration
+    float y_cur = 0.f, y_nxt = 0.f;
+    if (lane < my_rows) {
+        idx_cur = batch_row(t_mine, (uint32_t)i, p.k0, (uint32_t)p.m, p.keys);
+        y_cur = labels[idx_cur];
+        if (lane >= slots) bulk_prefetch_l2(A + (long long)idx_cur * d, row_bytes);   // not copied yet
+        if (p.steps > 1) {
+            idx_nxt = batch_row(t_mine, (uint32_t)i, p.k0 + 1u, (uint32_t)p.m, p.keys);
+            y_nxt = labels[idx_nxt];
+            bulk_prefetch_l2(A + (long long)idx_nxt * d, row_bytes);
+        }
+    }
+    if (lane == 0) {
+        for (int s = 0; s < slots; ++s) mbar_init(&bar[s], 1);
+        if (warp == 0) {
+            mbar_init(&sums_bar, 1);
+            mbar_init(&x_bar, 1);
+        }
+        mbar_init_fence();
+    }
+    __syncwarp();
+    // Row rho of local iteration it is position it * my_rows + rho of this warp's stream; position q
+    // goes through buffer q % depth, phase (q / depth) & 1 of its barrier.
+    int issued = 0, consumed = 0;
+    int issue_slot = 0, wait_slot = 0;
+    uint32_t wait_parity = 0u;
+    auto issue = [&](uint32_t idx) {   // whole warp calls; lane 0 starts the copy
+        if (lane == 0) {
+            mbar_arrive_expect_tx(&bar[issue_slot], row_bytes);
+            bulk_copy_g2s(mine + (size_t)issue_slot * d, A + (long long)idx * d, row_bytes, &bar[issue_slot]);
+        }
+        issue_slot = (issue_slot + 1 == depth) ? 0 : issue_slot + 1;
+        ++issued;
+    };
+    for (int rho = 0; rho < depth; ++rho) issue(__shfl_sync(0xFFFFFFFFu, idx_cur, rho));
+    // the rows of the iteration after the next: indices, labels, and the rows asked into L2
+    auto roll = [&](int it) {
+        idx_cur = idx_nxt;
+        y_cur = y_nxt;
+        if (it + 2 < p.steps && lane < my_rows) {
+            idx_nxt = batch_row(t_mine, (uint32_t)i, p.k0 + (uint32_t)(it + 2), (uint32_t)p.m, p.keys);
+            y_nxt = labels[idx_nxt];
+        }
+    };
+
+    ulonglong2 xr[kRunGroups];   // x_i, group lane + 32 j, as two packed pairs
+    const ulonglong2 zero2 = make_ulonglong2(0ull, 0ull);
+    {
+        const ulonglong2* x4 = reinterpret_cast<const ulonglong2*>(p.x_in + (long long)i * p.ldx);
+#pragma unroll
+        for (int j = 0; j < kRunGroups; ++j) {
+            const int g = lane + 32 * j;
+            xr[j] = (FULL || g < d4) ? x4[g] : zero2;
+        }
+    }
+    const bool finisher = tid < owned;   // finishes group g_lo + tid
+    float4 xo = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (finisher) xo = reinterpret_cast<const float4*>(p.x_in + (long long)i * p.ldx)[g_lo + tid];
+    cluster.sync();   // the partner's barriers are set up before anything is sent to them
+
+    bool failed = false;
+    int it = 0;
+    for (; it < p.steps; ++it) {
+        const long long k = (long long)p.k0 + it;
+        const uint32_t tag = (uint32_t)it + 1u;
+        const uint32_t phase = (uint32_t)it & 1u;
+        if (tid == 0) {   // what this iteration will send to this block
+            mbar_arrive_expect_tx(&sums_bar, (uint32_t)(chunks * owned) * 16u);
+            mbar_arrive_expect_tx(&x_bar, (uint32_t)d4 * 16u);
+        }
+        // ---- gradient sums of this warp's rows ----------------------------------------------------
+        ulonglong2 acc[kRunGroups];
+#pragma unroll
+        for (int j = 0; j < kRunGroups; ++j) acc[j] = zero2;
+        for (int rho = 0; rho < my_rows; ++rho) {
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&bar[wait_slot], wait_parity, kRunCopyTries))) {
+                failed = true;
+                break;
+            }
+            const ulonglong2* a4 = reinterpret_cast<const ulonglong2*>(mine + (size_t)wait_slot * d);
+            ulonglong2 a[kRunGroups];
+            f32x2_t z01 = 0ull, z23 = 0ull;   // the four running sums z0 .. z3 of the scalar form
+#pragma unroll
+            for (int j = 0; j < kRunGroups; ++j) {
+                const int g = lane + 32 * j;
+                a[j] = (FULL || g < d4) ? a4[g] : zero2;
+                z01 = fma2(a[j].x, xr[j].x, z01);
+                z23 = fma2(a[j].y, xr[j].y, z23);
+            }
+            const float2 za = unpack2(z01), zb = unpack2(z23);
+            const float z = warp_sum_f((za.x + za.y) + (zb.x + zb.y));   // every lane holds the sum
+            ++consumed;
+            if (++wait_slot == depth) {
+                wait_slot = 0;
+                wait_parity ^= 1u;
+            }
+            // the sum needed every lane's loads, so the buffer is free: start the copy of the row
+            // `depth` positions ahead (this iteration's, or the next one's) into it
+            const int ahead = rho + depth;
+            if (ahead < my_rows)
+                issue(__shfl_sync(0xFFFFFFFFu, idx_cur, ahead));
+            else if (it + 1 < p.steps)
+                issue(__shfl_sync(0xFFFFFFFFu, idx_nxt, ahead - my_rows));
+            // the rows of the next iteration that no buffer is free for yet: ask them into L2 now, one
+            // per row step (a burst of such requests is dropped more easily than a trickle)
+            if (rho + depth < my_rows && it + 1 < p.steps) {
+                const uint32_t later = __shfl_sync(0xFFFFFFFFu, idx_nxt, rho + depth);
+                if (lane == 0) bulk_prefetch_l2(A + (long long)later * d, row_bytes);
+            }
+            const float yr = __shfl_sync(0xFFFFFFFFu, y_cur, rho);
+            const float sc = -yr / (1.0f + expf(yr * z));
+            const f32x2_t sc2 = pack2(sc, sc);
+#pragma unroll
+            for (int j = 0; j < kRunGroups; ++j) {
+                acc[j].x = fma2(sc2, a[j].x, acc[j].x);
+                acc[j].y = fma2(sc2, a[j].y, acc[j].y);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kRunGroups; ++j) {
+            const int g = lane + 32 * j;
+            if (FULL || g < d4) reinterpret_cast<ulonglong2*>(red)[warp * d4 + g] = acc[j];
+        }
+        __syncthreads();
+        // ---- chunk sums (eight warps in order), sent to the block that finishes the group ---------
+        {
+            const int cl = tid >> 8, g = tid & 255;
+            const int cc = 2 * r + cl;
+            if (g < d4 && cc < chunks) {
+                const float4* src = red + (size_t)(cl * kRunChunkWarps) * d4 + g;
+                float4 sum = src[0];
+#pragma unroll
+                for (int ww = 1; ww < kRunChunkWarps; ++ww) add4_to(sum, src[(size_t)ww * d4]);
+                const int to = g >= h0 ? 1 : 0;
+                send4(pbuf_at[to] + (uint32_t)(cc * h0 + (g - (to ? h0 : 0))) * 16u, sums_bar_at[to], sum);
+            }
+        }
+        const bool finisher_warp = warp * 32 < owned;
+        if (!finisher_warp) roll(it);   // off the path that the next iteration waits for
+        // ---- gradient, local update, publication of this block's half of y_i ----------------------
+        const bool glob = p.H > 0 && ((k + 1) % p.H) == 0;
+        const int buf = glob ? gossip_bufs + (int)(((k + 1) / p.H) & 1) : it % gossip_bufs;
+        unsigned long long* ybuf = p.ytag + (size_t)buf * buf_words;
+        float4 yv = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (finisher) {
+            if (!wait_phase(&sums_bar, phase, stop)) failed = true;
+            float4 gs = pbuf[tid];
+            for (int cc = 1; cc < chunks; ++cc) add4_to(gs, pbuf[cc * h0 + tid]);
+            const float4 gr = make_float4(fmaf(gs.x, inv_batch, p.l2 * xo.x), fmaf(gs.y, inv_batch, p.l2 * xo.y),
+                                          fmaf(gs.z, inv_batch, p.l2 * xo.z), fmaf(gs.w, inv_batch, p.l2 * xo.w));
+            yv = make_float4(fmaf(-p.gamma, gr.x, xo.x), fmaf(-p.gamma, gr.y, xo.y), fmaf(-p.gamma, gr.z, xo.z),
+                             fmaf(-p.gamma, gr.w, xo.w));
+            if (!failed) publish4(ybuf + (size_t)i * d + 4 * (g_lo + tid), yv, tag);
+        }
+        // ---- mix ------------------------------------------------------------------------------------
+        float4 xp = yv;
+        if (glob) {
+            // Column mean in two hops.  The column groups of this half are dealt out over the nodes:
+            // block (i, r) takes local groups i, i + n, ...; it reads those groups of every node's row,
+            // forms their means exactly as the one-iteration kernels do (rows added in fp32 in groups
+            // of four, (y0 + y1) + (y2 + y3), the group sums in fp64 in row order) and publishes them;
+            // then every block reads the means of its half.  A block reads n * (groups / n) + groups
+            // words instead of n * groups.
+            const int mine_cnt = i < owned ? (owned - i + n - 1) / n : 0;   // groups this block averages
+            unsigned long long* means = p.ytag + (size_t)p.nbuf * buf_words + (size_t)(buf - gossip_bufs) * d;
+            __syncthreads();   // the reduction area is free: every chunk sum has been read out of it
+            if (tid < mine_cnt * n) {
+                const int j = tid / n, row = tid - j * n;
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (!read4(ybuf + (size_t)row * d + 4 * (g_lo + i + j * n), tag, stop, &v)) failed = true;
+                red[tid] = v;   // [j][row]
+            }
+            __syncthreads();
+            if (tid < mine_cnt) {
+                const float4* col = red + tid * n;
+                double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+                int q = 0;
+                for (; q + 4 <= n; q += 4) {
+                    float4 a = col[q], b = col[q + 2];
+                    add4_to(a, col[q + 1]);
+                    add4_to(b, col[q + 3]);
+                    add4_to(a, b);
+                    s0 += (double)a.x;
+                    s1 += (double)a.y;
+                    s2 += (double)a.z;
+                    s3 += (double)a.w;
+                }
+                const int rest = n - q;
+                if (rest >= 1) {
+                    float4 a = col[q];
+                    if (rest >= 2) add4_to(a, col[q + 1]);
+                    s0 += (double)a.x;
+                    s1 += (double)a.y;
+                    s2 += (double)a.z;
+                    s3 += (double)a.w;
+                }
+                if (rest == 3) {
+                    const float4 b = col[q + 2];
+                    s0 += (double)b.x;
+                    s1 += (double)b.y;
+                    s2 += (double)b.z;
+                    s3 += (double)b.w;
+                }
+                float4 mean;
+                if ((n & (n - 1)) == 0) {   // 1/n is exact: the product equals the quotient
+                    const double inv = 1.0 / (double)n;
+                    mean = make_float4((float)(s0 * inv), (float)(s1 * inv), (float)(s2 * inv), (float)(s3 * inv));
+                } else {
+                    const double dn_ = (double)n;
+                    mean = make_float4((float)(s0 / dn_), (float)(s1 / dn_), (float)(s2 / dn_), (float)(s3 / dn_));
+                }
+                publish4(means + 4 * (g_lo + i + tid * n), mean, tag);
+            }
+            if (finisher && !read4(means + 4 * (g_lo + tid), tag, stop, &xp)) failed = true;
+        } else if (finisher_warp) {
+            const int seg_last = min(warp * 32 + 31, owned - 1);
+            const unsigned long long* col = ybuf + 4 * (g_lo + min(tid, owned - 1));
+            const unsigned long long* gate = ybuf + 4 * (g_lo + seg_last) + 3;
+            if (p.topology == GPGA_TOPO_RING) {
+                const int up = (i == 0) ? n - 1 : i - 1, dn = (i == n - 1) ? 0 : i + 1;
+                float4 yu = yv, yd = yv;
+                if (lane < 2 && !wait_tag(gate + (size_t)(lane ? dn : up) * d, tag, stop)) failed = true;
+                __syncwarp();
+                if (finisher && !failed) {
+                    const bool ok_u = try4(col + (size_t)up * d, tag, &yu), ok_d = try4(col + (size_t)dn * d, tag, &yd);
+                    if (!ok_u && !read4(col + (size_t)up * d, tag, stop, &yu)) failed = true;
+                    if (!ok_d && !read4(col + (size_t)dn * d, tag, stop, &yd)) failed = true;
+                }
+                const float third = 0.333333343f;
+                xp = make_float4((yu.x + yv.x + yd.x) * third, (yu.y + yv.y + yd.y) * third,
+                                 (yu.z + yv.z + yd.z) * third, (yu.w + yv.w + yd.w) * third);
+            } else {
+                const int hop_log2 = p.log2n > 0 ? (int)(k % p.log2n) : 0;
+                const int peer = (i + (1 << hop_log2)) & (n - 1);
+                float4 yp = yv;
+                if (!read4_warp(finisher, col + (size_t)peer * d, gate + (size_t)peer * d, tag, stop, &yp)) failed = true;
+                xp = make_float4((yv.x + yp.x) * 0.5f, (yv.y + yp.y) * 0.5f, (yv.z + yp.z) * 0.5f,
+                                 (yv.w + yp.w) * 0.5f);
+            }
+        }
+        // ---- x_i^(k+1) to both blocks of the pair ---------------------------------------------------
+        if (finisher && !failed) {
+            const uint32_t off = (uint32_t)(g_lo + tid) * 16u;
+            send4(xnew_at[0] + off, x_bar_at[0], xp);
+            send4(xnew_at[1] + off, x_bar_at[1], xp);
+            if (it == p.steps - 1) reinterpret_cast<float4*>(p.x_out + (long long)i * p.ldx)[g_lo + tid] = xp;
+        }
+        if (finisher_warp) roll(it);
+        if (!failed && !wait_phase(&x_bar, phase, stop)) failed = true;
+        if (failed) {   // tell everyone; the partner's and the other nodes' waits end on the stop word
+            st_relaxed_gpu(p.stop, 1);
+            if (p.error_flag) atomicExch(p.error_flag, 1);
+        }
+        if (__syncthreads_or(failed)) break;
+#pragma unroll
+        for (int j = 0; j < kRunGroups; ++j) {
+            const int g = lane + 32 * j;
+            if (FULL || g < d4) xr[j] = reinterpret_cast<const ulonglong2*>(xnew)[g];
+        }
+        if (finisher) xo = xnew[g_lo + tid];
+    }
+    // Copies still in flight target this block's shared memory: give each a bounded chance to land
+    // (none is in flight after a run that went through).
+    for (int q = consumed; q < issued; ++q)
+        mbar_wait_bounded(&bar[q % depth], (uint32_t)(q / depth) & 1u, kRunCopyTries);
+    cluster.sync();   // neither block leaves while the other may still send to it
+}
+
+namespace {
+
+cudaError_t run_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attrs, int n, size_t smem, cudaStream_t s,
+                       bool cooperative)
+{
+    *cfg = cudaLaunchConfig_t{};
+    cfg->gridDim = dim3((unsigned)(2 * n));
+    cfg->blockDim = dim3(kRunThreads);
+    cfg->dynamicSmemBytes = smem;
+    cfg->stream = s;
+    attrs[0].id = cudaLaunchAttributeClusterDimension;
+    attrs[0].val.clusterDim.x = 2;
+    attrs[0].val.clusterDim.y = 1;
+    attrs[0].val.clusterDim.z = 1;
+    attrs[1].id = cudaLaunchAttributeCooperative;
+    attrs[1].val.cooperative = 1;
+    cfg->attrs = attrs;
+    cfg->numAttrs = cooperative ? 2 : 1;
+    static unsigned long long limit_set = 0, limit_set_full = 0;
+    const cudaError_t e = ensure_smem_limit(logreg_run_kernel<false>, kRunSmemLimit, limit_set);
+    return e != cudaSuccess ? e : ensure_smem_limit(logreg_run_kernel<true>, kRunSmemLimit, limit_set_full);
+}
+
+}  // namespace
+
+cudaError_t logreg_run_supported(int n, int d, int batch, int topology, long long H, bool* ok)
+{
+    *ok = false;
+    if (topology != GPGA_TOPO_RING && topology != GPGA_TOPO_EXP) return cudaSuccess;
+    if (d < 4 || d > kRunMaxD || (d & 3) != 0 || batch < 1 || batch > kRunChunkRows * kRunMaxChunks) return cudaSuccess;
+    if (n < 1 || n > kRunMaxNodes || H < 0 || H >= (1ll << 31)) return cudaSuccess;
+    const RunSmem plan = run_smem_plan(d);
+    if (plan.slots < 1) return cudaSuccess;
+    // all 2 n blocks must be resident at once: they wait for one another
+    static int max_clusters[64] = {0};   // per device, for the widest rows (the fewest blocks per SM)
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    int& cached = max_clusters[dev & 63];
+    if (cached == 0) {
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attrs[2];
+        e = run_config(&cfg, attrs, kRunMaxNodes, (size_t)kRunSmemLimit, nullptr, false);
+        if (e != cudaSuccess) return e;
+        int clusters = 0;
+        e = cudaOccupancyMaxActiveClusters(&clusters, logreg_run_kernel<false>, &cfg);
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            clusters = -1;   // the query is not available: do not use the kernel
+        }
+        cached = clusters > 0 ? clusters : -1;
+    }
+    *ok = cached >= n;
+    return cudaSuccess;
+}
+
+cudaError_t launch_logreg_run(const LogRunParams& p, cudaStream_t s)
+{
+    const RunSmem plan = run_smem_plan(p.d);
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attrs[2];
+    // Cooperative where the driver accepts it together with the cluster shape (the launch then fails
+    // instead of starting with blocks that cannot all be resident); otherwise a plain cluster launch,
+    // after the occupancy check in logreg_run_supported.
+    static int plain_only[64] = {0};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (!plain_only[dev & 63]) {
+        e = run_config(&cfg, attrs, p.n, plan.bytes, s, true);
+        if (e != cudaSuccess) return e;
+        e = cudaLaunchKernelEx(&cfg, p.d == kRunMaxD ? logreg_run_kernel<true> : logreg_run_kernel<false>, p, plan.slots,
+                               plan.red_f4);
+        if (e == cudaSuccess) return e;
+        if (e != cudaErrorNotSupported && e != cudaErrorInvalidValue && e != cudaErrorInvalidConfiguration) return e;
+        (void)cudaGetLastError();
+        plain_only[dev & 63] = 1;
+    }
+    e = run_config(&cfg, attrs, p.n, plan.bytes, s, false);
+    if (e != cudaSuccess) return e;
+    return cudaLaunchKernelEx(&cfg, p.d == kRunMaxD ? logreg_run_kernel<true> : logreg_run_kernel<false>, p, plan.slots,
+                              plan.red_f4);
+}
+
+}  // namespace gpga
