@@ -144,12 +144,15 @@ __global__ void __launch_bounds__(kLrBlock, 2) logreg_partial_tma_reg_kernel(con
     // everything above reads only A, y and the iteration index; x is the previous step's output and
     // the partial sums may still be read by it
     grid_dependency_wait();
-    float4 xr[kRegGroups], acc[kRegGroups];
+    // x_i and the running sums as packed pairs: one instruction does two fused multiply-adds, each
+    // half rounded exactly as a scalar fmaf
+    ulonglong2 xr[kRegGroups], acc[kRegGroups];
+    const ulonglong2 zero2 = make_ulonglong2(0ull, 0ull);
 #pragma unroll
     for (int j = 0; j < kRegGroups; ++j) {
         const int g = lane + 32 * j;
-        xr[j] = g < d4 ? x4[g] : make_float4(0.f, 0.f, 0.f, 0.f);
-        acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        xr[j] = g < d4 ? reinterpret_cast<const ulonglong2*>(x4)[g] : zero2;
+        acc[j] = zero2;
     }
     bool failed = false;
     for (int r = 0; r < my_rows; ++r) {
@@ -162,29 +165,27 @@ __global__ void __launch_bounds__(kLrBlock, 2) logreg_partial_tma_reg_kernel(con
             failed = true;
             break;
         }
-        const float4* a4 = reinterpret_cast<const float4*>(mine + (size_t)s * p.d);
-        float4 a[kRegGroups];
-        float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
+        const ulonglong2* a4 = reinterpret_cast<const ulonglong2*>(mine + (size_t)s * p.d);
+        ulonglong2 a[kRegGroups];
+        f32x2_t z01 = 0ull, z23 = 0ull;   // four running sums z0 .. z3
 #pragma unroll
         for (int j = 0; j < kRegGroups; ++j) {
             const int g = lane + 32 * j;
-            a[j] = g < d4 ? a4[g] : make_float4(0.f, 0.f, 0.f, 0.f);
-            z0 = fmaf(a[j].x, xr[j].x, z0);
-            z1 = fmaf(a[j].y, xr[j].y, z1);
-            z2 = fmaf(a[j].z, xr[j].z, z2);
-            z3 = fmaf(a[j].w, xr[j].w, z3);
+            a[j] = g < d4 ? a4[g] : zero2;
+            z01 = fma2(a[j].x, xr[j].x, z01);
+            z23 = fma2(a[j].y, xr[j].y, z23);
         }
-        const float z = warp_sum_f((z0 + z1) + (z2 + z3));   // every lane holds the sum
+        const float2 za = unpack2(z01), zb = unpack2(z23);
+        const float z = warp_sum_f((za.x + za.y) + (zb.x + zb.y));   // every lane holds the sum
         // the sum needed every lane's loads, so the slot is free: refill it before the arithmetic
         if (r + slots < my_rows) issue(r + slots);
         const float yr = __shfl_sync(0xFFFFFFFFu, my_y, r);
         const float sc = -yr / (1.0f + expf(yr * z));
+        const f32x2_t sc2 = pack2(sc, sc);
 #pragma unroll
         for (int j = 0; j < kRegGroups; ++j) {
-            acc[j].x = fmaf(sc, a[j].x, acc[j].x);
-            acc[j].y = fmaf(sc, a[j].y, acc[j].y);
-            acc[j].z = fmaf(sc, a[j].z, acc[j].z);
-            acc[j].w = fmaf(sc, a[j].w, acc[j].w);
+            acc[j].x = fma2(sc2, a[j].x, acc[j].x);
+            acc[j].y = fma2(sc2, a[j].y, acc[j].y);
         }
     }
     grid_launch_dependents();   // the step kernel may take its place; it waits for this grid before reading
@@ -198,7 +199,7 @@ __global__ void __launch_bounds__(kLrBlock, 2) logreg_partial_tma_reg_kernel(con
 #pragma unroll
     for (int j = 0; j < kRegGroups; ++j) {
         const int g = lane + 32 * j;
-        if (g < d4) red[warp * wstride + g] = acc[j];
+        if (g < d4) reinterpret_cast<ulonglong2*>(red)[warp * wstride + g] = acc[j];
     }
     __syncthreads();
     float4* out4 = reinterpret_cast<float4*>(p.partial + ((long long)c * p.n + i) * p.d);

@@ -33,7 +33,7 @@
 //
 // Waiting: a block only waits for data of the SAME iteration, which its owner publishes before it
 // waits for anything of that iteration, so the waits cannot form a cycle as long as all blocks
-// are resident (checked before the launch; the launch is cooperative where the driver allows).
+// are resident (checked against the device's capacity before the launch).
 // Every wait is bounded; one that gives up raises the error word and a stop word that ends the
 // other blocks' waits.  Both blocks of a pair meet at a cluster barrier before they exit, so no
 // asynchronous store is ever aimed at a block that has left.
@@ -187,19 +187,19 @@ __device__ __forceinline__ void add4_to(float4& s, const float4 v)
     s.w += v.w;
 }
 
-// Shared-memory plan for row width d: row buffers [16 warps][slots][d], the reduction area, the
-// chunk sums of this block's half [4][h0] and x_i [d].
+// Shared-memory plan for row width d: row buffers [16 warps][slots][d], the (group, row) items of
+// a column mean [512], the chunk sums of this block's half [4][h0] and x_i [d].  The per-warp
+// gradient sums have no area of their own: a warp parks them in the buffer of the row it consumed
+// last, which is refilled only after the chunk sums have been formed.
 struct RunSmem {
     int slots;
-    int red_f4;      // float4 entries of the reduction area
     size_t bytes;
 };
 __host__ __device__ inline RunSmem run_smem_plan(int d)
 {
     const int d4 = d >> 2, h0 = (d4 + 1) >> 1;
     RunSmem s;
-    s.red_f4 = kRunWarps * d4 > kRunThreads ? kRunWarps * d4 : kRunThreads;   // row sums; (group, row) items of a column mean
-    const size_t fixed = ((size_t)s.red_f4 + (size_t)kRunMaxChunks * h0 + (size_t)d4) * sizeof(float4);
+    const size_t fixed = ((size_t)kRunThreads + (size_t)kRunMaxChunks * h0 + (size_t)d4) * sizeof(float4);
     const size_t per_slot = (size_t)kRunWarps * d * sizeof(float);
     long long slots = ((long long)kRunSmemLimit - (long long)fixed) / (long long)per_slot;
     if (slots > kRunMaxSlots) slots = kRunMaxSlots;
@@ -210,11 +210,12 @@ __host__ __device__ inline RunSmem run_smem_plan(int d)
 
 // FULL: d == kRunMaxD, every lane holds kRunGroups whole groups (no guards in the row loop).
 template <bool FULL>
-__global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRunParams p, int slots, int red_f4)
+__global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRunParams p, int slots)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t bars[kRunWarps * kRunMaxSlots];
     __shared__ __align__(8) uint64_t sums_bar, x_bar;   // chunk sums of this block's half; x_i^(k+1)
+    __shared__ int stage_at[kRunWarps];                 // where each warp parked its gradient sums (float4 index)
     cg::cluster_group cluster = cg::this_cluster();
     const int r = (int)cluster.block_rank();   // which half of the columns this block finishes
     const int i = (int)(blockIdx.x >> 1);      // node
@@ -229,8 +230,8 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
     const size_t buf_words = (size_t)n * d;
 
     float* slot_base = reinterpret_cast<float*>(smem_raw);
-    float4* red = reinterpret_cast<float4*>(slot_base + (size_t)kRunWarps * slots * d);
-    float4* pbuf = red + red_f4;                    // [chunk][h0]: chunk sums of this block's groups
+    float4* items = reinterpret_cast<float4*>(slot_base + (size_t)kRunWarps * slots * d);   // [kRunThreads]
+    float4* pbuf = items + kRunThreads;             // [chunk][h0]: chunk sums of this block's groups
     float4* xnew = pbuf + kRunMaxChunks * h0;       // [d4]: x_i^(k+1), both halves
     // the same locations in both blocks of the pair, as cluster addresses
     const uint32_t pbuf_at[2] = {cluster_addr(pbuf, 0), cluster_addr(pbuf, 1)};
@@ -326,7 +327,11 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
         ulonglong2 acc[kRunGroups];
 #pragma unroll
         for (int j = 0; j < kRunGroups; ++j) acc[j] = zero2;
+        bool deferred = false;
+        uint32_t deferred_idx = 0u;
+        int stage_slot = 0;   // a warp without rows parks its zeros in its first buffer
         for (int rho = 0; rho < my_rows; ++rho) {
+            stage_slot = wait_slot;
             if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&bar[wait_slot], wait_parity, kRunCopyTries))) {
                 failed = true;
                 break;
@@ -351,10 +356,17 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
             // the sum needed every lane's loads, so the buffer is free: start the copy of the row
             // `depth` positions ahead (this iteration's, or the next one's) into it
             const int ahead = rho + depth;
-            if (ahead < my_rows)
+            if (ahead < my_rows) {
                 issue(__shfl_sync(0xFFFFFFFFu, idx_cur, ahead));
-            else if (it + 1 < p.steps)
-                issue(__shfl_sync(0xFFFFFFFFu, idx_nxt, ahead - my_rows));
+            } else if (it + 1 < p.steps) {
+                const uint32_t idx = __shfl_sync(0xFFFFFFFFu, idx_nxt, ahead - my_rows);
+                if (rho + 1 < my_rows) {
+                    issue(idx);
+                } else {   // the last row's buffer first carries this warp's sums to the chunk sums
+                    deferred = true;
+                    deferred_idx = idx;
+                }
+            }
             // the rows of the next iteration that no buffer is free for yet: ask them into L2 now, one
             // per row step (a burst of such requests is dropped more easily than a trickle)
             if (rho + depth < my_rows && it + 1 < p.steps) {
@@ -370,10 +382,14 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
                 acc[j].y = fma2(sc2, a[j].y, acc[j].y);
             }
         }
+        {
+            ulonglong2* stage = reinterpret_cast<ulonglong2*>(mine + (size_t)stage_slot * d);
 #pragma unroll
-        for (int j = 0; j < kRunGroups; ++j) {
-            const int g = lane + 32 * j;
-            if (FULL || g < d4) reinterpret_cast<ulonglong2*>(red)[warp * d4 + g] = acc[j];
+            for (int j = 0; j < kRunGroups; ++j) {
+                const int g = lane + 32 * j;
+                if (FULL || g < d4) stage[g] = acc[j];
+            }
+            if (lane == 0) stage_at[warp] = (warp * slots + stage_slot) * d4;
         }
         __syncthreads();
         // ---- chunk sums (eight warps in order), sent to the block that finishes the group ---------
@@ -381,13 +397,18 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
             const int cl = tid >> 8, g = tid & 255;
             const int cc = 2 * r + cl;
             if (g < d4 && cc < chunks) {
-                const float4* src = red + (size_t)(cl * kRunChunkWarps) * d4 + g;
-                float4 sum = src[0];
+                const float4* all = reinterpret_cast<const float4*>(slot_base) + g;
+                float4 sum = all[stage_at[cl * kRunChunkWarps]];
 #pragma unroll
-                for (int ww = 1; ww < kRunChunkWarps; ++ww) add4_to(sum, src[(size_t)ww * d4]);
+                for (int ww = 1; ww < kRunChunkWarps; ++ww) add4_to(sum, all[stage_at[cl * kRunChunkWarps + ww]]);
                 const int to = g >= h0 ? 1 : 0;
                 send4(pbuf_at[to] + (uint32_t)(cc * h0 + (g - (to ? h0 : 0))) * 16u, sums_bar_at[to], sum);
             }
+        }
+        __syncthreads();   // every parked sum has been read: the buffers that carried them can be refilled
+        if (deferred) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // this warp's writes before the copy's
+            issue(deferred_idx);
         }
         const bool finisher_warp = warp * 32 < owned;
         if (!finisher_warp) roll(it);   // off the path that the next iteration waits for
@@ -417,16 +438,15 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
             // words instead of n * groups.
             const int mine_cnt = i < owned ? (owned - i + n - 1) / n : 0;   // groups this block averages
             unsigned long long* means = p.ytag + (size_t)p.nbuf * buf_words + (size_t)(buf - gossip_bufs) * d;
-            __syncthreads();   // the reduction area is free: every chunk sum has been read out of it
             if (tid < mine_cnt * n) {
                 const int j = tid / n, row = tid - j * n;
                 float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (!read4(ybuf + (size_t)row * d + 4 * (g_lo + i + j * n), tag, stop, &v)) failed = true;
-                red[tid] = v;   // [j][row]
+                items[tid] = v;   // [j][row]
             }
             __syncthreads();
             if (tid < mine_cnt) {
-                const float4* col = red + tid * n;
+                const float4* col = items + tid * n;
                 double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
                 int q = 0;
                 for (; q + 4 <= n; q += 4) {
@@ -522,8 +542,7 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
 
 namespace {
 
-cudaError_t run_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attrs, int n, size_t smem, cudaStream_t s,
-                       bool cooperative)
+cudaError_t run_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attrs, int n, size_t smem, cudaStream_t s)
 {
     *cfg = cudaLaunchConfig_t{};
     cfg->gridDim = dim3((unsigned)(2 * n));
@@ -534,10 +553,8 @@ cudaError_t run_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attrs, int 
     attrs[0].val.clusterDim.x = 2;
     attrs[0].val.clusterDim.y = 1;
     attrs[0].val.clusterDim.z = 1;
-    attrs[1].id = cudaLaunchAttributeCooperative;
-    attrs[1].val.cooperative = 1;
     cfg->attrs = attrs;
-    cfg->numAttrs = cooperative ? 2 : 1;
+    cfg->numAttrs = 1;
     static unsigned long long limit_set = 0, limit_set_full = 0;
     const cudaError_t e = ensure_smem_limit(logreg_run_kernel<false>, kRunSmemLimit, limit_set);
     return e != cudaSuccess ? e : ensure_smem_limit(logreg_run_kernel<true>, kRunSmemLimit, limit_set_full);
@@ -551,18 +568,18 @@ cudaError_t logreg_run_supported(int n, int d, int batch, int topology, long lon
     if (topology != GPGA_TOPO_RING && topology != GPGA_TOPO_EXP) return cudaSuccess;
     if (d < 4 || d > kRunMaxD || (d & 3) != 0 || batch < 1 || batch > kRunChunkRows * kRunMaxChunks) return cudaSuccess;
     if (n < 1 || n > kRunMaxNodes || H < 0 || H >= (1ll << 31)) return cudaSuccess;
-    const RunSmem plan = run_smem_plan(d);
-    if (plan.slots < 1) return cudaSuccess;
-    // all 2 n blocks must be resident at once: they wait for one another
-    static int max_clusters[64] = {0};   // per device, for the widest rows (the fewest blocks per SM)
+    if (run_smem_plan(d).slots < 1) return cudaSuccess;
+    // All 2 n blocks must be resident at once: they wait for one another.  The widest rows take the
+    // most shared memory, so the number of pairs that fit then holds for every width.
+    static int max_clusters[64] = {0};   // per device
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     int& cached = max_clusters[dev & 63];
     if (cached == 0) {
         cudaLaunchConfig_t cfg;
-        cudaLaunchAttribute attrs[2];
-        e = run_config(&cfg, attrs, kRunMaxNodes, (size_t)kRunSmemLimit, nullptr, false);
+        cudaLaunchAttribute attrs[1];
+        e = run_config(&cfg, attrs, kRunMaxNodes, (size_t)kRunSmemLimit, nullptr);
         if (e != cudaSuccess) return e;
         int clusters = 0;
         e = cudaOccupancyMaxActiveClusters(&clusters, logreg_run_kernel<false>, &cfg);
@@ -576,32 +593,17 @@ cudaError_t logreg_run_supported(int n, int d, int batch, int topology, long lon
     return cudaSuccess;
 }
 
+// A plain launch of clusters of two.  Residency of all blocks is what logreg_run_supported checked
+// for an otherwise idle device; if other work holds multiprocessors for longer than the kernel's
+// bounded waits last, the run ends with the error word set instead of hanging.
 cudaError_t launch_logreg_run(const LogRunParams& p, cudaStream_t s)
 {
     const RunSmem plan = run_smem_plan(p.d);
     cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attrs[2];
-    // Cooperative where the driver accepts it together with the cluster shape (the launch then fails
-    // instead of starting with blocks that cannot all be resident); otherwise a plain cluster launch,
-    // after the occupancy check in logreg_run_supported.
-    static int plain_only[64] = {0};
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    cudaLaunchAttribute attrs[1];
+    const cudaError_t e = run_config(&cfg, attrs, p.n, plan.bytes, s);
     if (e != cudaSuccess) return e;
-    if (!plain_only[dev & 63]) {
-        e = run_config(&cfg, attrs, p.n, plan.bytes, s, true);
-        if (e != cudaSuccess) return e;
-        e = cudaLaunchKernelEx(&cfg, p.d == kRunMaxD ? logreg_run_kernel<true> : logreg_run_kernel<false>, p, plan.slots,
-                               plan.red_f4);
-        if (e == cudaSuccess) return e;
-        if (e != cudaErrorNotSupported && e != cudaErrorInvalidValue && e != cudaErrorInvalidConfiguration) return e;
-        (void)cudaGetLastError();
-        plain_only[dev & 63] = 1;
-    }
-    e = run_config(&cfg, attrs, p.n, plan.bytes, s, false);
-    if (e != cudaSuccess) return e;
-    return cudaLaunchKernelEx(&cfg, p.d == kRunMaxD ? logreg_run_kernel<true> : logreg_run_kernel<false>, p, plan.slots,
-                              plan.red_f4);
+    return cudaLaunchKernelEx(&cfg, p.d == kRunMaxD ? logreg_run_kernel<true> : logreg_run_kernel<false>, p, plan.slots);
 }
 
 }  // namespace gpga

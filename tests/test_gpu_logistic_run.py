@@ -1,7 +1,8 @@
 """gpga_run on the logistic objective (narrow states): many iterations in one launch, x_i resident
-on chip, neighbours' half-step rows exchanged through global memory with progress words.  Every
-sum is formed in the order of the one-iteration kernels, so a run must equal the same number of
-gpga_step calls bit for bit; parity with the oracle is checked on top."""
+on chip, neighbours' half-step rows exchanged through global memory as (value, iteration tag)
+words.  Every sum is formed in the order of the one-iteration kernels, so a run must equal the same
+number of gpga_step calls bit for bit; parity with the oracle is checked on top.  (With H = 1 or 2
+gpga_run keeps to single steps, which are as fast there.)"""
 import numpy as np
 import pytest
 
@@ -36,7 +37,7 @@ SHAPES = [(8, 256, 1024, 128), (16, 64, 512, 100), (5, 100, 260, 50), (4, 20, 4,
 
 
 @pytest.mark.parametrize("n,m,d,batch", SHAPES)
-@pytest.mark.parametrize("topo,H", [("ring", 4), ("ring", 0), ("ring", 1), ("exp", 3), ("exp", 0), ("ring", 2)])
+@pytest.mark.parametrize("topo,H", [("ring", 4), ("ring", 0), ("ring", 3), ("exp", 3), ("exp", 0), ("exp", 5)])
 def test_resident_run_equals_single_steps(topo, H, n, m, d, batch):
     if topo == "exp" and n & (n - 1):
         pytest.skip("the one-peer exponential graph needs n to be a power of two")
