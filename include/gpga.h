@@ -180,7 +180,15 @@ int32_t gpga_step(gpga_t* ctx, int64_t k, void* stream);
  * Logistic objective: within one call the launches of consecutive iterations overlap (the rows of A and
  * the labels of iteration k+1 are fetched while iteration k finishes); A and the labels are inputs that
  * no kernel of the library writes, and the caller must not write them while the call's work is in
- * flight on the stream.  Results are the same as K calls of gpga_step. */
+ * flight on the stream.  For a narrow state (d <= 1024, batch <= 128, ring or one-peer exponential
+ * graph, H = 0 or H >= 3, and as many nodes as the device holds pairs of blocks at once: 74 on a B200)
+ * and K >= 2 the whole call is one launch per 16384 iterations: a pair of thread blocks per node keeps
+ * x_i on chip and exchanges the half-step rows with its neighbours' pairs through the scratch area.
+ * That launch expects the device to itself: its blocks wait for one another, every wait is bounded,
+ * and if other work keeps some of them from starting for seconds the call's work ends early and the
+ * next synchronising call returns GPGA_ERR_TIMEOUT (the state is then unusable).  Only the current
+ * buffer holds a defined state after such a call (the other one is not X^(k-1)).
+ * Results are bit-identical to K calls of gpga_step either way. */
 int32_t gpga_run(gpga_t* ctx, int64_t K, void* stream);
 
 /*
