@@ -76,18 +76,22 @@ __device__ __forceinline__ float fast_cos(float x)
 //    -ln(1 - t) = t + t^2/2 + t^3/3 (t exact) is used instead.
 //  - Angle: evaluated at 2 pi (u2 - 1/2) in [-pi, pi), where the hardware sine and
 //    cosine are most accurate, then negated (cos(x + pi) = -cos x).
+// -2 ln u1 for u1 within 2^-10 of 1, from t = 1 - u1 = (2^24 - 1 - m) / 2^24 (exact): the series
+// -ln(1 - t) = t + t^2/2 + t^3/3.  Needed by one sample in a thousand, so it is kept out of line:
+// the common path does not carry its instructions.
+static __device__ __noinline__ float neg2ln_near_one(uint32_t m)
+{
+    const float t = (float)(0xFFFFFFu - m) * 0x1p-24f;
+    return t * (2.0f + t * (1.0f + t * 0.6666667f));
+}
+
 __device__ __forceinline__ float2 box_muller(uint32_t a, uint32_t b)
 {
     const uint32_t m = a >> 8;
-    float neg2ln;
-    if (m >= 0xFFFFFFu - 0x3FFFu) {
-        const float t = (float)(0xFFFFFFu - m) * 0x1p-24f;   // 1 - u1, exact
-        neg2ln = t * (2.0f + t * (1.0f + t * 0.6666667f));
-    } else {
-        // (the exact scaling to (0,1] first: the hardware log2 is most accurate near 1)
-        const float u1 = (float)(m + 1u) * 0x1p-24f;
-        neg2ln = -1.3862943611198906f * fast_lg2(u1);
-    }
+    // (the exact scaling to (0,1] first: the hardware log2 is most accurate near 1)
+    const float u1 = (float)(m + 1u) * 0x1p-24f;
+    float neg2ln = -1.3862943611198906f * fast_lg2(u1);
+    if (m >= 0xFFFFFFu - 0x3FFFu) neg2ln = neg2ln_near_one(m);
     const float r = fast_sqrt(neg2ln);
     const float ang = (float)((int)(b >> 8) - (1 << 23)) * 3.7450704e-07f;   // 2 pi / 2^24
     return make_float2(-r * fast_cos(ang), -r * fast_sin(ang));
@@ -141,6 +145,52 @@ __device__ __forceinline__ f32x2_t fma2(f32x2_t a, f32x2_t b, f32x2_t c)
     f32x2_t d;
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
     return d;
+}
+
+__device__ __forceinline__ f32x2_t add2(f32x2_t a, f32x2_t b)
+{
+    f32x2_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2_t sub2(f32x2_t a, f32x2_t b)
+{
+    f32x2_t d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2_t mul2(f32x2_t a, f32x2_t b)
+{
+    f32x2_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// Element-wise arithmetic on a group of four columns, two packed instructions each; every
+// component is rounded as the scalar operation of the same name would round it.
+__device__ __forceinline__ float4 join4(f32x2_t lo, f32x2_t hi)
+{
+    const float2 a = unpack2(lo), b = unpack2(hi);
+    return make_float4(a.x, a.y, b.x, b.y);
+}
+__device__ __forceinline__ float4 add4(float4 a, float4 b)
+{
+    return join4(add2(pack2(a.x, a.y), pack2(b.x, b.y)), add2(pack2(a.z, a.w), pack2(b.z, b.w)));
+}
+__device__ __forceinline__ float4 sub4(float4 a, float4 b)
+{
+    return join4(sub2(pack2(a.x, a.y), pack2(b.x, b.y)), sub2(pack2(a.z, a.w), pack2(b.z, b.w)));
+}
+__device__ __forceinline__ float4 scale4(float4 a, float s)
+{
+    const f32x2_t s2 = pack2(s, s);
+    return join4(mul2(pack2(a.x, a.y), s2), mul2(pack2(a.z, a.w), s2));
+}
+// s * a + b
+__device__ __forceinline__ float4 fma4(float s, float4 a, float4 b)
+{
+    const f32x2_t s2 = pack2(s, s);
+    return join4(fma2(s2, pack2(a.x, a.y), pack2(b.x, b.y)), fma2(s2, pack2(a.z, a.w), pack2(b.z, b.w)));
 }
 
 // ---- streaming (read-once / write-once) 128-bit accesses -------------------

@@ -13,15 +13,6 @@ namespace gpga {
 
 constexpr int kBlock = 256;
 
-__device__ __forceinline__ float4 add4(float4 a, float4 b)
-{
-    return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
-}
-__device__ __forceinline__ float4 scale4(float4 a, float s)
-{
-    return make_float4(a.x * s, a.y * s, a.z * s, a.w * s);
-}
-
 // One row's inputs for one column group, and x^(k+1/2) formed from them
 // (Algorithm 1: gradient, then the local update).  Loading and finishing are split
 // so that a thread can have the loads of several rows in flight before it needs any.
@@ -81,17 +72,10 @@ __device__ __forceinline__ float4 finish_row(const StepParams& p, const ColGroup
     if (MODE == GRAD_BUFFER) {
         g = r.b;
     } else {
-        g = make_float4(r.x.x - r.b.x, r.x.y - r.b.y, r.x.z - r.b.z, r.x.w - r.b.w);
-        if (MODE == GRAD_QUAD_NOISE) {
-            const float4 z = normal4(c.qg, (uint32_t)i, p.k, 0u, p.keys);
-            g.x = fmaf(p.sigma, z.x, g.x);
-            g.y = fmaf(p.sigma, z.y, g.y);
-            g.z = fmaf(p.sigma, z.z, g.z);
-            g.w = fmaf(p.sigma, z.w, g.w);
-        }
+        g = sub4(r.x, r.b);
+        if (MODE == GRAD_QUAD_NOISE) g = fma4(p.sigma, normal4(c.qg, (uint32_t)i, p.k, 0u, p.keys), g);
     }
-    return make_float4(fmaf(-p.gamma, g.x, r.x.x), fmaf(-p.gamma, g.y, r.x.y),
-                       fmaf(-p.gamma, g.z, r.x.z), fmaf(-p.gamma, g.w, r.x.w));
+    return fma4(-p.gamma, g, r.x);
 }
 
 template <int MODE, bool VEC>
@@ -149,9 +133,7 @@ __device__ __forceinline__ void stream_rows(const StepParams& p, const ColGroup&
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ float4 mix3(float4 a, float4 b, float4 c)
 {
-    const float third = 0.333333343f;
-    return make_float4((a.x + b.x + c.x) * third, (a.y + b.y + c.y) * third, (a.z + b.z + c.z) * third,
-                       (a.w + b.w + c.w) * third);
+    return scale4(add4(add4(a, b), c), 0.333333343f);
 }
 
 template <int MODE, bool VEC, int U, bool PIPE, int BLOCK, int MINB>

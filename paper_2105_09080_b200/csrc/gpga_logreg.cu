@@ -84,9 +84,10 @@ __global__ void __launch_bounds__(kLrBlock) logreg_partial_kernel(const LogregPa
     }
 }
 
-// Polls of an mbarrier before a kernel gives up on a bulk copy (each poll may block for a short,
-// hardware-defined time): far beyond any copy's latency, and finite.
-constexpr uint32_t kTmaMaxTries = 1u << 22;
+// Polls of an mbarrier before a kernel gives up on a bulk copy.  A poll of a phase that is not
+// complete blocks for about 4 microseconds (measured: 2000 polls of a barrier nobody completes take
+// 8.2 ms), so this is about one second: far beyond any copy's latency, and finite.
+constexpr uint32_t kTmaMaxTries = 1u << 18;
 
 // Narrow rows (d <= kRegMaxD): the batch rows are staged in shared memory by bulk asynchronous
 // copies (one 16-byte-aligned row of d floats per copy, completion counted on an mbarrier) and

@@ -57,8 +57,8 @@ constexpr int kRunChunkRows = 32, kRunChunkWarps = 8;   // the batch is cut as b
 constexpr int kRunMaxChunks = 2 * kRunWarps / kRunChunkWarps;   // 4: batch <= 128
 constexpr int kRunMaxNodes = 88;
 constexpr int kRunSmemLimit = 226 * 1024;       // dynamic; the static arrays take under 1 KB
-constexpr uint32_t kRunCopyTries = 1u << 22;    // polls of an mbarrier before a copy is given up
-constexpr uint32_t kRunPollTries = 1u << 21;    // reads of a published group (about a microsecond each)
+constexpr uint32_t kRunCopyTries = 1u << 18;    // polls of an mbarrier (about 4 us each while incomplete): about a second
+constexpr uint32_t kRunPollTries = 1u << 21;    // reads of a published word (half a microsecond or more each): a second or two
 
 __device__ __forceinline__ int ld_relaxed_gpu(const int* p)
 {

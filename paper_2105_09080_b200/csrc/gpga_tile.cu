@@ -31,17 +31,10 @@ __device__ __forceinline__ float4 tile_finish(const StepParams& p, float4 x, flo
     if (MODE == GRAD_BUFFER) {
         g = b;
     } else {
-        g = make_float4(x.x - b.x, x.y - b.y, x.z - b.z, x.w - b.w);
-        if (MODE == GRAD_QUAD_NOISE) {
-            const float4 z = normal4(p.q_base + (uint32_t)q, (uint32_t)i, k, 0u, p.keys);
-            g.x = fmaf(p.sigma, z.x, g.x);
-            g.y = fmaf(p.sigma, z.y, g.y);
-            g.z = fmaf(p.sigma, z.z, g.z);
-            g.w = fmaf(p.sigma, z.w, g.w);
-        }
+        g = sub4(x, b);
+        if (MODE == GRAD_QUAD_NOISE) g = fma4(p.sigma, normal4(p.q_base + (uint32_t)q, (uint32_t)i, k, 0u, p.keys), g);
     }
-    return make_float4(fmaf(-p.gamma, g.x, x.x), fmaf(-p.gamma, g.y, x.y), fmaf(-p.gamma, g.z, x.z),
-                       fmaf(-p.gamma, g.w, x.w));
+    return fma4(-p.gamma, g, x);
 }
 
 template <int MODE, bool VEC>
@@ -69,13 +62,7 @@ __device__ __forceinline__ float4 tile_half_step(const StepParams& p, int i, lon
     return tile_finish<MODE>(p, x, b, i, q, p.k);
 }
 
-__device__ __forceinline__ void acc4(float4& s, const float4 v)
-{
-    s.x += v.x;
-    s.y += v.y;
-    s.z += v.z;
-    s.w += v.w;
-}
+__device__ __forceinline__ void acc4(float4& s, const float4 v) { s = add4(s, v); }
 
 // x_i^(k+1) for cell (row i, group g) from the tile of Y.  `mix` is a GPGA_TOPO_* value or
 // TILE_MIX_GLOBAL.
@@ -125,13 +112,10 @@ __device__ __forceinline__ float4 tile_mix(const float4* ytile, int i, int g, in
     } else if (mix == GPGA_TOPO_RING) {
         const float4 up = ytile[(i == 0 ? n - 1 : i - 1) * tile_groups + g];
         const float4 dn = ytile[(i == n - 1 ? 0 : i + 1) * tile_groups + g];
-        const float third = 0.333333343f;
-        s = make_float4((up.x + s.x + dn.x) * third, (up.y + s.y + dn.y) * third, (up.z + s.z + dn.z) * third,
-                        (up.w + s.w + dn.w) * third);
+        s = scale4(add4(add4(up, s), dn), 0.333333343f);
     } else if (mix == GPGA_TOPO_EXP) {
         const float4 peer = ytile[((i + (1 << hop_log2)) & (n - 1)) * tile_groups + g];
-        s = make_float4((s.x + peer.x) * 0.5f, (s.y + peer.y) * 0.5f, (s.z + peer.z) * 0.5f,
-                        (s.w + peer.w) * 0.5f);
+        s = scale4(add4(s, peer), 0.5f);
     } else if (mix == GPGA_TOPO_GRID) {
         const int cols = grid_cols, rows = n / cols;
         const int a = i / cols, b = i - a * cols;
