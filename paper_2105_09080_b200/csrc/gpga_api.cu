@@ -216,7 +216,9 @@ int32_t do_step(gpga_ctx* c, int64_t k, bool global, cudaStream_t s, bool after_
 //    arithmetic bound (6.0-6.9e11 updates/s measured for n = 8 ... 64, 5.3e11 at n = 128) is above
 //    what the row-streaming kernels reach from HBM (at most 5.5e11, 4.9-5.3e11 at 0.8 GB of
 //    state), and the one extra pass over the state is amortised.  At n = 256 the two are equal,
-//    and wider n would go through the several-cells-per-thread kernel, which is far slower.
+//    and wider n would go through the several-cells-per-thread kernel, which is far slower.  A
+//    global-average iteration costs more on chip (the fp64 column mean: 3.99 against 3.07 ms at
+//    n = 64, d = 25,557,032) than a gossip iteration saves, so H = 1 and H = 2 keep to single steps.
 // A launch is kept to about half a second of work.
 constexpr int64_t kFusedStateBytes = 64ll << 20;
 constexpr int64_t kFusedSteps = 1024;
@@ -279,7 +281,8 @@ int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)
     if (c->topology == GPGA_TOPO_SPARSE && !c->sparse.row_ptr)
         return fail(c, GPGA_ERR_NOT_READY, "topology SPARSE needs gpga_set_weight_matrix");
     const bool fused = c->objective == GPGA_OBJ_QUADRATIC && K >= 2 && run_tile_supports(c->n) &&
-                       (12 * c->n * c->ld <= kFusedStateBytes || (c->n <= kFusedWideNodes && K >= kFusedMinSteps));
+                       (12 * c->n * c->ld <= kFusedStateBytes ||
+                        (c->n <= kFusedWideNodes && K >= kFusedMinSteps && (c->H == 0 || c->H >= 3)));
     int64_t per_launch = (int64_t)(kFusedUpdatesPerLaunch / ((double)c->n * (double)c->d));
     if (per_launch > kFusedSteps) per_launch = kFusedSteps;
     if (per_launch < 16) per_launch = 16;
