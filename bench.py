@@ -62,9 +62,9 @@ DEFAULT_WORKLOAD = "c3_ring_h4"
 NCU_TRAFFIC = {
     # kernel name: (traffic / algorithmic bytes, source digest); captured at n=64, d=2,097,192 and
     # n=16, d=8,388,608 -- one pass over three n x d arrays, so traffic scales with n x d
-    "step_ring_kernel": (0.977, "a5e0b622641a23d1"),
-    "step_exp_kernel": (0.976, "a5e0b622641a23d1"),
-    "step_global_kernel": (0.968, "a5e0b622641a23d1"),
+    "step_ring_kernel": (0.977, "3199e78917cf862e"),
+    "step_exp_kernel": (0.977, "3199e78917cf862e"),
+    "step_global_kernel": (0.968, "3199e78917cf862e"),
 }
 
 

@@ -186,6 +186,71 @@ __global__ void __launch_bounds__(BLOCK, MINB) step_exp_kernel(const StepParams 
     const int hop = 1 << hop_log2;
     const int lmask = (1 << len_log2) - 1;
     float4 first = make_float4(0.f, 0.f, 0.f, 0.f), prev = first;
+    const int n = (int)p.n;
+    if (U == 4 && n >= 4) {
+        // Batches of four consecutive steps of the walk (n and the cycle length L are powers of two).
+        // With L >= 4 a batch lies inside one cycle: rows row0 + u h, addressed from one base by
+        // multiples of h rows; with L = 2 it is two whole cycles: rows c, c + h, c + 1, c + 1 + h.
+        // Only the batch start is tracked (position in the cycle, first row), not every row.
+        const int L = 1 << len_log2;
+        const long long hop_ld = (long long)p.ld << hop_log2, hop_ldb = (long long)p.ldb << hop_log2;
+        const long long j0 = VEC ? 0 : c.j0;
+        auto load_at = [&](long long ox, long long ob) {
+            RowIn r;
+            r.x = load4<VEC>(c.x + ox, j0, p.d);
+            r.b = load4<VEC>(c.b + ob, j0, p.d);
+            return r;
+        };
+        auto store_at = [&](long long o, float4 v) { store4<VEC>(c.out + o, j0, p.d, v); };
+        auto half = [](float4 a, float4 b) { return scale4(add4(a, b), 0.5f); };
+        if (L >= 4) {
+            int s0 = 0, row0 = 0;
+            for (int t = 0; t < n; t += 4) {
+                const long long ox = (long long)row0 * p.ld, ob = (long long)row0 * p.ldb;
+                RowIn r[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) r[u] = load_at(ox + u * hop_ld, ob + u * hop_ldb);
+                float4 y = finish_row<MODE>(p, c, r[0], row0);
+                if (s0 == 0)
+                    first = y;
+                else
+                    store_at(ox - hop_ld, half(prev, y));
+                prev = y;
+#pragma unroll
+                for (int u = 1; u < 4; ++u) {
+                    y = finish_row<MODE>(p, c, r[u], row0 + (u << hop_log2));
+                    store_at(ox + (u - 1) * hop_ld, half(prev, y));
+                    prev = y;
+                }
+                s0 += 4;
+                if (s0 == L) {   // the cycle closes: its last row mixes with its first
+                    store_at(ox + 3 * hop_ld, half(prev, first));
+                    s0 = 0;
+                    row0 = (t + 4) >> len_log2;
+                } else {
+                    row0 += 4 << hop_log2;
+                }
+            }
+        } else {   // L == 2
+            for (int cyc = 0; cyc < hop; cyc += 2) {
+                const long long ox = (long long)cyc * p.ld, ob = (long long)cyc * p.ldb;
+                RowIn r[4];
+                r[0] = load_at(ox, ob);
+                r[1] = load_at(ox + hop_ld, ob + hop_ldb);
+                r[2] = load_at(ox + p.ld, ob + p.ldb);
+                r[3] = load_at(ox + p.ld + hop_ld, ob + p.ldb + hop_ldb);
+                const float4 y0 = finish_row<MODE>(p, c, r[0], cyc);
+                const float4 y1 = finish_row<MODE>(p, c, r[1], cyc + hop);
+                store_at(ox, half(y0, y1));
+                store_at(ox + hop_ld, half(y1, y0));
+                const float4 y2 = finish_row<MODE>(p, c, r[2], cyc + 1);
+                const float4 y3 = finish_row<MODE>(p, c, r[3], cyc + 1 + hop);
+                store_at(ox + p.ld, half(y2, y3));
+                store_at(ox + p.ld + hop_ld, half(y3, y2));
+            }
+        }
+        return;
+    }
     stream_rows<MODE, VEC, U, PIPE>(
         p, c, 0, [=](int t) { return (t >> len_log2) + ((t & lmask) << hop_log2); },
         [&](int t, int row, float4 cur) {
