@@ -7,7 +7,7 @@
 //  - the batch rows of A stream into per-warp shared-memory buffers by bulk asynchronous
 //    copies, the copies of the next iteration's rows (their indices depend only on the seed,
 //    the node and the iteration) already in flight while this iteration is reduced and mixed,
-//    and every row asked into L2 more than an iteration before it is copied;
+//    and the rows that no buffer is free for asked into L2 an iteration before they are copied;
 //  - the per-warp gradient sums are added in shared memory; the chunk sums go to the block that
 //    finishes the column group by asynchronous stores into its shared memory, which count
 //    themselves off on an mbarrier there (no cluster-wide barrier in the loop); each block
@@ -288,7 +288,7 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
         ++issued;
     };
     for (int rho = 0; rho < depth; ++rho) issue(__shfl_sync(0xFFFFFFFFu, idx_cur, rho));
-    // the rows of the iteration after the next: indices, labels, and the rows asked into L2
+    // the rows of the iteration after the next: indices and labels
     auto roll = [&](int it) {
         idx_cur = idx_nxt;
         y_cur = y_nxt;
@@ -368,7 +368,9 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
                 }
             }
             // the rows of the next iteration that no buffer is free for yet: ask them into L2 now, one
-            // per row step (a burst of such requests is dropped more easily than a trickle)
+            // per row step (a copy of a row that is in L2 lands in about 640 cycles instead of 1100;
+            // asking for every row of the next iteration here was measured and is slower: the requests
+            // then compete with the copies this iteration is waiting for)
             if (rho + depth < my_rows && it + 1 < p.steps) {
                 const uint32_t later = __shfl_sync(0xFFFFFFFFu, idx_nxt, rho + depth);
                 if (lane == 0) bulk_prefetch_l2(A + (long long)later * d, row_bytes);
