@@ -295,25 +295,21 @@ __global__ void __launch_bounds__(kTileBlock) run_cell_kernel(const StepParams p
                 }
             }
             __syncthreads();
-            if (c < tile_groups && q_first + c < p.Q) {      // thread c: the mean of column group c
+            // thread c: component c & 3 of the mean of column group c >> 2 (four threads per group: the
+            // fp64 chain of a component is what this step waits for, and the four are independent)
+            for (int cc = c; cc < 4 * tile_groups; cc += blockDim.x) {   // (a block of n < 4 rows has fewer threads)
+                const int gg = cc >> 2, comp = cc & 3;
+                if (q_first + gg >= p.Q) continue;
                 const int addends = full + (rest >= 1 ? 1 : 0) + (rest == 3 ? 1 : 0);
-                double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
-                for (int j = 0; j < addends; ++j) {
-                    const float4 v = gsum[j * tile_groups + c];
-                    s0 += (double)v.x;
-                    s1 += (double)v.y;
-                    s2 += (double)v.z;
-                    s3 += (double)v.w;
-                }
-                float4 m;
-                if ((n & (n - 1)) == 0) {   // 1/n is exact: the product equals the quotient
-                    const double inv = 1.0 / (double)n;
-                    m = make_float4((float)(s0 * inv), (float)(s1 * inv), (float)(s2 * inv), (float)(s3 * inv));
-                } else {
-                    const double dn = (double)n;
-                    m = make_float4((float)(s0 / dn), (float)(s1 / dn), (float)(s2 / dn), (float)(s3 / dn));
-                }
-                gmean[c] = m;
+                const float* v = reinterpret_cast<const float*>(gsum + gg) + comp;
+                double sum = 0.0;
+                for (int j = 0; j < addends; ++j) sum += (double)v[(size_t)j * tile_groups * 4];
+                float m;
+                if ((n & (n - 1)) == 0)   // 1/n is exact: the product equals the quotient
+                    m = (float)(sum * (1.0 / (double)n));
+                else
+                    m = (float)(sum / (double)n);
+                reinterpret_cast<float*>(gmean + gg)[comp] = m;
             }
             __syncthreads();
             if (own) x = gmean[g];
