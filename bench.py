@@ -36,6 +36,7 @@ WORKLOADS = {
     "c1_ring_h4": dict(n=8, d=65_536, topo="ring", H=4, gamma=0.1, sigma=0.1, K=32, x0="zero", x0_std=1.0, b_shift=0.0),
     "c2_exp_h8": dict(n=32, d=1_048_576, topo="exp", H=8, gamma=0.05, sigma=0.1, K=64, x0="zero", x0_std=1.0, b_shift=0.0),
     "c3_ring_h4": dict(n=64, d=25_557_032, topo="ring", H=4, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),
+    "c3_ring_h2": dict(n=64, d=25_557_032, topo="ring", H=2, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),
     "c3_ring_h16": dict(n=64, d=25_557_032, topo="ring", H=16, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),
     "c3_ring_hinf": dict(n=64, d=25_557_032, topo="ring", H=0, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),
     "c3_exp_h4": dict(n=64, d=25_557_032, topo="exp", H=4, gamma=0.01, sigma=0.01, K=50, x0="shared", x0_std=0.1, b_shift=0.5),

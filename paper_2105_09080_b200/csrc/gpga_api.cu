@@ -217,8 +217,8 @@ int32_t do_step(gpga_ctx* c, int64_t k, bool global, cudaStream_t s, bool after_
 //    what the row-streaming kernels reach from HBM (at most 5.5e11, 4.9-5.3e11 at 0.8 GB of
 //    state), and the one extra pass over the state is amortised.  At n = 256 the two are equal,
 //    and wider n would go through the several-cells-per-thread kernel, which is far slower.  A
-//    global-average iteration costs more on chip (the fp64 column mean: 3.99 against 3.07 ms at
-//    n = 64, d = 25,557,032) than a gossip iteration saves, so H = 1 and H = 2 keep to single steps.
+//    global-average iteration costs a little more on chip (the fp64 column mean: 3.15 against
+//    3.02 ms at n = 64, d = 25,557,032), so H = 1 keeps to single steps (H = 2: 2.66 against 3.04).
 // A launch is kept to about half a second of work.
 constexpr int64_t kFusedStateBytes = 64ll << 20;
 constexpr int64_t kFusedSteps = 1024;
@@ -282,7 +282,7 @@ int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)
         return fail(c, GPGA_ERR_NOT_READY, "topology SPARSE needs gpga_set_weight_matrix");
     const bool fused = c->objective == GPGA_OBJ_QUADRATIC && K >= 2 && run_tile_supports(c->n) &&
                        (12 * c->n * c->ld <= kFusedStateBytes ||
-                        (c->n <= kFusedWideNodes && K >= kFusedMinSteps && (c->H == 0 || c->H >= 3)));
+                        (c->n <= kFusedWideNodes && K >= kFusedMinSteps && c->H != 1));
     int64_t per_launch = (int64_t)(kFusedUpdatesPerLaunch / ((double)c->n * (double)c->d));
     if (per_launch > kFusedSteps) per_launch = kFusedSteps;
     if (per_launch < 16) per_launch = 16;
