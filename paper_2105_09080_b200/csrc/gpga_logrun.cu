@@ -447,45 +447,25 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
                 items[tid] = v;   // [j][row]
             }
             __syncthreads();
-            if (tid < mine_cnt) {
-                const float4* col = items + tid * n;
-                double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+            if (tid < 4 * mine_cnt) {   // four threads per column group, one per component
+                const int j = tid >> 2, comp = tid & 3;
+                const float* col = reinterpret_cast<const float*>(items + j * n) + comp;   // [row * 4]
+                double sum = 0.0;
                 int q = 0;
-                for (; q + 4 <= n; q += 4) {
-                    float4 a = col[q], b = col[q + 2];
-                    add4_to(a, col[q + 1]);
-                    add4_to(b, col[q + 3]);
-                    add4_to(a, b);
-                    s0 += (double)a.x;
-                    s1 += (double)a.y;
-                    s2 += (double)a.z;
-                    s3 += (double)a.w;
-                }
+                for (; q + 4 <= n; q += 4)
+                    sum += (double)((col[4 * q] + col[4 * (q + 1)]) + (col[4 * (q + 2)] + col[4 * (q + 3)]));
                 const int rest = n - q;
-                if (rest >= 1) {
-                    float4 a = col[q];
-                    if (rest >= 2) add4_to(a, col[q + 1]);
-                    s0 += (double)a.x;
-                    s1 += (double)a.y;
-                    s2 += (double)a.z;
-                    s3 += (double)a.w;
-                }
-                if (rest == 3) {
-                    const float4 b = col[q + 2];
-                    s0 += (double)b.x;
-                    s1 += (double)b.y;
-                    s2 += (double)b.z;
-                    s3 += (double)b.w;
-                }
-                float4 mean;
-                if ((n & (n - 1)) == 0) {   // 1/n is exact: the product equals the quotient
-                    const double inv = 1.0 / (double)n;
-                    mean = make_float4((float)(s0 * inv), (float)(s1 * inv), (float)(s2 * inv), (float)(s3 * inv));
-                } else {
-                    const double dn_ = (double)n;
-                    mean = make_float4((float)(s0 / dn_), (float)(s1 / dn_), (float)(s2 / dn_), (float)(s3 / dn_));
-                }
-                publish4(means + 4 * (g_lo + i + tid * n), mean, tag);
+                if (rest >= 1) sum += (double)(rest >= 2 ? col[4 * q] + col[4 * (q + 1)] : col[4 * q]);
+                if (rest == 3) sum += (double)col[4 * (q + 2)];
+                float mean;
+                if ((n & (n - 1)) == 0)   // 1/n is exact: the product equals the quotient
+                    mean = (float)(sum * (1.0 / (double)n));
+                else
+                    mean = (float)(sum / (double)n);
+                // one (value, tag) word per component
+                const unsigned long long word = ((unsigned long long)tag << 32) | __float_as_uint(mean);
+                asm volatile("st.relaxed.gpu.global.b64 [%0], %1;" ::"l"(means + 4 * (g_lo + i + j * n) + comp), "l"(word)
+                             : "memory");
             }
             if (finisher && !read4(means + 4 * (g_lo + tid), tag, stop, &xp)) failed = true;
         } else if (finisher_warp) {
