@@ -100,3 +100,18 @@ def test_resident_run_in_place_and_long():
     a, b = g.get_x().cpu().numpy(), ref.get_x().cpu().numpy()
     assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), float(np.abs(a - b).max())
     assert g.consensus_distance() == ref.consensus_distance()
+
+
+def test_resident_run_is_cut_into_launches_of_16384_iterations():
+    """A longer run takes two launches (the tags restart with each launch, its buffers are cleared
+    before it); still bit-identical to single steps."""
+    n, m, d, batch, K = 4, 64, 64, 8, (1 << 14) + 10
+    A, y = logistic_inputs(n, m, d, SEED + 9)
+    X0 = np.zeros((n, d), dtype=np.float32)
+    run, stepped = _pair(n, m, d, batch, "ring", 4, X0, A, y, gamma=0.05)
+    run.run(K)
+    assert run.launch_count() == 2 and run.get_k() == K
+    for k in range(K):
+        stepped.step(k)
+    a, b = run.get_x().cpu().numpy(), stepped.get_x().cpu().numpy()
+    assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), float(np.abs(a - b).max())
