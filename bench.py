@@ -314,9 +314,9 @@ def run_ours(args, w, name):
         traffic = NCU_TRAFFIC[dominant][0] * algo_bytes
     if resident:
         # Compute-bound: X and b stay on chip.  Peak = SMs x 128 lanes/clk x max SM clock / lane
-        # operations per update (43 = the 172 warp instructions that run_cell_kernel executes per warp
+        # operations per update (42 = the 169 warp instructions that run_cell_kernel executes per warp
         # and iteration, ncu smsp__inst_executed, over the 4 updates of a thread).
-        alu_peak = 148 * 128 * (clocks.get("sm_max_mhz") or 1965) * 1e6 / 43.0
+        alu_peak = 148 * 128 * (clocks.get("sm_max_mhz") or 1965) * 1e6 / 42.0
         rate = n * d / (kernels[dominant] * 1e-3)
         roofline = {"bound": "alu", "kernel": dominant, "achieved": rate / 1e9, "peak": alu_peak / 1e9,
                     "unit": "G node-param updates/s", "frac": rate / alu_peak, "traffic": None,
