@@ -20,6 +20,10 @@
  *    an n x d matrix is at index i * ld + j (64-bit).
  *  - `stream` arguments are a cudaStream_t passed as void* (NULL = default
  *    stream).  Calls are asynchronous on that stream unless stated otherwise.
+ *  - Kernels are launched on the device that is current in the calling thread.
+ *    All buffers of a handle, and the streams given with it, must belong to that
+ *    device; make it current (cudaSetDevice) before every call on the handle.  A
+ *    handle is used from one host thread at a time.
  *  - Random numbers are Philox4x32-10 (Salmon et al., SC'11) keyed by
  *    key = (seed low word, seed high word), counter = (column >> 2, node i,
  *    iteration k, stream id); the four output words give four normals for
@@ -204,6 +208,9 @@ int32_t gpga_run(gpga_t* ctx, int64_t K, void* stream);
  * bit-identical to bind + gpga_run), and on return the bound device buffers hold the whole X^(K).
  * Work already queued on `stream` is waited for; the internal streams and events are created on
  * the first call and released by gpga_destroy.
+ * Not re-entrant: while the call runs, the handle's view (d, column offset, buffer pointers) is
+ * narrowed to the chunk in hand and put back before it returns, so no other call on the same
+ * handle (gpga_get_x included) may run beside it from another host thread.
  */
 int32_t gpga_run_host(gpga_t* ctx, const float* x0_host, const float* data_host, int64_t K,
                       float* x_out_host, void* stream);
@@ -304,14 +311,29 @@ int32_t gpga_normal_fill(uint64_t seed, uint32_t stream_id, uint32_t k, uint32_t
  *
  * Behaviour to rely on:
  *  - It calls no allocating routine.  The first call on a device resolves the array's
- *    address (a symbol lookup); make that first call before any stream capture begins.
+ *    address (a symbol lookup); with CUDA's lazy module loading that first lookup or launch
+ *    is also when the driver loads the library's device code and sets the array aside, and
+ *    it may synchronise the device.  So make one warm-up call per device at start-up,
+ *    before any stream capture begins and outside the region that must not stall; from
+ *    the second call on, a call leaves the device's free memory unchanged.
+ *  - The kernels run on the device that is current when the call is made and use that
+ *    device's copy of the array: A_dev, y_dev, x_dev and G_dev must all be memory of that
+ *    device (or managed memory) and `stream` a stream of it.  The call checks the pointers
+ *    (a query, not an allocation) and returns INVALID_ARG, launching nothing, otherwise.
  *  - Asynchronous on `stream`.  All calls on a device share the one array, which keeps the
  *    previous call's contents; each call writes every element it later reads, so nothing
  *    has to be cleared, but calls that overlap on the GPU race.  Issue them on one stream.
- *  - Errors: INVALID_ARG for NULL or misaligned pointers and out-of-range sizes;
- *    UNSUPPORTED when the problem needs more than GPGA_NOALLOC_SCRATCH_BYTES (the need is
- *    reported in *needed_bytes_host; use gpga_step with a bound scratch buffer instead);
- *    CUDA if a CUDA call fails.
+ *  - Errors: INVALID_ARG for NULL or misaligned pointers, out-of-range sizes and buffers
+ *    that are not the current device's; UNSUPPORTED when the problem needs more than
+ *    GPGA_NOALLOC_SCRATCH_BYTES (the need is reported in *needed_bytes_host; use gpga_step
+ *    with a bound scratch buffer instead); CUDA if a CUDA call fails (also: no device).
+ *  - There is no handle, hence no error word for a later call to report.  The gradient
+ *    kernels for d <= 8192 wait, a bounded number of polls (about a second), for the
+ *    asynchronous copies of the batch rows; should such a wait give up, the block writes
+ *    NaN over its slice of the partial sums, so the affected rows of G are NaN (never the
+ *    previous call's values) while the status already returned stays GPGA_OK.  A caller
+ *    that must know checks G for NaN; the handle path reports the same event as
+ *    GPGA_ERR_TIMEOUT.
  */
 #define GPGA_NOALLOC_SCRATCH_BYTES (4 * 1024 * 1024)
 int32_t gpga_logistic_gradient_noalloc(const float* A_dev, const float* y_dev, const float* x_dev,

@@ -50,55 +50,54 @@ _lib = None
 def load(path):
     """Load an oracle shared library (the built one, or a deliberately broken copy that a test
     compiled to see whether the pins notice) and declare its signatures."""
-    if True:
-        L = C.CDLL(str(path))
-        i64, i32, u32, u64, f64 = C.c_int64, C.c_int32, C.c_uint32, C.c_uint64, C.c_double
-        P = C.c_void_p
-        L.gpga_oracle_philox4x32_10.argtypes = [P, P, P]
-        L.gpga_oracle_philox4x32_10.restype = None
-        L.gpga_oracle_box_muller.argtypes = [u32, u32, P]
-        L.gpga_oracle_box_muller.restype = None
-        L.gpga_oracle_normal4.argtypes = [u64, u32, u32, u32, u32, P]
-        L.gpga_oracle_normal4.restype = None
-        L.gpga_oracle_is_global.argtypes = [i64, i64]
-        L.gpga_oracle_is_global.restype = i32
-        L.gpga_oracle_exp_hop.argtypes = [i64, i64]
-        L.gpga_oracle_exp_hop.restype = i64
-        L.gpga_oracle_quadratic_half_step.argtypes = [i64, i64, i64, f64, f64, u64, i64, P, P, P]
-        L.gpga_oracle_quadratic_half_step.restype = None
-        L.gpga_oracle_gradient_half_step.argtypes = [i64, i64, f64, P, P, P]
-        L.gpga_oracle_gradient_half_step.restype = None
-        L.gpga_oracle_mix_ring.argtypes = [i64, i64, P, P]
-        L.gpga_oracle_mix_ring.restype = None
-        L.gpga_oracle_mix_exp.argtypes = [i64, i64, i64, P, P]
-        L.gpga_oracle_mix_exp.restype = None
-        L.gpga_oracle_mix_global.argtypes = [i64, i64, P, P]
-        L.gpga_oracle_mix_global.restype = None
-        L.gpga_oracle_mix_grid.argtypes = [i64, i64, i64, P, P]
-        L.gpga_oracle_mix_grid.restype = None
-        L.gpga_oracle_mix_static_exp.argtypes = [i64, i64, P, P]
-        L.gpga_oracle_mix_static_exp.restype = None
-        L.gpga_oracle_consensus_distance.argtypes = [i64, i64, P]
-        L.gpga_oracle_consensus_distance.restype = f64
-        L.gpga_oracle_batch_indices.argtypes = [u64, i64, i64, i64, i64, P]
-        L.gpga_oracle_batch_indices.restype = None
-        L.gpga_oracle_logistic_loss.argtypes = [i64, i64, P, P, P, f64]
-        L.gpga_oracle_logistic_loss.restype = f64
-        L.gpga_oracle_logistic_grad.argtypes = [i64, P, P, P, i64, P, f64, P]
-        L.gpga_oracle_logistic_grad.restype = None
-        L.gpga_oracle_logistic_gradient_matrix.argtypes = [i64, i64, i64, i64, u64, i64, P, P, P,
-                                                           f64, P]
-        L.gpga_oracle_logistic_gradient_matrix.restype = None
-        L.gpga_oracle_init_b.argtypes = [i64, i64, i64, u64, f64, P]
-        L.gpga_oracle_init_b.restype = None
-        L.gpga_oracle_init_x0.argtypes = [i64, i64, i64, u64, i32, f64, P]
-        L.gpga_oracle_init_x0.restype = None
-        L.gpga_oracle_aga_update.argtypes = [i64, i64, i64, f64, P, P]
-        L.gpga_oracle_aga_update.restype = None
-        L.gpga_oracle_box_muller_many.argtypes = [P, P, i64, P]
-        L.gpga_oracle_box_muller_many.restype = None
-        L.gpga_oracle_quadratic_mean_loss.argtypes = [i64, i64, P, P]
-        L.gpga_oracle_quadratic_mean_loss.restype = f64
+    L = C.CDLL(str(path))
+    i64, i32, u32, u64, f64 = C.c_int64, C.c_int32, C.c_uint32, C.c_uint64, C.c_double
+    P = C.c_void_p
+    L.gpga_oracle_philox4x32_10.argtypes = [P, P, P]
+    L.gpga_oracle_philox4x32_10.restype = None
+    L.gpga_oracle_box_muller.argtypes = [u32, u32, P]
+    L.gpga_oracle_box_muller.restype = None
+    L.gpga_oracle_normal4.argtypes = [u64, u32, u32, u32, u32, P]
+    L.gpga_oracle_normal4.restype = None
+    L.gpga_oracle_is_global.argtypes = [i64, i64]
+    L.gpga_oracle_is_global.restype = i32
+    L.gpga_oracle_exp_hop.argtypes = [i64, i64]
+    L.gpga_oracle_exp_hop.restype = i64
+    L.gpga_oracle_quadratic_half_step.argtypes = [i64, i64, i64, f64, f64, u64, i64, P, P, P]
+    L.gpga_oracle_quadratic_half_step.restype = None
+    L.gpga_oracle_gradient_half_step.argtypes = [i64, i64, f64, P, P, P]
+    L.gpga_oracle_gradient_half_step.restype = None
+    L.gpga_oracle_mix_ring.argtypes = [i64, i64, P, P]
+    L.gpga_oracle_mix_ring.restype = None
+    L.gpga_oracle_mix_exp.argtypes = [i64, i64, i64, P, P]
+    L.gpga_oracle_mix_exp.restype = None
+    L.gpga_oracle_mix_global.argtypes = [i64, i64, P, P]
+    L.gpga_oracle_mix_global.restype = None
+    L.gpga_oracle_mix_grid.argtypes = [i64, i64, i64, P, P]
+    L.gpga_oracle_mix_grid.restype = None
+    L.gpga_oracle_mix_static_exp.argtypes = [i64, i64, P, P]
+    L.gpga_oracle_mix_static_exp.restype = None
+    L.gpga_oracle_consensus_distance.argtypes = [i64, i64, P]
+    L.gpga_oracle_consensus_distance.restype = f64
+    L.gpga_oracle_batch_indices.argtypes = [u64, i64, i64, i64, i64, P]
+    L.gpga_oracle_batch_indices.restype = None
+    L.gpga_oracle_logistic_loss.argtypes = [i64, i64, P, P, P, f64]
+    L.gpga_oracle_logistic_loss.restype = f64
+    L.gpga_oracle_logistic_grad.argtypes = [i64, P, P, P, i64, P, f64, P]
+    L.gpga_oracle_logistic_grad.restype = None
+    L.gpga_oracle_logistic_gradient_matrix.argtypes = [i64, i64, i64, i64, u64, i64, P, P, P,
+                                                       f64, P]
+    L.gpga_oracle_logistic_gradient_matrix.restype = None
+    L.gpga_oracle_init_b.argtypes = [i64, i64, i64, u64, f64, P]
+    L.gpga_oracle_init_b.restype = None
+    L.gpga_oracle_init_x0.argtypes = [i64, i64, i64, u64, i32, f64, P]
+    L.gpga_oracle_init_x0.restype = None
+    L.gpga_oracle_aga_update.argtypes = [i64, i64, i64, f64, P, P]
+    L.gpga_oracle_aga_update.restype = None
+    L.gpga_oracle_box_muller_many.argtypes = [P, P, i64, P]
+    L.gpga_oracle_box_muller_many.restype = None
+    L.gpga_oracle_quadratic_mean_loss.argtypes = [i64, i64, P, P]
+    L.gpga_oracle_quadratic_mean_loss.restype = f64
     return L
 
 

@@ -130,6 +130,17 @@ class Gpga:
         if st != GPGA_OK:
             raise GpgaError(st, lib().gpga_last_error(self._h).decode())
 
+    def _sp(self, stream):
+        """Stream pointer for a launch; the handle's device must be the current one (the library
+        launches on the current device and never switches it)."""
+        dev = getattr(self, "device", None)
+        if dev is not None:
+            import torch
+            if torch.cuda.current_device() != dev.index:
+                raise GpgaError(GPGA_ERR_INVALID_ARG,
+                                f"buffers live on {dev} but cuda:{torch.cuda.current_device()} is current")
+        return _stream_ptr(stream)
+
     def close(self):
         if self._h:
             lib().gpga_destroy(self._h)
@@ -171,6 +182,9 @@ class Gpga:
             scratch = torch.empty(self.scratch_bytes(), dtype=torch.uint8, device=x_a.device)
         for t in (x_a, x_b, data) + ((labels,) if labels is not None else ()):
             assert t.is_cuda and t.is_contiguous() and t.dtype == torch.float32
+            assert t.device == x_a.device, "all buffers of one handle must live on one device"
+        assert scratch.device == x_a.device, "all buffers of one handle must live on one device"
+        self.device = x_a.device
         self._keep = [x_a, x_b, data, labels, scratch]
         self.x_bufs = (x_a, x_b)
         self._check(lib().gpga_bind(self._h, x_a.data_ptr(), x_b.data_ptr(), data.data_ptr(),
@@ -192,41 +206,41 @@ class Gpga:
 
     # -- the path
     def init_from_seed(self, x0_kind=GPGA_X0_ZERO, x0_std=1.0, b_shift=0.0, stream=None):
-        self._check(lib().gpga_init_from_seed(self._h, x0_kind, x0_std, b_shift, _stream_ptr(stream)))
+        self._check(lib().gpga_init_from_seed(self._h, x0_kind, x0_std, b_shift, self._sp(stream)))
 
     def step(self, k, stream=None):
-        self._check(lib().gpga_step(self._h, k, _stream_ptr(stream)))
+        self._check(lib().gpga_step(self._h, k, self._sp(stream)))
 
     def run(self, K, stream=None):
-        self._check(lib().gpga_run(self._h, K, _stream_ptr(stream)))
+        self._check(lib().gpga_run(self._h, K, self._sp(stream)))
 
     def run_host(self, x0_host, data_host, K, x_out_host, stream=None):
         """x0_host, data_host, x_out_host: CPU float32 torch tensors (pinned for speed)."""
         self._check(lib().gpga_run_host(self._h, x0_host.data_ptr(), data_host.data_ptr(), K,
-                                        x_out_host.data_ptr(), _stream_ptr(stream)))
+                                        x_out_host.data_ptr(), self._sp(stream)))
 
     def consensus_distance(self, stream=None) -> float:
         out = C.c_double()
-        self._check(lib().gpga_consensus_distance(self._h, _stream_ptr(stream), C.byref(out)))
+        self._check(lib().gpga_consensus_distance(self._h, self._sp(stream), C.byref(out)))
         return out.value
 
     def mean_loss(self, stream=None) -> float:
         out = C.c_double()
-        self._check(lib().gpga_mean_loss(self._h, _stream_ptr(stream), C.byref(out)))
+        self._check(lib().gpga_mean_loss(self._h, self._sp(stream), C.byref(out)))
         return out.value
 
     def global_loss(self, stream=None) -> float:
         out = C.c_double()
-        self._check(lib().gpga_global_loss(self._h, _stream_ptr(stream), C.byref(out)))
+        self._check(lib().gpga_global_loss(self._h, self._sp(stream), C.byref(out)))
         return out.value
 
     def selftest_bounded_wait(self, stream=None):
-        self._check(lib().gpga_selftest_bounded_wait(self._h, _stream_ptr(stream)))
+        self._check(lib().gpga_selftest_bounded_wait(self._h, self._sp(stream)))
 
     def run_adaptive(self, K, H_init, warmup_iters, stream=None, max_periods=4096):
         periods = (_i64 * max_periods)()
         count = _i64()
-        self._check(lib().gpga_run_adaptive(self._h, K, H_init, warmup_iters, _stream_ptr(stream),
+        self._check(lib().gpga_run_adaptive(self._h, K, H_init, warmup_iters, self._sp(stream),
                                             periods, max_periods, C.byref(count)))
         return [int(periods[t]) for t in range(min(count.value, max_periods))]
 
@@ -305,8 +319,14 @@ def logistic_gradient_noalloc(A, y, x, batch, l2, seed, k, out=None, stream=None
     n, m, d = A.shape
     if out is None:
         out = torch.empty((n, d), dtype=torch.float32, device=A.device)
+    # the library runs on the current device with that device's scratch array: all tensors must
+    # live on one device, which is made current for the call
+    devices = {t.device for t in (A, y, x, out)}
+    if len(devices) != 1 or not A.is_cuda:
+        raise ValueError(f"A, y, x and out must be CUDA tensors on one device, got {sorted(map(str, devices))}")
     need = _i64()
-    st = lib().gpga_logistic_gradient_noalloc(A.data_ptr(), y.data_ptr(), x.data_ptr(), x.stride(0), n, d, m,
-                                              batch, l2, seed, k, out.data_ptr(), _stream_ptr(stream),
-                                              C.byref(need))
+    with torch.cuda.device(A.device):
+        st = lib().gpga_logistic_gradient_noalloc(A.data_ptr(), y.data_ptr(), x.data_ptr(), x.stride(0), n, d, m,
+                                                  batch, l2, seed, k, out.data_ptr(), _stream_ptr(stream),
+                                                  C.byref(need))
     return st, int(need.value), out

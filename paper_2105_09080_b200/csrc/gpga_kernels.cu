@@ -328,7 +328,6 @@ struct ExpTune { static constexpr int U = 4; static constexpr bool PIPE = false;
 struct GlobalTune { static constexpr int U = 4; static constexpr bool PIPE = false; static constexpr int BLOCK = 256; static constexpr int MINB = 4; };
 constexpr int kSmallBlock = 64;   // small problems: narrow blocks spread the column groups over more SMs
 
-#ifndef GPGA_TUNING_HARNESS
 #define GPGA_DISPATCH(kernel, T, p, mode, vec, s)                                                      \
     do {                                                                                               \
         const bool small = (p).Q < 148LL * 4 * T::BLOCK;                                               \
@@ -358,7 +357,6 @@ cudaError_t launch_step_global(const StepParams& p, int mode, bool vec, cudaStre
 {
     GPGA_DISPATCH(step_global_kernel, GlobalTune, p, mode, vec, s);
 }
-#endif  // GPGA_TUNING_HARNESS
 
 // ---------------------------------------------------------------------------
 // Consensus distance sum_j sum_i (x_ij - xbar_j)^2.  One pass over X: with

@@ -89,6 +89,16 @@ __global__ void __launch_bounds__(kLrBlock) logreg_partial_kernel(const LogregPa
 // 8.2 ms), so this is about one second: far beyond any copy's latency, and finite.
 constexpr uint32_t kTmaMaxTries = 1u << 18;
 
+// A block whose bounded wait gave up and that was given no error word to raise writes NaN over its
+// slice of the chunk partials (whole block calls): the sum over chunks, and so the gradient row of
+// node i, is then NaN instead of whatever an earlier call left in that slice.
+__device__ __forceinline__ void poison_partial(const LogregParams& p, int i, int c)
+{
+    float4* out4 = reinterpret_cast<float4*>(p.partial + ((long long)c * p.n + i) * p.d);
+    const float q = __int_as_float(0x7FC00000);
+    for (int g = threadIdx.x; g < (int)(p.d >> 2); g += blockDim.x) out4[g] = make_float4(q, q, q, q);
+}
+
 // Narrow rows (d <= kRegMaxD): the batch rows are staged in shared memory by bulk asynchronous
 // copies (one 16-byte-aligned row of d floats per copy, completion counted on an mbarrier) and
 // every warp runs its own pipeline -- it draws the indices of its rows (rows warp, warp + 8, ...
@@ -191,7 +201,11 @@ __global__ void __launch_bounds__(kLrBlock, 2) logreg_partial_tma_reg_kernel(con
     }
     grid_launch_dependents();   // the step kernel may take its place; it waits for this grid before reading
     if (__syncthreads_or(failed)) {
-        if (threadIdx.x == 0 && p.error_flag) atomicExch(p.error_flag, 1);
+        if (p.error_flag) {
+            if (threadIdx.x == 0) atomicExch(p.error_flag, 1);
+        } else {
+            poison_partial(p, i, c);   // no error word to raise: make the result visibly invalid, never stale
+        }
         return;
     }
     // every copy has landed and been read: park the per-warp sums in each warp's first slot
@@ -340,7 +354,10 @@ __global__ void __launch_bounds__(kLrBlock, 2) logreg_partial_tma_cols_kernel(co
         }
     }
     grid_launch_dependents();   // the step kernel may take its place; it waits for this grid before reading
-    if (failed) return;
+    if (failed) {   // block-uniform
+        if (!p.error_flag) poison_partial(p, i, c);
+        return;
+    }
     float4* out4 = reinterpret_cast<float4*>(p.partial + ((long long)c * p.n + i) * p.d);
 #pragma unroll
     for (int u = 0; u < J; ++u) {

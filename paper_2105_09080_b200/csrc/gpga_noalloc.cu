@@ -14,7 +14,16 @@
 //
 // Things a user must know:
 //  * The first call on each device looks up the array's device address (a symbol query,
-//    not an allocation).  Make that first call outside any CUDA stream capture.
+//    not an allocation).  Under CUDA's lazy module loading that first query or launch is also
+//    when the driver loads this library's device code and sets the array aside, and it may
+//    synchronise the device.  Make that first call at start-up, outside any CUDA stream
+//    capture and outside the region that must not stall.
+//  * All four buffers must belong to the device that is current when the call is made; the
+//    call checks this (a pointer query) and launches nothing otherwise.
+//  * There is no handle and so no error word.  If a bounded wait inside the gradient kernel
+//    gives up (an asynchronous row copy that does not complete within about a second), the
+//    block writes NaN over its slice of the partial sums, so the affected rows of G come
+//    out NaN rather than stale; the status, returned at launch time, is still GPGA_OK.
 //  * Every call on a device uses the same array.  It holds whatever the previous call
 //    left; each call overwrites every element before reading it, so nothing needs to be
 //    cleared -- but two calls that overlap on the GPU (different streams, or different
@@ -39,12 +48,10 @@ constexpr int kMaxDevices = 64;
 std::mutex g_setup_mutex;
 float* g_scratch_addr[kMaxDevices] = {nullptr};
 
-// Device address of the scratch array on the current device, looked up once per device.
-cudaError_t static_scratch(float** out)
+// Device address of the scratch array on device `dev` (the current one), looked up once per device.
+cudaError_t static_scratch(int dev, float** out)
 {
-    int dev = -1;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
+    cudaError_t e;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     std::lock_guard<std::mutex> lock(g_setup_mutex);
     if (!g_scratch_addr[dev]) {
@@ -55,6 +62,21 @@ cudaError_t static_scratch(float** out)
     }
     *out = g_scratch_addr[dev];
     return cudaSuccess;
+}
+
+// The kernels run on the current device and use that device's copy of the scratch array, so every
+// buffer must be memory that device owns (or managed memory).  A pointer query, not an allocation.
+// A buffer of another GPU would be an illegal address there -- or, with peer access enabled, would
+// quietly work while the partial sums land in the wrong device's array.
+bool on_device(const void* p, int dev)
+{
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, p) != cudaSuccess) {
+        (void)cudaGetLastError();   // a pointer CUDA does not know: not an error of the context
+        return false;
+    }
+    if (a.type == cudaMemoryTypeManaged) return true;
+    return a.type == cudaMemoryTypeDevice && a.device == dev;
 }
 
 }  // namespace
@@ -77,8 +99,13 @@ int32_t gpga_logistic_gradient_noalloc(const float* A_dev, const float* y_dev, c
     const long long need = (long long)logreg_chunks(batch) * n * d;
     if (needed_bytes_host) *needed_bytes_host = need * 4;
     if (need > kStaticScratchFloats) return GPGA_ERR_UNSUPPORTED;   // larger than the built-in scratch
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return GPGA_ERR_CUDA;
+    if (!on_device(A_dev, dev) || !on_device(y_dev, dev) || !on_device(x_dev, dev) || !on_device(G_dev, dev))
+        return GPGA_ERR_INVALID_ARG;   // not this device's memory: nothing is launched
     float* scratch = nullptr;
-    cudaError_t e = static_scratch(&scratch);
+    e = static_scratch(dev, &scratch);
     if (e != cudaSuccess) return GPGA_ERR_CUDA;
     LogregParams p;
     p.A = A_dev;
@@ -87,7 +114,7 @@ int32_t gpga_logistic_gradient_noalloc(const float* A_dev, const float* y_dev, c
     p.ldx = ldx;
     p.partial = scratch;
     p.G = G_dev;
-    p.error_flag = nullptr;
+    p.error_flag = nullptr;   // no handle, no error word: a block whose bounded wait gives up writes NaN instead
     p.n = n; p.d = d; p.m = m; p.batch = batch;
     p.k = (uint32_t)k;
     p.l2 = l2;

@@ -141,3 +141,24 @@ def test_generator_surface_argument_checks(L):
     assert L.gpga_philox_words(None, 0, 0, 4, None, None) == pkg.GPGA_ERR_INVALID_ARG
     assert L.gpga_box_muller_words(None, None, -1, None, None) == pkg.GPGA_ERR_INVALID_ARG
     assert L.gpga_normal_fill(1, 0, 0, 0, 0, 8, None, None) == pkg.GPGA_ERR_INVALID_ARG
+
+
+def test_noalloc_entry_point_checks_arguments_before_any_launch(L):
+    """Sizes are judged first (no CUDA call), then the pointers are looked up: addresses that are
+    not the current device's memory -- or no device at all, as on a CPU-only box -- end the call
+    with a status and nothing is launched."""
+    a, y, x, g = 0x10000, 0x20000, 0x30000, 0x40000       # fake aligned addresses, never dereferenced
+    need = C.c_int64(-1)
+    call = L.gpga_logistic_gradient_noalloc
+    assert call(a, y, x, 64, 4, 64, 16, 8, 0.0, 1, 0, g + 4, None, C.byref(need)) == pkg.GPGA_ERR_INVALID_ARG
+    assert call(a, y, x, 60, 4, 64, 16, 8, 0.0, 1, 0, g, None, C.byref(need)) == pkg.GPGA_ERR_INVALID_ARG   # ldx < d
+    assert call(a, y, x, 64, 4, 66, 16, 8, 0.0, 1, 0, g, None, C.byref(need)) == pkg.GPGA_ERR_INVALID_ARG   # d % 4
+    assert call(a, y, x, 64, 4, 64, 16, 8, -1.0, 1, 0, g, None, C.byref(need)) == pkg.GPGA_ERR_INVALID_ARG
+    assert call(a, y, x, 64, 4, 64, 16, 8, 0.0, 1, -1, g, None, C.byref(need)) == pkg.GPGA_ERR_INVALID_ARG
+    # too large for the built-in scratch: refused with the need reported, before any CUDA call
+    assert call(a, y, x, 4096, 64, 4096, 64, 256, 0.0, 1, 0, g, None, C.byref(need)) == pkg.GPGA_ERR_UNSUPPORTED
+    assert need.value == 8 * 64 * 4096 * 4 > binding.GPGA_NOALLOC_SCRATCH_BYTES
+    # sizes fine, pointers not device memory of a current device
+    st = call(a, y, x, 64, 4, 64, 16, 8, 0.0, 1, 0, g, None, C.byref(need))
+    assert st in (pkg.GPGA_ERR_INVALID_ARG, pkg.GPGA_ERR_CUDA)
+    assert need.value == 1 * 4 * 64 * 4

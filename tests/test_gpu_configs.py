@@ -156,21 +156,69 @@ def test_logistic_steps(topo, n, m, d, batch):
     assert abs(g.global_loss() - f_glob) <= 1e-4 * abs(f_glob)
 
 
-def test_config_5_logistic_reduced_iterations():
-    # n=64, m=4096, d=1024, batch 128, l2=1e-4, gamma=0.1; the oracle covers the first 40 of
-    # the 2000 iterations in seconds (ring, H=4 and exp, H=16)
-    n, m, d, batch = 64, 4096, 1024, 128
+@pytest.fixture(scope="module")
+def c5_data():
+    """The convex workload's data set (n = 64 nodes, m = 4096 samples of d = 1024 features) once
+    for all sweep points: fp32 for the GPU, and the same values widened to fp64 once for the
+    oracle (which otherwise converts all of A on every iteration)."""
+    torch = _torch()
+    n, m, d = 64, 4096, 1024
     A, y = logistic_inputs(n, m, d, SEED)
-    X0 = np.zeros((n, d), dtype=np.float32)
-    for topo, H in (("ring", 4), ("exp", 16)):
-        g, p = _make_logistic(n, m, d, batch, topo, H, 0.1, 1e-4, SEED, A, y, X0)
-        g.run(40)
-        want = o.run(p, X0, 0, 40)
-        ok, worst = close(g.get_x().cpu().numpy(), want, TOL_RUN)
-        assert ok, (topo, worst)
-        xi = o.consensus_distance(want)
-        assert abs(g.consensus_distance() - xi) <= 1e-4 * xi + 1e-12
-        g.close()
+    return dict(n=n, m=m, d=d, A=A, y=y, A64=A.astype(np.float64), y64=y.astype(np.float64),
+                A_dev=torch.from_numpy(A).cuda(), y_dev=torch.from_numpy(y).cuda())
+
+
+# the ten (topology, H) points of the sweep; H = 0 encodes H = infinity (pure gossip)
+C5_POINTS = [(topo, H) for topo in ("ring", "exp") for H in (1, 4, 16, 64, 0)]
+# (501 and 1502 fall between global averages for every finite H > 1 of the sweep)
+C5_CHECKPOINTS = (200, 501, 1000, 1502, 2000)
+
+
+@pytest.mark.parametrize("topo,H", C5_POINTS)
+def test_config_5_logistic_sweep_full_length(c5_data, topo, H):
+    """Every point of the sweep for its whole K = 2000 iterations (batch 128, l2 = 1e-4,
+    gamma = 0.1, X0 = 0) against the oracle, with the state, the consensus distance and the global
+    loss f(xbar) of problem (1) compared at k = 0, 200, 501, 1000, 1502 and 2000."""
+    torch = _torch()
+    c = c5_data
+    n, m, d, batch, l2, gamma = c["n"], c["m"], c["d"], 128, 1e-4, 0.1
+    g = pkg.Gpga(n, d, TOPO[topo][0], H, gamma, SEED)
+    g.set_objective(pkg.GPGA_OBJ_LOGISTIC, l2=l2, m=m, batch=batch)
+    xa = torch.zeros((n, d), dtype=torch.float32, device="cuda")
+    g.bind(xa, torch.empty_like(xa), c["A_dev"], c["y_dev"])
+    p = o.Problem(TOPO[topo][1], H, gamma, SEED, objective="logistic", data=c["A64"], labels=c["y64"], l2=l2,
+                  batch=batch)
+    want = np.zeros((n, d), dtype=np.float32)
+    f0 = o.global_logistic_loss(c["A64"], c["y64"], np.zeros(d), l2)
+    assert abs(f0 - np.log(2.0)) < 1e-12                     # loss at x = 0
+    assert abs(g.global_loss() - f0) <= 1e-6 * f0
+    k = 0
+    losses = [f0]
+    for k_next in C5_CHECKPOINTS:
+        g.run(k_next - k)
+        want = o.run(p, want, k, k_next - k)
+        k = k_next
+        got = g.get_x().cpu().numpy()
+        ok, worst = close(got, want, TOL_RUN)
+        assert ok, (topo, H, k, worst)
+        # the consensus-distance kernel against the oracle on the very state the GPU holds
+        xi_gpu = g.consensus_distance()
+        xi_same = o.consensus_distance(got)
+        assert abs(xi_gpu - xi_same) <= 1e-5 * xi_same, (topo, H, k, xi_gpu, xi_same)
+        # and against the oracle's own trajectory: sqrt(Xi) is the norm ||X - Xbar||_F, so the two
+        # differ by at most the norm of the difference of the states
+        xi_traj = o.consensus_distance(want)
+        gap = np.linalg.norm(got.astype(np.float64) - want.astype(np.float64))
+        assert abs(np.sqrt(xi_gpu) - np.sqrt(xi_traj)) <= gap * (1 + 1e-6) + 1e-12, (topo, H, k, xi_gpu, xi_traj)
+        if H and k % H == 0:
+            assert xi_gpu == 0.0 and xi_traj == 0.0           # rows identical after a global average
+        else:
+            assert xi_traj > 0.0 and xi_gpu > 0.0
+        f = o.global_logistic_loss(c["A64"], c["y64"], want.astype(np.float64).mean(0), l2)
+        assert abs(g.global_loss() - f) <= 1e-5 * f, (topo, H, k)
+        losses.append(f)
+    assert all(b < a for a, b in zip(losses, losses[1:]))     # the loss at the average keeps falling
+    g.close()
 
 
 # ------------------------------------------------------------------ Gossip-AGA

@@ -43,7 +43,18 @@ def _free_gib():
     return free / 2**30
 
 
-def _run_case(bufs, n, d, topo, H, gamma, sigma, K, x0_kind, x0_std, b_shift, offs, one_step_ks, ld=None):
+def _oracle_xi_of_device_state(x, d, chunk=1 << 20):
+    """Consensus distance of the state the GPU holds, recomputed by the oracle: X is downloaded in
+    column chunks and the oracle's value of every chunk is added up (the distance
+    sum_j sum_i (x_ij - xbar_j)^2 of Section 4 is a sum over columns)."""
+    total = 0.0
+    for c0 in range(0, d, chunk):
+        total += o.consensus_distance(x[:, c0:min(d, c0 + chunk)].cpu().numpy())
+    return total
+
+
+def _run_case(bufs, n, d, topo, H, gamma, sigma, K, x0_kind, x0_std, b_shift, offs, one_step_ks, ld=None,
+              check_xi=False):
     xa, xb, b, scratch = bufs
     ld = ld or d
     xa, xb, b = (t.view(-1)[:n * ld].view(n, ld) for t in (xa, xb, b))
@@ -80,6 +91,12 @@ def _run_case(bufs, n, d, topo, H, gamma, sigma, K, x0_kind, x0_std, b_shift, of
     assert np.isfinite(xi) and xi >= 0.0
     if H and K % H == 0:
         assert xi == 0.0            # ended on a global average: rows bit-identical
+    elif check_xi:
+        # the whole n x d state through the oracle: the kernel's strided pass over all column
+        # groups and its 64-bit element offsets, on a state whose rows differ
+        want = _oracle_xi_of_device_state(x, d)
+        assert want > 0.0
+        assert abs(xi - want) <= 1e-5 * want, (topo, H, xi, want)
     g.close()
 
 
@@ -100,8 +117,10 @@ def test_config_3_resnet50_sized():
             ks = [0]
             if H == 4:
                 ks = [0, 3] if topo == "ring" else [0, 1, 2, 3, 4, 5]   # hops 1..32; k=3 is global
+            # K = 50 ends between global averages for H = 16 and for pure gossip
             _run_case((xa, xb, b, scratch), n, d, topo, H, gamma, sigma, K,
-                      pkg.GPGA_X0_SHARED_NORMAL, 0.1, 0.5, offs, ks, ld=ld)
+                      pkg.GPGA_X0_SHARED_NORMAL, 0.1, 0.5, offs, ks, ld=ld,
+                      check_xi=(topo, H) in (("ring", 16), ("exp", 0)))
     # the dense layout (row stride d, rows not 128-byte aligned) once as well
     _run_case((xa, xb, b, scratch), n, d, "ring", 4, gamma, sigma, 8, pkg.GPGA_X0_SHARED_NORMAL, 0.1, 0.5,
               offs, [0], ld=d)
@@ -173,6 +192,10 @@ def test_config_4_bert_large_sized():
     offs = _blocks(d, 48, np.random.default_rng(4))
     _run_case((xa, xb, b, scratch), n, d, "exp", H, gamma, sigma, K, pkg.GPGA_X0_ZERO, 1.0, 0.0,
               offs, [0, 1, 2, 3])
+    # K = 18 ends two gossip steps after a global average: a non-zero consensus distance over
+    # n d > 2^32 elements, recomputed by the oracle from the downloaded state
+    _run_case((xa, xb, b, scratch), n, d, "exp", H, gamma, sigma, 18, pkg.GPGA_X0_ZERO, 1.0, 0.0,
+              offs[::6], [], check_xi=True)
     # a run of 32 iterations goes through the multi-iteration launch: 10.5 M strips of 8 column groups
     _run_case((xa, xb, b, scratch), n, d, "exp", H, gamma, sigma, 32, pkg.GPGA_X0_ZERO, 1.0, 0.0,
               offs[::2], [])

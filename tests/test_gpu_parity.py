@@ -261,7 +261,10 @@ def test_step_is_a_pure_function_and_resume_is_exact():
 
 
 # ------------------------------------------------------------------ consensus distance
-@pytest.mark.parametrize("n,d", [(1, 8), (2, 5), (8, 4100), (64, 777), (16, 100000)])
+# (8, 1_300_000) and (3, 1_250_003): more column groups than 1184 blocks of 256 threads cover in one
+# pass (d > 1.21 M), so every thread strides to a second group -- 128-bit and scalar paths
+@pytest.mark.parametrize("n,d", [(1, 8), (2, 5), (8, 4100), (64, 777), (16, 100000), (8, 1_300_000),
+                                 (3, 1_250_003)])
 def test_consensus_distance(n, d):
     X0, B = quadratic_inputs(n, d, 400 + n, x0="per_node")
     g, _ = make_quadratic(n, d, "ring", 0, 0.1, 1, 0.0, X0, B)
