@@ -5,18 +5,28 @@ A "step" is one iteration of Algorithm 1 over the whole n x d state: the fused
 local-update + gossip kernel, or the fused local-update + global-average kernel on
 every H-th iteration.  Prints one JSON line (rank 0).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3_ring_h4] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4_exp_h4] [--impl reference]
+
+Default workload: the BERT-Large-sized configuration (n = 16, d = 335,141,888, one-peer
+exponential graph, H = 4; 64.35 GB per step), or the ResNet-50-sized ring configuration when
+three 21.45 GB buffers do not fit the device; `config.workload` says which.  Beside the
+headline the line carries one roofline cell per target kernel and size (`cells`), a
+seconds-long loop with the sampled clocks (`sustained`), and one gpga_run call.
 
 Multi-GPU: the state is sharded by columns (columns evolve independently), one
 process per GPU, no data-path collective; every rank holds a full-width shard of a
-problem N times wider (weak scaling).
+problem N times wider (weak scaling).  `--gpus N` without a torchrun environment starts
+the N ranks itself.
 """
 from __future__ import annotations
 
 import argparse
 import hashlib
 import json
+import math
 import os
+import socket
+import subprocess
 import sys
 import threading
 import time
@@ -55,7 +65,9 @@ for _topo in ("ring", "exp"):
     for _H in (1, 4, 16, 64, 0):
         WORKLOADS[f"c5_{_topo}_h{_H or 'inf'}"] = dict(objective="logistic", n=64, d=1024, m=4096, batch=128, l2=1e-4,
                                                         topo=_topo, H=_H, gamma=0.1, K=2000)
-DEFAULT_WORKLOAD = "c3_ring_h4"
+DEFAULT_WORKLOAD = "c4_exp_h4"        # the largest single-GPU configuration
+FALLBACK_WORKLOAD = "c3_ring_h4"      # when three n x d buffers of the default do not fit the device
+NOMINAL_PEAK_GBS = 8000.0             # the HBM3e figure the 75 % target is quoted against
 
 # DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), as a multiple of the algorithmic bytes of the captured launch, with
@@ -87,7 +99,8 @@ def measured_peak_gbs():
 
 
 class ClockSampler(threading.Thread):
-    """Samples SM clock and clock-event reasons through NVML (read-only) while the timed region runs."""
+    """Samples SM clock and clock-event reasons through NVML (read-only) while a timed region runs.
+    One thread for the whole run; `begin()` opens a section, `end()` closes it and returns its summary."""
 
     def __init__(self, index: int, period_s: float = 0.02):
         super().__init__(daemon=True)
@@ -95,6 +108,7 @@ class ClockSampler(threading.Thread):
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._halt = threading.Event()
         self.active = threading.Event()
+        self.ready = threading.Event()
         self.error = None
 
     def run(self):
@@ -111,25 +125,40 @@ class ClockSampler(threading.Thread):
                         names.setdefault(v, attr.replace("nvmlClocksEventReason", "").replace("nvmlClocksThrottleReason", ""))
             get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
                 nv.nvmlDeviceGetCurrentClocksThrottleReasons
+            self.ready.set()
             while not self._halt.is_set():
                 if self.active.is_set():
-                    self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                    mhz = nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)
                     mask = get_reasons(h)
-                    for bit, nm in names.items():
-                        if mask & bit and bit.bit_count() == 1:
-                            self.reasons.add(nm)
+                    if self.active.is_set():
+                        self.samples.append(mhz)
+                        for bit, nm in names.items():
+                            if mask & bit and bit.bit_count() == 1:
+                                self.reasons.add(nm)
                 time.sleep(self.period)
             nv.nvmlShutdown()
         except Exception as exc:          # NVML missing: report it, do not fail the run
             self.error = repr(exc)
+            self.ready.set()
 
-    def finish(self):
-        self._halt.set()
-        self.join(timeout=2)
+    def begin(self):
+        if not self.is_alive() and not self._halt.is_set():
+            self.start()
+            self.ready.wait(timeout=5)
+        self.samples, self.reasons = [], set()
+        self.active.set()
+
+    def end(self):
+        self.active.clear()
         s = sorted(self.samples)
         return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
                 "reasons": sorted(r for r in self.reasons if r not in ("GpuIdle", "None")),
                 "samples": len(s), **({"error": self.error} if self.error else {})}
+
+    def finish(self):
+        self._halt.set()
+        if self.is_alive():
+            self.join(timeout=2)
 
 
 def physical_gpu_index(local: int) -> int:
@@ -173,7 +202,7 @@ def cpu_baseline(w, target_s=12.0):
                       f"{w['n']} rows, {t:.1f} s; columns are independent so throughput scales linearly in d"}
 
 
-def run_reference(args, w, name):
+def run_reference(args, w, name, choice=None):
     """--impl reference: the oracle on the host cores; each step = one iteration on a bounded slice."""
     from oracle import gpga_oracle as o
     rank = int(os.environ.get("RANK", "0"))
@@ -206,7 +235,7 @@ def run_reference(args, w, name):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": workload_config(name, w, args.gpus),
+        "data": "synthetic", "config": workload_config(name, w, args.gpus, choice),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": o.num_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
@@ -216,19 +245,146 @@ def padded_stride(d):
     return (d + 31) // 32 * 32
 
 
-def workload_config(name, w, n_gpus):
-    return {"workload": f"{name}: n={w['n']} nodes x d={w['d']} fp32, {w['topo']} topology, H={w['H'] or 'inf'}, "
-                        f"gamma={w['gamma']}, sigma={w['sigma']}, quadratic objective, seed {SEED}",
-            "l2_flush": f"none needed: each step streams {BYTES_PER_UPDATE * w['n'] * w['d'] / 1e9:.2f} GB, larger than the 126 MB L2"
-                        if BYTES_PER_UPDATE * w['n'] * w['d'] > 4 * 126e6 else "state fits in L2; reported as L2-resident",
-            "layout": f"row-major fp32, row stride {padded_stride(w['d'])} floats (rows padded to 128 B)",
-            "sharding": f"columns, {n_gpus} shard(s) of d columns each, no collective"}
+def workload_config(name, w, n_gpus, note=None):
+    cfg = {"workload": f"{name}: n={w['n']} nodes x d={w['d']} fp32, {w['topo']} topology, H={w['H'] or 'inf'}, "
+                       f"gamma={w['gamma']}, sigma={w['sigma']}, quadratic objective, seed {SEED}",
+           "l2_flush": f"none needed: each step streams {BYTES_PER_UPDATE * w['n'] * w['d'] / 1e9:.2f} GB, larger than the 126 MB L2"
+                       if BYTES_PER_UPDATE * w['n'] * w['d'] > 4 * 126e6 else "state fits in L2; reported as L2-resident",
+           "layout": f"row-major fp32, row stride {padded_stride(w['d'])} floats (rows padded to 128 B)",
+           "sharding": f"columns, {n_gpus} shard(s) of d columns each, no collective"}
+    if note:
+        cfg["choice"] = note
+    return cfg
+
+
+def state_bytes(w):
+    return 3 * w["n"] * padded_stride(w["d"]) * 4
+
+
+def resolve_workload(args, torch=None, dist=None):
+    """The workload to run: the one asked for, else the largest single-GPU configuration when three
+    of its n x d buffers fit the device (every rank's), else the ResNet-50-sized one."""
+    if args.workload:
+        return args.workload, None
+    fits = 1
+    if torch is not None and torch.cuda.is_available():
+        free, _ = torch.cuda.mem_get_info()
+        fits = int(free >= state_bytes(WORKLOADS[DEFAULT_WORKLOAD]) + (3 << 30))
+        if dist is not None:
+            t = torch.tensor([fits], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MIN)
+            fits = int(t.item())
+    if fits:
+        return DEFAULT_WORKLOAD, "default: the largest configuration that fits one GPU"
+    return FALLBACK_WORKLOAD, (f"fallback: 3 x {state_bytes(WORKLOADS[DEFAULT_WORKLOAD]) / 3e9:.2f} GB of "
+                               f"{DEFAULT_WORKLOAD} do not fit the free device memory")
+
+
+# ---------------------------------------------------------------------------------
+# Arithmetic the method itself needs per node-parameter update (quadratic objective with noise),
+# counted from the generator's published definition and Algorithm 1 -- not from any kernel:
+#   Philox4x32-10, one call per 4 updates: 10 rounds x (2 wide multiplies + 2 three-input xors)  -> 10 per update
+#   Box-Muller, one pair per 2 updates: 2 int->float conversions, 2 scalings of the uniforms,
+#     lg2, the multiply by -2 ln 2, sqrt, sin, cos, 2 products r cos, r sin = 11                  -> 5.5 per update,
+#     of which the 4 special-function evaluations                                                -> 2 per update
+#   stochastic gradient and local update: x - b, fma(sigma, z, .), fma(-gamma, g, x)             -> 3 per update
+#   mix: ring 2 adds + 1 multiply = 3; one-peer exponential 1 add + 1 multiply = 2; global
+#     average 1 add per update (+ 1/n of a division)                                             -> 3 / 2 / 1
+# An SM issues 4 warp instructions per clock (128 lane operations) and evaluates 16 special
+# functions per clock (four per scheduler), the per-SM figures of CUDA's arithmetic-throughput table.
+# ---------------------------------------------------------------------------------
+LANE_OPS_PHILOX, LANE_OPS_BOX_MULLER, LANE_OPS_UPDATE = 10.0, 5.5, 3.0
+LANE_OPS_MIX = {"ring": 3.0, "exp": 2.0, "global": 1.0}
+XU_OPS_PER_UPDATE = 2.0
+SM_COUNT, ISSUE_LANES_PER_CLK, XU_LANES_PER_CLK = 148, 128, 16
+
+
+def method_lane_ops(w):
+    share_global = (1.0 / w["H"]) if w["H"] else 0.0
+    mix = share_global * LANE_OPS_MIX["global"] + (1.0 - share_global) * LANE_OPS_MIX[w["topo"]]
+    noise = LANE_OPS_PHILOX + LANE_OPS_BOX_MULLER if w["sigma"] else 0.0
+    return noise + LANE_OPS_UPDATE + mix
+
+
+def alu_roofline(w, rate, kernel, sm_max_mhz, achieved_gbs):
+    """Compute-bound roofline of a state that stays on chip: the rate against what the issue slots and
+    the special-function units allow for the method's own operation count."""
+    hz = (sm_max_mhz or 1965) * 1e6
+    ops = method_lane_ops(w)
+    peak_issue = SM_COUNT * ISSUE_LANES_PER_CLK * hz / ops
+    peak_xu = SM_COUNT * XU_LANES_PER_CLK * hz / XU_OPS_PER_UPDATE if w["sigma"] else float("inf")
+    peak = min(peak_issue, peak_xu)
+    return {"bound": "alu", "kernel": kernel, "achieved": rate / 1e9, "peak": peak / 1e9,
+            "unit": "G node-param updates/s", "frac": rate / peak, "traffic": None,
+            "binding_unit": "issue slots" if peak_issue <= peak_xu else "special-function units",
+            "method_lane_ops_per_update": ops, "frac_of_issue_peak": rate / peak_issue,
+            "frac_of_special_function_peak": (rate / peak_xu) if w["sigma"] else None,
+            "peak_kind": f"derived: {SM_COUNT} SMs x {ISSUE_LANES_PER_CLK} lanes/clk (special functions: "
+                         f"{XU_LANES_PER_CLK}/clk) x {hz / 1e6:.0f} MHz / the method's operations per update",
+            "note": "state resident on chip across iterations; HBM is touched once per launch",
+            "effective_GB/s_at_12B_per_update": achieved_gbs}
+
+
+# one roofline cell per target kernel and size: name, n, d, topology, H (0: gossip only, 1: global average only)
+C3_D, C4_D = 25_557_032, 335_141_888
+CELLS = [("c3_ring", 64, C3_D, "ring", 0, "shared", 0.1, 0.5), ("c3_exp", 64, C3_D, "exp", 0, "shared", 0.1, 0.5),
+         ("c3_global", 64, C3_D, "ring", 1, "shared", 0.1, 0.5),
+         ("c4_exp", 16, C4_D, "exp", 0, "zero", 1.0, 0.0), ("c4_global", 16, C4_D, "exp", 1, "zero", 1.0, 0.0)]
+
+
+def timed_steps(torch, g, steps):
+    """`steps` calls of gpga_step, one CUDA event pair each, on torch's current stream (the stream the
+    kernels are launched on); returns the per-step milliseconds."""
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    k0 = g.get_k()
+    ev[0].record()
+    for s in range(steps):
+        g.step(k0 + s)
+        ev[s + 1].record()
+    torch.cuda.synchronize()
+    return [ev[s].elapsed_time(ev[s + 1]) for s in range(steps)]
+
+
+def median(v):
+    v = sorted(v)
+    return v[len(v) // 2] if v else None
+
+
+def loop_for(torch, g, sampler, seconds, est_ms):
+    """Step loop of about `seconds` with the clocks sampled beside it."""
+    steps = int(max(8, min(20000, math.ceil(seconds * 1e3 / max(est_ms, 1e-3)))))
+    sampler.begin()
+    ms = timed_steps(torch, g, steps)
+    clocks = sampler.end()
+    return ms, clocks
+
+
+def run_cell(torch, pkg, bufs, spec, sampler, seconds, peak):
+    name, n, d, topo, H, x0, x0_std, b_shift = spec
+    ld = padded_stride(d)
+    if bufs[0].numel() < n * ld:
+        return {"skipped": "the bound buffers are smaller than this state"}
+    views = [t.view(-1)[:n * ld].view(n, ld) for t in bufs]
+    g = pkg.Gpga(n, d, {"ring": pkg.GPGA_TOPO_RING, "exp": pkg.GPGA_TOPO_EXP}[topo], H, 0.01, SEED)
+    g.set_objective(pkg.GPGA_OBJ_QUADRATIC, sigma=0.01)
+    g.set_row_stride(ld)
+    g.bind(*views)
+    g.init_from_seed({"zero": pkg.GPGA_X0_ZERO, "shared": pkg.GPGA_X0_SHARED_NORMAL}[x0], x0_std, b_shift)
+    est = median(timed_steps(torch, g, 3))
+    ms, clocks = loop_for(torch, g, sampler, seconds, est)
+    g.close()
+    med, algo = median(ms), BYTES_PER_UPDATE * n * d
+    gbs = algo / (med * 1e-3) / 1e9
+    return {"kernel": "step_global_kernel" if H == 1 else f"step_{topo}_kernel", "n": n, "d": d, "steps": len(ms),
+            "ms": med, "GB/s": gbs, "frac": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_PEAK_GBS,
+            "sm_mhz": clocks["sm_mhz"], "reasons": clocks["reasons"],
+            "ms_x_mhz": med * clocks["sm_mhz"] if clocks["sm_mhz"] else None}
 
 
 # ---------------------------------------------------------------------------------
 # CUDA arm
 # ---------------------------------------------------------------------------------
-def run_ours(args, w, name):
+def run_ours(args):
     import torch
     import paper_2105_09080_b200 as pkg
 
@@ -242,6 +398,17 @@ def run_ours(args, w, name):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    name, choice = resolve_workload(args, torch, dist)
+    w = WORKLOADS[name]
+    if w.get("objective") == "logistic":
+        if dist is not None:
+            dist.destroy_process_group()
+        if rank == 0:
+            run_logistic(args, w, name)
+        return
+    resident = BYTES_PER_UPDATE * w["n"] * padded_stride(w["d"]) <= (64 << 20)
+    if args.steps is None:
+        args.steps = 100_000 if resident else 200
 
     n, d = w["n"], w["d"]
     topo = {"ring": pkg.GPGA_TOPO_RING, "exp": pkg.GPGA_TOPO_EXP}[w["topo"]]
@@ -261,43 +428,44 @@ def run_ours(args, w, name):
             dist.barrier()
             torch.cuda.synchronize()
 
+    def max_over_ranks(ms):
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
     # A state of at most 64 MB is advanced many iterations per launch by gpga_run (strips resident
-    # in shared memory): one call, no per-step events.  Larger states: one launch per step.
-    resident = BYTES_PER_UPDATE * n * padded_stride(d) <= (64 << 20)
-    events = [torch.cuda.Event(enable_timing=True) for _ in range(2 if resident else args.steps + 1)]
+    # on chip): one call, no per-step events.  Larger states: one launch per step.
     if resident:
         g.run(max(args.warmup, 2))      # the same multi-iteration kernel as the timed call
     else:
         for _ in range(args.warmup):
             g.step(g.get_k())
-    barrier()
     sampler = ClockSampler(physical_gpu_index(local))
-    sampler.start()
+    barrier()
     launches0 = g.launch_count()
     k_first = g.get_k()
-    sampler.active.set()
-    events[0].record()
+    sampler.begin()
     if resident:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
         g.run(args.steps)
-        events[-1].record()
+        e1.record()
+        barrier()
+        per_step, elapsed_ms = [], e0.elapsed_time(e1)
     else:
-        for s in range(args.steps):
-            g.step(k_first + s)
-            events[s + 1].record()
-    barrier()
-    sampler.active.clear()
-    clocks = sampler.finish()
+        per_step = timed_steps(torch, g, args.steps)
+        barrier()
+        elapsed_ms = sum(per_step)
+    clocks = sampler.end()
     launches = g.launch_count() - launches0
-    elapsed_ms = events[0].elapsed_time(events[-1])
-    per_step = [] if resident else [events[s].elapsed_time(events[s + 1]) for s in range(args.steps)]
-    if dist is not None:
-        t = torch.tensor([elapsed_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = max_over_ranks(elapsed_ms)
 
     # per-kernel durations from the per-step events (one kernel per step)
-    glob = [ms for s, ms in enumerate(per_step) if w["H"] and (k_first + s + 1) % w["H"] == 0]
-    goss = [ms for s, ms in enumerate(per_step) if not (w["H"] and (k_first + s + 1) % w["H"] == 0)]
+    is_glob = lambda k: bool(w["H"]) and (k + 1) % w["H"] == 0
+    glob = [ms for s, ms in enumerate(per_step) if is_glob(k_first + s)]
+    goss = [ms for s, ms in enumerate(per_step) if not is_glob(k_first + s)]
     peak, peak_kind = measured_peak_gbs()
     algo_bytes = BYTES_PER_UPDATE * n * d
     kernels = {}
@@ -312,25 +480,39 @@ def run_ours(args, w, name):
     traffic = None
     if dominant in NCU_TRAFFIC and NCU_TRAFFIC[dominant][1] == kernel_source_digest():
         traffic = NCU_TRAFFIC[dominant][0] * algo_bytes
+    sustained, cells = None, None
     if resident:
-        # Compute-bound: X and b stay on chip.  Peak = SMs x 128 lanes/clk x max SM clock / lane
-        # operations per update (42 = the 169 warp instructions that run_cell_kernel executes per warp
-        # and iteration, ncu smsp__inst_executed, over the 4 updates of a thread).
-        alu_peak = 148 * 128 * (clocks.get("sm_max_mhz") or 1965) * 1e6 / 42.0
-        rate = n * d / (kernels[dominant] * 1e-3)
-        roofline = {"bound": "alu", "kernel": dominant, "achieved": rate / 1e9, "peak": alu_peak / 1e9,
-                    "unit": "G node-param updates/s", "frac": rate / alu_peak, "traffic": None,
-                    "note": "state resident in shared memory across iterations; HBM is touched once per launch",
-                    "effective_GB/s_at_12B_per_update": achieved}
+        roofline = alu_roofline(w, n * d / (kernels[dominant] * 1e-3), dominant, clocks.get("sm_max_mhz"), achieved)
     else:
-      roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
-                "algorithmic_bytes_per_launch": algo_bytes,
-                "per_kernel": {nm: {"ms": ms, "GB/s": algo_bytes / (ms * 1e-3) / 1e9,
-                                    "frac": algo_bytes / (ms * 1e-3) / 1e9 / peak} for nm, ms in kernels.items()},
-                "frac_of_nominal_8TBs": achieved / 8000.0}
+        roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                    "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
+                    "algorithmic_bytes_per_launch": algo_bytes,
+                    "frac_of_nominal_8TBs": achieved / NOMINAL_PEAK_GBS}
+        for nm, ms in kernels.items():      # flat: one scalar per kernel of the timed loop
+            roofline[f"{nm}_ms"] = ms
+            roofline[f"{nm}_GBs"] = algo_bytes / (ms * 1e-3) / 1e9
+        # the same loop for seconds, not milliseconds: what the board sustains under its power cap
+        barrier()
+        ms, sclk = loop_for(torch, g, sampler, args.sustained_seconds, elapsed_ms / args.steps)
+        med = max_over_ranks(median(ms))
+        sustained = {"seconds": sum(ms) * 1e-3, "steps": len(ms), "median_ms_per_step": med,
+                     "value": n * d * world / (med * 1e-3), "GB/s": algo_bytes / (med * 1e-3) / 1e9,
+                     "frac": algo_bytes / (med * 1e-3) / 1e9 / peak,
+                     "frac_of_nominal_8TBs": algo_bytes / (med * 1e-3) / 1e9 / NOMINAL_PEAK_GBS,
+                     "sm_mhz": sclk["sm_mhz"], "reasons": sclk["reasons"], "clock_samples": sclk["samples"],
+                     "ms_x_mhz": med * sclk["sm_mhz"] if sclk["sm_mhz"] else None}
+        if world == 1 and not args.no_cells and state_bytes(w) >= state_bytes(WORKLOADS[FALLBACK_WORKLOAD]):
+            cells = {}
+            for spec in CELLS:
+                cells[spec[0]] = run_cell(torch, pkg, (xa, xb, b), spec, sampler, args.cell_seconds, peak)
+                c = cells[spec[0]]
+                if "GB/s" in c:     # flat copies inside `roofline`
+                    roofline[f"cell_{spec[0]}_GBs"] = c["GB/s"]
+                    roofline[f"cell_{spec[0]}_frac_of_nominal_8TBs"] = c["frac_of_nominal_8TBs"]
+            g.init_from_seed(kind, w["x0_std"], w["b_shift"])     # the cells used the same buffers
+            for _ in range(3):
+                g.step(g.get_k())
 
-    # end to end through the host entry point: pinned host buffers in, K iterations, result out
     # the consensus-distance diagnostic (off the timed loop): one pass over X, 4 bytes per element
     c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     g.consensus_distance()
@@ -344,48 +526,46 @@ def run_ours(args, w, name):
                  "note": "includes the result read-back and stream synchronisation",
                  "launches": g.launch_count() - launches_c}
 
-    # the same iterations through gpga_run: for n <= 128 and long runs it advances many iterations
-    # per launch with the cells on chip, so its rate is not tied to 12 bytes per update
+    # one gpga_run call over the configuration's own run length (at least 32 iterations): for
+    # n <= 128 and runs that long it advances many iterations per launch with the cells on chip, so
+    # its rate is not tied to 12 bytes per update
     run_info = None
     if not resident:
+        K_run = max(w["K"], 32)
         barrier()
         r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         launches_r = g.launch_count()
         r0.record()
-        g.run(args.steps)
+        g.run(K_run)
         r1.record()
         barrier()
-        run_ms = r0.elapsed_time(r1)
-        if dist is not None:
-            t = torch.tensor([run_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            run_ms = float(t.item())
-        run_info = {"value": n * d * args.steps * world / (run_ms * 1e-3), "unit": UNIT, "iterations": args.steps,
-                    "ms_per_iteration": run_ms / args.steps, "launches": g.launch_count() - launches_r,
-                    "note": "one gpga_run call over the same number of iterations, after the timed loop; "
-                            "reported beside `value`, which times one launch per iteration"}
+        run_ms = max_over_ranks(r0.elapsed_time(r1))
+        run_info = {"value": n * d * K_run * world / (run_ms * 1e-3), "unit": UNIT, "iterations": K_run,
+                    "ms_per_iteration": run_ms / K_run, "launches": g.launch_count() - launches_r,
+                    "note": "one gpga_run call, after the timed loop; `value` above times one launch per iteration"}
 
     e2e = None
     if not args.no_e2e:
         try:
-            e2e = run_e2e(torch, g, w, dist)
+            e2e = run_e2e(torch, pkg, (xa, xb, b), w, dist, rank)
         except Exception as exc:     # e.g. not enough pinnable host memory for the host copies
             e2e = {"value": None, "unit": UNIT, "error": repr(exc)[:200]}
+    sampler.finish()
 
     value = n * d * args.steps * world / (elapsed_ms * 1e-3)
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": workload_config(name, w, world), "hbm_gbs": value * BYTES_PER_UPDATE / 1e9 / world,
+            "config": workload_config(name, w, world, choice), "hbm_gbs": value * BYTES_PER_UPDATE / 1e9 / world,
             "roofline": roofline, "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
-            "consensus_distance": consensus, "gpga_run": run_info}
+            "sustained": sustained, "cells": cells, "consensus_distance": consensus, "gpga_run": run_info}
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             try:
                 line["cpu_baseline"] = cpu_baseline(w)
             except Exception as exc:
                 line["cpu_baseline"] = {"value": None, "unit": UNIT, "kind": "oracle", "error": repr(exc)[:200]}
-        print(json.dumps(line))
+        print(json.dumps(line), flush=True)
     g.close()
     if dist is not None:
         dist.destroy_process_group()
@@ -409,16 +589,15 @@ def run_logistic(args, w, name):
     g.run(max(args.warmup, 50))         # the same back-to-back launches as the timed call
     torch.cuda.synchronize()
     sampler = ClockSampler(physical_gpu_index(int(os.environ.get("LOCAL_RANK", "0"))))
-    sampler.start()
     launches0 = g.launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler.active.set()
+    sampler.begin()
     e0.record()
     g.run(args.steps)
     e1.record()
     torch.cuda.synchronize()
-    sampler.active.clear()
-    clocks = sampler.finish()
+    clocks = sampler.end()
+    sampler.finish()
     ms = e0.elapsed_time(e1)
     launches = g.launch_count() - launches0
     if launches < args.steps:      # gpga_run took the many-iterations-per-launch kernel
@@ -472,13 +651,38 @@ def run_logistic(args, w, name):
     print(json.dumps(line))
 
 
-def run_e2e(torch, g, w, dist):
+def host_memory_available():
+    try:
+        for ln in open("/proc/meminfo"):
+            if ln.startswith("MemAvailable:"):
+                return int(ln.split()[1]) * 1024
+    except OSError:
+        pass
+    return None
+
+
+def e2e_columns(n, d, world):
+    """Columns of the end-to-end job: all d when the three pinned host buffers of every rank fit in
+    70 % of the host's available memory, else as many as do (a multiple of 32, at least 4096)."""
+    avail = host_memory_available()
+    need = 3 * n * d * 4 * world
+    if avail is None or need <= 0.7 * avail:
+        return d
+    cols = int(0.7 * avail / world / (3 * n * 4)) // 32 * 32
+    return max(4096, min(d, cols))
+
+
+def run_e2e(torch, pkg, bufs, w, dist, rank):
+    """The configuration's K iterations through gpga_run_host: pinned host X0 and b in, X^(K) out."""
+    from paper_2105_09080_b200.sharding import weak_shard_offset
     n, d, K = w["n"], w["d"], w["K"]
+    world = dist.get_world_size() if dist is not None else 1
+    cols = e2e_columns(n, d, world)
     problem = None
     try:
-        x0 = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
-        bh = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
-        out = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+        x0 = torch.empty((n, cols), dtype=torch.float32, pin_memory=True)
+        bh = torch.empty((n, cols), dtype=torch.float32, pin_memory=True)
+        out = torch.empty((n, cols), dtype=torch.float32, pin_memory=True)
     except Exception as exc:        # not enough pinnable host memory on this rank
         problem = repr(exc)[:200]
     if dist is not None:            # every rank must take the same branch before the next collective
@@ -488,10 +692,17 @@ def run_e2e(torch, g, w, dist):
             problem = "another rank could not pin its host buffers"
     if problem:
         return {"value": None, "unit": UNIT, "error": problem}
+    ld = padded_stride(cols)
+    views = [t.view(-1)[:n * ld].view(n, ld) for t in bufs]
+    g = pkg.Gpga(n, cols, {"ring": pkg.GPGA_TOPO_RING, "exp": pkg.GPGA_TOPO_EXP}[w["topo"]], w["H"], w["gamma"], SEED)
+    g.set_objective(pkg.GPGA_OBJ_QUADRATIC, sigma=w["sigma"])
+    g.set_column_offset(weak_shard_offset(rank, d))
+    g.set_row_stride(ld)
+    g.bind(*views)
     # host copies of the seeded inputs (downloaded once, outside the timed region)
     g.init_from_seed({"zero": 0, "shared": 1}[w["x0"]], w["x0_std"], w["b_shift"])
-    x0.copy_(g.x_bufs[0][:, :d])
-    bh.copy_(g._keep[2][:, :d])
+    x0.copy_(views[0][:, :cols])
+    bh.copy_(views[2][:, :cols])
     torch.cuda.synchronize()
     g.run_host(x0, bh, K, out)                      # warm-up job
     if dist is not None:
@@ -505,20 +716,67 @@ def run_e2e(torch, g, w, dist):
     e1.record()
     torch.cuda.synchronize()
     dt = e0.elapsed_time(e1) * 1e-3                 # device time, copies included
-    world = 1
+    g.close()
     if dist is not None:
         t = torch.tensor([dt], device="cuda", dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         dt = float(t.item())
-        world = dist.get_world_size()
-    return {"value": n * d * K * jobs * world / dt, "unit": UNIT,
-            "h2d_bytes_per_step": 2 * n * d * 4 / K, "d2h_bytes_per_step": n * d * 4 / K,
-            "job": f"gpga_run_host: pinned host X0 and b copied in ({2 * n * d * 4 / 1e9:.2f} GB), K={K} iterations, "
-                   f"X copied out ({n * d * 4 / 1e9:.2f} GB); bytes per step are the job's bytes / K",
+    width = "all" if cols == d else f"the first {cols} of"
+    return {"value": n * cols * K * jobs * world / dt, "unit": UNIT,
+            "h2d_bytes_per_step": 2 * n * cols * 4 / K, "d2h_bytes_per_step": n * cols * 4 / K,
+            "job": f"gpga_run_host on {width} {d} columns: pinned host X0 and b copied in "
+                   f"({2 * n * cols * 4 / 1e9:.2f} GB), K={K} iterations, X copied out ({n * cols * 4 / 1e9:.2f} GB); "
+                   f"bytes per step are the job's bytes / K",
             "seconds_per_job": dt / jobs}
 
 
-def main():
+def run_dry(args):
+    """--dry-run: the multi-rank plumbing without CUDA (gloo): every rank takes its column shard,
+    the ranks meet at a barrier, a per-rank number is reduced with MAX as the timing is, and rank 0
+    prints one JSON line.  Used by the CPU tests of the launch path."""
+    import torch
+    import torch.distributed as dist
+    from paper_2105_09080_b200.sharding import weak_shard_offset
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    name = args.workload or DEFAULT_WORKLOAD
+    w = WORKLOADS[name]
+    if world > 1:
+        dist.init_process_group("gloo")
+    shard = (rank, weak_shard_offset(rank, w["d"]), w["d"])
+    shards, slowest = [shard], float(rank + 1)
+    if world > 1:
+        shards = [None] * world
+        dist.all_gather_object(shards, shard)
+        dist.barrier()
+        t = torch.tensor([slowest], dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        slowest = float(t.item())
+    if rank == 0:
+        print(json.dumps({"dry_run": True, "metric": METRIC, "unit": UNIT, "n_gpus": world, "value": None,
+                          "config": workload_config(name, w, world), "scaling": "weak",
+                          "shards": [list(x) for x in sorted(shards)], "max_over_ranks": slowest}), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def spawn_ranks(n_ranks, argv):
+    """Start n_ranks copies of this script, one per GPU, the way the multi-GPU contract launches it."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_ranks}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), str(Path(__file__).resolve())] + list(argv)
+    return subprocess.call(cmd)
+
+
+def main(argv=None):
+    argv = list(sys.argv[1:] if argv is None else argv)
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None,
@@ -526,29 +784,41 @@ def main():
                          "logistic workload, so that the timed region lasts milliseconds, not microseconds)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default=None, choices=sorted(WORKLOADS),
+                    help=f"default: {DEFAULT_WORKLOAD}, or {FALLBACK_WORKLOAD} when it does not fit the device")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    args = ap.parse_args()
+    ap.add_argument("--no-cells", action="store_true", help="skip the per-kernel roofline cells")
+    ap.add_argument("--sustained-seconds", type=float, default=2.0)
+    ap.add_argument("--cell-seconds", type=float, default=1.0)
+    ap.add_argument("--dry-run", action="store_true", help="multi-rank plumbing only, on CPU with gloo")
+    args = ap.parse_args(argv)
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
-    w = WORKLOADS[args.workload]
-    if args.steps is None:
+    under_launcher = "WORLD_SIZE" in os.environ and "RANK" in os.environ
+    if args.gpus > 1 and not under_launcher and args.impl == "ours":
+        sys.exit(spawn_ranks(args.gpus, argv))       # one process per GPU; rank 0 prints the line
+    if args.dry_run:
+        return run_dry(args)
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) != 0:
+            return                                    # rank 0 alone runs the oracle
+        torch = None
+        try:
+            import torch
+        except Exception:
+            pass
+        name, choice = resolve_workload(args, torch)
+        w = WORKLOADS[name]
         if w.get("objective") == "logistic":
-            args.steps = 2000
-        elif BYTES_PER_UPDATE * w["n"] * padded_stride(w["d"]) <= (64 << 20):
-            args.steps = 100_000
-        else:
-            args.steps = 200
-    if w.get("objective") == "logistic":
-        if args.impl == "reference":
             print(json.dumps({"impl": "reference", "unavailable": "reference arm is defined for the quadratic workloads"}))
-        else:
-            run_logistic(args, w, args.workload)
-    elif args.impl == "reference":
-        run_reference(args, w, args.workload)
-    else:
-        run_ours(args, w, args.workload)
+            return
+        if args.steps is None:
+            args.steps = 20
+        return run_reference(args, w, name, choice)
+    if args.steps is None and args.workload and WORKLOADS[args.workload].get("objective") == "logistic":
+        args.steps = 2000
+    run_ours(args)
 
 
 if __name__ == "__main__":
