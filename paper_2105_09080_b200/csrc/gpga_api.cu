@@ -14,6 +14,11 @@
 
 using namespace gpga;
 
+// Scratch layout: [reduction partials | result double | G | gradient chunk partials | published rows]
+struct ScratchLayout {
+    int64_t slots = 0, partials_off = 0, result_off = 0, G_off = 0, chunk_off = 0, ytag_off = 0, ytag_bytes = 0, total = 0;
+};
+
 struct gpga_ctx {
     int64_t n = 0, d = 0, H = 0;
     int32_t topology = 0;
@@ -30,6 +35,7 @@ struct gpga_ctx {
     const float* labels = nullptr;
     char* scratch = nullptr;
     int64_t scratch_bytes = 0;
+    ScratchLayout L;   // layout of the scratch area, fixed by gpga_bind (the host entry narrows d per chunk)
     int cur = 0;
     int64_t k = 0;
     int64_t launches = 0;
@@ -76,15 +82,14 @@ int log2_floor(int64_t v) { int t = 0; while ((int64_t(1) << (t + 1)) <= v) ++t;
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
 
-// Scratch layout: [reduction partials | result double | G | gradient chunk partials | published rows]
-struct ScratchLayout {
-    int64_t partials_off = 0, result_off = 0, G_off = 0, chunk_off = 0, ytag_off = 0, ytag_bytes = 0, total = 0;
-};
 ScratchLayout scratch_layout(const gpga_ctx* c)
 {
     ScratchLayout L;
     int64_t slots = kMaxReduceBlocks;
     if (c->n > slots) slots = c->n;
+    // the consensus distance writes one partial per 256 column groups
+    if (consensus_blocks((c->d + 3) / 4) > slots) slots = consensus_blocks((c->d + 3) / 4);
+    L.slots = slots;
     L.partials_off = 0;
     L.result_off = round_up(slots * 8, 256);
     L.total = L.result_off + 256;
@@ -119,7 +124,7 @@ int32_t check_ready(gpga_ctx* c)
 
 LogregParams logreg_params(const gpga_ctx* c, int64_t k)
 {
-    const ScratchLayout L = scratch_layout(c);
+    const ScratchLayout& L = c->L;
     LogregParams lp;
     lp.A = c->data;
     lp.y = c->labels;
@@ -234,7 +239,7 @@ constexpr int64_t kLogRunSteps = 1 << 14;   // per launch: about a tenth of a se
 
 int32_t run_logistic_resident(gpga_ctx* c, int64_t K, cudaStream_t s)
 {
-    const ScratchLayout L = scratch_layout(c);
+    const ScratchLayout& L = c->L;
     const int64_t k_end = c->k + K;
     cudaError_t e;
     if (!c->flag_cleared) {
@@ -292,7 +297,7 @@ int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)
         bool ok = false;
         const cudaError_t e = logreg_run_supported((int)c->n, (int)c->d, (int)c->batch, c->topology, c->H, &ok);
         if (e != cudaSuccess) return cuda_fail(c, e, "occupancy query");
-        if (ok && scratch_layout(c).ytag_bytes > 0) return run_logistic_resident(c, K, s);
+        if (ok && c->L.ytag_bytes > 0) return run_logistic_resident(c, K, s);
     }
     if (!fused) {
         for (int64_t k = c->k; k < k_end; ++k) {
@@ -328,7 +333,7 @@ int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)
 
 int32_t mean_loss_async(gpga_ctx* c, cudaStream_t s, double** result_dev)
 {
-    const ScratchLayout L = scratch_layout(c);
+    const ScratchLayout& L = c->L;
     double* partials = reinterpret_cast<double*>(c->scratch + L.partials_off);
     double* result = reinterpret_cast<double*>(c->scratch + L.result_off);
     cudaError_t e;
@@ -487,6 +492,7 @@ int32_t gpga_bind(gpga_t* c, void* x_a, void* x_b, void* data, const void* label
     c->labels = static_cast<const float*>(labels);
     c->scratch = static_cast<char*>(scratch);
     c->scratch_bytes = scratch_bytes;
+    c->L = scratch_layout(c);
     c->cur = 0;
     c->k = 0;
     c->bound = true;
@@ -637,7 +643,7 @@ int32_t gpga_consensus_distance(gpga_t* c, void* stream, double* out_host)
     if (st) return st;
     if (!out_host) return fail(c, GPGA_ERR_INVALID_ARG, "out_host is NULL");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const ScratchLayout L = scratch_layout(c);
+    const ScratchLayout& L = c->L;
     double* partials = reinterpret_cast<double*>(c->scratch + L.partials_off);
     double* result = reinterpret_cast<double*>(c->scratch + L.result_off);
     cudaError_t e = launch_consensus(c->x[c->cur], c->n, c->d, c->ld, vec_ok(c), partials, result, s);
@@ -664,17 +670,15 @@ int32_t gpga_global_loss(gpga_t* c, void* stream, double* out_host)
     if (st) return st;
     if (!out_host) return fail(c, GPGA_ERR_INVALID_ARG, "out_host is NULL");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const ScratchLayout L = scratch_layout(c);
+    const ScratchLayout& L = c->L;
     double* partials = reinterpret_cast<double*>(c->scratch + L.partials_off);
     double* result = reinterpret_cast<double*>(c->scratch + L.result_off);
     cudaError_t e;
     if (c->objective == GPGA_OBJ_LOGISTIC) {
         // xbar borrows the gradient buffer, which is dead between iterations
         float* xbar = reinterpret_cast<float*>(c->scratch + L.G_off);
-        int64_t slots = kMaxReduceBlocks;
-        if (c->n > slots) slots = c->n;
         e = launch_logistic_global_loss(c->data, c->labels, c->x[c->cur], c->ld, c->n, c->d, c->m, c->l2, xbar,
-                                        partials, slots, result, s);
+                                        partials, L.slots, result, s);
         c->launches += 3;
     } else {
         e = launch_quadratic_global_loss(c->x[c->cur], c->data, c->n, c->d, c->ld, vec_ok(c), partials, result, s);
@@ -689,7 +693,7 @@ int32_t gpga_selftest_bounded_wait(gpga_t* c, void* stream)
     int32_t st = check_ready(c);
     if (st) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    int* flag = reinterpret_cast<int*>(c->scratch + scratch_layout(c).result_off + 8);
+    int* flag = reinterpret_cast<int*>(c->scratch + c->L.result_off + 8);
     cudaError_t e = cudaMemsetAsync(flag, 0, sizeof(int), s);
     if (e != cudaSuccess) return cuda_fail(c, e, "error word clear");
     c->flag_cleared = true;

@@ -136,11 +136,9 @@ __device__ __forceinline__ float4 mix3(float4 a, float4 b, float4 c)
     return scale4(add4(add4(a, b), c), 0.333333343f);
 }
 
-template <int MODE, bool VEC, int U, bool PIPE, int BLOCK, int MINB>
-__global__ void __launch_bounds__(BLOCK, MINB) step_ring_kernel(const StepParams p)
+template <int MODE, bool VEC, int U, bool PIPE>
+__device__ __forceinline__ void ring_columns(const StepParams& p, long long q)
 {
-    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (q >= p.Q) return;
     const ColGroup c = col_group<VEC>(p, q);
     const int n = (int)p.n;
     if (n <= 2) {
@@ -169,6 +167,16 @@ __global__ void __launch_bounds__(BLOCK, MINB) step_ring_kernel(const StepParams
     store_row<VEC>(p, c, 0, mix3(b, y0, y1));
 }
 
+// The grid holds one thread per column group.  (Cutting the grid of a state of a few waves to one
+// resident wave, every thread taking several groups a grid apart, measured slower: n = 32,
+// d = 2^20: 75.8 against 70.7 us per launch; n = 32, d = 2^21: 150 against 132 us.)
+template <int MODE, bool VEC, int U, bool PIPE, int BLOCK, int MINB>
+__global__ void __launch_bounds__(BLOCK, MINB) step_ring_kernel(const StepParams p)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q < p.Q) ring_columns<MODE, VEC, U, PIPE>(p, q);
+}
+
 // ---------------------------------------------------------------------------
 // One-peer exponential graph: x_i^(k+1) = (y_i + y_{(i+h) mod n}) / 2, h = 2^t.
 // i -> i + h splits the nodes into h cycles of length n/h; walking a cycle needs
@@ -176,11 +184,9 @@ __global__ void __launch_bounds__(BLOCK, MINB) step_ring_kernel(const StepParams
 // noise generated) once.  Step t of the flattened walk visits row
 // (t / L) + (t mod L) * h with L = n / h.
 // ---------------------------------------------------------------------------
-template <int MODE, bool VEC, int U, bool PIPE, int BLOCK, int MINB>
-__global__ void __launch_bounds__(BLOCK, MINB) step_exp_kernel(const StepParams p)
+template <int MODE, bool VEC, int U, bool PIPE>
+__device__ __forceinline__ void exp_columns(const StepParams& p, long long q)
 {
-    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (q >= p.Q) return;
     const ColGroup c = col_group<VEC>(p, q);
     const int len_log2 = p.len_log2, hop_log2 = p.hop_log2;
     const int hop = 1 << hop_log2;
@@ -264,6 +270,13 @@ __global__ void __launch_bounds__(BLOCK, MINB) step_exp_kernel(const StepParams 
         });
 }
 
+template <int MODE, bool VEC, int U, bool PIPE, int BLOCK, int MINB>
+__global__ void __launch_bounds__(BLOCK, MINB) step_exp_kernel(const StepParams p)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q < p.Q) exp_columns<MODE, VEC, U, PIPE>(p, q);
+}
+
 // ---------------------------------------------------------------------------
 // Global average: m_j = (1/n) sum_i y_ij, written to every row.  Rows are added
 // pairwise in fp32 in groups of four, (y0 + y1) + (y2 + y3), and the group sums are
@@ -271,11 +284,9 @@ __global__ void __launch_bounds__(BLOCK, MINB) step_exp_kernel(const StepParams 
 // roundings, so the mean is within a few 1e-8 (1 + |y|) of the exact one; and when all
 // rows are equal every group sum (v, 2v or 4v) is exact, so the mean is exactly v.
 // ---------------------------------------------------------------------------
-template <int MODE, bool VEC, int U, bool PIPE, int BLOCK, int MINB>
-__global__ void __launch_bounds__(BLOCK, MINB) step_global_kernel(const StepParams p)
+template <int MODE, bool VEC, int U, bool PIPE>
+__device__ __forceinline__ void global_columns(const StepParams& p, long long q)
 {
-    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (q >= p.Q) return;
     const ColGroup c = col_group<VEC>(p, q);
     double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
@@ -316,6 +327,13 @@ __global__ void __launch_bounds__(BLOCK, MINB) step_global_kernel(const StepPara
                                  (float)(s3 / inv));
 #pragma unroll 4
     for (int i = 0; i < n; ++i) store_row<VEC>(p, c, i, m);
+}
+
+template <int MODE, bool VEC, int U, bool PIPE, int BLOCK, int MINB>
+__global__ void __launch_bounds__(BLOCK, MINB) step_global_kernel(const StepParams p)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q < p.Q) global_columns<MODE, VEC, U, PIPE>(p, q);
 }
 
 static inline unsigned grid_for(long long Q, int block) { return (unsigned)((Q + block - 1) / block); }
@@ -360,12 +378,25 @@ cudaError_t launch_step_global(const StepParams& p, int mode, bool vec, cudaStre
 
 // ---------------------------------------------------------------------------
 // Consensus distance sum_j sum_i (x_ij - xbar_j)^2.  One pass over X: with
-// e_i = x_i - x_0 (exact in fp64), sum_i (x_i - xbar)^2 = sum e_i^2 - (sum e_i)^2 / n;
-// shifting by row 0 keeps the subtraction benign when the rows are nearly equal.
+// e_i = x_i - x_0, sum_i (x_i - xbar)^2 = sum e_i^2 - (sum e_i)^2 / n; shifting by row 0 keeps
+// the subtraction benign when the rows are nearly equal.  e_i is formed in fp32: exact when x_i
+// and x_0 are within a factor of two of each other (the nearly-consensual case, where it matters),
+// one rounding of 2^-24 relative otherwise.  Rows are taken in groups of four: e and e^2 are added
+// pairwise in fp32 inside a group, (e0 + e1) + (e2 + e3), and the group sums are accumulated in
+// fp64 -- a quarter of the conversions and fp64 additions of an all-fp64 pass, at a relative error of
+// a few 1e-7.  Like the step kernels, one thread owns a group of four columns and keeps the loads
+// of four rows in flight; one block covers 256 adjacent column groups (a contiguous window in
+// every row), writes one partial, and a second kernel adds the partials in a fixed order.
 // ---------------------------------------------------------------------------
 constexpr int kReduceBlock = 256;
 
-int consensus_blocks(long long Q)
+long long consensus_blocks(long long Q)
+{
+    const long long b = (Q + kReduceBlock - 1) / kReduceBlock;
+    return b < 1 ? 1 : b;
+}
+
+int reduce_blocks(long long Q)
 {
     long long b = (Q + kReduceBlock - 1) / kReduceBlock;
     if (b > kMaxReduceBlocks) b = kMaxReduceBlocks;
@@ -373,23 +404,48 @@ int consensus_blocks(long long Q)
     return (int)b;
 }
 
+__device__ __forceinline__ float4 mul4(float4 a, float4 b)
+{
+    return join4(mul2(pack2(a.x, a.y), pack2(b.x, b.y)), mul2(pack2(a.z, a.w), pack2(b.z, b.w)));
+}
+// a * a + c, component-wise
+__device__ __forceinline__ float4 sqadd4(float4 a, float4 c)
+{
+    return join4(fma2(pack2(a.x, a.y), pack2(a.x, a.y), pack2(c.x, c.y)),
+                 fma2(pack2(a.z, a.w), pack2(a.z, a.w), pack2(c.z, c.w)));
+}
+
 template <bool VEC>
-__global__ void __launch_bounds__(kReduceBlock, 3) consensus_kernel(const float* __restrict__ x,
+__global__ void __launch_bounds__(kReduceBlock, 4) consensus_kernel(const float* __restrict__ x,
                                                                  long long n, long long d,
-                                                                 long long ld, long long Q,
+                                                                 long long ld, long long Q, int slabs,
                                                                  double* __restrict__ partials)
 {
     double acc = 0.0;
-    for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < Q;
-         q += (long long)gridDim.x * blockDim.x) {
+    // a block covers `slabs` adjacent slabs of 256 column groups (more than one when n is small, so
+    // that a block lives long enough to amortise its start and its reduction)
+    for (int sl = 0; sl < slabs; ++sl) {
+        const long long q = ((long long)blockIdx.x * slabs + sl) * blockDim.x + threadIdx.x;
+        if (q >= Q) break;
         const long long j0 = q * 4;
-        const float4 r0 = load4<VEC>(x, j0, d);
+        const float* col = VEC ? x + j0 : x;       // load4<true> ignores j0 and d
+        const long long jv = VEC ? 0 : j0;
+        const float4 r0 = load4<VEC>(col, jv, d);
         double s1[4] = {0, 0, 0, 0}, s2[4] = {0, 0, 0, 0};
-#pragma unroll 4
-        for (long long i = 1; i < n; ++i) {
-            const float4 v = load4<VEC>(x + i * ld, j0, d);
-            const double e0 = (double)v.x - (double)r0.x, e1 = (double)v.y - (double)r0.y;
-            const double e2 = (double)v.z - (double)r0.z, e3 = (double)v.w - (double)r0.w;
+        long long i = 1;
+        for (; i + 4 <= n; i += 4) {
+            float4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v[u] = load4<VEC>(col + (i + u) * ld, jv, d);
+            const float4 e0 = sub4(v[0], r0), e1 = sub4(v[1], r0), e2 = sub4(v[2], r0), e3 = sub4(v[3], r0);
+            const float4 sum = add4(add4(e0, e1), add4(e2, e3));
+            const float4 sq = add4(sqadd4(e1, mul4(e0, e0)), sqadd4(e3, mul4(e2, e2)));
+            s1[0] += (double)sum.x; s1[1] += (double)sum.y; s1[2] += (double)sum.z; s1[3] += (double)sum.w;
+            s2[0] += (double)sq.x; s2[1] += (double)sq.y; s2[2] += (double)sq.z; s2[3] += (double)sq.w;
+        }
+        for (; i < n; ++i) {   // at most three rows left
+            const float4 e = sub4(load4<VEC>(col + i * ld, jv, d), r0);
+            const double e0 = (double)e.x, e1 = (double)e.y, e2 = (double)e.z, e3 = (double)e.w;
             s1[0] += e0; s2[0] = fma(e0, e0, s2[0]);
             s1[1] += e1; s2[1] = fma(e1, e1, s2[1]);
             s1[2] += e2; s2[2] = fma(e2, e2, s2[2]);
@@ -417,16 +473,34 @@ __global__ void final_sum_kernel(const double* __restrict__ partials, int count,
     if (threadIdx.x == 0) *result = v * scale;
 }
 
+// The same for many partials: thread t of one 1024-thread block adds partials t, t + 1024, ... in
+// that order, then the block's fixed shuffle / shared-memory tree.  Independent of scheduling.
+__global__ void __launch_bounds__(1024) final_sum_wide_kernel(const double* __restrict__ partials, long long count,
+                                                              double* __restrict__ result)
+{
+    double v = 0.0;
+    for (long long t = threadIdx.x; t < count; t += 1024) v += partials[t];
+    v = block_sum(v);
+    if (threadIdx.x == 0) *result = v;
+}
+
 cudaError_t launch_consensus(const float* x, long long n, long long d, long long ld, bool vec, double* partials,
                              double* result, cudaStream_t s)
 {
     const long long Q = (d + 3) / 4;
-    const int blocks = consensus_blocks(Q);
+    // about 64 rows' worth of loads per thread: n >= 64 one slab, n = 16 four, at most 8
+    int slabs = (int)(64 / (n < 1 ? 1 : n));
+    slabs = slabs < 1 ? 1 : (slabs > 8 ? 8 : slabs);
+    if (consensus_blocks(Q) < 148 * 16) slabs = 1;   // small states: keep every SM busy
+    const long long blocks = (consensus_blocks(Q) + slabs - 1) / slabs;
     if (vec)
-        consensus_kernel<true><<<blocks, kReduceBlock, 0, s>>>(x, n, d, ld, Q, partials);
+        consensus_kernel<true><<<(unsigned)blocks, kReduceBlock, 0, s>>>(x, n, d, ld, Q, slabs, partials);
     else
-        consensus_kernel<false><<<blocks, kReduceBlock, 0, s>>>(x, n, d, ld, Q, partials);
-    final_sum_kernel<<<1, 32, 0, s>>>(partials, blocks, 1.0, result);
+        consensus_kernel<false><<<(unsigned)blocks, kReduceBlock, 0, s>>>(x, n, d, ld, Q, slabs, partials);
+    if (blocks <= 4096)
+        final_sum_kernel<<<1, 32, 0, s>>>(partials, (int)blocks, 1.0, result);
+    else
+        final_sum_wide_kernel<<<1, 1024, 0, s>>>(partials, blocks, result);
     return cudaGetLastError();
 }
 
@@ -462,7 +536,7 @@ cudaError_t launch_quadratic_loss(const float* x, const float* b, long long n, l
                                   bool vec, double* partials, double* result, cudaStream_t s)
 {
     const long long Q = (d + 3) / 4;
-    const int blocks = consensus_blocks(Q);
+    const int blocks = reduce_blocks(Q);
     if (vec)
         quadratic_loss_kernel<true><<<blocks, kReduceBlock, 0, s>>>(x, b, n, d, ld, Q, partials);
     else

@@ -46,9 +46,12 @@ cudaError_t launch_step_global(const StepParams& p, int mode, bool vec, cudaStre
 cudaError_t launch_step_tile(const StepParams& p, int mode, bool vec, int mix, cudaStream_t s);
 bool tile_supports(long long n);   // the n rows of one column group fit the shared-memory tile
 
-// Consensus distance: partials (one double per block) then a fixed-order final sum.
-constexpr int kMaxReduceBlocks = 148 * 8;   // capacity of the partials array, in doubles
-int consensus_blocks(long long Q);
+// Consensus distance: partials (one double per block of 256 column groups) then a fixed-order final
+// sum.  consensus_blocks(Q) is the number of partials it writes; the loss reductions use a
+// grid-stride pass of at most kMaxReduceBlocks blocks (reduce_blocks).
+constexpr int kMaxReduceBlocks = 148 * 8;
+long long consensus_blocks(long long Q);
+int reduce_blocks(long long Q);
 cudaError_t launch_consensus(const float* x, long long n, long long d, long long ld, bool vec, double* partials,
                              double* result, cudaStream_t s);
 // (1/n) sum_i 1/2 ||x_i - b_i||^2, same two-stage reduction.

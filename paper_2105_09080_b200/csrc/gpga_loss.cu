@@ -66,7 +66,7 @@ cudaError_t launch_quadratic_global_loss(const float* x, const float* b, long lo
                                          bool vec, double* partials, double* result, cudaStream_t s)
 {
     const long long Q = (d + 3) / 4;
-    const int blocks = consensus_blocks(Q);
+    const int blocks = reduce_blocks(Q);
     if (vec)
         quadratic_global_loss_kernel<true><<<blocks, kLossBlock, 0, s>>>(x, b, n, d, ld, Q, partials);
     else

@@ -109,7 +109,7 @@ def test_config_3_resnet50_sized():
     xa = torch.empty((n, ld), dtype=torch.float32, device="cuda")
     xb = torch.empty_like(xa)
     b = torch.empty_like(xa)
-    scratch = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+    scratch = torch.empty(4 << 20, dtype=torch.uint8, device="cuda")   # >= gpga_scratch_bytes at these sizes
     offs = _blocks(d, 64, np.random.default_rng(3))
     assert d % 128 == 40 and offs[-1] + BLOCK == d
     for topo in ("ring", "exp"):
@@ -188,7 +188,7 @@ def test_config_4_bert_large_sized():
     xa = torch.empty((n, d), dtype=torch.float32, device="cuda")
     xb = torch.empty_like(xa)
     b = torch.empty_like(xa)
-    scratch = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+    scratch = torch.empty(4 << 20, dtype=torch.uint8, device="cuda")   # >= gpga_scratch_bytes at these sizes
     offs = _blocks(d, 48, np.random.default_rng(4))
     _run_case((xa, xb, b, scratch), n, d, "exp", H, gamma, sigma, K, pkg.GPGA_X0_ZERO, 1.0, 0.0,
               offs, [0, 1, 2, 3])
