@@ -252,6 +252,66 @@ int32_t gpga_run_adaptive(gpga_t* ctx, int64_t K, int64_t H_init, int64_t warmup
                           int64_t* num_periods_host);
 
 /*
+ * Node sharding: the deployment of Section 3, where the n nodes live on several devices, a gossip
+ * step exchanges the half-step vectors x^(k+1/2) of neighbouring nodes and the global average is
+ * an All-Reduce ("All-Reduce v.s. multiple Gossips"); the appendix's implementation details: on
+ * the one-peer exponential graph a worker sends one copy of its parameters and receives one.
+ * Here a shard is a handle holding n consecutive nodes (all d columns) of an (n * shards)-node
+ * problem; quadratic objective, ring or one-peer exponential graph.  One iteration k on a shard:
+ *     gpga_shard_export(k, send)   forms what other shards need of this shard's half-step
+ *     -- the caller delivers the messages gpga_shard_plan lists (copies, or send/recv and an
+ *        all-gather of a communication library) --
+ *     gpga_shard_step(k, recv)     local update + mix of the local rows with what was received
+ * Results equal the unsharded iteration's (same operations in the same order; the column mean adds
+ * the shards' fp64 sums in shard order).  Send and receive buffers are caller-owned device memory,
+ * 16-byte aligned, gpga_shard_exchange_bytes() each; an exchanged row is ceil(d/4)*4 floats.
+ * The library reads remote rows only from the receive buffer in this device's own memory.
+ */
+enum { GPGA_SHARD_RING = 0, GPGA_SHARD_EXP = 1, GPGA_SHARD_GLOBAL = 2 };
+
+typedef struct gpga_shard_plan {
+    int32_t kind;            /* what iteration k is: GPGA_SHARD_RING / EXP (a gossip step) or GLOBAL */
+    int32_t messages;        /* point-to-point messages this shard sends, and as many it receives:
+                                ring 2 (first row up, last row down), exponential graph 1, global 0 */
+    int32_t send_to[2];      /* message m goes to this shard ...                                    */
+    int32_t recv_from[2];    /* ... and received message m comes from this one                     */
+    int64_t send_offset[2];  /* byte offset of message m in this shard's send buffer               */
+    int64_t dst_offset[2];   /* byte offset in the DESTINATION's receive buffer where it lands     */
+    int64_t recv_offset[2];  /* byte offset in this shard's receive buffer of received message m   */
+    int64_t bytes[2];        /* size of sent message m (received message m has the same size)      */
+    int64_t gather_bytes;    /* GLOBAL: bytes of one shard's column sums (ceil(d/4)*4 doubles at the
+                                start of its send buffer); the receive buffer holds every shard's,
+                                shard s at offset s * gather_bytes (an all-gather)                  */
+    int64_t hop;             /* exponential graph: 2^(k mod log2 n)                                 */
+} gpga_shard_plan_t;
+
+/* Who exchanges what at iteration k (host logic only; Algorithm 1's schedule, the ring's two
+ * neighbours, the exponential graph's partner (i + 2^(k mod log2 n)) mod n).  With hop h and n_l
+ * nodes per shard the partner rows of a shard are the first min(h, n_l) rows of the shard
+ * max(1, h / n_l) places ahead.  With one shard every message goes to the shard itself.
+ * Errors: INVALID_ARG / UNSUPPORTED as for gpga_create and gpga_set_node_shard. */
+int32_t gpga_shard_plan(int32_t topology, int64_t H, int64_t n_total, int64_t shards, int64_t shard, int64_t d,
+                        int64_t k, gpga_shard_plan_t* out);
+
+/* Declares that this handle's n nodes are nodes shard*n .. (shard+1)*n - 1 of an (n*shards)-node
+ * problem (the node index keys the noise generator).  Errors: UNSUPPORTED for another objective or
+ * topology, for the exponential graph with a number of shards that is not a power of two, and for
+ * several shards of a node count that is not a multiple of four. */
+int32_t gpga_set_node_shard(gpga_t* ctx, int64_t shards, int64_t shard);
+
+/* Bytes each of the send and the receive buffer must have (the largest message set of any iteration). */
+int64_t gpga_shard_exchange_bytes(const gpga_t* ctx);
+
+/* First half of iteration k on this shard: writes the outgoing messages (gpga_shard_plan's
+ * send_offset / bytes, or the column sums) to send_dev.  Asynchronous on `stream`. */
+int32_t gpga_shard_export(gpga_t* ctx, int64_t k, void* send_dev, void* stream);
+
+/* Second half: Algorithm 1's update and mix for the local rows, with recv_dev holding the received
+ * messages (recv_offset) or all shards' column sums.  Reads the current buffer, writes the other,
+ * flips them and sets the counter to k + 1, like gpga_step.  Asynchronous on `stream`. */
+int32_t gpga_shard_step(gpga_t* ctx, int64_t k, const void* recv_dev, void* stream);
+
+/*
  * Self-test of the in-kernel wait limit (no counterpart in the paper): launches one block that
  * waits, a bounded number of polls, on a barrier that nothing will ever complete.  The wait must
  * give up and raise the handle's device error word, so that the NEXT synchronising call
@@ -259,6 +319,18 @@ int32_t gpga_run_adaptive(gpga_t* ctx, int64_t K, int64_t H_init, int64_t warmup
  * which the handle stays in that state.  Nothing faults, traps or hangs.  For tests only.
  */
 int32_t gpga_selftest_bounded_wait(gpga_t* ctx, void* stream);
+
+/*
+ * Self-test of the waits between blocks of the one-launch logistic kernel (no counterpart in the
+ * paper).  Needs a bound logistic handle on the ring with n >= 2 that gpga_run would hand to that
+ * kernel (d <= 1024, batch <= 128).  Launches node 0's pair of blocks alone, with wait limits of a
+ * few thousand polls: the rows of its neighbours are never published, so its waits give up after
+ * some milliseconds, raise the handle's error word, and both blocks leave together.  The NEXT
+ * synchronising call returns GPGA_ERR_TIMEOUT and the handle stays in that state (its X is not
+ * advanced).  Nothing faults, traps or hangs.  For tests only.
+ * Errors: UNSUPPORTED for any other handle.
+ */
+int32_t gpga_selftest_run_wait(gpga_t* ctx, void* stream);
 
 /* Accessors.  gpga_get_x returns the device pointer of the current state buffer. */
 int32_t gpga_get_x(const gpga_t* ctx, void** x_cur);

@@ -55,6 +55,12 @@ SIGNATURES = {
     "gpga_mean_loss": (_i32, [_P, _P, C.POINTER(C.c_double)]),
     "gpga_global_loss": (_i32, [_P, _P, C.POINTER(C.c_double)]),
     "gpga_selftest_bounded_wait": (_i32, [_P, _P]),
+    "gpga_selftest_run_wait": (_i32, [_P, _P]),
+    "gpga_shard_plan": (_i32, [_i32, _i64, _i64, _i64, _i64, _i64, _i64, _P]),
+    "gpga_set_node_shard": (_i32, [_P, _i64, _i64]),
+    "gpga_shard_exchange_bytes": (_i64, [_P]),
+    "gpga_shard_export": (_i32, [_P, _i64, _P, _P]),
+    "gpga_shard_step": (_i32, [_P, _i64, _P, _P]),
     "gpga_run_adaptive": (_i32, [_P, _i64, _i64, _i64, _P, C.POINTER(_i64), _i64, C.POINTER(_i64)]),
     "gpga_get_x": (_i32, [_P, C.POINTER(_P)]),
     "gpga_get_k": (_i32, [_P, C.POINTER(_i64)]),
@@ -236,6 +242,9 @@ class Gpga:
 
     def selftest_bounded_wait(self, stream=None):
         self._check(lib().gpga_selftest_bounded_wait(self._h, self._sp(stream)))
+
+    def selftest_run_wait(self, stream=None):
+        self._check(lib().gpga_selftest_run_wait(self._h, self._sp(stream)))
 
     def run_adaptive(self, K, H_init, warmup_iters, stream=None, max_periods=4096):
         periods = (_i64 * max_periods)()

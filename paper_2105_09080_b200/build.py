@@ -10,7 +10,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libgpga.so"
-SOURCES = ["gpga_api.cu", "gpga_kernels.cu", "gpga_tile.cu", "gpga_logreg.cu", "gpga_logrun.cu", "gpga_noalloc.cu", "gpga_loss.cu"]
+SOURCES = ["gpga_api.cu", "gpga_kernels.cu", "gpga_tile.cu", "gpga_logreg.cu", "gpga_logrun.cu", "gpga_noalloc.cu", "gpga_loss.cu", "gpga_shard.cu"]
 
 
 def nvcc_path() -> str:

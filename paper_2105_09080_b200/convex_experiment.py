@@ -1,14 +1,26 @@
-"""The paper's convex experiment (Section 5.1) on the library: distributed logistic regression
-over a ring of n = 20 / 50 / 100 nodes, d = 10, M = 8000 samples per node, non-iid data,
-step size 0.2 halved every 1000 iterations, comparing parallel SGD (H = 1), Gossip SGD
-(H = infinity) and Gossip-PGA (H = 16).
+"""The paper's convex experiment (Section 5.1 and the appendix's additional experiments) on the
+library: distributed logistic regression over n = 20 / 50 / 100 nodes, d = 10, M = 8000 samples
+per node, step size 0.2 halved every 1000 iterations, repeated over many trials, comparing
+parallel SGD (a global average every iteration), Gossip SGD (H = infinity), Gossip-PGA (H = 16)
+and Local SGD (W = I between global averages), on the ring, the grid and the static exponential
+graph, with non-iid or iid data.
 
-    python -m paper_2105_09080_b200.convex_experiment [--trials 5] [--iters 6000] [--out runs.jsonl]
+    python -m paper_2105_09080_b200.convex_experiment [--sizes 20 50 100] [--trials 50] [--iters 6000]
+           [--topology ring|grid|static_exp] [--period 16] [--iid] [--out runs.jsonl]
 
-Prints one JSON line per (n, method) with the global loss f(xbar) and the consensus distance
-every `--every` iterations, averaged over the trials (different seeds for data order and
-mini-batches).  The data recipe follows the paper; the mini-batch size, which the paper does
-not state, is an option.  Everything numerical runs in the library's kernels.
+All trials of one (n, method) run as ONE problem: T independent copies of the n-node network are
+the diagonal blocks of a (T n)-node weight matrix given to the library in CSR form (topology
+SPARSE), each node with its own data, so a sweep is one launch sequence instead of T.  The
+global-averaging step of Algorithm 1 is then a matrix too (1/n on every node of the same copy):
+the driver hands the library the gossip matrix for the gossip iterations and the averaging matrix
+for the iterations with mod(k + 1, H) = 0.  Per-trial diagnostics (the loss f(xbar) of problem (1)
+at the copy's node average, and its consensus distance) come from small handles bound to each
+copy's rows of the same buffers.  Everything numerical runs in the library's kernels.
+
+Prints one JSON line per (n, method): mean and standard deviation over the trials of the loss and of
+the consensus distance every `--every` iterations, and the transient stage read off the curves (the
+last recorded iteration at which the method's mean loss is still apart from parallel SGD's).
+The data recipe follows the paper; the mini-batch size, which the paper does not state, is an option.
 """
 from __future__ import annotations
 
@@ -19,63 +31,166 @@ import sys
 import numpy as np
 
 from . import binding as B
+from . import topologies
 from .inputs import convex_experiment_inputs
 
-METHODS = {"parallel_sgd": 1, "gossip_sgd": 0, "gossip_pga": 16}
+# method -> (weight matrix of the gossip iterations, uses the period)
+METHODS = {"parallel_sgd": ("average", False), "gossip_sgd": (None, False), "gossip_pga": (None, True),
+           "local_sgd": ("none", True)}
+MAX_NODES = 4096        # what topology SPARSE takes
 
 
-def run_one(A_dev, y_dev, topology, H, iters, every, batch, seed, gamma0=0.2, halve_every=1000):
+def _to_device(arrays, device):
     import torch
-    n, m, d = A_dev.shape
-    g = B.Gpga(n, d, topology, H, gamma0, seed)
-    g.set_objective(B.GPGA_OBJ_LOGISTIC, l2=0.0, m=m, batch=batch)
-    xa = torch.zeros((n, d), device=A_dev.device)
-    g.bind(xa, torch.empty_like(xa), A_dev, y_dev)
-    loss, cons = [g.global_loss()], [g.consensus_distance()]
+    return tuple(torch.from_numpy(a).to(device) for a in arrays)
+
+
+class BatchedTrials:
+    """T copies of an n-node problem as one (T n)-node problem with a block-diagonal W."""
+
+    def __init__(self, A_dev, y_dev, n, topology, batch, seed, gamma0=0.2, halve_every=1000, grid_cols=0):
+        import torch
+        N, m, d = A_dev.shape
+        assert N % n == 0 and N <= MAX_NODES
+        self.n, self.trials, self.m, self.d, self.batch = n, N // n, m, d, batch
+        self.gamma0, self.halve_every = gamma0, halve_every
+        self.A, self.y = A_dev, y_dev
+        dev = A_dev.device
+        self.W = {name: _to_device(topologies.csr(name, n, self.trials, grid_cols), dev)
+                  for name in {topology, "average", "none"}}
+        self.topology = topology
+        self.g = B.Gpga(N, d, B.GPGA_TOPO_SPARSE, 0, gamma0, seed)
+        self.g.set_objective(B.GPGA_OBJ_LOGISTIC, l2=0.0, m=m, batch=batch)
+        self.xa = torch.zeros((N, d), device=dev)
+        self.xb = torch.empty_like(self.xa)
+        self.scratch = torch.empty(self.g.scratch_bytes(), dtype=torch.uint8, device=dev)
+        self.g.bind(self.xa, self.xb, A_dev, y_dev, scratch=self.scratch)
+        # one small handle per copy, for the copy's own loss and consensus distance
+        self.diag = []
+        for t in range(self.trials):
+            h = B.Gpga(n, d, B.GPGA_TOPO_RING, 0, gamma0, seed)
+            h.set_objective(B.GPGA_OBJ_LOGISTIC, l2=0.0, m=m, batch=batch)
+            self.diag.append((h, torch.empty(h.scratch_bytes(), dtype=torch.uint8, device=dev)))
+
+    def reset(self):
+        self.xa.zero_()
+        self.g.bind(self.xa, self.xb, self.A, self.y, scratch=self.scratch)       # x_a current, counter 0
+
+    def diagnostics(self):
+        """(loss at the node average, consensus distance) of every copy's current state."""
+        cur = self.g.get_x()
+        other = self.xb if cur.data_ptr() == self.xa.data_ptr() else self.xa
+        n = self.n
+        loss, cons = np.empty(self.trials), np.empty(self.trials)
+        for t, (h, scratch) in enumerate(self.diag):
+            rows = slice(t * n, (t + 1) * n)
+            h.bind(cur[rows], other[rows], self.A[rows], self.y[rows], scratch=scratch)
+            loss[t] = h.global_loss()
+            cons[t] = h.consensus_distance()
+        return loss, cons
+
+    def run(self, method, period, iters, every):
+        """Iterations 0 .. iters-1 of `method`; returns (iterations, loss[record][trial], cons[record][trial])."""
+        gossip_name, periodic = METHODS[method]
+        gossip = self.W[gossip_name or self.topology]
+        H = period if periodic else 0
+        self.reset()
+        marks, loss, cons = [0], [], []
+        l0, c0 = self.diagnostics()
+        loss.append(l0)
+        cons.append(c0)
+        k = 0
+        while k < iters:
+            self.g.set_gamma(self.gamma0 * 0.5 ** (k // self.halve_every))
+            stop = min(iters, (k // every + 1) * every, (k // self.halve_every + 1) * self.halve_every)
+            if H and (k + 1) % H == 0:           # Algorithm 1: global average when mod(k + 1, H) = 0
+                self.g.set_weight_matrix(*self.W["average"])
+                self.g.run(1)
+                k += 1
+            else:
+                if H:
+                    stop = min(stop, (k + 1 + H - 1) // H * H - 1)     # up to the next averaging iteration
+                self.g.set_weight_matrix(*gossip)
+                self.g.run(stop - k)
+                k = stop
+            if k % every == 0 or k == iters:
+                l, c = self.diagnostics()
+                marks.append(k)
+                loss.append(l)
+                cons.append(c)
+        return marks, np.array(loss), np.array(cons)
+
+    def close(self):
+        self.g.close()
+        for h, _ in self.diag:
+            h.close()
+
+
+def transient_stage(marks, loss, reference):
+    """Last recorded iteration at which the mean loss over trials is still apart from the
+    reference method's (beyond three standard errors of the two means), 0 if never."""
+    mean, ref = loss.mean(1), reference.mean(1)
+    sem = np.sqrt(loss.var(1) / loss.shape[1] + reference.var(1) / reference.shape[1])
+    apart = np.abs(mean - ref) > 3.0 * sem + 1e-12
+    idx = np.nonzero(apart)[0]
+    return int(marks[idx[-1]]) if idx.size else 0
+
+
+def run_size(n, trials, iters, every, batch, samples, iid, topology, period, methods, seed=1, device="cuda"):
+    """All methods for one network size; trials go in batches of at most MAX_NODES // n copies."""
+    import torch
+    per_batch = max(1, min(trials, MAX_NODES // n))
+    out = {name: ([], [], None) for name in methods}
     done = 0
-    while done < iters:
-        g.set_gamma(gamma0 * 0.5 ** (done // halve_every))
-        next_record = min((done // every + 1) * every, iters)
-        next_halving = (done // halve_every + 1) * halve_every
-        step = min(next_record, next_halving) - done
-        g.run(step)
-        done += step
-        if done == next_record:
-            loss.append(g.global_loss())
-            cons.append(g.consensus_distance())
-    g.close()
-    return np.array(loss), np.array(cons)
+    while done < trials:
+        T = min(per_batch, trials - done)
+        parts = [convex_experiment_inputs(n, samples, 10, seed=1000 * n + done + t, iid=iid) for t in range(T)]
+        A = torch.from_numpy(np.concatenate([p[0] for p in parts])).to(device)
+        y = torch.from_numpy(np.concatenate([p[1] for p in parts])).to(device)
+        bt = BatchedTrials(A, y, n, topology, batch, seed + done)
+        for name in methods:
+            marks, loss, cons = bt.run(name, period, iters, every)
+            out[name][0].append(loss)
+            out[name][1].append(cons)
+            out[name] = (out[name][0], out[name][1], marks)
+        bt.close()
+        done += T
+    return {name: (marks, np.concatenate(l, axis=1), np.concatenate(c, axis=1)) for name, (l, c, marks) in out.items()}
 
 
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--sizes", type=int, nargs="+", default=[20, 50, 100])
-    ap.add_argument("--trials", type=int, default=5)
+    ap.add_argument("--trials", type=int, default=50)
     ap.add_argument("--iters", type=int, default=6000)
     ap.add_argument("--every", type=int, default=200)
     ap.add_argument("--batch", type=int, default=8)
     ap.add_argument("--samples", type=int, default=8000)
+    ap.add_argument("--period", type=int, default=16)
     ap.add_argument("--iid", action="store_true")
     ap.add_argument("--topology", default="ring", choices=["ring", "grid", "static_exp"])
+    ap.add_argument("--methods", nargs="+", default=list(METHODS), choices=list(METHODS))
     ap.add_argument("--out", default="")
     args = ap.parse_args(argv)
     import torch
     if not torch.cuda.is_available():
         raise RuntimeError("the experiment needs a CUDA device (there is no CPU fallback)")
-    topo = {"ring": B.GPGA_TOPO_RING, "grid": B.GPGA_TOPO_GRID, "static_exp": B.GPGA_TOPO_STATIC_EXP}[args.topology]
+    methods = list(args.methods)
+    if "parallel_sgd" not in methods:
+        methods.insert(0, "parallel_sgd")        # the reference curve of the transient stage
     sink = open(args.out, "w") if args.out else sys.stdout
     for n in args.sizes:
-        A, y = convex_experiment_inputs(n, args.samples, 10, seed=1000 + n, iid=args.iid)
-        A_dev, y_dev = torch.from_numpy(A).cuda(), torch.from_numpy(y).cuda()
-        for name, H in METHODS.items():
-            runs = [run_one(A_dev, y_dev, topo, H, args.iters, args.every, args.batch, seed=trial + 1)
-                    for trial in range(args.trials)]
-            loss = np.mean([r[0] for r in runs], axis=0)
-            cons = np.mean([r[1] for r in runs], axis=0)
-            sink.write(json.dumps({"n": n, "method": name, "H": H or "inf", "topology": args.topology,
-                                   "iid": args.iid, "trials": args.trials, "batch": args.batch,
-                                   "iterations": list(range(0, args.iters + 1, args.every)),
-                                   "global_loss": loss.tolist(), "consensus_distance": cons.tolist()}) + "\n")
+        res = run_size(n, args.trials, args.iters, args.every, args.batch, args.samples, args.iid, args.topology,
+                       args.period, methods)
+        ref = res["parallel_sgd"][1]
+        for name in methods:
+            marks, loss, cons = res[name]
+            sink.write(json.dumps({
+                "n": n, "method": name, "period": args.period if METHODS[name][1] else None,
+                "topology": args.topology, "iid": args.iid, "trials": args.trials, "batch": args.batch,
+                "iterations": marks, "loss_mean": loss.mean(1).tolist(), "loss_std": loss.std(1).tolist(),
+                "consensus_mean": cons.mean(1).tolist(), "consensus_std": cons.std(1).tolist(),
+                "transient_stage": transient_stage(marks, loss, ref)}) + "\n")
             sink.flush()
     if args.out:
         sink.close()

@@ -10,6 +10,7 @@
 #include "gpga_logreg.cuh"
 #include "gpga_logrun.cuh"
 #include "gpga_loss.cuh"
+#include "gpga_shard.cuh"
 #include "gpga_tile.cuh"
 
 using namespace gpga;
@@ -30,6 +31,7 @@ struct gpga_ctx {
     int64_t grid_cols = 0;
     int64_t col0 = 0;
     int64_t ld = 0;   // row stride of X and b in floats
+    int64_t shards = 1, shard = 0;   // node sharding: this handle holds nodes shard * n .. (shard + 1) * n - 1
     float* x[2] = {nullptr, nullptr};
     float* data = nullptr;
     const float* labels = nullptr;
@@ -700,6 +702,202 @@ int32_t gpga_selftest_bounded_wait(gpga_t* c, void* stream)
     e = launch_bounded_wait_selftest(flag, s);
     c->launches += 1;
     if (e != cudaSuccess) return cuda_fail(c, e, "self-test launch");
+    return GPGA_OK;
+}
+
+// Node 0's pair of blocks of the one-launch logistic kernel, alone, with short wait limits: its
+// neighbours' rows are never published, so its waits run out; it raises the error and stop words and
+// both blocks leave through their common barrier.
+int32_t gpga_selftest_run_wait(gpga_t* c, void* stream)
+{
+    int32_t st = check_ready(c);
+    if (st) return st;
+    bool ok = false;
+    if (c->objective == GPGA_OBJ_LOGISTIC && c->topology == GPGA_TOPO_RING && c->n >= 2 && c->L.ytag_bytes > 0) {
+        const cudaError_t q = logreg_run_supported((int)c->n, (int)c->d, (int)c->batch, c->topology, 0, &ok);
+        if (q != cudaSuccess) return cuda_fail(c, q, "occupancy query");
+    }
+    if (!ok) return fail(c, GPGA_ERR_UNSUPPORTED, "needs a logistic ring problem with n >= 2 that the one-launch kernel takes");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const ScratchLayout& L = c->L;
+    LogRunParams p;
+    p.A = c->data;
+    p.y = c->labels;
+    p.x_in = c->x[c->cur];
+    p.x_out = c->x[c->cur];
+    p.ldx = c->ld;
+    p.ytag = reinterpret_cast<unsigned long long*>(c->scratch + L.ytag_off);
+    p.nbuf = 2 + logreg_run_buffers(0, log2_floor(c->n));
+    p.stop = reinterpret_cast<int*>(c->scratch + L.partials_off);
+    p.error_flag = reinterpret_cast<int*>(c->scratch + L.result_off + 8);
+    p.n = (int)c->n; p.d = (int)c->d; p.m = (int)c->m; p.batch = (int)c->batch;
+    p.k0 = 0u;
+    p.steps = 2;
+    p.topology = c->topology;
+    p.H = 0;
+    p.log2n = log2_floor(c->n);
+    p.gamma = c->gamma; p.l2 = c->l2;
+    p.keys = c->keys;
+    p.poll_tries = 4096u;      // a few milliseconds
+    p.launch_nodes = 1;
+    cudaError_t e = cudaMemsetAsync(p.error_flag, 0, sizeof(int), s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(p.stop, 0, sizeof(int), s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(p.ytag, 0, (size_t)L.ytag_bytes, s);
+    if (e != cudaSuccess) return cuda_fail(c, e, "self-test clear");
+    c->flag_cleared = true;
+    e = launch_logreg_run(p, s);
+    c->launches += 1;
+    if (e != cudaSuccess) return cuda_fail(c, e, "self-test launch");
+    return GPGA_OK;
+}
+
+// ---- node sharding ------------------------------------------------------------------------------
+namespace {
+
+int64_t shard_row_bytes(int64_t d) { return (d + 3) / 4 * 16; }   // one exchanged row: whole groups of four floats
+
+ShardParams shard_params(const gpga_ctx* c, int64_t k)
+{
+    ShardParams p;
+    p.x = c->x[c->cur];
+    p.b = c->data;
+    p.out = c->x[c->cur ^ 1];
+    p.n = c->n; p.n_total = c->n * c->shards; p.row0 = c->shard * c->n;
+    p.d = c->d; p.ld = c->ld; p.Q = (c->d + 3) / 4;
+    p.q_base = (uint32_t)(c->col0 >> 2);
+    p.k = (uint32_t)k;
+    p.gamma = c->gamma; p.sigma = c->sigma;
+    p.keys = c->keys;
+    return p;
+}
+
+int32_t shard_ready(gpga_ctx* c, int64_t k)
+{
+    int32_t st = check_ready(c);
+    if (st) return st;
+    if (c->objective != GPGA_OBJ_QUADRATIC || (c->topology != GPGA_TOPO_RING && c->topology != GPGA_TOPO_EXP))
+        return fail(c, GPGA_ERR_UNSUPPORTED, "node sharding: quadratic objective on the ring or the one-peer exponential graph");
+    if (k < 0 || k >= (int64_t(1) << 32)) return fail(c, GPGA_ERR_INVALID_ARG, "k must be in [0, 2^32)");
+    return GPGA_OK;
+}
+
+}  // namespace
+
+int32_t gpga_shard_plan(int32_t topology, int64_t H, int64_t n_total, int64_t shards, int64_t shard, int64_t d,
+                        int64_t k, gpga_shard_plan_t* out)
+{
+    if (!out) return fail(nullptr, GPGA_ERR_INVALID_ARG, "out is NULL");
+    *out = gpga_shard_plan_t{};
+    if (topology != GPGA_TOPO_RING && topology != GPGA_TOPO_EXP)
+        return fail(nullptr, GPGA_ERR_UNSUPPORTED, "node sharding: ring or one-peer exponential graph");
+    if (H < 0 || n_total < 1 || n_total >= (int64_t(1) << 31) || shards < 1 || n_total % shards != 0 || shard < 0 ||
+        shard >= shards || d < 1 || k < 0)
+        return fail(nullptr, GPGA_ERR_INVALID_ARG, "need H >= 0, shards dividing n_total, 0 <= shard < shards, d >= 1, k >= 0");
+    if (topology == GPGA_TOPO_EXP && (!is_pow2(n_total) || !is_pow2(shards)))
+        return fail(nullptr, GPGA_ERR_UNSUPPORTED, "the one-peer exponential graph needs n and the number of shards to be powers of two");
+    const int64_t n_l = n_total / shards, row = shard_row_bytes(d);
+    const int32_t up = (int32_t)((shard + shards - 1) % shards), dn = (int32_t)((shard + 1) % shards);
+    if (is_global_step(k, H)) {   // every shard's column sums to every shard, in shard order
+        out->kind = GPGA_SHARD_GLOBAL;
+        out->gather_bytes = (d + 3) / 4 * 4 * (int64_t)sizeof(double);
+        return GPGA_OK;
+    }
+    if (topology == GPGA_TOPO_RING) {
+        out->kind = GPGA_SHARD_RING;
+        out->messages = 2;
+        // message 0: this shard's first row goes up (it is the lower neighbour of the shard above's last
+        // node); message 1: its last row goes down.  Received: slot 0 = the row above, slot 1 = the row below.
+        out->send_to[0] = up; out->send_offset[0] = 0;   out->dst_offset[0] = row; out->bytes[0] = row;
+        out->send_to[1] = dn; out->send_offset[1] = row; out->dst_offset[1] = 0;   out->bytes[1] = row;
+        out->recv_from[0] = up; out->recv_offset[0] = 0;
+        out->recv_from[1] = dn; out->recv_offset[1] = row;
+        return GPGA_OK;
+    }
+    const int tau = log2_floor(n_total);
+    const int64_t hop = tau > 0 ? (int64_t(1) << (k % tau)) : 1;
+    const int64_t he = hop < n_l ? hop : n_l;              // rows that cross the shard boundary
+    const int64_t ahead = hop < n_l ? 1 : hop / n_l;       // the partner rows live this many shards ahead
+    out->kind = GPGA_SHARD_EXP;
+    out->hop = hop;
+    out->messages = 1;
+    out->send_to[0] = (int32_t)(((shard - ahead) % shards + shards) % shards);
+    out->recv_from[0] = (int32_t)((shard + ahead) % shards);
+    out->bytes[0] = he * row;
+    return GPGA_OK;
+}
+
+int32_t gpga_set_node_shard(gpga_t* c, int64_t shards, int64_t shard)
+{
+    if (!c) return fail(nullptr, GPGA_ERR_NOT_READY, "NULL handle");
+    if (shards < 1 || shard < 0 || shard >= shards || c->n * shards >= (int64_t(1) << 31))
+        return fail(c, GPGA_ERR_INVALID_ARG, "need shards >= 1, 0 <= shard < shards, n * shards < 2^31");
+    if (c->objective != GPGA_OBJ_QUADRATIC || (c->topology != GPGA_TOPO_RING && c->topology != GPGA_TOPO_EXP))
+        return fail(c, GPGA_ERR_UNSUPPORTED, "node sharding: quadratic objective on the ring or the one-peer exponential graph");
+    if (c->topology == GPGA_TOPO_EXP && !is_pow2(shards))
+        return fail(c, GPGA_ERR_UNSUPPORTED, "the one-peer exponential graph needs a power-of-two number of shards");
+    if (shards > 1 && (c->n % 4) != 0)
+        return fail(c, GPGA_ERR_UNSUPPORTED, "with several shards a shard holds a multiple of four nodes (the column mean adds rows in groups of four)");
+    c->shards = shards;
+    c->shard = shard;
+    return GPGA_OK;
+}
+
+int64_t gpga_shard_exchange_bytes(const gpga_t* c)
+{
+    if (!c) return 0;
+    const int64_t row = shard_row_bytes(c->d);
+    int64_t rows = c->n > 2 ? c->n : 2;
+    int64_t bytes = rows * row;
+    const int64_t sums = c->shards * ((c->d + 3) / 4 * 4) * (int64_t)sizeof(double);
+    return bytes > sums ? bytes : sums;
+}
+
+int32_t gpga_shard_export(gpga_t* c, int64_t k, void* send_dev, void* stream)
+{
+    int32_t st = shard_ready(c, k);
+    if (st) return st;
+    if (!send_dev || !aligned16(send_dev)) return fail(c, GPGA_ERR_INVALID_ARG, "send buffer must be a 16-byte aligned device pointer");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const ShardParams p = shard_params(c, k);
+    const bool vec = vec_ok(c);
+    cudaError_t e;
+    if (is_global_step(k, c->H)) {
+        e = launch_shard_export_sums(p, vec, static_cast<double*>(send_dev), s);
+    } else if (c->topology == GPGA_TOPO_RING) {
+        // the first and the last local row (one and the same when the shard holds a single node)
+        e = launch_shard_export_rows(p, vec, static_cast<float*>(send_dev), 0, (int)(c->n - 1), 2, s);
+    } else {
+        const int tau = log2_floor(p.n_total);
+        const int64_t hop = tau > 0 ? (int64_t(1) << (k % tau)) : 1;
+        e = launch_shard_export_rows(p, vec, static_cast<float*>(send_dev), 0, 1, (int)(hop < c->n ? hop : c->n), s);
+    }
+    c->launches += 1;
+    if (e != cudaSuccess) return cuda_fail(c, e, "shard export launch");
+    return GPGA_OK;
+}
+
+int32_t gpga_shard_step(gpga_t* c, int64_t k, const void* recv_dev, void* stream)
+{
+    int32_t st = shard_ready(c, k);
+    if (st) return st;
+    if (!recv_dev || !aligned16(recv_dev)) return fail(c, GPGA_ERR_INVALID_ARG, "receive buffer must be a 16-byte aligned device pointer");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const ShardParams p = shard_params(c, k);
+    const bool vec = vec_ok(c);
+    cudaError_t e;
+    if (is_global_step(k, c->H)) {
+        e = launch_shard_global(p, vec, static_cast<const double*>(recv_dev), (int)c->shards, s);
+    } else if (c->topology == GPGA_TOPO_RING) {
+        e = launch_shard_ring(p, vec, static_cast<const float*>(recv_dev), s);
+    } else {
+        const int tau = log2_floor(p.n_total);
+        const int64_t hop = tau > 0 ? (int64_t(1) << (k % tau)) : 1;
+        e = launch_shard_exp(p, vec, static_cast<const float*>(recv_dev), (int)(hop < c->n ? hop : c->n), s);
+    }
+    c->launches += 1;
+    if (e != cudaSuccess) return cuda_fail(c, e, "shard step launch");
+    c->cur ^= 1;
+    c->k = k + 1;
     return GPGA_OK;
 }
 

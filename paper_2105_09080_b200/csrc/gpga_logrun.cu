@@ -57,8 +57,6 @@ constexpr int kRunChunkRows = 32, kRunChunkWarps = 8;   // the batch is cut as b
 constexpr int kRunMaxChunks = 2 * kRunWarps / kRunChunkWarps;   // 4: batch <= 128
 constexpr int kRunMaxNodes = 88;
 constexpr int kRunSmemLimit = 226 * 1024;       // dynamic; the static arrays take under 1 KB
-constexpr uint32_t kRunCopyTries = 1u << 18;    // polls of an mbarrier (about 4 us each while incomplete): about a second
-constexpr uint32_t kRunPollTries = 1u << 21;    // reads of a published word (half a microsecond or more each): a second or two
 
 __device__ __forceinline__ int ld_relaxed_gpu(const int* p)
 {
@@ -82,11 +80,12 @@ __device__ __forceinline__ void publish4(unsigned long long* dst, float4 v, uint
     asm volatile("st.relaxed.gpu.global.v2.b64 [%0], {%1, %2};" ::"l"(dst), "l"(w0), "l"(w1) : "memory");
     asm volatile("st.relaxed.gpu.global.v2.b64 [%0], {%1, %2};" ::"l"(dst + 2), "l"(w2), "l"(w3) : "memory");
 }
-// Reads the group until all four tags equal `tag`.  Gives up after kRunPollTries reads, or as soon
+// Reads the group until all four tags equal `tag`.  Gives up after `tries` reads, or as soon
 // as *stop is set; returns false then (v is not meaningful).
-__device__ __forceinline__ bool read4(const unsigned long long* src, uint32_t tag, const int* stop, float4* v)
+__device__ __forceinline__ bool read4(const unsigned long long* src, uint32_t tag, const int* stop, uint32_t tries,
+                                      float4* v)
 {
-    for (uint32_t t = 0; t < kRunPollTries; ++t) {
+    for (uint32_t t = 0; t < tries; ++t) {
         unsigned long long w0, w1, w2, w3;
         asm volatile("ld.relaxed.gpu.global.v2.b64 {%0, %1}, [%2];" : "=l"(w0), "=l"(w1) : "l"(src) : "memory");
         asm volatile("ld.relaxed.gpu.global.v2.b64 {%0, %1}, [%2];" : "=l"(w2), "=l"(w3) : "l"(src + 2) : "memory");
@@ -114,9 +113,9 @@ __device__ __forceinline__ bool try4(const unsigned long long* src, uint32_t tag
            (uint32_t)(w3 >> 32) == tag;
 }
 // Polls one word until its tag equals `tag` (bounded, ends on the stop word).
-__device__ __forceinline__ bool wait_tag(const unsigned long long* word, uint32_t tag, const int* stop)
+__device__ __forceinline__ bool wait_tag(const unsigned long long* word, uint32_t tag, const int* stop, uint32_t tries)
 {
-    for (uint32_t t = 0; t < kRunPollTries; ++t) {
+    for (uint32_t t = 0; t < tries; ++t) {
         unsigned long long w;
         asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];" : "=l"(w) : "l"(word) : "memory");
         if ((uint32_t)(w >> 32) == tag) return true;
@@ -130,12 +129,12 @@ __device__ __forceinline__ bool wait_tag(const unsigned long long* word, uint32_
 // case that its words are not there yet).  One poller per warp keeps the polling traffic small.
 // The whole warp must call.
 __device__ __forceinline__ bool read4_warp(bool active, const unsigned long long* src, const unsigned long long* gate,
-                                           uint32_t tag, const int* stop, float4* v)
+                                           uint32_t tag, const int* stop, uint32_t tries, float4* v)
 {
     int ok = 1;
     if ((threadIdx.x & 31) == 0) {
         ok = 0;
-        for (uint32_t t = 0; t < kRunPollTries; ++t) {
+        for (uint32_t t = 0; t < tries; ++t) {
             unsigned long long w;
             asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];" : "=l"(w) : "l"(gate) : "memory");
             if ((uint32_t)(w >> 32) == tag) {
@@ -147,7 +146,7 @@ __device__ __forceinline__ bool read4_warp(bool active, const unsigned long long
     }
     ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
     if (!ok) return false;
-    return active ? read4(src, tag, stop, v) : true;
+    return active ? read4(src, tag, stop, tries, v) : true;
 }
 
 // ---- counted asynchronous stores into a block of the pair (distributed shared memory) ----------
@@ -168,11 +167,11 @@ __device__ __forceinline__ void send4(uint32_t dst, uint32_t bar, float4 v)
                  "r"(__float_as_uint(v.w)), "r"(bar)
                  : "memory");
 }
-// Waits for the phase of `bar` with the given parity; gives up after kRunCopyTries polls, or as soon
+// Waits for the phase of `bar` with the given parity; gives up after `tries` polls, or as soon
 // as *stop is set.
-__device__ __forceinline__ bool wait_phase(uint64_t* bar, uint32_t parity, const int* stop)
+__device__ __forceinline__ bool wait_phase(uint64_t* bar, uint32_t parity, const int* stop, uint32_t tries)
 {
-    for (uint32_t t = 0; t < kRunCopyTries; ++t) {
+    for (uint32_t t = 0; t < tries; ++t) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((t & 255u) == 255u && ld_relaxed_gpu(stop) != 0) return false;
     }
@@ -332,7 +331,7 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
         int stage_slot = 0;   // a warp without rows parks its zeros in its first buffer
         for (int rho = 0; rho < my_rows; ++rho) {
             stage_slot = wait_slot;
-            if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&bar[wait_slot], wait_parity, kRunCopyTries))) {
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&bar[wait_slot], wait_parity, p.copy_tries))) {
                 failed = true;
                 break;
             }
@@ -420,7 +419,7 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
         unsigned long long* ybuf = p.ytag + (size_t)buf * buf_words;
         float4 yv = make_float4(0.f, 0.f, 0.f, 0.f);
         if (finisher) {
-            if (!wait_phase(&sums_bar, phase, stop)) failed = true;
+            if (!wait_phase(&sums_bar, phase, stop, p.copy_tries)) failed = true;
             float4 gs = pbuf[tid];
             for (int cc = 1; cc < chunks; ++cc) add4_to(gs, pbuf[cc * h0 + tid]);
             const float4 gr = make_float4(fmaf(gs.x, inv_batch, p.l2 * xo.x), fmaf(gs.y, inv_batch, p.l2 * xo.y),
@@ -443,7 +442,7 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
             if (tid < mine_cnt * n) {
                 const int j = tid / n, row = tid - j * n;
                 float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (!read4(ybuf + (size_t)row * d + 4 * (g_lo + i + j * n), tag, stop, &v)) failed = true;
+                if (!read4(ybuf + (size_t)row * d + 4 * (g_lo + i + j * n), tag, stop, p.poll_tries, &v)) failed = true;
                 items[tid] = v;   // [j][row]
             }
             __syncthreads();
@@ -467,7 +466,7 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
                 asm volatile("st.relaxed.gpu.global.b64 [%0], %1;" ::"l"(means + 4 * (g_lo + i + j * n) + comp), "l"(word)
                              : "memory");
             }
-            if (finisher && !read4(means + 4 * (g_lo + tid), tag, stop, &xp)) failed = true;
+            if (finisher && !read4(means + 4 * (g_lo + tid), tag, stop, p.poll_tries, &xp)) failed = true;
         } else if (finisher_warp) {
             const int seg_last = min(warp * 32 + 31, owned - 1);
             const unsigned long long* col = ybuf + 4 * (g_lo + min(tid, owned - 1));
@@ -475,12 +474,12 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
             if (p.topology == GPGA_TOPO_RING) {
                 const int up = (i == 0) ? n - 1 : i - 1, dn = (i == n - 1) ? 0 : i + 1;
                 float4 yu = yv, yd = yv;
-                if (lane < 2 && !wait_tag(gate + (size_t)(lane ? dn : up) * d, tag, stop)) failed = true;
+                if (lane < 2 && !wait_tag(gate + (size_t)(lane ? dn : up) * d, tag, stop, p.poll_tries)) failed = true;
                 __syncwarp();
                 if (finisher && !failed) {
                     const bool ok_u = try4(col + (size_t)up * d, tag, &yu), ok_d = try4(col + (size_t)dn * d, tag, &yd);
-                    if (!ok_u && !read4(col + (size_t)up * d, tag, stop, &yu)) failed = true;
-                    if (!ok_d && !read4(col + (size_t)dn * d, tag, stop, &yd)) failed = true;
+                    if (!ok_u && !read4(col + (size_t)up * d, tag, stop, p.poll_tries, &yu)) failed = true;
+                    if (!ok_d && !read4(col + (size_t)dn * d, tag, stop, p.poll_tries, &yd)) failed = true;
                 }
                 const float third = 0.333333343f;
                 xp = make_float4((yu.x + yv.x + yd.x) * third, (yu.y + yv.y + yd.y) * third,
@@ -489,7 +488,7 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
                 const int hop_log2 = p.log2n > 0 ? (int)(k % p.log2n) : 0;
                 const int peer = (i + (1 << hop_log2)) & (n - 1);
                 float4 yp = yv;
-                if (!read4_warp(finisher, col + (size_t)peer * d, gate + (size_t)peer * d, tag, stop, &yp)) failed = true;
+                if (!read4_warp(finisher, col + (size_t)peer * d, gate + (size_t)peer * d, tag, stop, p.poll_tries, &yp)) failed = true;
                 xp = make_float4((yv.x + yp.x) * 0.5f, (yv.y + yp.y) * 0.5f, (yv.z + yp.z) * 0.5f,
                                  (yv.w + yp.w) * 0.5f);
             }
@@ -502,7 +501,7 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
             if (it == p.steps - 1) reinterpret_cast<float4*>(p.x_out + (long long)i * p.ldx)[g_lo + tid] = xp;
         }
         if (finisher_warp) roll(it);
-        if (!failed && !wait_phase(&x_bar, phase, stop)) failed = true;
+        if (!failed && !wait_phase(&x_bar, phase, stop, p.copy_tries)) failed = true;
         if (failed) {   // tell everyone; the partner's and the other nodes' waits end on the stop word
             st_relaxed_gpu(p.stop, 1);
             if (p.error_flag) atomicExch(p.error_flag, 1);
@@ -518,7 +517,7 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
     // Copies still in flight target this block's shared memory: give each a bounded chance to land
     // (none is in flight after a run that went through).
     for (int q = consumed; q < issued; ++q)
-        mbar_wait_bounded(&bar[q % depth], (uint32_t)(q / depth) & 1u, kRunCopyTries);
+        mbar_wait_bounded(&bar[q % depth], (uint32_t)(q / depth) & 1u, p.copy_tries);
     cluster.sync();   // neither block leaves while the other may still send to it
 }
 
@@ -583,7 +582,8 @@ cudaError_t launch_logreg_run(const LogRunParams& p, cudaStream_t s)
     const RunSmem plan = run_smem_plan(p.d);
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attrs[1];
-    const cudaError_t e = run_config(&cfg, attrs, p.n, plan.bytes, s);
+    // (launch_nodes < n only in the self-test of the bounded waits: the rows of the nodes left out are never published)
+    const cudaError_t e = run_config(&cfg, attrs, p.launch_nodes > 0 ? p.launch_nodes : p.n, plan.bytes, s);
     if (e != cudaSuccess) return e;
     return cudaLaunchKernelEx(&cfg, p.d == kRunMaxD ? logreg_run_kernel<true> : logreg_run_kernel<false>, p, plan.slots);
 }

@@ -7,6 +7,8 @@
 
 namespace gpga {
 
+constexpr uint32_t kLogRunCopyTries = 1u << 18, kLogRunPollTries = 1u << 21;
+
 struct LogRunParams {
     const float* A;       // n x m x d
     const float* y;       // n x m, +-1
@@ -26,6 +28,11 @@ struct LogRunParams {
     int log2n;            // one-peer exponential graph: hops cycle through 2^0 .. 2^(log2n - 1)
     float gamma, l2;
     PhiloxKeys keys;
+    // Limits of the kernel's waits: polls of an mbarrier (about 4 us each while incomplete) and reads
+    // of a published word (half a microsecond or more each); the defaults make a wait last a second or
+    // two before it gives up.  Shorter limits are for the self-test of the give-up path.
+    uint32_t copy_tries = kLogRunCopyTries, poll_tries = kLogRunPollTries;
+    int launch_nodes = 0;   // > 0: launch only the pairs of nodes 0 .. launch_nodes - 1 (self-test only)
 };
 
 // Buffers of half-step rows the kernel cycles through.  A block overwrites the row it published

@@ -1,0 +1,240 @@
+// Node-sharded Gossip-PGA: the n nodes (rows of X) are split over several devices, each
+// holding n_l = n / shards consecutive nodes and all d columns -- the deployment of Section 3,
+// where a gossip step exchanges half-step parameter vectors x^(k+1/2) between neighbouring nodes
+// and the global average is an All-Reduce.  One iteration of Algorithm 1 on a shard is two
+// kernels with an exchange between them:
+//
+//   export : form the half-step rows y = x - gamma g that OTHER shards need (ring: the first and
+//            the last local row; one-peer exponential graph with hop h: the first min(h, n_l)
+//            local rows; global average: the shard's column sums over its rows) -> send buffer
+//   -- the caller moves send buffers into the peers' receive buffers (a copy, or NCCL) --
+//   step   : the fused local update + mix over the local rows, reading what was received where
+//            a neighbour is not local (ring: the row above the first and below the last local
+//            row; exponential graph: the partner rows; global average: all shards' column sums)
+//
+// Every result is formed by the operations, in the order, of the unsharded kernels (ring:
+// (up + self) + down; exponential graph: (y_i + y_partner) / 2; column mean: rows added pairwise
+// in fp32 in groups of four, group sums accumulated in fp64 in row order -- shard boundaries
+// fall on multiples of four rows -- and the shards' fp64 sums added in shard order), so a
+// sharded run agrees with the unsharded one bit for bit whenever the fp64 accumulation of a
+// column is exact (always, unless magnitudes inside one column differ by more than 2^29), and to
+// one fp64 rounding otherwise.  Remote rows are only ever read from this device's own memory.
+#include "gpga_shard.cuh"
+
+namespace gpga {
+
+namespace {
+
+constexpr int kShardBlock = 256;
+
+struct Group {
+    long long j0;   // first local column
+    uint32_t qg;    // global group index (first counter word of the generator)
+};
+
+__device__ __forceinline__ Group group_of(const ShardParams& p, long long q)
+{
+    Group g;
+    g.j0 = q * 4;
+    g.qg = p.q_base + (uint32_t)q;
+    return g;
+}
+
+// Half-step value of local row i for one column group (Algorithm 1: gradient, local update).
+template <bool NOISE, bool VEC>
+__device__ __forceinline__ float4 half_step_row(const ShardParams& p, const Group& g, int i)
+{
+    const float4 x = load4<VEC>(p.x + (long long)i * p.ld, g.j0, p.d);
+    const float4 b = load4<VEC>(p.b + (long long)i * p.ld, g.j0, p.d);
+    float4 gr = sub4(x, b);
+    if (NOISE) gr = fma4(p.sigma, normal4(g.qg, (uint32_t)(p.row0 + i), p.k, 0u, p.keys), gr);
+    return fma4(-p.gamma, gr, x);
+}
+
+template <bool VEC>
+__device__ __forceinline__ float4 load_dense(const float* buf, long long row, const ShardParams& p, const Group& g)
+{
+    // exchange buffers are dense: row stride d4 * 4 floats (d rounded up to a whole group)
+    const long long pitch = p.Q * 4;
+    return load4<true>(buf + row * pitch + g.j0, 0, 0);
+}
+__device__ __forceinline__ void store_dense(float* buf, long long row, const ShardParams& p, const Group& g, float4 v)
+{
+    store4<true>(buf + row * p.Q * 4 + g.j0, 0, 0, v);
+}
+
+template <bool VEC>
+__device__ __forceinline__ void store_out(const ShardParams& p, const Group& g, int i, float4 v)
+{
+    store4<VEC>(p.out + (long long)i * p.ld, g.j0, p.d, v);
+}
+
+__device__ __forceinline__ float4 mix3(float4 a, float4 b, float4 c)
+{
+    return scale4(add4(add4(a, b), c), 0.333333343f);
+}
+__device__ __forceinline__ float4 half(float4 a, float4 b) { return scale4(add4(a, b), 0.5f); }
+
+// ---- export ------------------------------------------------------------------------------------
+// send[t][:] = half-step of local row first + t * stride, t < rows.
+template <bool NOISE, bool VEC>
+__global__ void __launch_bounds__(kShardBlock) shard_export_rows_kernel(const ShardParams p, float* __restrict__ send,
+                                                                         int first, int stride, int rows)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.Q) return;
+    const Group g = group_of(p, q);
+    for (int t = 0; t < rows; ++t) store_dense(send, t, p, g, half_step_row<NOISE, VEC>(p, g, first + t * stride));
+}
+
+// Column sums of the half-step over the local rows, as the global-average kernel forms them:
+// rows pairwise in fp32 in groups of four, groups in fp64 in row order.  sums[4 q .. 4 q + 3].
+template <bool NOISE, bool VEC>
+__global__ void __launch_bounds__(kShardBlock) shard_export_sums_kernel(const ShardParams p, double* __restrict__ sums)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.Q) return;
+    const Group g = group_of(p, q);
+    double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+    const int n = (int)p.n;
+    int i = 0;
+    for (; i + 4 <= n; i += 4) {
+        const float4 y0 = half_step_row<NOISE, VEC>(p, g, i), y1 = half_step_row<NOISE, VEC>(p, g, i + 1);
+        const float4 y2 = half_step_row<NOISE, VEC>(p, g, i + 2), y3 = half_step_row<NOISE, VEC>(p, g, i + 3);
+        const float4 t = add4(add4(y0, y1), add4(y2, y3));
+        s0 += (double)t.x; s1 += (double)t.y; s2 += (double)t.z; s3 += (double)t.w;
+    }
+    const int rest = n - i;   // an unfinished last group (only when the shard is the whole problem)
+    if (rest >= 1) {
+        float4 a = half_step_row<NOISE, VEC>(p, g, i);
+        if (rest >= 2) a = add4(a, half_step_row<NOISE, VEC>(p, g, i + 1));
+        s0 += (double)a.x; s1 += (double)a.y; s2 += (double)a.z; s3 += (double)a.w;
+    }
+    if (rest == 3) {
+        const float4 b = half_step_row<NOISE, VEC>(p, g, i + 2);
+        s0 += (double)b.x; s1 += (double)b.y; s2 += (double)b.z; s3 += (double)b.w;
+    }
+    double* o = sums + 4 * q;
+    o[0] = s0; o[1] = s1; o[2] = s2; o[3] = s3;
+}
+
+// ---- step --------------------------------------------------------------------------------------
+// Ring: recv[0] = half-step of the node above local row 0, recv[1] = of the node below the last.
+template <bool NOISE, bool VEC>
+__global__ void __launch_bounds__(kShardBlock, 4) shard_ring_kernel(const ShardParams p, const float* __restrict__ recv)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.Q) return;
+    const Group g = group_of(p, q);
+    const int n = (int)p.n;
+    float4 a = load_dense<VEC>(recv, 0, p, g);
+    float4 b = half_step_row<NOISE, VEC>(p, g, 0);
+#pragma unroll 4
+    for (int i = 1; i < n; ++i) {
+        const float4 v = half_step_row<NOISE, VEC>(p, g, i);
+        store_out<VEC>(p, g, i - 1, mix3(a, b, v));
+        a = b;
+        b = v;
+    }
+    store_out<VEC>(p, g, n - 1, mix3(a, b, load_dense<VEC>(recv, 1, p, g)));
+}
+
+// One-peer exponential graph with hop h: he = min(h, n_l) chains c, c + he, c + 2 he, ... of local
+// rows; a row's partner is the next row of its chain, the last row's partner is recv[c] (the
+// partner shard's row c).  Each local row is read, and its noise generated, once.
+template <bool NOISE, bool VEC>
+__global__ void __launch_bounds__(kShardBlock, 4) shard_exp_kernel(const ShardParams p, const float* __restrict__ recv,
+                                                                    int he)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.Q) return;
+    const Group g = group_of(p, q);
+    const int n = (int)p.n;
+    for (int c = 0; c < he; ++c) {
+        float4 prev = half_step_row<NOISE, VEC>(p, g, c);
+        int row = c;
+#pragma unroll 4
+        for (int nxt = c + he; nxt < n; nxt += he) {
+            const float4 y = half_step_row<NOISE, VEC>(p, g, nxt);
+            store_out<VEC>(p, g, row, half(prev, y));
+            prev = y;
+            row = nxt;
+        }
+        store_out<VEC>(p, g, row, half(prev, load_dense<VEC>(recv, c, p, g)));
+    }
+}
+
+// Global average: recv holds `parts` vectors of column sums (4 Q doubles each), one per shard in
+// shard order; mean = (sum of the parts in that order) / n_total, rounded once, to every local row.
+template <bool VEC>
+__global__ void __launch_bounds__(kShardBlock) shard_global_kernel(const ShardParams p, const double* __restrict__ recv,
+                                                                    int parts)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.Q) return;
+    const Group g = group_of(p, q);
+    double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+    for (int t = 0; t < parts; ++t) {
+        const double* v = recv + ((long long)t * p.Q + q) * 4;
+        s0 += v[0]; s1 += v[1]; s2 += v[2]; s3 += v[3];
+    }
+    const double inv = (double)p.n_total;
+    const float4 m = make_float4((float)(s0 / inv), (float)(s1 / inv), (float)(s2 / inv), (float)(s3 / inv));
+    const int n = (int)p.n;
+    for (int i = 0; i < n; ++i) store_out<VEC>(p, g, i, m);
+}
+
+unsigned grid_of(long long Q) { return (unsigned)((Q + kShardBlock - 1) / kShardBlock); }
+
+}  // namespace
+
+#define GPGA_SHARD_LAUNCH(kernel, noise, vec, ...)                                           \
+    do {                                                                                     \
+        if (noise) {                                                                         \
+            if (vec) kernel<true, true><<<grid_of(p.Q), kShardBlock, 0, s>>>(__VA_ARGS__);   \
+            else kernel<true, false><<<grid_of(p.Q), kShardBlock, 0, s>>>(__VA_ARGS__);      \
+        } else {                                                                             \
+            if (vec) kernel<false, true><<<grid_of(p.Q), kShardBlock, 0, s>>>(__VA_ARGS__);  \
+            else kernel<false, false><<<grid_of(p.Q), kShardBlock, 0, s>>>(__VA_ARGS__);     \
+        }                                                                                    \
+    } while (0)
+
+cudaError_t launch_shard_export_rows(const ShardParams& p, bool vec, float* send, int first, int stride, int rows,
+                                     cudaStream_t s)
+{
+    const bool noise = p.sigma != 0.f;
+    GPGA_SHARD_LAUNCH(shard_export_rows_kernel, noise, vec, p, send, first, stride, rows);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_shard_export_sums(const ShardParams& p, bool vec, double* sums, cudaStream_t s)
+{
+    const bool noise = p.sigma != 0.f;
+    GPGA_SHARD_LAUNCH(shard_export_sums_kernel, noise, vec, p, sums);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_shard_ring(const ShardParams& p, bool vec, const float* recv, cudaStream_t s)
+{
+    const bool noise = p.sigma != 0.f;
+    GPGA_SHARD_LAUNCH(shard_ring_kernel, noise, vec, p, recv);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_shard_exp(const ShardParams& p, bool vec, const float* recv, int he, cudaStream_t s)
+{
+    const bool noise = p.sigma != 0.f;
+    GPGA_SHARD_LAUNCH(shard_exp_kernel, noise, vec, p, recv, he);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_shard_global(const ShardParams& p, bool vec, const double* recv, int parts, cudaStream_t s)
+{
+    if (vec)
+        shard_global_kernel<true><<<grid_of(p.Q), kShardBlock, 0, s>>>(p, recv, parts);
+    else
+        shard_global_kernel<false><<<grid_of(p.Q), kShardBlock, 0, s>>>(p, recv, parts);
+    return cudaGetLastError();
+}
+
+}  // namespace gpga

@@ -1,0 +1,37 @@
+// Launchers of the node-sharded iteration (defined in gpga_shard.cu).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gpga_device.cuh"
+
+namespace gpga {
+
+struct ShardParams {
+    const float* x;      // X^(k), the shard's n x d rows, row stride ld
+    const float* b;      // targets b, same layout
+    float* out;          // X^(k+1), same layout (may be x: every kernel reads a row before it writes it)
+    long long n;         // local rows (nodes of this shard)
+    long long n_total;   // nodes of the whole problem
+    long long row0;      // global index of local row 0 (second counter word of the generator)
+    long long d, ld;
+    long long Q;         // column groups of four: ceil(d / 4); exchange buffers have rows of 4 Q floats
+    uint32_t q_base;     // global index of local group 0 (column offset / 4)
+    uint32_t k;          // iteration index
+    float gamma, sigma;
+    PhiloxKeys keys;
+};
+
+// export: half-step rows first, first + stride, ... (rows of them) into the dense send buffer
+cudaError_t launch_shard_export_rows(const ShardParams& p, bool vec, float* send, int first, int stride, int rows,
+                                     cudaStream_t s);
+// export: the shard's column sums of the half-step (4 Q doubles)
+cudaError_t launch_shard_export_sums(const ShardParams& p, bool vec, double* sums, cudaStream_t s);
+// step: ring with recv = [row above local row 0 | row below the last local row]
+cudaError_t launch_shard_ring(const ShardParams& p, bool vec, const float* recv, cudaStream_t s);
+// step: one-peer exponential graph, he = min(hop, local rows); recv = the partner shard's rows 0 .. he-1
+cudaError_t launch_shard_exp(const ShardParams& p, bool vec, const float* recv, int he, cudaStream_t s);
+// step: global average from `parts` vectors of column sums in shard order
+cudaError_t launch_shard_global(const ShardParams& p, bool vec, const double* recv, int parts, cudaStream_t s);
+
+}  // namespace gpga

@@ -1,0 +1,129 @@
+"""Node-sharded Gossip-PGA: the n nodes split over several devices, as in the paper's own deployment
+(Section 3: gossip between neighbouring nodes, All-Reduce for the global average; appendix,
+implementation details: one parameter copy sent and one received per one-peer step).
+
+The arithmetic of a shard's iteration is the library's (`gpga_shard_export`, `gpga_shard_step`), the
+schedule of who sends what to whom is the library's too (`gpga_shard_plan`).  This module only
+moves the messages: between shards that live in one process (`exchange_local`: one copy per
+message) or between ranks of a `torch.distributed` group (`exchange_dist`: isend / irecv for the
+gossip messages, an all-gather of the column sums for the global average; NCCL on GPUs, gloo on CPU).
+"""
+from __future__ import annotations
+
+import ctypes as C
+
+from . import binding as B
+
+
+class ShardPlan(C.Structure):
+    """Mirror of gpga_shard_plan_t."""
+    _fields_ = [("kind", C.c_int32), ("messages", C.c_int32), ("send_to", C.c_int32 * 2), ("recv_from", C.c_int32 * 2),
+                ("send_offset", C.c_int64 * 2), ("dst_offset", C.c_int64 * 2), ("recv_offset", C.c_int64 * 2),
+                ("bytes", C.c_int64 * 2), ("gather_bytes", C.c_int64), ("hop", C.c_int64)]
+
+
+GPGA_SHARD_RING, GPGA_SHARD_EXP, GPGA_SHARD_GLOBAL = 0, 1, 2
+
+
+def shard_plan(topology, H, n_total, shards, shard, d, k) -> ShardPlan:
+    plan = ShardPlan()
+    st = B.lib().gpga_shard_plan(topology, H, n_total, shards, shard, d, k, C.byref(plan))
+    if st != B.GPGA_OK:
+        raise B.GpgaError(st, B.lib().gpga_last_error(None).decode())
+    return plan
+
+
+class NodeShard:
+    """One shard on the current CUDA device: a handle over n_total / shards nodes and its exchange
+    buffers (uint8 tensors `send` and `recv`)."""
+
+    def __init__(self, n_total, d, topology, H, gamma, seed, shards, shard, sigma=0.0, ld=None, col0=0,
+                 device="cuda"):
+        import torch
+        assert n_total % shards == 0
+        self.n_total, self.d, self.topology, self.H = n_total, d, topology, H
+        self.shards, self.shard, self.n = shards, shard, n_total // shards
+        self.g = B.Gpga(self.n, d, topology, H, gamma, seed)
+        self.g.set_objective(B.GPGA_OBJ_QUADRATIC, sigma=sigma)
+        if ld:
+            self.g.set_row_stride(ld)
+        if col0:
+            self.g.set_column_offset(col0)
+        self.g._check(B.lib().gpga_set_node_shard(self.g._h, shards, shard))
+        nbytes = int(B.lib().gpga_shard_exchange_bytes(self.g._h))
+        self.send = torch.zeros(nbytes, dtype=torch.uint8, device=device)
+        self.recv = torch.zeros(nbytes, dtype=torch.uint8, device=device)
+
+    def bind(self, x_a, x_b, b):
+        self.g.bind(x_a, x_b, b)
+
+    def plan(self, k) -> ShardPlan:
+        return shard_plan(self.topology, self.H, self.n_total, self.shards, self.shard, self.d, k)
+
+    def export(self, k, stream=None):
+        self.g._check(B.lib().gpga_shard_export(self.g._h, k, self.send.data_ptr(), self.g._sp(stream)))
+
+    def step(self, k, stream=None):
+        self.g._check(B.lib().gpga_shard_step(self.g._h, k, self.recv.data_ptr(), self.g._sp(stream)))
+
+    def get_x(self):
+        return self.g.get_x()
+
+    def close(self):
+        self.g.close()
+
+
+def exchange_local(shards, k):
+    """Deliver iteration k's messages between shards of one process: one copy per message (the
+    column sums of a global average: one copy per pair of shards).  `shards[s]` is shard s; each has
+    `.send`, `.recv` (uint8 tensors) and `.plan(k)`."""
+    for src in shards:
+        plan = src.plan(k)
+        if plan.kind == GPGA_SHARD_GLOBAL:
+            nb = plan.gather_bytes
+            for dst in shards:
+                dst.recv[src.shard * nb:(src.shard + 1) * nb].copy_(src.send[:nb], non_blocking=True)
+            continue
+        for m in range(plan.messages):
+            dst = shards[plan.send_to[m]]
+            lo, nb = plan.send_offset[m], plan.bytes[m]
+            dst.recv[plan.dst_offset[m]:plan.dst_offset[m] + nb].copy_(src.send[lo:lo + nb], non_blocking=True)
+
+
+def exchange_dist(shard, k, group=None):
+    """Deliver iteration k's messages of this rank's shard through torch.distributed: rank r holds
+    shard r.  Gossip messages go point to point (all sends and receives of the iteration posted
+    together), the column sums of a global average by an all-gather in rank order."""
+    import torch.distributed as dist
+    plan = shard.plan(k)
+    if plan.kind == GPGA_SHARD_GLOBAL:
+        nb = plan.gather_bytes
+        world = dist.get_world_size(group)
+        dist.all_gather([shard.recv[r * nb:(r + 1) * nb] for r in range(world)], shard.send[:nb], group=group)
+        return
+    me, ops, local = dist.get_rank(group), [], []
+    for m in range(plan.messages):
+        lo, nb = plan.send_offset[m], plan.bytes[m]
+        if plan.send_to[m] == me:       # a neighbour in the same shard (one shard, or a two-shard ring's both sides)
+            local.append((plan.dst_offset[m], lo, nb))
+        else:
+            ops.append(dist.P2POp(dist.isend, shard.send[lo:lo + nb], plan.send_to[m], group=group, tag=m))
+    for m in range(plan.messages):
+        if plan.recv_from[m] != me:
+            lo = plan.recv_offset[m]
+            # the sender's message index for this slot: ring slot 0 (row above) is the upper shard's message 1
+            tag = (1 - m) if plan.kind == GPGA_SHARD_RING else m
+            ops.append(dist.P2POp(dist.irecv, shard.recv[lo:lo + plan.bytes[m]], plan.recv_from[m], group=group, tag=tag))
+    for dst, lo, nb in local:
+        shard.recv[dst:dst + nb].copy_(shard.send[lo:lo + nb])
+    if ops:
+        for req in dist.batch_isend_irecv(ops):
+            req.wait()
+
+
+def run_dist(shard, K, k0=0, group=None):
+    """K iterations of this rank's shard: export, exchange, step."""
+    for k in range(k0, k0 + K):
+        shard.export(k)
+        exchange_dist(shard, k, group)
+        shard.step(k)

@@ -304,22 +304,6 @@ def test_multi_iteration_launch_is_chunked_for_long_runs():
     assert ok, worst
 
 
-def test_convex_experiment_driver_small():
-    """The Section 5.1 experiment driver at a reduced size: periodic global averaging keeps the
-    nodes closer to consensus than plain gossip, and all methods reduce the global loss."""
-    torch = _torch()
-    from paper_2105_09080_b200 import convex_experiment as ce
-    from paper_2105_09080_b200.inputs import convex_experiment_inputs
-    A, y = convex_experiment_inputs(20, 400, 10, seed=3)
-    A_dev, y_dev = torch.from_numpy(A).cuda(), torch.from_numpy(y).cuda()
-    out = {name: ce.run_one(A_dev, y_dev, pkg.GPGA_TOPO_RING, H, 600, 100, 8, seed=1, halve_every=250)
-           for name, H in ce.METHODS.items()}
-    for loss, cons in out.values():
-        assert len(loss) == 7 and loss[-1] < loss[0]
-    assert np.all(out["parallel_sgd"][1] == 0.0)
-    assert out["gossip_pga"][1][1:].mean() < out["gossip_sgd"][1][1:].mean()
-
-
 @pytest.mark.parametrize("n,d", [(9, 40), (30, 1030), (16, 20_004)])
 def test_general_sparse_weight_matrix(n, d):
     """Topology SPARSE: Metropolis weights of a random connected graph, given in CSR form."""

@@ -115,3 +115,43 @@ def test_resident_run_is_cut_into_launches_of_16384_iterations():
         stepped.step(k)
     a, b = run.get_x().cpu().numpy(), stepped.get_x().cpu().numpy()
     assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), float(np.abs(a - b).max())
+
+
+def test_waits_between_blocks_give_up_and_report_timeout():
+    """Node 0's pair of blocks launched alone with wait limits of a few thousand polls: its
+    neighbours' rows never appear, so its waits run out, the error word is raised, both blocks
+    of the pair leave, and the next synchronising call returns GPGA_ERR_TIMEOUT.  Nothing hangs
+    or faults: the device runs the next problem as before."""
+    import time
+    import torch
+    n, m, d, batch = 2, 64, 256, 64
+    A, y = logistic_inputs(n, m, d, SEED)
+    X0 = np.zeros((n, d), dtype=np.float32)
+    run, stepped = _pair(n, m, d, batch, "ring", 0, X0, A, y)
+    run.run(4)                                           # the kernel itself works on this problem
+    for k in range(4):
+        stepped.step(k)
+    assert np.array_equal(run.get_x().cpu().numpy(), stepped.get_x().cpu().numpy())
+    assert run.consensus_distance() >= 0.0
+    t0 = time.perf_counter()
+    run.selftest_run_wait()
+    with pytest.raises(pkg.GpgaError) as err:
+        run.consensus_distance()
+    assert err.value.status == pkg.GPGA_ERR_TIMEOUT
+    assert time.perf_counter() - t0 < 5.0                # milliseconds of polling, not the seconds of the defaults
+    with pytest.raises(pkg.GpgaError) as err:           # sticky
+        run.run(2)
+    assert err.value.status == pkg.GPGA_ERR_TIMEOUT
+    run.close()
+    torch.cuda.synchronize()
+    # a handle that the kernel does not take is turned away
+    with pytest.raises(pkg.GpgaError) as err:
+        stepped_exp = _pair(2, m, d, batch, "exp", 0, X0, A, y)[0]
+        stepped_exp.selftest_run_wait()
+    assert err.value.status == pkg.GPGA_ERR_UNSUPPORTED
+    # the device is as before: a fresh pair of handles agrees again
+    run2, stepped2 = _pair(n, m, d, batch, "ring", 3, X0, A, y)
+    run2.run(7)
+    for k in range(7):
+        stepped2.step(k)
+    assert np.array_equal(run2.get_x().cpu().numpy(), stepped2.get_x().cpu().numpy())
