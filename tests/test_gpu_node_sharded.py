@@ -1,0 +1,114 @@
+"""Node-sharded Gossip-PGA on ONE device: the n nodes are split into shards of consecutive rows,
+each shard a handle of its own; per iteration every shard exports what its neighbours need,
+the messages are delivered by one device-to-device copy each, and every shard steps.  The result
+must equal the unsharded run of the same problem bit for bit -- ring, every hop of the one-peer
+exponential graph (hops inside a shard and hops that span shards) and the global average -- and
+match the oracle within the parity tolerances."""
+import numpy as np
+import pytest
+
+import paper_2105_09080_b200 as pkg
+from oracle import gpga_oracle as o
+from paper_2105_09080_b200 import node_sharded as ns
+from paper_2105_09080_b200.inputs import quadratic_inputs
+from test_gpu_parity import TOL_RUN, TOL_STEP, TOPO, close, make_quadratic
+
+pytestmark = pytest.mark.gpu
+
+SEED = 20210509
+
+
+def _sharded_run(n, d, topo, H, gamma, sigma, X0, B, shards, K, col0=0, check_first=None):
+    import torch
+    n_l = n // shards
+    parts = []
+    for s in range(shards):
+        sh = ns.NodeShard(n, d, TOPO[topo][0], H, gamma, SEED, shards, s, sigma=sigma, col0=col0)
+        rows = slice(s * n_l, (s + 1) * n_l)
+        xa = torch.from_numpy(np.ascontiguousarray(X0[rows])).cuda()
+        sh.bind(xa, torch.empty_like(xa), torch.from_numpy(np.ascontiguousarray(B[rows])).cuda())
+        parts.append(sh)
+    for k in range(K):
+        for sh in parts:
+            sh.export(k)
+        ns.exchange_local(parts, k)
+        for sh in parts:
+            sh.step(k)
+        if check_first is not None and k == 0:
+            check_first(np.concatenate([sh.get_x().cpu().numpy() for sh in parts]))
+    out = np.concatenate([sh.get_x().cpu().numpy() for sh in parts])
+    assert all(sh.g.get_k() == K for sh in parts)
+    for sh in parts:
+        sh.close()
+    return out
+
+
+# d = 4104: the unsharded run goes through the shared-memory tile kernel; d = 19456: through the
+# row-streaming kernels; d = 1031: the scalar path (rows neither aligned nor whole groups)
+@pytest.mark.parametrize("d", [4104, 19456, 1031])
+@pytest.mark.parametrize("topo,H,n,shards", [("ring", 4, 16, 2), ("ring", 0, 16, 4), ("ring", 3, 8, 1), ("ring", 5, 24, 3),
+                                             ("exp", 3, 16, 2), ("exp", 0, 16, 4), ("exp", 5, 32, 4), ("exp", 4, 8, 1),
+                                             ("exp", 0, 8, 2)])
+def test_sharded_run_is_bit_identical_to_the_unsharded_run(topo, H, n, shards, d):
+    gamma, sigma, K = 0.1, 0.3, 13          # 13 iterations: every hop of the exponential graph, several global averages
+    X0, B = quadratic_inputs(n, d, SEED + n + d, x0="per_node")
+    g, p = make_quadratic(n, d, topo, H, gamma, SEED, sigma, X0, B)
+    first = {}
+
+    def one_step(x):
+        first["x"] = x
+
+    got = _sharded_run(n, d, topo, H, gamma, sigma, X0, B, shards, K, check_first=one_step)
+    g.step(0)
+    assert np.array_equal(first["x"].view(np.uint32), g.get_x().cpu().numpy().view(np.uint32))
+    ok, worst = close(first["x"], o.step(p, X0, 0), TOL_STEP)
+    assert ok, worst
+    for k in range(1, K):
+        g.step(k)
+    want = g.get_x().cpu().numpy()
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), float(np.abs(got - want).max())
+    ok, worst = close(got, o.run(p, X0, 0, K), TOL_RUN)
+    assert ok, worst
+    if H and K % H == 0:
+        assert np.all(got == got[0])
+    g.close()
+
+
+def test_sharded_run_with_a_column_offset_and_no_noise():
+    n, d, shards, K = 16, 2052, 4, 6
+    X0, B = quadratic_inputs(n, d, 5, x0="per_node")
+    for sigma, col0 in ((0.0, 0), (0.2, 8192)):
+        g, _ = make_quadratic(n, d, "exp", 3, 0.05, SEED, sigma, X0, B, col0=col0)
+        g.run(K)
+        got = _sharded_run(n, d, "exp", 3, 0.05, sigma, X0, B, shards, K, col0=col0)
+        assert np.array_equal(got, g.get_x().cpu().numpy())
+        g.close()
+
+
+def test_plan_and_argument_checks():
+    L = pkg.lib()
+    # two shards of 8 nodes, 16-node exponential graph: hops 1, 2, 4 stay next door, hop 8 is one shard ahead
+    for k, hop, rows in ((0, 1, 1), (1, 2, 2), (2, 4, 4), (3, 8, 8), (4, 1, 1)):
+        plan = ns.shard_plan(pkg.GPGA_TOPO_EXP, 0, 16, 2, 0, 40, k)
+        assert (plan.kind, plan.hop, plan.messages) == (ns.GPGA_SHARD_EXP, hop, 1)
+        assert plan.bytes[0] == rows * 40 * 4 and plan.send_to[0] == 1 and plan.recv_from[0] == 1
+    # eight shards of 4 nodes, 32 nodes: hop 16 is four shards ahead, hop 2 is the next shard
+    plan = ns.shard_plan(pkg.GPGA_TOPO_EXP, 0, 32, 8, 1, 8, 4)
+    assert plan.hop == 16 and plan.recv_from[0] == 5 and plan.send_to[0] == 5 and plan.bytes[0] == 4 * 8 * 4
+    plan = ns.shard_plan(pkg.GPGA_TOPO_EXP, 0, 32, 8, 1, 8, 1)
+    assert plan.hop == 2 and plan.recv_from[0] == 2 and plan.send_to[0] == 0 and plan.bytes[0] == 2 * 8 * 4
+    # ring: first row up, last row down; d = 10 travels as 12 floats
+    plan = ns.shard_plan(pkg.GPGA_TOPO_RING, 4, 12, 3, 0, 10, 0)
+    assert (plan.kind, plan.messages) == (ns.GPGA_SHARD_RING, 2)
+    assert list(plan.send_to) == [2, 1] and list(plan.recv_from) == [2, 1]
+    assert list(plan.bytes) == [48, 48] and list(plan.send_offset) == [0, 48] and list(plan.dst_offset) == [48, 0]
+    plan = ns.shard_plan(pkg.GPGA_TOPO_RING, 4, 12, 3, 0, 10, 3)          # mod(k + 1, H) = 0
+    assert plan.kind == ns.GPGA_SHARD_GLOBAL and plan.messages == 0 and plan.gather_bytes == 12 * 8
+    with pytest.raises(pkg.GpgaError):
+        ns.shard_plan(pkg.GPGA_TOPO_EXP, 0, 16, 3, 0, 8, 0)               # 3 shards of a 16-node exponential graph
+    with pytest.raises(pkg.GpgaError):
+        ns.shard_plan(pkg.GPGA_TOPO_GRID, 0, 16, 2, 0, 8, 0)
+    # a shard of several holds a multiple of four nodes
+    with pytest.raises(pkg.GpgaError) as err:
+        ns.NodeShard(12, 64, pkg.GPGA_TOPO_RING, 4, 0.1, 1, 2, 0)
+    assert err.value.status == pkg.GPGA_ERR_UNSUPPORTED

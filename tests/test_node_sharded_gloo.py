@@ -1,0 +1,142 @@
+"""The exchange schedule of node-sharded Gossip-PGA over ranks: world_size 2 (and 4), gloo on CPU.
+Each rank holds a shard of consecutive nodes and computes with the oracle; what is under test is
+the plan (who sends which rows to whom at which iteration: the ring's two neighbours, the partner
+shard of every hop of the one-peer exponential graph, the all-gather of the global average) and
+the torch.distributed delivery of the messages.  A wrong neighbour, offset or hop changes the
+result by O(1); the comparison with the unsharded oracle run allows only the fp32 rounding of the
+exchanged rows."""
+import os
+import socket
+
+import numpy as np
+import pytest
+
+import paper_2105_09080_b200 as pkg
+from oracle import gpga_oracle as o
+from paper_2105_09080_b200 import node_sharded as ns
+from paper_2105_09080_b200.inputs import quadratic_inputs
+
+TOPOLOGY = {"ring": (pkg.GPGA_TOPO_RING, o.TOPO_RING), "exp": (pkg.GPGA_TOPO_EXP, o.TOPO_EXP)}
+
+
+class OracleShard:
+    """A shard whose arithmetic is the oracle's: exported rows are the fp64 half-step rounded to the
+    fp32 the messages carry; the mix uses the received rows where the neighbour is not local."""
+
+    def __init__(self, n_total, d, topo, H, gamma, sigma, seed, shards, shard, X0, B):
+        import torch
+        self.n_total, self.d, self.topology, self.H = n_total, d, TOPOLOGY[topo][0], H
+        self.topo, self.gamma, self.sigma, self.seed = topo, gamma, sigma, seed
+        self.shards, self.shard, self.n = shards, shard, n_total // shards
+        rows = slice(shard * self.n, (shard + 1) * self.n)
+        self.X, self.B = X0[rows].astype(np.float32), B[rows].astype(np.float64)
+        self.q4 = (d + 3) // 4 * 4
+        nbytes = max(max(self.n, 2) * self.q4 * 4, shards * self.q4 * 8)
+        self.send = torch.zeros(nbytes, dtype=torch.uint8)
+        self.recv = torch.zeros(nbytes, dtype=torch.uint8)
+
+    def plan(self, k):
+        return ns.shard_plan(self.topology, self.H, self.n_total, self.shards, self.shard, self.d, k)
+
+    def _half_step(self, k):
+        """fp64 half-step of the local rows: the rows sit at their global positions of a full-height
+        matrix so that the oracle keys the noise by the global node index."""
+        full_x = np.zeros((self.n_total, self.d))
+        full_b = np.zeros((self.n_total, self.d))
+        rows = slice(self.shard * self.n, (self.shard + 1) * self.n)
+        full_x[rows], full_b[rows] = self.X, self.B
+        return o.quadratic_half_step(full_x, full_b, self.gamma, self.sigma, self.seed, k)[rows]
+
+    def export(self, k):
+        plan, Y = self.plan(k), self._half_step(k)
+        self.Y = Y
+        if plan.kind == ns.GPGA_SHARD_GLOBAL:
+            sums = np.zeros(self.q4)
+            sums[:self.d] = Y.sum(0)
+            self.send[:self.q4 * 8] = _bytes(sums)
+            return
+        if plan.kind == ns.GPGA_SHARD_RING:
+            out = Y[[0, self.n - 1]]
+        else:
+            out = Y[:min(plan.hop, self.n)]
+        msg = np.zeros((out.shape[0], self.q4), dtype=np.float32)
+        msg[:, :self.d] = out
+        self.send[:msg.nbytes] = _bytes(msg)
+
+    def step(self, k):
+        plan, Y, n, d = self.plan(k), self.Y, self.n, self.d
+        if plan.kind == ns.GPGA_SHARD_GLOBAL:
+            parts = np.frombuffer(self.recv.numpy()[:self.shards * self.q4 * 8].tobytes(), dtype=np.float64)
+            total = parts.reshape(self.shards, self.q4).sum(0)[:d]
+            Z = np.repeat((total / self.n_total)[None, :], n, axis=0)
+        else:
+            rows = 2 if plan.kind == ns.GPGA_SHARD_RING else min(plan.hop, n)
+            got = np.frombuffer(self.recv.numpy()[:rows * self.q4 * 4].tobytes(), dtype=np.float32)
+            got = got.reshape(rows, self.q4)[:, :d].astype(np.float64)
+            if plan.kind == ns.GPGA_SHARD_RING:
+                ext = np.concatenate([got[:1], Y, got[1:]])          # row above, local rows, row below
+                Z = (ext[:-2] + ext[1:-1] + ext[2:]) / 3.0
+            else:
+                he = rows
+                partner = np.concatenate([Y[he:], got]) if he < n else got
+                Z = (Y + partner) / 2.0
+        self.X = Z.astype(np.float32)
+
+
+def _bytes(a):
+    import torch
+    return torch.frombuffer(bytearray(np.ascontiguousarray(a).tobytes()), dtype=torch.uint8)
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def _worker(rank, world, port, topo, H, n, d, K, out_dir):
+    import torch.distributed as dist
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    X0, B = quadratic_inputs(n, d, 7, x0="per_node")
+    shard = OracleShard(n, d, topo, H, 0.1, 0.4, 11, world, rank, X0, B)
+    ns.run_dist(shard, K)
+    gathered = [None] * world
+    dist.all_gather_object(gathered, (rank, shard.X))
+    if rank == 0:
+        np.save(os.path.join(out_dir, "full.npy"), np.concatenate([x for _, x in sorted(gathered, key=lambda t: t[0])]))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("topo,H,n,world", [("ring", 4, 8, 2), ("exp", 3, 16, 2), ("exp", 0, 16, 4), ("ring", 0, 12, 3)])
+def test_ranks_exchange_the_right_rows(tmp_path, topo, H, n, world):
+    import torch.multiprocessing as mp
+    d, K = 10, 9
+    mp.spawn(_worker, args=(world, _free_port(), topo, H, n, d, K, str(tmp_path)), nprocs=world, join=True)
+    X0, B = quadratic_inputs(n, d, 7, x0="per_node")
+    want = o.run(o.Problem(TOPOLOGY[topo][1], H, 0.1, 11, sigma=0.4, data=B), X0, 0, K)
+    got = np.load(tmp_path / "full.npy")
+    assert got.shape == want.shape
+    # the exchanged half-step rows travel as fp32: a relative 6e-8 per exchanged row and iteration
+    assert np.abs(got - want).max() <= 2e-6 * (1 + np.abs(want).max())
+
+
+def test_one_process_delivery_matches_the_plan():
+    """exchange_local with four oracle shards in this process, ring and exponential graph."""
+    n, d, K, shards = 16, 6, 7, 4
+    X0, B = quadratic_inputs(n, d, 3, x0="per_node")
+    for topo, H in (("ring", 3), ("exp", 0), ("exp", 4)):
+        parts = [OracleShard(n, d, topo, H, 0.2, 0.1, 5, shards, s, X0, B) for s in range(shards)]
+        for k in range(K):
+            for sh in parts:
+                sh.export(k)
+            ns.exchange_local(parts, k)
+            for sh in parts:
+                sh.step(k)
+        got = np.concatenate([sh.X for sh in parts])
+        want = o.run(o.Problem(TOPOLOGY[topo][1], H, 0.2, 5, sigma=0.1, data=B), X0, 0, K)
+        assert np.abs(got - want).max() <= 2e-6 * (1 + np.abs(want).max()), (topo, H)
