@@ -18,8 +18,9 @@ at the copy's node average, and its consensus distance) come from small handles 
 copy's rows of the same buffers.  Everything numerical runs in the library's kernels.
 
 Prints one JSON line per (n, method): mean and standard deviation over the trials of the loss and of
-the consensus distance every `--every` iterations, and the transient stage read off the curves (the
-last recorded iteration at which the method's mean loss is still apart from parallel SGD's).
+the consensus distance every `--every` iterations, the loss in excess of parallel SGD's (a paired
+difference: all methods of a trial share its data and mini-batch draws) and the transient stage read
+off the curves (the last recorded iteration at which that excess is still apart from zero).
 The data recipe follows the paper; the mini-batch size, which the paper does not state, is an option.
 """
 from __future__ import annotations
@@ -126,12 +127,22 @@ class BatchedTrials:
             h.close()
 
 
+def excess_over(loss, reference):
+    """Per record: mean and standard error over trials of loss - reference, trial by trial (the
+    trials of two methods share data sets and mini-batch draws, so the difference is paired)."""
+    diff = loss - reference
+    return diff.mean(1), diff.std(1) / np.sqrt(diff.shape[1])
+
+
 def transient_stage(marks, loss, reference):
-    """Last recorded iteration at which the mean loss over trials is still apart from the
-    reference method's (beyond three standard errors of the two means), 0 if never."""
-    mean, ref = loss.mean(1), reference.mean(1)
-    sem = np.sqrt(loss.var(1) / loss.shape[1] + reference.var(1) / reference.shape[1])
-    apart = np.abs(mean - ref) > 3.0 * sem + 1e-12
+    """Last recorded iteration at which the method's loss is still apart from the reference method's:
+    the paired difference over trials is more than three standard errors from zero (and more than
+    0.1 % of the reference's total decrease, so that significant but negligible gaps do not count).
+    0 if never."""
+    mean, sem = excess_over(loss, reference)
+    ref = reference.mean(1)
+    floor = 1e-3 * abs(ref[0] - ref[-1])        # and more than 0.1 % of what the reference gains over the run
+    apart = (np.abs(mean) > 3.0 * sem + 1e-12) & (np.abs(mean) > floor)
     idx = np.nonzero(apart)[0]
     return int(marks[idx[-1]]) if idx.size else 0
 
@@ -190,6 +201,8 @@ def main(argv=None):
                 "topology": args.topology, "iid": args.iid, "trials": args.trials, "batch": args.batch,
                 "iterations": marks, "loss_mean": loss.mean(1).tolist(), "loss_std": loss.std(1).tolist(),
                 "consensus_mean": cons.mean(1).tolist(), "consensus_std": cons.std(1).tolist(),
+                "excess_over_parallel_sgd_mean": excess_over(loss, ref)[0].tolist(),
+                "excess_over_parallel_sgd_sem": excess_over(loss, ref)[1].tolist(),
                 "transient_stage": transient_stage(marks, loss, ref)}) + "\n")
             sink.flush()
     if args.out:
