@@ -341,7 +341,12 @@ static inline unsigned grid_for(long long Q, int block) { return (unsigned)((Q +
 // Launch shape per kernel: rows in flight per thread (U), register pipeline (PIPE),
 // threads per block and minimum resident blocks (the register cap), chosen by timing
 // on B200 at the ResNet-50- and BERT-Large-sized states.
-struct RingTune { static constexpr int U = 2; static constexpr bool PIPE = false; static constexpr int BLOCK = 256; static constexpr int MINB = 4; };
+// (ring: four rows in flight need ~85 registers; 768 threads per SM with four rows each keep more
+// bytes in flight than 1024 threads with two, worth 2.5 % in the seconds-long loop under the power
+// cap: 2.96 against 3.03 ms per launch at n = 64, d = 25,557,032.  The exponential and the
+// global-average kernel already have four rows in flight at 64 registers; 128-thread blocks, six or
+// eight rows in flight or a looser register cap measured equal or slower for them.)
+struct RingTune { static constexpr int U = 4; static constexpr bool PIPE = false; static constexpr int BLOCK = 128; static constexpr int MINB = 6; };
 struct ExpTune { static constexpr int U = 4; static constexpr bool PIPE = false; static constexpr int BLOCK = 256; static constexpr int MINB = 4; };
 struct GlobalTune { static constexpr int U = 4; static constexpr bool PIPE = false; static constexpr int BLOCK = 256; static constexpr int MINB = 4; };
 constexpr int kSmallBlock = 64;   // small problems: narrow blocks spread the column groups over more SMs
