@@ -303,7 +303,9 @@ int32_t gpga_set_node_shard(gpga_t* ctx, int64_t shards, int64_t shard);
 int64_t gpga_shard_exchange_bytes(const gpga_t* ctx);
 
 /* First half of iteration k on this shard: writes the outgoing messages (gpga_shard_plan's
- * send_offset / bytes, or the column sums) to send_dev.  Asynchronous on `stream`. */
+ * send_offset / bytes, or the column sums) to send_dev.  Asynchronous on `stream`.  Leave the send
+ * buffer as it is until gpga_shard_step of the same iteration has run: when every local row was
+ * exported (a hop of at least n nodes) the step takes the half-step rows from there. */
 int32_t gpga_shard_export(gpga_t* ctx, int64_t k, void* send_dev, void* stream);
 
 /* Second half: Algorithm 1's update and mix for the local rows, with recv_dev holding the received

@@ -32,6 +32,8 @@ struct gpga_ctx {
     int64_t col0 = 0;
     int64_t ld = 0;   // row stride of X and b in floats
     int64_t shards = 1, shard = 0;   // node sharding: this handle holds nodes shard * n .. (shard + 1) * n - 1
+    const void* exported = nullptr;  // send buffer of the last gpga_shard_export and its iteration
+    int64_t exported_k = -1;
     float* x[2] = {nullptr, nullptr};
     float* data = nullptr;
     const float* labels = nullptr;
@@ -873,6 +875,8 @@ int32_t gpga_shard_export(gpga_t* c, int64_t k, void* send_dev, void* stream)
     }
     c->launches += 1;
     if (e != cudaSuccess) return cuda_fail(c, e, "shard export launch");
+    c->exported = send_dev;
+    c->exported_k = k;
     return GPGA_OK;
 }
 
@@ -892,9 +896,14 @@ int32_t gpga_shard_step(gpga_t* c, int64_t k, const void* recv_dev, void* stream
     } else {
         const int tau = log2_floor(p.n_total);
         const int64_t hop = tau > 0 ? (int64_t(1) << (k % tau)) : 1;
-        e = launch_shard_exp(p, vec, static_cast<const float*>(recv_dev), (int)(hop < c->n ? hop : c->n), s);
+        if (hop >= c->n && c->exported && c->exported_k == k)   // every row was exported: take the half-steps from there
+            e = launch_shard_exp_exported(p, vec, static_cast<const float*>(c->exported),
+                                          static_cast<const float*>(recv_dev), s);
+        else
+            e = launch_shard_exp(p, vec, static_cast<const float*>(recv_dev), (int)(hop < c->n ? hop : c->n), s);
     }
     c->launches += 1;
+    c->exported_k = -1;
     if (e != cudaSuccess) return cuda_fail(c, e, "shard step launch");
     c->cur ^= 1;
     c->k = k + 1;

@@ -40,16 +40,35 @@ __device__ __forceinline__ Group group_of(const ShardParams& p, long long q)
     return g;
 }
 
-// Half-step value of local row i for one column group (Algorithm 1: gradient, local update).
+// One local row's inputs for one column group, and the half-step formed from them (Algorithm 1:
+// gradient, local update).  Loading and finishing are split so that a thread can issue the loads of
+// several rows before it stores anything: the output may alias the input (in-place update), so the
+// compiler cannot move a load above a store by itself.
+struct RowIn {
+    float4 x, b;
+};
+template <bool VEC>
+__device__ __forceinline__ RowIn load_row(const ShardParams& p, const Group& g, int i)
+{
+    RowIn r;
+    r.x = load4<VEC>(p.x + (long long)i * p.ld, g.j0, p.d);
+    r.b = load4<VEC>(p.b + (long long)i * p.ld, g.j0, p.d);
+    return r;
+}
+template <bool NOISE>
+__device__ __forceinline__ float4 finish_row(const ShardParams& p, const Group& g, const RowIn& r, int i)
+{
+    float4 gr = sub4(r.x, r.b);
+    if (NOISE) gr = fma4(p.sigma, normal4(g.qg, (uint32_t)(p.row0 + i), p.k, 0u, p.keys), gr);
+    return fma4(-p.gamma, gr, r.x);
+}
 template <bool NOISE, bool VEC>
 __device__ __forceinline__ float4 half_step_row(const ShardParams& p, const Group& g, int i)
 {
-    const float4 x = load4<VEC>(p.x + (long long)i * p.ld, g.j0, p.d);
-    const float4 b = load4<VEC>(p.b + (long long)i * p.ld, g.j0, p.d);
-    float4 gr = sub4(x, b);
-    if (NOISE) gr = fma4(p.sigma, normal4(g.qg, (uint32_t)(p.row0 + i), p.k, 0u, p.keys), gr);
-    return fma4(-p.gamma, gr, x);
+    return finish_row<NOISE>(p, g, load_row<VEC>(p, g, i), i);
 }
+
+constexpr int kRowsInFlight = 4;
 
 template <bool VEC>
 __device__ __forceinline__ float4 load_dense(const float* buf, long long row, const ShardParams& p, const Group& g)
@@ -84,7 +103,16 @@ __global__ void __launch_bounds__(kShardBlock) shard_export_rows_kernel(const Sh
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (q >= p.Q) return;
     const Group g = group_of(p, q);
-    for (int t = 0; t < rows; ++t) store_dense(send, t, p, g, half_step_row<NOISE, VEC>(p, g, first + t * stride));
+    int t = 0;
+    for (; t + kRowsInFlight <= rows; t += kRowsInFlight) {
+        RowIn r[kRowsInFlight];
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) r[u] = load_row<VEC>(p, g, first + (t + u) * stride);
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u)
+            store_dense(send, t + u, p, g, finish_row<NOISE>(p, g, r[u], first + (t + u) * stride));
+    }
+    for (; t < rows; ++t) store_dense(send, t, p, g, half_step_row<NOISE, VEC>(p, g, first + t * stride));
 }
 
 // Column sums of the half-step over the local rows, as the global-average kernel forms them:
@@ -99,8 +127,11 @@ __global__ void __launch_bounds__(kShardBlock) shard_export_sums_kernel(const Sh
     const int n = (int)p.n;
     int i = 0;
     for (; i + 4 <= n; i += 4) {
-        const float4 y0 = half_step_row<NOISE, VEC>(p, g, i), y1 = half_step_row<NOISE, VEC>(p, g, i + 1);
-        const float4 y2 = half_step_row<NOISE, VEC>(p, g, i + 2), y3 = half_step_row<NOISE, VEC>(p, g, i + 3);
+        RowIn r[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) r[u] = load_row<VEC>(p, g, i + u);
+        const float4 y0 = finish_row<NOISE>(p, g, r[0], i), y1 = finish_row<NOISE>(p, g, r[1], i + 1);
+        const float4 y2 = finish_row<NOISE>(p, g, r[2], i + 2), y3 = finish_row<NOISE>(p, g, r[3], i + 3);
         const float4 t = add4(add4(y0, y1), add4(y2, y3));
         s0 += (double)t.x; s1 += (double)t.y; s2 += (double)t.z; s3 += (double)t.w;
     }
@@ -120,47 +151,106 @@ __global__ void __launch_bounds__(kShardBlock) shard_export_sums_kernel(const Sh
 
 // ---- step --------------------------------------------------------------------------------------
 // Ring: recv[0] = half-step of the node above local row 0, recv[1] = of the node below the last.
+// A three-row window slides down the local rows, four rows' loads in flight.
 template <bool NOISE, bool VEC>
-__global__ void __launch_bounds__(kShardBlock, 4) shard_ring_kernel(const ShardParams p, const float* __restrict__ recv)
+__global__ void __launch_bounds__(kShardBlock, 3) shard_ring_kernel(const ShardParams p, const float* __restrict__ recv)
 {
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (q >= p.Q) return;
     const Group g = group_of(p, q);
     const int n = (int)p.n;
     float4 a = load_dense<VEC>(recv, 0, p, g);
+    const float4 below = load_dense<VEC>(recv, 1, p, g);
     float4 b = half_step_row<NOISE, VEC>(p, g, 0);
-#pragma unroll 4
-    for (int i = 1; i < n; ++i) {
+    int i = 1;
+    for (; i + kRowsInFlight <= n; i += kRowsInFlight) {
+        RowIn r[kRowsInFlight];
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) r[u] = load_row<VEC>(p, g, i + u);
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) {
+            const float4 v = finish_row<NOISE>(p, g, r[u], i + u);
+            store_out<VEC>(p, g, i + u - 1, mix3(a, b, v));
+            a = b;
+            b = v;
+        }
+    }
+    for (; i < n; ++i) {
         const float4 v = half_step_row<NOISE, VEC>(p, g, i);
         store_out<VEC>(p, g, i - 1, mix3(a, b, v));
         a = b;
         b = v;
     }
-    store_out<VEC>(p, g, n - 1, mix3(a, b, load_dense<VEC>(recv, 1, p, g)));
+    store_out<VEC>(p, g, n - 1, mix3(a, b, below));
 }
 
-// One-peer exponential graph with hop h: he = min(h, n_l) chains c, c + he, c + 2 he, ... of local
-// rows; a row's partner is the next row of its chain, the last row's partner is recv[c] (the
-// partner shard's row c).  Each local row is read, and its noise generated, once.
+// One-peer exponential graph with hop h: he = min(h, n_l) chains c, c + he, c + 2 he, ... of
+// L = n_l / he local rows (powers of two); a row's partner is the next row of its chain, the last
+// row's partner is recv[c] (the partner shard's row c).  The walk visits step t = c L + s (chain c,
+// position s) at row c + s he, four steps' loads in flight; each local row is read, and its noise
+// generated, once.
 template <bool NOISE, bool VEC>
-__global__ void __launch_bounds__(kShardBlock, 4) shard_exp_kernel(const ShardParams p, const float* __restrict__ recv,
-                                                                    int he)
+__global__ void __launch_bounds__(kShardBlock, 3) shard_exp_kernel(const ShardParams p, const float* __restrict__ recv,
+                                                                    int he_log2, int len_log2)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.Q) return;
+    const Group g = group_of(p, q);
+    const int n = (int)p.n, lmask = (1 << len_log2) - 1;
+    auto row_of = [=](int t) { return (t >> len_log2) + ((t & lmask) << he_log2); };
+    float4 prev = make_float4(0.f, 0.f, 0.f, 0.f);
+    int prev_row = 0;
+    auto visit = [&](int t, int row, float4 y) {
+        const int s = t & lmask;
+        if (s != 0) store_out<VEC>(p, g, prev_row, half(prev, y));
+        if (s == lmask) store_out<VEC>(p, g, row, half(y, load_dense<VEC>(recv, t >> len_log2, p, g)));
+        prev = y;
+        prev_row = row;
+    };
+    int t = 0;
+    for (; t + kRowsInFlight <= n; t += kRowsInFlight) {
+        RowIn r[kRowsInFlight];
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) r[u] = load_row<VEC>(p, g, row_of(t + u));
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) {
+            const int row = row_of(t + u);
+            visit(t + u, row, finish_row<NOISE>(p, g, r[u], row));
+        }
+    }
+    for (; t < n; ++t) {
+        const int row = row_of(t);
+        visit(t, row, half_step_row<NOISE, VEC>(p, g, row));
+    }
+}
+
+// The same when every local row's partner is remote (hop >= n_l) and the rows' half-steps are still in
+// the send buffer the export wrote: x_i^(k+1) = (send[i] + recv[i]) / 2, 12 bytes per update.
+__global__ void __launch_bounds__(kShardBlock) shard_exp_exported_kernel(const ShardParams p, const float* __restrict__ own,
+                                                                          const float* __restrict__ recv, bool vec)
 {
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (q >= p.Q) return;
     const Group g = group_of(p, q);
     const int n = (int)p.n;
-    for (int c = 0; c < he; ++c) {
-        float4 prev = half_step_row<NOISE, VEC>(p, g, c);
-        int row = c;
-#pragma unroll 4
-        for (int nxt = c + he; nxt < n; nxt += he) {
-            const float4 y = half_step_row<NOISE, VEC>(p, g, nxt);
-            store_out<VEC>(p, g, row, half(prev, y));
-            prev = y;
-            row = nxt;
+    int i = 0;
+    for (; i + kRowsInFlight <= n; i += kRowsInFlight) {
+        float4 y[kRowsInFlight], z[kRowsInFlight];
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) {
+            y[u] = load_dense<true>(own, i + u, p, g);
+            z[u] = load_dense<true>(recv, i + u, p, g);
         }
-        store_out<VEC>(p, g, row, half(prev, load_dense<VEC>(recv, c, p, g)));
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) {
+            if (vec) store_out<true>(p, g, i + u, half(y[u], z[u]));
+            else store_out<false>(p, g, i + u, half(y[u], z[u]));
+        }
+    }
+    for (; i < n; ++i) {
+        const float4 v = half(load_dense<true>(own, i, p, g), load_dense<true>(recv, i, p, g));
+        if (vec) store_out<true>(p, g, i, v);
+        else store_out<false>(p, g, i, v);
     }
 }
 
@@ -224,7 +314,16 @@ cudaError_t launch_shard_ring(const ShardParams& p, bool vec, const float* recv,
 cudaError_t launch_shard_exp(const ShardParams& p, bool vec, const float* recv, int he, cudaStream_t s)
 {
     const bool noise = p.sigma != 0.f;
-    GPGA_SHARD_LAUNCH(shard_exp_kernel, noise, vec, p, recv, he);
+    int he_log2 = 0, len_log2 = 0;
+    while ((1 << (he_log2 + 1)) <= he) ++he_log2;
+    while (((long long)he << (len_log2 + 1)) <= p.n) ++len_log2;
+    GPGA_SHARD_LAUNCH(shard_exp_kernel, noise, vec, p, recv, he_log2, len_log2);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_shard_exp_exported(const ShardParams& p, bool vec, const float* own, const float* recv, cudaStream_t s)
+{
+    shard_exp_exported_kernel<<<grid_of(p.Q), kShardBlock, 0, s>>>(p, own, recv, vec);
     return cudaGetLastError();
 }
 

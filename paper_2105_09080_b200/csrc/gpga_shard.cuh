@@ -31,6 +31,8 @@ cudaError_t launch_shard_export_sums(const ShardParams& p, bool vec, double* sum
 cudaError_t launch_shard_ring(const ShardParams& p, bool vec, const float* recv, cudaStream_t s);
 // step: one-peer exponential graph, he = min(hop, local rows); recv = the partner shard's rows 0 .. he-1
 cudaError_t launch_shard_exp(const ShardParams& p, bool vec, const float* recv, int he, cudaStream_t s);
+// step: the same when hop >= local rows and `own` still holds this shard's exported half-step rows
+cudaError_t launch_shard_exp_exported(const ShardParams& p, bool vec, const float* own, const float* recv, cudaStream_t s);
 // step: global average from `parts` vectors of column sums in shard order
 cudaError_t launch_shard_global(const ShardParams& p, bool vec, const double* recv, int parts, cudaStream_t s);
 
