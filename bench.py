@@ -102,13 +102,14 @@ class ClockSampler(threading.Thread):
     """Samples SM clock and clock-event reasons through NVML (read-only) while a timed region runs.
     One thread for the whole run; `begin()` opens a section, `end()` closes it and returns its summary."""
 
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.005):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._halt = threading.Event()
         self.active = threading.Event()
         self.ready = threading.Event()
+        self.once = threading.Event()      # one more sample, asked for by end() when a region was too short for any
         self.error = None
 
     def run(self):
@@ -127,14 +128,15 @@ class ClockSampler(threading.Thread):
                 nv.nvmlDeviceGetCurrentClocksThrottleReasons
             self.ready.set()
             while not self._halt.is_set():
-                if self.active.is_set():
+                if self.active.is_set() or self.once.is_set():
                     mhz = nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)
                     mask = get_reasons(h)
-                    if self.active.is_set():
+                    if self.active.is_set() or self.once.is_set():
                         self.samples.append(mhz)
                         for bit, nm in names.items():
                             if mask & bit and bit.bit_count() == 1:
                                 self.reasons.add(nm)
+                    self.once.clear()
                 time.sleep(self.period)
             nv.nvmlShutdown()
         except Exception as exc:          # NVML missing: report it, do not fail the run
@@ -150,6 +152,12 @@ class ClockSampler(threading.Thread):
 
     def end(self):
         self.active.clear()
+        if not self.samples and self.is_alive() and not self.error:
+            # the region ended before the first sample: take one now, the work has only just drained
+            self.once.set()
+            t0 = time.time()
+            while self.once.is_set() and time.time() - t0 < 0.5:
+                time.sleep(0.001)
         s = sorted(self.samples)
         return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
                 "reasons": sorted(r for r in self.reasons if r not in ("GpuIdle", "None")),
