@@ -140,3 +140,47 @@ def test_one_process_delivery_matches_the_plan():
         got = np.concatenate([sh.X for sh in parts])
         want = o.run(o.Problem(TOPOLOGY[topo][1], H, 0.2, 5, sigma=0.1, data=B), X0, 0, K)
         assert np.abs(got - want).max() <= 2e-6 * (1 + np.abs(want).max()), (topo, H)
+
+
+def test_plan_is_consistent_for_every_shape():
+    """Host logic only, exhaustively over small shapes: every message a shard sends is one its
+    destination expects (same size, landing where the destination reads it), and the rows a shard
+    receives are the rows its local nodes' neighbours live in."""
+    row = lambda d: (d + 3) // 4 * 16
+    for d in (8, 10):
+        for n in (4, 8, 16, 32, 64):
+            for shards in (1, 2, 4, 8, 16):
+                if n % shards or (n // shards) % 4 and shards > 1:
+                    continue
+                n_l = n // shards
+                for k in range(0, 14):
+                    plans = [ns.shard_plan(pkg.GPGA_TOPO_EXP, 0, n, shards, g, d, k) for g in range(shards)]
+                    hop = plans[0].hop
+                    assert hop == 1 << (k % max(1, n.bit_length() - 1))
+                    he = min(hop, n_l)
+                    for g, p in enumerate(plans):
+                        assert (p.kind, p.messages, p.bytes[0]) == (ns.GPGA_SHARD_EXP, 1, he * row(d))
+                        src = p.recv_from[0]
+                        assert plans[src].send_to[0] == g and plans[src].bytes[0] == p.bytes[0]
+                        # local node i = n_l - he + c (the last he rows) has its partner (i + hop) mod n at row c of `src`
+                        for c in range(he):
+                            partner = (g * n_l + n_l - he + c + hop) % n
+                            assert partner == src * n_l + c, (n, shards, k, g, c)
+                        # and every other local node's partner is local
+                        for i in range(n_l - he):
+                            assert g * n_l <= (g * n_l + i + hop) % n < (g + 1) * n_l
+        for n, shards in ((8, 1), (8, 2), (12, 3), (64, 4), (64, 16), (20, 5)):
+            n_l = n // shards
+            plans = [ns.shard_plan(pkg.GPGA_TOPO_RING, 4, n, shards, g, d, 0) for g in range(shards)]
+            for g, p in enumerate(plans):
+                assert (p.kind, p.messages) == (ns.GPGA_SHARD_RING, 2)
+                assert p.recv_from[0] == (g - 1) % shards and p.recv_from[1] == (g + 1) % shards
+                for m in (0, 1):
+                    dst = plans[p.send_to[m]]
+                    assert dst.recv_from[1 - m] == g                      # my first row is my upper neighbour's "row below"
+                    assert p.dst_offset[m] == dst.recv_offset[1 - m] and p.bytes[m] == row(d)
+                # the row above local row 0 is the last row of shard g-1; the row below the last is row 0 of shard g+1
+                assert (g * n_l - 1) % n == ((g - 1) % shards) * n_l + n_l - 1
+                assert ((g + 1) * n_l) % n == ((g + 1) % shards) * n_l
+            glob = ns.shard_plan(pkg.GPGA_TOPO_RING, 4, n, shards, 0, d, 3)
+            assert glob.kind == ns.GPGA_SHARD_GLOBAL and glob.gather_bytes == (d + 3) // 4 * 4 * 8
