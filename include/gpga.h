@@ -313,6 +313,17 @@ int32_t gpga_shard_export(gpga_t* ctx, int64_t k, void* send_dev, void* stream);
  * flips them and sets the counter to k + 1, like gpga_step.  Asynchronous on `stream`. */
 int32_t gpga_shard_step(gpga_t* ctx, int64_t k, const void* recv_dev, void* stream);
 
+/* gpga_shard_step in two parts, so that the exchange overlaps the bulk of the arithmetic (double
+ * buffer only: x_a != x_b).  gpga_shard_step_interior writes the rows of X^(k+1) whose neighbours
+ * are all local -- ring: rows 1 .. n-2; exponential graph with hop h < n: rows 0 .. n-h-1; none for a
+ * global average or a hop of at least n nodes (then it launches nothing) -- and needs nothing
+ * received, so it can run while the messages of gpga_shard_export travel on another stream.
+ * gpga_shard_step_boundary then writes the remaining rows from recv_dev, flips the buffers and
+ * sets the counter to k + 1.  Together they give exactly gpga_shard_step's result.
+ * Errors: as gpga_shard_step; UNSUPPORTED for the in-place update. */
+int32_t gpga_shard_step_interior(gpga_t* ctx, int64_t k, void* stream);
+int32_t gpga_shard_step_boundary(gpga_t* ctx, int64_t k, const void* recv_dev, void* stream);
+
 /*
  * Self-test of the in-kernel wait limit (no counterpart in the paper): launches one block that
  * waits, a bounded number of polls, on a barrier that nothing will ever complete.  The wait must

@@ -61,6 +61,8 @@ SIGNATURES = {
     "gpga_shard_exchange_bytes": (_i64, [_P]),
     "gpga_shard_export": (_i32, [_P, _i64, _P, _P]),
     "gpga_shard_step": (_i32, [_P, _i64, _P, _P]),
+    "gpga_shard_step_interior": (_i32, [_P, _i64, _P]),
+    "gpga_shard_step_boundary": (_i32, [_P, _i64, _P, _P]),
     "gpga_run_adaptive": (_i32, [_P, _i64, _i64, _i64, _P, C.POINTER(_i64), _i64, C.POINTER(_i64)]),
     "gpga_get_x": (_i32, [_P, C.POINTER(_P)]),
     "gpga_get_k": (_i32, [_P, C.POINTER(_i64)]),

@@ -880,27 +880,46 @@ int32_t gpga_shard_export(gpga_t* c, int64_t k, void* send_dev, void* stream)
     return GPGA_OK;
 }
 
-int32_t gpga_shard_step(gpga_t* c, int64_t k, const void* recv_dev, void* stream)
+namespace {
+
+// Second half of a shard's iteration, whole or in two parts (see ShardPart).
+int32_t shard_step_part(gpga_ctx* c, int64_t k, const void* recv_dev, int part, cudaStream_t s)
 {
     int32_t st = shard_ready(c, k);
     if (st) return st;
-    if (!recv_dev || !aligned16(recv_dev)) return fail(c, GPGA_ERR_INVALID_ARG, "receive buffer must be a 16-byte aligned device pointer");
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (part != SHARD_INTERIOR && (!recv_dev || !aligned16(recv_dev)))
+        return fail(c, GPGA_ERR_INVALID_ARG, "receive buffer must be a 16-byte aligned device pointer");
+    if (part != SHARD_ALL && c->x[0] == c->x[1])
+        return fail(c, GPGA_ERR_UNSUPPORTED, "the two-part step needs the double buffer (x_a != x_b)");
     const ShardParams p = shard_params(c, k);
     const bool vec = vec_ok(c);
-    cudaError_t e;
-    if (is_global_step(k, c->H)) {
+    const int tau = log2_floor(p.n_total);
+    const int64_t hop = tau > 0 ? (int64_t(1) << (k % tau)) : 1;
+    const bool global = is_global_step(k, c->H);
+    const bool ring = c->topology == GPGA_TOPO_RING;
+    // rows that need nothing remote: ring 1 .. n - 2, exponential graph 0 .. n - hop - 1; none for a
+    // global average or a hop of at least n nodes
+    const bool has_interior = !global && (ring ? c->n >= 3 : hop < c->n);
+    cudaError_t e = cudaSuccess;
+    if (part == SHARD_INTERIOR) {
+        if (has_interior) {
+            e = ring ? launch_shard_ring(p, vec, nullptr, SHARD_INTERIOR, s)
+                     : launch_shard_exp(p, vec, nullptr, (int)hop, SHARD_INTERIOR, s);
+            c->launches += 1;
+        }
+        if (e != cudaSuccess) return cuda_fail(c, e, "shard step launch");
+        return GPGA_OK;   // the buffers flip when the boundary part has run
+    }
+    const int rest = (part == SHARD_BOUNDARY && has_interior) ? SHARD_BOUNDARY : SHARD_ALL;
+    if (global) {
         e = launch_shard_global(p, vec, static_cast<const double*>(recv_dev), (int)c->shards, s);
-    } else if (c->topology == GPGA_TOPO_RING) {
-        e = launch_shard_ring(p, vec, static_cast<const float*>(recv_dev), s);
+    } else if (ring) {
+        e = launch_shard_ring(p, vec, static_cast<const float*>(recv_dev), rest, s);
+    } else if (hop >= c->n && c->exported && c->exported_k == k) {   // every row was exported: take the half-steps from there
+        e = launch_shard_exp_exported(p, vec, static_cast<const float*>(c->exported),
+                                      static_cast<const float*>(recv_dev), s);
     } else {
-        const int tau = log2_floor(p.n_total);
-        const int64_t hop = tau > 0 ? (int64_t(1) << (k % tau)) : 1;
-        if (hop >= c->n && c->exported && c->exported_k == k)   // every row was exported: take the half-steps from there
-            e = launch_shard_exp_exported(p, vec, static_cast<const float*>(c->exported),
-                                          static_cast<const float*>(recv_dev), s);
-        else
-            e = launch_shard_exp(p, vec, static_cast<const float*>(recv_dev), (int)(hop < c->n ? hop : c->n), s);
+        e = launch_shard_exp(p, vec, static_cast<const float*>(recv_dev), (int)(hop < c->n ? hop : c->n), rest, s);
     }
     c->launches += 1;
     c->exported_k = -1;
@@ -908,6 +927,23 @@ int32_t gpga_shard_step(gpga_t* c, int64_t k, const void* recv_dev, void* stream
     c->cur ^= 1;
     c->k = k + 1;
     return GPGA_OK;
+}
+
+}  // namespace
+
+int32_t gpga_shard_step(gpga_t* c, int64_t k, const void* recv_dev, void* stream)
+{
+    return shard_step_part(c, k, recv_dev, SHARD_ALL, static_cast<cudaStream_t>(stream));
+}
+
+int32_t gpga_shard_step_interior(gpga_t* c, int64_t k, void* stream)
+{
+    return shard_step_part(c, k, nullptr, SHARD_INTERIOR, static_cast<cudaStream_t>(stream));
+}
+
+int32_t gpga_shard_step_boundary(gpga_t* c, int64_t k, const void* recv_dev, void* stream)
+{
+    return shard_step_part(c, k, recv_dev, SHARD_BOUNDARY, static_cast<cudaStream_t>(stream));
 }
 
 int32_t gpga_run_adaptive(gpga_t* c, int64_t K, int64_t H_init, int64_t warmup_iters, void* stream,

@@ -152,15 +152,18 @@ __global__ void __launch_bounds__(kShardBlock) shard_export_sums_kernel(const Sh
 // ---- step --------------------------------------------------------------------------------------
 // Ring: recv[0] = half-step of the node above local row 0, recv[1] = of the node below the last.
 // A three-row window slides down the local rows, four rows' loads in flight.
+// interior = true: only the rows whose neighbours are both local (1 .. n - 2); recv is not read.
 template <bool NOISE, bool VEC>
-__global__ void __launch_bounds__(kShardBlock, 3) shard_ring_kernel(const ShardParams p, const float* __restrict__ recv)
+__global__ void __launch_bounds__(kShardBlock, 3) shard_ring_kernel(const ShardParams p, const float* __restrict__ recv,
+                                                                     bool interior)
 {
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (q >= p.Q) return;
     const Group g = group_of(p, q);
     const int n = (int)p.n;
-    float4 a = load_dense<VEC>(recv, 0, p, g);
-    const float4 below = load_dense<VEC>(recv, 1, p, g);
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 a = interior ? zero : load_dense<VEC>(recv, 0, p, g);
+    const float4 below = interior ? zero : load_dense<VEC>(recv, 1, p, g);
     float4 b = half_step_row<NOISE, VEC>(p, g, 0);
     int i = 1;
     for (; i + kRowsInFlight <= n; i += kRowsInFlight) {
@@ -170,18 +173,41 @@ __global__ void __launch_bounds__(kShardBlock, 3) shard_ring_kernel(const ShardP
 #pragma unroll
         for (int u = 0; u < kRowsInFlight; ++u) {
             const float4 v = finish_row<NOISE>(p, g, r[u], i + u);
-            store_out<VEC>(p, g, i + u - 1, mix3(a, b, v));
+            if (!interior || i + u > 1) store_out<VEC>(p, g, i + u - 1, mix3(a, b, v));
             a = b;
             b = v;
         }
     }
     for (; i < n; ++i) {
         const float4 v = half_step_row<NOISE, VEC>(p, g, i);
-        store_out<VEC>(p, g, i - 1, mix3(a, b, v));
+        if (!interior || i > 1) store_out<VEC>(p, g, i - 1, mix3(a, b, v));
         a = b;
         b = v;
     }
-    store_out<VEC>(p, g, n - 1, mix3(a, b, below));
+    if (!interior) store_out<VEC>(p, g, n - 1, mix3(a, b, below));
+}
+
+// The two rows of a ring shard that have a remote neighbour: row 0 (the node above it is recv[0])
+// and row n - 1 (the node below it is recv[1]); reads local rows 0, 1, n - 2, n - 1.
+template <bool NOISE, bool VEC>
+__global__ void __launch_bounds__(kShardBlock) shard_ring_boundary_kernel(const ShardParams p, const float* __restrict__ recv)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.Q) return;
+    const Group g = group_of(p, q);
+    const int n = (int)p.n;
+    const float4 above = load_dense<VEC>(recv, 0, p, g), below = load_dense<VEC>(recv, 1, p, g);
+    const RowIn r0 = load_row<VEC>(p, g, 0), r1 = load_row<VEC>(p, g, n > 1 ? 1 : 0);
+    const RowIn r2 = load_row<VEC>(p, g, n > 1 ? n - 2 : 0), r3 = load_row<VEC>(p, g, n - 1);
+    const float4 y0 = finish_row<NOISE>(p, g, r0, 0);
+    if (n == 1) {
+        store_out<VEC>(p, g, 0, mix3(above, y0, below));
+        return;
+    }
+    const float4 y1 = finish_row<NOISE>(p, g, r1, 1);
+    const float4 yl2 = finish_row<NOISE>(p, g, r2, n - 2), yl1 = finish_row<NOISE>(p, g, r3, n - 1);
+    store_out<VEC>(p, g, 0, mix3(above, y0, y1));
+    store_out<VEC>(p, g, n - 1, mix3(yl2, yl1, below));
 }
 
 // One-peer exponential graph with hop h: he = min(h, n_l) chains c, c + he, c + 2 he, ... of
@@ -191,7 +217,7 @@ __global__ void __launch_bounds__(kShardBlock, 3) shard_ring_kernel(const ShardP
 // generated, once.
 template <bool NOISE, bool VEC>
 __global__ void __launch_bounds__(kShardBlock, 3) shard_exp_kernel(const ShardParams p, const float* __restrict__ recv,
-                                                                    int he_log2, int len_log2)
+                                                                    int he_log2, int len_log2, bool interior)
 {
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (q >= p.Q) return;
@@ -203,7 +229,7 @@ __global__ void __launch_bounds__(kShardBlock, 3) shard_exp_kernel(const ShardPa
     auto visit = [&](int t, int row, float4 y) {
         const int s = t & lmask;
         if (s != 0) store_out<VEC>(p, g, prev_row, half(prev, y));
-        if (s == lmask) store_out<VEC>(p, g, row, half(y, load_dense<VEC>(recv, t >> len_log2, p, g)));
+        if (s == lmask && !interior) store_out<VEC>(p, g, row, half(y, load_dense<VEC>(recv, t >> len_log2, p, g)));
         prev = y;
         prev_row = row;
     };
@@ -222,6 +248,32 @@ __global__ void __launch_bounds__(kShardBlock, 3) shard_exp_kernel(const ShardPa
         const int row = row_of(t);
         visit(t, row, half_step_row<NOISE, VEC>(p, g, row));
     }
+}
+
+// The last he local rows of the exponential graph's shard, whose partners are recv[0 .. he - 1].
+template <bool NOISE, bool VEC>
+__global__ void __launch_bounds__(kShardBlock) shard_exp_boundary_kernel(const ShardParams p, const float* __restrict__ recv,
+                                                                          int he)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.Q) return;
+    const Group g = group_of(p, q);
+    const int first = (int)p.n - he;
+    int c = 0;
+    for (; c + kRowsInFlight <= he; c += kRowsInFlight) {
+        RowIn r[kRowsInFlight];
+        float4 z[kRowsInFlight];
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) {
+            r[u] = load_row<VEC>(p, g, first + c + u);
+            z[u] = load_dense<VEC>(recv, c + u, p, g);
+        }
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u)
+            store_out<VEC>(p, g, first + c + u, half(finish_row<NOISE>(p, g, r[u], first + c + u), z[u]));
+    }
+    for (; c < he; ++c)
+        store_out<VEC>(p, g, first + c, half(half_step_row<NOISE, VEC>(p, g, first + c), load_dense<VEC>(recv, c, p, g)));
 }
 
 // The same when every local row's partner is remote (hop >= n_l) and the rows' half-steps are still in
@@ -304,20 +356,27 @@ cudaError_t launch_shard_export_sums(const ShardParams& p, bool vec, double* sum
     return cudaGetLastError();
 }
 
-cudaError_t launch_shard_ring(const ShardParams& p, bool vec, const float* recv, cudaStream_t s)
+cudaError_t launch_shard_ring(const ShardParams& p, bool vec, const float* recv, int part, cudaStream_t s)
 {
     const bool noise = p.sigma != 0.f;
-    GPGA_SHARD_LAUNCH(shard_ring_kernel, noise, vec, p, recv);
+    if (part == SHARD_BOUNDARY)
+        GPGA_SHARD_LAUNCH(shard_ring_boundary_kernel, noise, vec, p, recv);
+    else
+        GPGA_SHARD_LAUNCH(shard_ring_kernel, noise, vec, p, recv, part == SHARD_INTERIOR);
     return cudaGetLastError();
 }
 
-cudaError_t launch_shard_exp(const ShardParams& p, bool vec, const float* recv, int he, cudaStream_t s)
+cudaError_t launch_shard_exp(const ShardParams& p, bool vec, const float* recv, int he, int part, cudaStream_t s)
 {
     const bool noise = p.sigma != 0.f;
+    if (part == SHARD_BOUNDARY) {
+        GPGA_SHARD_LAUNCH(shard_exp_boundary_kernel, noise, vec, p, recv, he);
+        return cudaGetLastError();
+    }
     int he_log2 = 0, len_log2 = 0;
     while ((1 << (he_log2 + 1)) <= he) ++he_log2;
     while (((long long)he << (len_log2 + 1)) <= p.n) ++len_log2;
-    GPGA_SHARD_LAUNCH(shard_exp_kernel, noise, vec, p, recv, he_log2, len_log2);
+    GPGA_SHARD_LAUNCH(shard_exp_kernel, noise, vec, p, recv, he_log2, len_log2, part == SHARD_INTERIOR);
     return cudaGetLastError();
 }
 

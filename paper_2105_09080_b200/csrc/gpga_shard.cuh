@@ -27,10 +27,13 @@ cudaError_t launch_shard_export_rows(const ShardParams& p, bool vec, float* send
                                      cudaStream_t s);
 // export: the shard's column sums of the half-step (4 Q doubles)
 cudaError_t launch_shard_export_sums(const ShardParams& p, bool vec, double* sums, cudaStream_t s);
+// Which rows a gossip step kernel writes: all of them, only those whose neighbours are all local
+// (so that they can be formed while the messages are still travelling), or only the others.
+enum ShardPart { SHARD_ALL = 0, SHARD_INTERIOR = 1, SHARD_BOUNDARY = 2 };
 // step: ring with recv = [row above local row 0 | row below the last local row]
-cudaError_t launch_shard_ring(const ShardParams& p, bool vec, const float* recv, cudaStream_t s);
+cudaError_t launch_shard_ring(const ShardParams& p, bool vec, const float* recv, int part, cudaStream_t s);
 // step: one-peer exponential graph, he = min(hop, local rows); recv = the partner shard's rows 0 .. he-1
-cudaError_t launch_shard_exp(const ShardParams& p, bool vec, const float* recv, int he, cudaStream_t s);
+cudaError_t launch_shard_exp(const ShardParams& p, bool vec, const float* recv, int he, int part, cudaStream_t s);
 // step: the same when hop >= local rows and `own` still holds this shard's exported half-step rows
 cudaError_t launch_shard_exp_exported(const ShardParams& p, bool vec, const float* own, const float* recv, cudaStream_t s);
 // step: global average from `parts` vectors of column sums in shard order

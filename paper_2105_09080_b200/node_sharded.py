@@ -66,6 +66,14 @@ class NodeShard:
     def step(self, k, stream=None):
         self.g._check(B.lib().gpga_shard_step(self.g._h, k, self.recv.data_ptr(), self.g._sp(stream)))
 
+    def step_interior(self, k, stream=None):
+        """The rows of X^(k+1) that need nothing received (can run while the messages travel)."""
+        self.g._check(B.lib().gpga_shard_step_interior(self.g._h, k, self.g._sp(stream)))
+
+    def step_boundary(self, k, stream=None):
+        """The remaining rows, from the receive buffer; completes iteration k."""
+        self.g._check(B.lib().gpga_shard_step_boundary(self.g._h, k, self.recv.data_ptr(), self.g._sp(stream)))
+
     def get_x(self):
         return self.g.get_x()
 
@@ -127,3 +135,23 @@ def run_dist(shard, K, k0=0, group=None):
         shard.export(k)
         exchange_dist(shard, k, group)
         shard.step(k)
+
+
+def run_dist_overlapped(shard, K, k0=0, group=None):
+    """The same with the exchange on a stream of its own, overlapped with the rows that need nothing
+    received: export -> [exchange on the side stream | interior rows on the main stream] -> boundary
+    rows.  CUDA shards on the double buffer only."""
+    import torch
+    main = torch.cuda.current_stream()
+    side = torch.cuda.Stream()
+    exported, delivered = torch.cuda.Event(), torch.cuda.Event()
+    for k in range(k0, k0 + K):
+        shard.export(k)
+        exported.record(main)
+        with torch.cuda.stream(side):
+            side.wait_event(exported)
+            exchange_dist(shard, k, group)
+            delivered.record(side)
+        shard.step_interior(k)
+        main.wait_event(delivered)
+        shard.step_boundary(k)

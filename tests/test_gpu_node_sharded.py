@@ -18,7 +18,7 @@ pytestmark = pytest.mark.gpu
 SEED = 20210509
 
 
-def _sharded_run(n, d, topo, H, gamma, sigma, X0, B, shards, K, col0=0, check_first=None):
+def _sharded_run(n, d, topo, H, gamma, sigma, X0, B, shards, K, col0=0, check_first=None, mode="whole"):
     import torch
     n_l = n // shards
     parts = []
@@ -31,9 +31,21 @@ def _sharded_run(n, d, topo, H, gamma, sigma, X0, B, shards, K, col0=0, check_fi
     for k in range(K):
         for sh in parts:
             sh.export(k)
-        ns.exchange_local(parts, k)
-        for sh in parts:
-            sh.step(k)
+        if mode == "whole":
+            ns.exchange_local(parts, k)
+            for sh in parts:
+                sh.step(k)
+        else:
+            # the step in two parts; "early": the rows that need nothing received are formed BEFORE the
+            # messages are delivered (they must not depend on them)
+            if mode == "split":
+                ns.exchange_local(parts, k)
+            for sh in parts:
+                sh.step_interior(k)
+            if mode == "early":
+                ns.exchange_local(parts, k)
+            for sh in parts:
+                sh.step_boundary(k)
         if check_first is not None and k == 0:
             check_first(np.concatenate([sh.get_x().cpu().numpy() for sh in parts]))
     out = np.concatenate([sh.get_x().cpu().numpy() for sh in parts])
@@ -71,6 +83,25 @@ def test_sharded_run_is_bit_identical_to_the_unsharded_run(topo, H, n, shards, d
     assert ok, worst
     if H and K % H == 0:
         assert np.all(got == got[0])
+    g.close()
+
+
+@pytest.mark.parametrize("mode", ["split", "early"])
+@pytest.mark.parametrize("topo,H,n,shards,d", [("ring", 4, 16, 2, 4104), ("ring", 0, 16, 4, 1031), ("ring", 3, 8, 1, 4104),
+                                               ("ring", 5, 8, 2, 64), ("exp", 3, 16, 2, 4104), ("exp", 0, 32, 4, 1031),
+                                               ("exp", 5, 8, 1, 19456), ("exp", 0, 8, 2, 64)])
+def test_two_part_step_equals_the_whole_step(topo, H, n, shards, d, mode):
+    """gpga_shard_step_interior + gpga_shard_step_boundary (the form that lets the exchange overlap
+    the arithmetic) against the unsharded run, bit for bit; in the "early" order the interior rows are
+    formed while the receive buffers still hold the previous iteration's messages."""
+    gamma, sigma, K = 0.1, 0.3, 11
+    X0, B = quadratic_inputs(n, d, SEED + n + d + 1, x0="per_node")
+    g, _ = make_quadratic(n, d, topo, H, gamma, SEED, sigma, X0, B)
+    for k in range(K):
+        g.step(k)
+    want = g.get_x().cpu().numpy()
+    got = _sharded_run(n, d, topo, H, gamma, sigma, X0, B, shards, K, mode=mode)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), float(np.abs(got - want).max())
     g.close()
 
 
@@ -112,3 +143,14 @@ def test_plan_and_argument_checks():
     with pytest.raises(pkg.GpgaError) as err:
         ns.NodeShard(12, 64, pkg.GPGA_TOPO_RING, 4, 0.1, 1, 2, 0)
     assert err.value.status == pkg.GPGA_ERR_UNSUPPORTED
+    # the two-part step needs the double buffer
+    import torch
+    sh = ns.NodeShard(8, 64, pkg.GPGA_TOPO_RING, 4, 0.1, 1, 2, 0)
+    x = torch.zeros((4, 64), device="cuda")
+    sh.bind(x, x, torch.zeros((4, 64), device="cuda"))
+    sh.export(0)
+    with pytest.raises(pkg.GpgaError) as err:
+        sh.step_interior(0)
+    assert err.value.status == pkg.GPGA_ERR_UNSUPPORTED
+    sh.step(0)                                              # the whole step works in place
+    sh.close()
