@@ -659,6 +659,63 @@ def run_logistic(args, w, name):
     print(json.dumps(line))
 
 
+def run_node_shard(args):
+    """--node-shards G: the two kernels of ONE shard of the node-sharded iteration (n / G consecutive
+    nodes, all d columns) timed per iteration: export, then step.  The exchange between shards is not
+    part of it (one GPU): the receive buffer keeps whatever it holds."""
+    import torch
+    import paper_2105_09080_b200 as pkg
+    from paper_2105_09080_b200 import node_sharded as ns
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    name = args.workload or FALLBACK_WORKLOAD
+    w = WORKLOADS[name]
+    G, n, d = args.node_shards, w["n"], w["d"]
+    n_l, ld = n // G, padded_stride(w["d"])
+    topo = {"ring": pkg.GPGA_TOPO_RING, "exp": pkg.GPGA_TOPO_EXP}[w["topo"]]
+    sh = ns.NodeShard(n, d, topo, w["H"], w["gamma"], SEED, G, min(1, G - 1), sigma=w["sigma"], ld=ld)
+    xa = torch.randn((n_l, ld), device="cuda") * 0.1
+    sh.bind(xa, torch.empty_like(xa), torch.randn((n_l, ld), device="cuda"))
+    steps = args.steps or 100
+    for k in range(args.warmup):
+        sh.export(k)
+        sh.step(k)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(physical_gpu_index(int(os.environ.get("LOCAL_RANK", "0"))))
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * steps + 1)]
+    kinds = []
+    sampler.begin()
+    ev[0].record()
+    for s_ in range(steps):
+        k = args.warmup + s_
+        plan = sh.plan(k)
+        kinds.append("global" if plan.kind == ns.GPGA_SHARD_GLOBAL else
+                     (f"exp_hop{plan.hop}" if plan.kind == ns.GPGA_SHARD_EXP else "ring"))
+        sh.export(k)
+        ev[2 * s_ + 1].record()
+        sh.step(k)
+        ev[2 * s_ + 2].record()
+    torch.cuda.synchronize()
+    clocks = sampler.end()
+    sampler.finish()
+    per = {}
+    for s_, kind in enumerate(kinds):
+        per.setdefault(kind, []).append((ev[2 * s_].elapsed_time(ev[2 * s_ + 1]), ev[2 * s_ + 1].elapsed_time(ev[2 * s_ + 2])))
+    table = {kind: {"iterations": len(v), "export_ms": median([a for a, _ in v]), "step_ms": median([b for _, b in v]),
+                    "GB/s_at_12_bytes_per_update": BYTES_PER_UPDATE * n_l * d / (median([a + b for a, b in v]) * 1e-3) / 1e9}
+             for kind, v in per.items()}
+    total_ms = ev[0].elapsed_time(ev[-1])
+    print(json.dumps({"metric": METRIC, "value": n_l * d * steps / (total_ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+                      "steps": steps, "warmup": args.warmup, "ms_per_step": total_ms / steps, "higher_is_better": True,
+                      "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": f"{name}: shard {min(1, G - 1)} of {G} ({n_l} of n={n} nodes x d={d} fp32, "
+                                             f"{w['topo']} topology, H={w['H'] or 'inf'}), export + step kernels of the "
+                                             f"node-sharded iteration; the exchange between shards is not timed"},
+                      "per_kind": table, "clocks": clocks, "gpu_launches": sh.g.launch_count()}), flush=True)
+    sh.close()
+
+
 def host_memory_available():
     try:
         for ln in open("/proc/meminfo"):
@@ -800,6 +857,8 @@ def main(argv=None):
     ap.add_argument("--sustained-seconds", type=float, default=2.0)
     ap.add_argument("--cell-seconds", type=float, default=1.0)
     ap.add_argument("--dry-run", action="store_true", help="multi-rank plumbing only, on CPU with gloo")
+    ap.add_argument("--node-shards", type=int, default=0,
+                    help="time the export + step kernels of one shard of a node-sharded run with this many shards")
     args = ap.parse_args(argv)
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
@@ -808,6 +867,8 @@ def main(argv=None):
         sys.exit(spawn_ranks(args.gpus, argv))       # one process per GPU; rank 0 prints the line
     if args.dry_run:
         return run_dry(args)
+    if args.node_shards:
+        return run_node_shard(args)
     if args.impl == "reference":
         if int(os.environ.get("RANK", "0")) != 0:
             return                                    # rank 0 alone runs the oracle
