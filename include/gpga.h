@@ -199,7 +199,8 @@ int32_t gpga_run(gpga_t* ctx, int64_t K, void* stream);
  * Same as gpga_run with HOST buffers (quadratic objective): copies x0_host and data_host
  * (dense n*d fp32 each) into the bound device buffers (row stride ld), resets the counter to 0, runs K
  * iterations, copies X^(K) to x_out_host and returns when all of that is done.  Host buffers
- * should be pinned for full copy speed.
+ * should be pinned for full copy speed.  x0_host may be NULL: X^(0) = 0 on every node (Algorithm 1
+ * asks for equal initial rows; zero is the common choice), filled on the device, nothing uploaded.
  * Columns of X evolve independently (W mixes rows; gradient and noise are element-wise and keyed by
  * the absolute column), so a state above 64 MB with d % 4 == 0 moves through the call as column
  * chunks (a sixteenth of a buffer, between 16 and 128 MB): the upload of one chunk, the K iterations of the one before

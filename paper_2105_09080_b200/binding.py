@@ -223,8 +223,10 @@ class Gpga:
         self._check(lib().gpga_run(self._h, K, self._sp(stream)))
 
     def run_host(self, x0_host, data_host, K, x_out_host, stream=None):
-        """x0_host, data_host, x_out_host: CPU float32 torch tensors (pinned for speed)."""
-        self._check(lib().gpga_run_host(self._h, x0_host.data_ptr(), data_host.data_ptr(), K,
+        """x0_host, data_host, x_out_host: CPU float32 torch tensors (pinned for speed); x0_host may be
+        None for X^(0) = 0."""
+        self._check(lib().gpga_run_host(self._h, x0_host.data_ptr() if x0_host is not None else None,
+                                        data_host.data_ptr(), K,
                                         x_out_host.data_ptr(), self._sp(stream)))
 
     def consensus_distance(self, stream=None) -> float:

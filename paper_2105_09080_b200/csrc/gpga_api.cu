@@ -574,7 +574,7 @@ int32_t gpga_run_host(gpga_t* c, const float* x0_host, const float* data_host, i
     int32_t st = check_ready(c);
     if (st) return st;
     if (c->objective != GPGA_OBJ_QUADRATIC) return fail(c, GPGA_ERR_UNSUPPORTED, "host entry is for the quadratic objective");
-    if (!x0_host || !data_host || !x_out_host) return fail(c, GPGA_ERR_INVALID_ARG, "NULL host buffer");
+    if (!data_host || !x_out_host) return fail(c, GPGA_ERR_INVALID_ARG, "NULL host buffer");
     if (K < 0) return fail(c, GPGA_ERR_INVALID_ARG, "K must be >= 0");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t host_pitch = (size_t)c->d * sizeof(float), pitch = (size_t)c->ld * sizeof(float);
@@ -609,7 +609,10 @@ int32_t gpga_run_host(gpga_t* c, const float* x0_host, const float* data_host, i
         const int64_t j0 = ch * width;
         const int64_t w = (d_full - j0 < width) ? d_full - j0 : width;
         const size_t wb = (size_t)w * sizeof(float);
-        e = cudaMemcpy2DAsync(x0_full + j0, pitch, x0_host + j0, host_pitch, wb, (size_t)c->n, cudaMemcpyHostToDevice, c->up);
+        if (x0_host)
+            e = cudaMemcpy2DAsync(x0_full + j0, pitch, x0_host + j0, host_pitch, wb, (size_t)c->n, cudaMemcpyHostToDevice, c->up);
+        else   // X^(0) = 0 on every node: nothing to upload (all-zero bits are 0.0f)
+            e = cudaMemset2DAsync(x0_full + j0, pitch, 0, wb, (size_t)c->n, c->up);
         if (e == cudaSuccess)
             e = cudaMemcpy2DAsync(data_full + j0, pitch, data_host + j0, host_pitch, wb, (size_t)c->n, cudaMemcpyHostToDevice, c->up);
         if (e == cudaSuccess) e = cudaEventRecord(ev[1 + 2 * ch], c->up);

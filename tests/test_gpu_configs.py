@@ -109,6 +109,32 @@ def test_run_host_equals_device_run():
     out = torch.empty((n, d), dtype=torch.float32).pin_memory()
     g2.run_host(torch.from_numpy(X0).pin_memory(), torch.from_numpy(B).pin_memory(), K, out)
     assert np.array_equal(out.numpy(), dev)
+    # X0 = NULL means X^(0) = 0, filled on the device: the same run (X0 is zero here), whatever the
+    # device buffers held before
+    g2.x_bufs[0].fill_(7.0)
+    g2.x_bufs[1].fill_(-3.0)
+    out.fill_(float("nan"))
+    g2.run_host(None, torch.from_numpy(B).pin_memory(), K, out)
+    assert np.array_equal(out.numpy(), dev)
+
+
+def test_run_host_zero_start_through_the_chunked_pipeline():
+    """A state above 64 MB moves through the host entry as column chunks; with X0 = NULL every chunk
+    of X^(0) is zeroed on the device instead of uploaded.  Same result as the resident run from zeros."""
+    torch = _torch()
+    n, d, K = 8, 3_000_000, 5
+    B = np.random.default_rng(SEED).standard_normal((n, d), dtype=np.float32)
+    X0 = np.zeros((n, d), dtype=np.float32)
+    g, _ = make_quadratic(n, d, "exp", 3, 0.05, SEED, 0.1, X0, B)
+    g.run(K)
+    dev = g.get_x().cpu().numpy()
+    g.x_bufs[0].fill_(1.5)
+    g.x_bufs[1].fill_(2.5)
+    out = torch.full((n, d), float("nan"), dtype=torch.float32).pin_memory()
+    g.run_host(None, torch.from_numpy(B).pin_memory(), K, out)
+    assert np.array_equal(out.numpy(), dev)
+    assert np.array_equal(g.get_x().cpu().numpy(), dev)
+    g.close()
 
 
 # ------------------------------------------------------------------ logistic objective
