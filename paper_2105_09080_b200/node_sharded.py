@@ -116,10 +116,14 @@ def exchange_dist(shard, k, group=None):
             local.append((plan.dst_offset[m], lo, nb))
         else:
             ops.append(dist.P2POp(dist.isend, shard.send[lo:lo + nb], plan.send_to[m], group=group, tag=m))
-    for m in range(plan.messages):
+    # Receives are posted in the order of the SENDER's message index: ring slot 0 (the row above) is the
+    # upper shard's message 1, slot 1 its lower shard's message 0.  A backend without tags (NCCL) pairs
+    # the messages of two ranks in posting order, which matters when both neighbours are one rank
+    # (a ring of two shards); a backend with tags (gloo) gets the index as the tag.
+    slots = range(plan.messages - 1, -1, -1) if plan.kind == GPGA_SHARD_RING else range(plan.messages)
+    for m in slots:
         if plan.recv_from[m] != me:
             lo = plan.recv_offset[m]
-            # the sender's message index for this slot: ring slot 0 (row above) is the upper shard's message 1
             tag = (1 - m) if plan.kind == GPGA_SHARD_RING else m
             ops.append(dist.P2POp(dist.irecv, shard.recv[lo:lo + plan.bytes[m]], plan.recv_from[m], group=group, tag=tag))
     for dst, lo, nb in local:
