@@ -98,10 +98,11 @@ def exchange_local(shards, k):
             dst.recv[plan.dst_offset[m]:plan.dst_offset[m] + nb].copy_(src.send[lo:lo + nb], non_blocking=True)
 
 
-def exchange_dist(shard, k, group=None):
+def exchange_dist(shard, k, group=None, tags=True):
     """Deliver iteration k's messages of this rank's shard through torch.distributed: rank r holds
     shard r.  Gossip messages go point to point (all sends and receives of the iteration posted
-    together), the column sums of a global average by an all-gather in rank order."""
+    together), the column sums of a global average by an all-gather in rank order.  tags=False posts
+    every message with tag 0, i.e. relies on posting order alone, as a backend without tags does."""
     import torch.distributed as dist
     plan = shard.plan(k)
     if plan.kind == GPGA_SHARD_GLOBAL:
@@ -115,7 +116,7 @@ def exchange_dist(shard, k, group=None):
         if plan.send_to[m] == me:       # a neighbour in the same shard (one shard, or a two-shard ring's both sides)
             local.append((plan.dst_offset[m], lo, nb))
         else:
-            ops.append(dist.P2POp(dist.isend, shard.send[lo:lo + nb], plan.send_to[m], group=group, tag=m))
+            ops.append(dist.P2POp(dist.isend, shard.send[lo:lo + nb], plan.send_to[m], group=group, tag=m if tags else 0))
     # Receives are posted in the order of the SENDER's message index: ring slot 0 (the row above) is the
     # upper shard's message 1, slot 1 its lower shard's message 0.  A backend without tags (NCCL) pairs
     # the messages of two ranks in posting order, which matters when both neighbours are one rank
@@ -124,7 +125,7 @@ def exchange_dist(shard, k, group=None):
     for m in slots:
         if plan.recv_from[m] != me:
             lo = plan.recv_offset[m]
-            tag = (1 - m) if plan.kind == GPGA_SHARD_RING else m
+            tag = ((1 - m) if plan.kind == GPGA_SHARD_RING else m) if tags else 0
             ops.append(dist.P2POp(dist.irecv, shard.recv[lo:lo + plan.bytes[m]], plan.recv_from[m], group=group, tag=tag))
     for dst, lo, nb in local:
         shard.recv[dst:dst + nb].copy_(shard.send[lo:lo + nb])
@@ -133,11 +134,11 @@ def exchange_dist(shard, k, group=None):
             req.wait()
 
 
-def run_dist(shard, K, k0=0, group=None):
+def run_dist(shard, K, k0=0, group=None, tags=True):
     """K iterations of this rank's shard: export, exchange, step."""
     for k in range(k0, k0 + K):
         shard.export(k)
-        exchange_dist(shard, k, group)
+        exchange_dist(shard, k, group, tags)
         shard.step(k)
 
 

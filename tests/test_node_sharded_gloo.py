@@ -96,14 +96,14 @@ def _free_port():
     return port
 
 
-def _worker(rank, world, port, topo, H, n, d, K, out_dir):
+def _worker(rank, world, port, topo, H, n, d, K, out_dir, tags=True):
     import torch.distributed as dist
     os.environ["MASTER_ADDR"] = "127.0.0.1"
     os.environ["MASTER_PORT"] = str(port)
     dist.init_process_group("gloo", rank=rank, world_size=world)
     X0, B = quadratic_inputs(n, d, 7, x0="per_node")
     shard = OracleShard(n, d, topo, H, 0.1, 0.4, 11, world, rank, X0, B)
-    ns.run_dist(shard, K)
+    ns.run_dist(shard, K, tags=tags)
     gathered = [None] * world
     dist.all_gather_object(gathered, (rank, shard.X))
     if rank == 0:
@@ -122,6 +122,19 @@ def test_ranks_exchange_the_right_rows(tmp_path, topo, H, n, world):
     got = np.load(tmp_path / "full.npy")
     assert got.shape == want.shape
     # the exchanged half-step rows travel as fp32: a relative 6e-8 per exchanged row and iteration
+    assert np.abs(got - want).max() <= 2e-6 * (1 + np.abs(want).max())
+
+
+def test_two_shard_ring_without_tags(tmp_path):
+    """Both neighbours of a shard are the same rank in a ring of two shards; a backend without message
+    tags pairs sends and receives by posting order alone.  With every tag forced to 0 the run must
+    still be right."""
+    import torch.multiprocessing as mp
+    n, d, K, world = 8, 10, 7, 2
+    mp.spawn(_worker, args=(world, _free_port(), "ring", 3, n, d, K, str(tmp_path), False), nprocs=world, join=True)
+    X0, B = quadratic_inputs(n, d, 7, x0="per_node")
+    want = o.run(o.Problem(o.TOPO_RING, 3, 0.1, 11, sigma=0.4, data=B), X0, 0, K)
+    got = np.load(tmp_path / "full.npy")
     assert np.abs(got - want).max() <= 2e-6 * (1 + np.abs(want).max())
 
 
