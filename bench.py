@@ -6,6 +6,7 @@ local-update + gossip kernel, or the fused local-update + global-average kernel 
 every H-th iteration.  Prints one JSON line (rank 0).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4_exp_h4] [--impl reference]
+    python bench.py --workload c3_ring_h4 --node-shards 4      # one shard's kernels of the node-sharded mode
 
 Default workload: the BERT-Large-sized configuration (n = 16, d = 335,141,888, one-peer
 exponential graph, H = 4; 64.35 GB per step), or the ResNet-50-sized ring configuration when
@@ -671,7 +672,11 @@ def run_node_shard(args):
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
     name = args.workload or FALLBACK_WORKLOAD
     w = WORKLOADS[name]
+    if w.get("objective") == "logistic":
+        raise SystemExit("--node-shards: the node-sharded iteration covers the quadratic workloads")
     G, n, d = args.node_shards, w["n"], w["d"]
+    if n % G:
+        raise SystemExit(f"--node-shards {G} does not divide n = {n}")
     n_l, ld = n // G, padded_stride(w["d"])
     topo = {"ring": pkg.GPGA_TOPO_RING, "exp": pkg.GPGA_TOPO_EXP}[w["topo"]]
     sh = ns.NodeShard(n, d, topo, w["H"], w["gamma"], SEED, G, min(1, G - 1), sigma=w["sigma"], ld=ld)
