@@ -258,7 +258,9 @@ int32_t gpga_run_adaptive(gpga_t* ctx, int64_t K, int64_t H_init, int64_t warmup
  * an All-Reduce ("All-Reduce v.s. multiple Gossips"); the appendix's implementation details: on
  * the one-peer exponential graph a worker sends one copy of its parameters and receives one.
  * Here a shard is a handle holding n consecutive nodes (all d columns) of an (n * shards)-node
- * problem; quadratic objective, ring or one-peer exponential graph.  One iteration k on a shard:
+ * problem; ring or one-peer exponential graph; quadratic objective, or the logistic one (the
+ * shard binds its own nodes' A and labels; gpga_shard_export first forms the mini-batch gradient
+ * of the local nodes, their draws keyed by the global node index).  One iteration k on a shard:
  *     gpga_shard_export(k, send)   forms what other shards need of this shard's half-step
  *     -- the caller delivers the messages gpga_shard_plan lists (copies, or send/recv and an
  *        all-gather of a communication library) --
@@ -295,8 +297,8 @@ int32_t gpga_shard_plan(int32_t topology, int64_t H, int64_t n_total, int64_t sh
                         int64_t k, gpga_shard_plan_t* out);
 
 /* Declares that this handle's n nodes are nodes shard*n .. (shard+1)*n - 1 of an (n*shards)-node
- * problem (the node index keys the noise generator).  Errors: UNSUPPORTED for another objective or
- * topology, for the exponential graph with a number of shards that is not a power of two, and for
+ * problem (the node index keys the noise generator and the mini-batch draws).  Errors: UNSUPPORTED
+ * for another topology, for the exponential graph with a number of shards that is not a power of two, and for
  * several shards of a node count that is not a multiple of four. */
 int32_t gpga_set_node_shard(gpga_t* ctx, int64_t shards, int64_t shard);
 

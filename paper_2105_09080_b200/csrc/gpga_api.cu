@@ -34,6 +34,7 @@ struct gpga_ctx {
     int64_t shards = 1, shard = 0;   // node sharding: this handle holds nodes shard * n .. (shard + 1) * n - 1
     const void* exported = nullptr;  // send buffer of the last gpga_shard_export and its iteration
     int64_t exported_k = -1;
+    int64_t shard_grad_k = -1;       // iteration whose logistic gradient matrix sits in the scratch area
     float* x[2] = {nullptr, nullptr};
     float* data = nullptr;
     const float* labels = nullptr;
@@ -138,6 +139,7 @@ LogregParams logreg_params(const gpga_ctx* c, int64_t k)
     lp.error_flag = reinterpret_cast<int*>(c->scratch + L.result_off + 8);
     lp.partial = reinterpret_cast<float*>(c->scratch + L.chunk_off);
     lp.n = c->n; lp.d = c->d; lp.m = c->m; lp.batch = c->batch;
+    lp.node0 = c->shard * c->n;
     lp.k = (uint32_t)k;
     lp.l2 = c->l2;
     lp.keys = c->keys;
@@ -497,6 +499,8 @@ int32_t gpga_bind(gpga_t* c, void* x_a, void* x_b, void* data, const void* label
     c->scratch = static_cast<char*>(scratch);
     c->scratch_bytes = scratch_bytes;
     c->L = scratch_layout(c);
+    c->exported_k = -1;
+    c->shard_grad_k = -1;
     c->cur = 0;
     c->k = 0;
     c->bound = true;
@@ -766,6 +770,13 @@ ShardParams shard_params(const gpga_ctx* c, int64_t k)
     ShardParams p;
     p.x = c->x[c->cur];
     p.b = c->data;
+    p.ldb = c->ld;
+    p.grad = c->sigma != 0.f ? SHARD_GRAD_QUAD_NOISE : SHARD_GRAD_QUAD;
+    if (c->objective == GPGA_OBJ_LOGISTIC) {   // the gradient matrix G of this iteration (shard_gradient)
+        p.b = reinterpret_cast<const float*>(c->scratch + c->L.G_off);
+        p.ldb = c->d;
+        p.grad = SHARD_GRAD_BUFFER;
+    }
     p.out = c->x[c->cur ^ 1];
     p.n = c->n; p.n_total = c->n * c->shards; p.row0 = c->shard * c->n;
     p.d = c->d; p.ld = c->ld; p.Q = (c->d + 3) / 4;
@@ -780,9 +791,28 @@ int32_t shard_ready(gpga_ctx* c, int64_t k)
 {
     int32_t st = check_ready(c);
     if (st) return st;
-    if (c->objective != GPGA_OBJ_QUADRATIC || (c->topology != GPGA_TOPO_RING && c->topology != GPGA_TOPO_EXP))
-        return fail(c, GPGA_ERR_UNSUPPORTED, "node sharding: quadratic objective on the ring or the one-peer exponential graph");
+    if (c->topology != GPGA_TOPO_RING && c->topology != GPGA_TOPO_EXP)
+        return fail(c, GPGA_ERR_UNSUPPORTED, "node sharding: ring or one-peer exponential graph");
     if (k < 0 || k >= (int64_t(1) << 32)) return fail(c, GPGA_ERR_INVALID_ARG, "k must be in [0, 2^32)");
+    return GPGA_OK;
+}
+
+// Logistic objective: the mini-batch gradient matrix of the local nodes at iteration k (their draws
+// keyed by the global node index), once per iteration, into the scratch area.
+int32_t shard_gradient(gpga_ctx* c, int64_t k, cudaStream_t s)
+{
+    if (c->objective != GPGA_OBJ_LOGISTIC || c->shard_grad_k == k) return GPGA_OK;
+    LogregParams lp = logreg_params(c, k);
+    cudaError_t e = cudaSuccess;
+    if (!c->flag_cleared) {
+        e = cudaMemsetAsync(lp.error_flag, 0, sizeof(int), s);
+        if (e != cudaSuccess) return cuda_fail(c, e, "error word clear");
+        c->flag_cleared = true;
+    }
+    e = launch_logreg_grad(lp, s);
+    c->launches += 2;
+    if (e != cudaSuccess) return cuda_fail(c, e, "logistic gradient launch");
+    c->shard_grad_k = k;
     return GPGA_OK;
 }
 
@@ -836,8 +866,8 @@ int32_t gpga_set_node_shard(gpga_t* c, int64_t shards, int64_t shard)
     if (!c) return fail(nullptr, GPGA_ERR_NOT_READY, "NULL handle");
     if (shards < 1 || shard < 0 || shard >= shards || c->n * shards >= (int64_t(1) << 31))
         return fail(c, GPGA_ERR_INVALID_ARG, "need shards >= 1, 0 <= shard < shards, n * shards < 2^31");
-    if (c->objective != GPGA_OBJ_QUADRATIC || (c->topology != GPGA_TOPO_RING && c->topology != GPGA_TOPO_EXP))
-        return fail(c, GPGA_ERR_UNSUPPORTED, "node sharding: quadratic objective on the ring or the one-peer exponential graph");
+    if (c->topology != GPGA_TOPO_RING && c->topology != GPGA_TOPO_EXP)
+        return fail(c, GPGA_ERR_UNSUPPORTED, "node sharding: ring or one-peer exponential graph");
     if (c->topology == GPGA_TOPO_EXP && !is_pow2(shards))
         return fail(c, GPGA_ERR_UNSUPPORTED, "the one-peer exponential graph needs a power-of-two number of shards");
     if (shards > 1 && (c->n % 4) != 0)
@@ -863,6 +893,8 @@ int32_t gpga_shard_export(gpga_t* c, int64_t k, void* send_dev, void* stream)
     if (st) return st;
     if (!send_dev || !aligned16(send_dev)) return fail(c, GPGA_ERR_INVALID_ARG, "send buffer must be a 16-byte aligned device pointer");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = shard_gradient(c, k, s);
+    if (st) return st;
     const ShardParams p = shard_params(c, k);
     const bool vec = vec_ok(c);
     cudaError_t e;
@@ -894,6 +926,8 @@ int32_t shard_step_part(gpga_ctx* c, int64_t k, const void* recv_dev, int part, 
         return fail(c, GPGA_ERR_INVALID_ARG, "receive buffer must be a 16-byte aligned device pointer");
     if (part != SHARD_ALL && c->x[0] == c->x[1])
         return fail(c, GPGA_ERR_UNSUPPORTED, "the two-part step needs the double buffer (x_a != x_b)");
+    st = shard_gradient(c, k, s);   // normally formed by the export of this iteration already
+    if (st) return st;
     const ShardParams p = shard_params(c, k);
     const bool vec = vec_ok(c);
     const int tau = log2_floor(p.n_total);
@@ -926,6 +960,7 @@ int32_t shard_step_part(gpga_ctx* c, int64_t k, const void* recv_dev, int part, 
     }
     c->launches += 1;
     c->exported_k = -1;
+    c->shard_grad_k = -1;   // the state moves on: the gradient matrix belongs to the old one
     if (e != cudaSuccess) return cuda_fail(c, e, "shard step launch");
     c->cur ^= 1;
     c->k = k + 1;

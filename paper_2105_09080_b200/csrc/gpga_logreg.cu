@@ -30,7 +30,7 @@ __global__ void __launch_bounds__(kLrBlock) logreg_partial_kernel(const LogregPa
     const float* x = p.x + (long long)i * p.ldx;
     for (int j = threadIdx.x; j < p.d; j += blockDim.x) xs[j] = x[j];
     if (threadIdx.x < nrows)
-        rows[threadIdx.x] = batch_row((uint32_t)(t0 + threadIdx.x), (uint32_t)i, p.k, (uint32_t)p.m, p.keys);
+        rows[threadIdx.x] = batch_row((uint32_t)(t0 + threadIdx.x), (uint32_t)(i + p.node0), p.k, (uint32_t)p.m, p.keys);
     if (threadIdx.x < nrows) ys[threadIdx.x] = y[rows[threadIdx.x]];
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(kLrBlock, 2) logreg_partial_tma_reg_kernel(con
     uint32_t my_idx = 0u;
     float my_y = 0.f;
     if (lane < my_rows) {
-        my_idx = batch_row((uint32_t)(t0 + warp + lane * kRegWarps), (uint32_t)i, p.k, (uint32_t)p.m, p.keys);
+        my_idx = batch_row((uint32_t)(t0 + warp + lane * kRegWarps), (uint32_t)(i + p.node0), p.k, (uint32_t)p.m, p.keys);
         my_y = y[my_idx];
     }
     if (lane == 0) {
@@ -264,7 +264,7 @@ __global__ void __launch_bounds__(kLrBlock, 2) logreg_partial_tma_cols_kernel(co
     const int d4 = (int)(p.d >> 2);
     const uint32_t row_bytes = (uint32_t)p.d * 4u;
     if (threadIdx.x < nrows)
-        rows[threadIdx.x] = batch_row((uint32_t)(t0 + threadIdx.x), (uint32_t)i, p.k, (uint32_t)p.m, p.keys);
+        rows[threadIdx.x] = batch_row((uint32_t)(t0 + threadIdx.x), (uint32_t)(i + p.node0), p.k, (uint32_t)p.m, p.keys);
     if (threadIdx.x == 0) {
         mbar_init(&bar[0], 1);
         mbar_init(&bar[1], 1);
@@ -400,7 +400,7 @@ __global__ void __launch_bounds__(kLrBlock) logreg_loss_kernel(const LogregParam
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     double acc = 0.0;
     for (int t = warp; t < (int)p.batch; t += nwarps) {
-        const uint32_t r = batch_row((uint32_t)t, (uint32_t)i, p.k, (uint32_t)p.m, p.keys);
+        const uint32_t r = batch_row((uint32_t)t, (uint32_t)(i + p.node0), p.k, (uint32_t)p.m, p.keys);
         double z = 0.0;
         for (int j = lane; j < (int)p.d; j += 32) z = fma((double)A[(long long)r * p.d + j], (double)x[j], z);
         z = warp_sum(z);

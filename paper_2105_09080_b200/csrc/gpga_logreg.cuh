@@ -18,6 +18,7 @@ struct LogregParams {
     float* G;         // n x d
     int* error_flag;  // set to 1 if a bounded wait inside a kernel gave up (may be NULL)
     long long n, d, m, batch;
+    long long node0 = 0;   // global index of local node 0 (node sharding): keys the mini-batch draws
     uint32_t k;
     float l2;
     PhiloxKeys keys;

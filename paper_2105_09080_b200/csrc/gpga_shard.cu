@@ -52,17 +52,22 @@ __device__ __forceinline__ RowIn load_row(const ShardParams& p, const Group& g, 
 {
     RowIn r;
     r.x = load4<VEC>(p.x + (long long)i * p.ld, g.j0, p.d);
-    r.b = load4<VEC>(p.b + (long long)i * p.ld, g.j0, p.d);
+    r.b = load4<VEC>(p.b + (long long)i * p.ldb, g.j0, p.d);
     return r;
 }
-template <bool NOISE>
+template <int NOISE>   // a ShardGrad
 __device__ __forceinline__ float4 finish_row(const ShardParams& p, const Group& g, const RowIn& r, int i)
 {
-    float4 gr = sub4(r.x, r.b);
-    if (NOISE) gr = fma4(p.sigma, normal4(g.qg, (uint32_t)(p.row0 + i), p.k, 0u, p.keys), gr);
+    float4 gr;
+    if (NOISE == SHARD_GRAD_BUFFER) {
+        gr = r.b;   // the gradient was formed by another kernel (logistic objective)
+    } else {
+        gr = sub4(r.x, r.b);
+        if (NOISE == SHARD_GRAD_QUAD_NOISE) gr = fma4(p.sigma, normal4(g.qg, (uint32_t)(p.row0 + i), p.k, 0u, p.keys), gr);
+    }
     return fma4(-p.gamma, gr, r.x);
 }
-template <bool NOISE, bool VEC>
+template <int NOISE, bool VEC>
 __device__ __forceinline__ float4 half_step_row(const ShardParams& p, const Group& g, int i)
 {
     return finish_row<NOISE>(p, g, load_row<VEC>(p, g, i), i);
@@ -96,7 +101,7 @@ __device__ __forceinline__ float4 half(float4 a, float4 b) { return scale4(add4(
 
 // ---- export ------------------------------------------------------------------------------------
 // send[t][:] = half-step of local row first + t * stride, t < rows.
-template <bool NOISE, bool VEC>
+template <int NOISE, bool VEC>
 __global__ void __launch_bounds__(kShardBlock) shard_export_rows_kernel(const ShardParams p, float* __restrict__ send,
                                                                          int first, int stride, int rows)
 {
@@ -117,7 +122,7 @@ __global__ void __launch_bounds__(kShardBlock) shard_export_rows_kernel(const Sh
 
 // Column sums of the half-step over the local rows, as the global-average kernel forms them:
 // rows pairwise in fp32 in groups of four, groups in fp64 in row order.  sums[4 q .. 4 q + 3].
-template <bool NOISE, bool VEC>
+template <int NOISE, bool VEC>
 __global__ void __launch_bounds__(kShardBlock) shard_export_sums_kernel(const ShardParams p, double* __restrict__ sums)
 {
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -153,7 +158,7 @@ __global__ void __launch_bounds__(kShardBlock) shard_export_sums_kernel(const Sh
 // Ring: recv[0] = half-step of the node above local row 0, recv[1] = of the node below the last.
 // A three-row window slides down the local rows, four rows' loads in flight.
 // interior = true: only the rows whose neighbours are both local (1 .. n - 2); recv is not read.
-template <bool NOISE, bool VEC>
+template <int NOISE, bool VEC>
 __global__ void __launch_bounds__(kShardBlock, 3) shard_ring_kernel(const ShardParams p, const float* __restrict__ recv,
                                                                      bool interior)
 {
@@ -189,7 +194,7 @@ __global__ void __launch_bounds__(kShardBlock, 3) shard_ring_kernel(const ShardP
 
 // The two rows of a ring shard that have a remote neighbour: row 0 (the node above it is recv[0])
 // and row n - 1 (the node below it is recv[1]); reads local rows 0, 1, n - 2, n - 1.
-template <bool NOISE, bool VEC>
+template <int NOISE, bool VEC>
 __global__ void __launch_bounds__(kShardBlock) shard_ring_boundary_kernel(const ShardParams p, const float* __restrict__ recv)
 {
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -215,7 +220,7 @@ __global__ void __launch_bounds__(kShardBlock) shard_ring_boundary_kernel(const 
 // row's partner is recv[c] (the partner shard's row c).  The walk visits step t = c L + s (chain c,
 // position s) at row c + s he, four steps' loads in flight; each local row is read, and its noise
 // generated, once.
-template <bool NOISE, bool VEC>
+template <int NOISE, bool VEC>
 __global__ void __launch_bounds__(kShardBlock, 3) shard_exp_kernel(const ShardParams p, const float* __restrict__ recv,
                                                                     int he_log2, int len_log2, bool interior)
 {
@@ -251,7 +256,7 @@ __global__ void __launch_bounds__(kShardBlock, 3) shard_exp_kernel(const ShardPa
 }
 
 // The last he local rows of the exponential graph's shard, whose partners are recv[0 .. he - 1].
-template <bool NOISE, bool VEC>
+template <int NOISE, bool VEC>
 __global__ void __launch_bounds__(kShardBlock) shard_exp_boundary_kernel(const ShardParams p, const float* __restrict__ recv,
                                                                           int he)
 {
@@ -330,35 +335,38 @@ unsigned grid_of(long long Q) { return (unsigned)((Q + kShardBlock - 1) / kShard
 
 }  // namespace
 
-#define GPGA_SHARD_LAUNCH(kernel, noise, vec, ...)                                           \
-    do {                                                                                     \
-        if (noise) {                                                                         \
-            if (vec) kernel<true, true><<<grid_of(p.Q), kShardBlock, 0, s>>>(__VA_ARGS__);   \
-            else kernel<true, false><<<grid_of(p.Q), kShardBlock, 0, s>>>(__VA_ARGS__);      \
-        } else {                                                                             \
-            if (vec) kernel<false, true><<<grid_of(p.Q), kShardBlock, 0, s>>>(__VA_ARGS__);  \
-            else kernel<false, false><<<grid_of(p.Q), kShardBlock, 0, s>>>(__VA_ARGS__);     \
-        }                                                                                    \
+#define GPGA_SHARD_LAUNCH(kernel, noise, vec, ...)                                                                   \
+    do {                                                                                                             \
+        if (noise == SHARD_GRAD_QUAD_NOISE) {                                                                        \
+            if (vec) kernel<SHARD_GRAD_QUAD_NOISE, true><<<grid_of(p.Q), kShardBlock, 0, s>>>(__VA_ARGS__);          \
+            else kernel<SHARD_GRAD_QUAD_NOISE, false><<<grid_of(p.Q), kShardBlock, 0, s>>>(__VA_ARGS__);             \
+        } else if (noise == SHARD_GRAD_QUAD) {                                                                       \
+            if (vec) kernel<SHARD_GRAD_QUAD, true><<<grid_of(p.Q), kShardBlock, 0, s>>>(__VA_ARGS__);                \
+            else kernel<SHARD_GRAD_QUAD, false><<<grid_of(p.Q), kShardBlock, 0, s>>>(__VA_ARGS__);                   \
+        } else {                                                                                                     \
+            if (vec) kernel<SHARD_GRAD_BUFFER, true><<<grid_of(p.Q), kShardBlock, 0, s>>>(__VA_ARGS__);              \
+            else kernel<SHARD_GRAD_BUFFER, false><<<grid_of(p.Q), kShardBlock, 0, s>>>(__VA_ARGS__);                 \
+        }                                                                                                            \
     } while (0)
 
 cudaError_t launch_shard_export_rows(const ShardParams& p, bool vec, float* send, int first, int stride, int rows,
                                      cudaStream_t s)
 {
-    const bool noise = p.sigma != 0.f;
+    const int noise = p.grad;
     GPGA_SHARD_LAUNCH(shard_export_rows_kernel, noise, vec, p, send, first, stride, rows);
     return cudaGetLastError();
 }
 
 cudaError_t launch_shard_export_sums(const ShardParams& p, bool vec, double* sums, cudaStream_t s)
 {
-    const bool noise = p.sigma != 0.f;
+    const int noise = p.grad;
     GPGA_SHARD_LAUNCH(shard_export_sums_kernel, noise, vec, p, sums);
     return cudaGetLastError();
 }
 
 cudaError_t launch_shard_ring(const ShardParams& p, bool vec, const float* recv, int part, cudaStream_t s)
 {
-    const bool noise = p.sigma != 0.f;
+    const int noise = p.grad;
     if (part == SHARD_BOUNDARY)
         GPGA_SHARD_LAUNCH(shard_ring_boundary_kernel, noise, vec, p, recv);
     else
@@ -368,7 +376,7 @@ cudaError_t launch_shard_ring(const ShardParams& p, bool vec, const float* recv,
 
 cudaError_t launch_shard_exp(const ShardParams& p, bool vec, const float* recv, int he, int part, cudaStream_t s)
 {
-    const bool noise = p.sigma != 0.f;
+    const int noise = p.grad;
     if (part == SHARD_BOUNDARY) {
         GPGA_SHARD_LAUNCH(shard_exp_boundary_kernel, noise, vec, p, recv, he);
         return cudaGetLastError();

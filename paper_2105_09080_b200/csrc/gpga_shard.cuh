@@ -7,9 +7,14 @@
 
 namespace gpga {
 
+// How a shard kernel gets the stochastic gradient of a row.
+enum ShardGrad { SHARD_GRAD_QUAD = 0, SHARD_GRAD_QUAD_NOISE = 1, SHARD_GRAD_BUFFER = 2 };
+
 struct ShardParams {
     const float* x;      // X^(k), the shard's n x d rows, row stride ld
-    const float* b;      // targets b, same layout
+    const float* b;      // quadratic: targets b, row stride ldb = ld; BUFFER: the gradient matrix G, row stride ldb
+    long long ldb;
+    int grad;            // a ShardGrad
     float* out;          // X^(k+1), same layout (may be x: every kernel reads a row before it writes it)
     long long n;         // local rows (nodes of this shard)
     long long n_total;   // nodes of the whole problem

@@ -38,13 +38,17 @@ class NodeShard:
     buffers (uint8 tensors `send` and `recv`)."""
 
     def __init__(self, n_total, d, topology, H, gamma, seed, shards, shard, sigma=0.0, ld=None, col0=0,
-                 device="cuda"):
+                 device="cuda", logistic=None):
+        """logistic: None for the quadratic objective, else dict(l2=..., m=..., batch=...)."""
         import torch
         assert n_total % shards == 0
         self.n_total, self.d, self.topology, self.H = n_total, d, topology, H
         self.shards, self.shard, self.n = shards, shard, n_total // shards
         self.g = B.Gpga(self.n, d, topology, H, gamma, seed)
-        self.g.set_objective(B.GPGA_OBJ_QUADRATIC, sigma=sigma)
+        if logistic:
+            self.g.set_objective(B.GPGA_OBJ_LOGISTIC, l2=logistic["l2"], m=logistic["m"], batch=logistic["batch"])
+        else:
+            self.g.set_objective(B.GPGA_OBJ_QUADRATIC, sigma=sigma)
         if ld:
             self.g.set_row_stride(ld)
         if col0:
@@ -54,8 +58,9 @@ class NodeShard:
         self.send = torch.zeros(nbytes, dtype=torch.uint8, device=device)
         self.recv = torch.zeros(nbytes, dtype=torch.uint8, device=device)
 
-    def bind(self, x_a, x_b, b):
-        self.g.bind(x_a, x_b, b)
+    def bind(self, x_a, x_b, data, labels=None):
+        """data: the local nodes' b (quadratic) or A (logistic, with their labels)."""
+        self.g.bind(x_a, x_b, data, labels)
 
     def plan(self, k) -> ShardPlan:
         return shard_plan(self.topology, self.H, self.n_total, self.shards, self.shard, self.d, k)

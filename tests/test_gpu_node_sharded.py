@@ -154,3 +154,53 @@ def test_plan_and_argument_checks():
     assert err.value.status == pkg.GPGA_ERR_UNSUPPORTED
     sh.step(0)                                              # the whole step works in place
     sh.close()
+
+
+@pytest.mark.parametrize("topo,H,n,shards,m,d,batch", [("ring", 4, 8, 2, 64, 256, 40), ("exp", 3, 16, 4, 32, 1024, 128),
+                                                         ("ring", 0, 12, 3, 40, 2052, 33), ("exp", 0, 8, 2, 24, 64, 8),
+                                                         ("ring", 3, 8, 1, 64, 256, 40)])
+def test_logistic_objective_sharded_by_nodes(topo, H, n, shards, m, d, batch):
+    """The logistic workload split by nodes (every shard binds its own nodes' samples and labels;
+    mini-batch draws keyed by the global node index): bit-identical to the unsharded steps, and within
+    tolerance of the oracle."""
+    import torch
+    from paper_2105_09080_b200.inputs import logistic_inputs
+    gamma, l2, K = 0.1, 1e-4, 9
+    A, y = logistic_inputs(n, m, d, SEED + n)
+    rng = np.random.default_rng(n + d)
+    X0 = (0.1 * rng.standard_normal((n, d))).astype(np.float32)
+    g = pkg.Gpga(n, d, TOPO[topo][0], H, gamma, SEED)
+    g.set_objective(pkg.GPGA_OBJ_LOGISTIC, l2=l2, m=m, batch=batch)
+    xa = torch.from_numpy(X0).cuda()
+    g.bind(xa, torch.empty_like(xa), torch.from_numpy(A).cuda(), torch.from_numpy(y).cuda())
+    for k in range(K):
+        g.step(k)
+    want = g.get_x().cpu().numpy()
+    n_l = n // shards
+    parts = []
+    for s in range(shards):
+        rows = slice(s * n_l, (s + 1) * n_l)
+        sh = ns.NodeShard(n, d, TOPO[topo][0], H, gamma, SEED, shards, s, logistic=dict(l2=l2, m=m, batch=batch))
+        x = torch.from_numpy(np.ascontiguousarray(X0[rows])).cuda()
+        sh.bind(x, torch.empty_like(x), torch.from_numpy(np.ascontiguousarray(A[rows])).cuda(),
+                torch.from_numpy(np.ascontiguousarray(y[rows])).cuda())
+        parts.append(sh)
+    for k in range(K):
+        for sh in parts:
+            sh.export(k)
+        ns.exchange_local(parts, k)
+        for sh in parts:
+            if k % 2:
+                sh.step(k)
+            else:                       # the two-part form as well
+                sh.step_interior(k)
+                sh.step_boundary(k)
+    got = np.concatenate([sh.get_x().cpu().numpy() for sh in parts])
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), float(np.abs(got - want).max())
+    p = o.Problem(TOPO[topo][1], H, gamma, SEED, objective="logistic", data=A.astype(np.float64),
+                  labels=y.astype(np.float64), l2=l2, batch=batch)
+    ok, worst = close(got, o.run(p, X0, 0, K), TOL_RUN)
+    assert ok, worst
+    for sh in parts:
+        sh.close()
+    g.close()
