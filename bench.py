@@ -909,6 +909,11 @@ def main(argv=None):
         args.warmup = 3
     under_launcher = "WORLD_SIZE" in os.environ and "RANK" in os.environ
     if args.gpus > 1 and not under_launcher and args.impl == "ours":
+        if not args.dry_run:
+            import torch
+            have = torch.cuda.device_count() if torch.cuda.is_available() else 0
+            if have < args.gpus:
+                raise SystemExit(f"bench.py --gpus {args.gpus}: this machine shows {have} CUDA device(s)")
         sys.exit(spawn_ranks(args.gpus, argv))       # one process per GPU; rank 0 prints the line
     if args.dry_run:
         return run_dry(args)
