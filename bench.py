@@ -551,6 +551,7 @@ def run_ours(args):
                 if "GB/s" in c:     # flat copies inside `roofline`
                     roofline[f"cell_{spec[0]}_GBs"] = c["GB/s"]
                     roofline[f"cell_{spec[0]}_frac_of_nominal_8TBs"] = c["frac_of_nominal_8TBs"]
+                    roofline[f"cell_{spec[0]}_sm_mhz"] = c["sm_mhz"]
             cells["c5_ring_h4"] = run_logistic_cell(torch, pkg, sampler, peak)
             roofline["cell_c5_ring_h4_us_per_iteration"] = cells["c5_ring_h4"]["us_per_iteration"]
             roofline["cell_c5_ring_h4_frac"] = cells["c5_ring_h4"]["frac"]
