@@ -162,3 +162,33 @@ def test_noalloc_entry_point_checks_arguments_before_any_launch(L):
     st = call(a, y, x, 64, 4, 64, 16, 8, 0.0, 1, 0, g, None, C.byref(need))
     assert st in (pkg.GPGA_ERR_INVALID_ARG, pkg.GPGA_ERR_CUDA)
     assert need.value == 1 * 4 * 64 * 4
+
+
+def test_header_is_plain_c_and_a_c_program_links_against_the_library(tmp_path, L):
+    """include/gpga.h compiles as C99 and as C++, and a C program that only includes it can create and
+    destroy a handle and read the exchange plan through the shared library (no CUDA device needed)."""
+    import shutil
+    import subprocess
+    header = ROOT / "include" / "gpga.h"
+    if not shutil.which("gcc"):
+        pytest.skip("no C compiler")
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-x", "c", str(header)],
+                   check=True)
+    if shutil.which("g++"):
+        subprocess.run(["g++", "-std=c++11", "-fsyntax-only", "-x", "c++", str(header)], check=True)
+    src = tmp_path / "use.c"
+    src.write_text('#include <stdio.h>\n#include "gpga.h"\n'
+                   'int main(void) {\n'
+                   '    gpga_t* h = 0;\n'
+                   '    if (gpga_create(8, 64, GPGA_TOPO_RING, 4, 0.1f, 1u, &h) != GPGA_OK) return 1;\n'
+                   '    if (gpga_step(h, 0, 0) != GPGA_ERR_NOT_READY) return 2;\n'
+                   '    gpga_shard_plan_t plan;\n'
+                   '    if (gpga_shard_plan(GPGA_TOPO_EXP, 0, 16, 2, 0, 40, 3, &plan) != GPGA_OK) return 3;\n'
+                   '    printf("%d %lld %lld\\n", (int)plan.kind, (long long)plan.hop, (long long)plan.bytes[0]);\n'
+                   '    return gpga_destroy(h);\n}\n')
+    exe = tmp_path / "use"
+    lib = binding.LIB_PATH
+    subprocess.run(["gcc", "-std=c99", "-I", str(header.parent), str(src), "-o", str(exe), str(lib),
+                    f"-Wl,-rpath,{lib.parent}", "-lstdc++", "-lm", "-ldl", "-lpthread", "-lrt"], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()
+    assert out == ["1", "8", str(8 * 40 * 4)]
