@@ -243,7 +243,9 @@ __global__ void __launch_bounds__(kTileBlock) run_tile_kernel(const StepParams p
 // through shared memory, in two tiles used alternately so that one barrier per iteration is
 // enough (a tile is rewritten two iterations later, and every thread passes the barrier in
 // between only after its reads of it).  Same arithmetic per element as run_tile_kernel.
-template <int MODE, bool VEC>
+// TOPO: GPGA_TOPO_RING or GPGA_TOPO_EXP specialise the gossip mix (neighbour offsets formed once, the
+// cell's own half-step taken from its register); -1 takes the general tile_mix.
+template <int MODE, bool VEC, int TOPO>
 __global__ void __launch_bounds__(kTileBlock) run_cell_kernel(const StepParams p, int topology, long long H,
                                                               long long phase0, int hop0, int steps,
                                                               int tile_groups, int log2n, const SparseW sw)
@@ -261,17 +263,28 @@ __global__ void __launch_bounds__(kTileBlock) run_cell_kernel(const StepParams p
         x = load4<VEC>(p.x + (long long)i * p.ld, q * 4, p.d);
         b = load4<VEC>(p.b + (long long)i * p.ldb, q * 4, p.d);
     }
-    long long phase = phase0;   // (k + 1) mod H, global average when it is 0
+    // Iterations left until the next global average (phase0 = (k + 1) mod H of the first iteration, a
+    // global average when it is 0), as 32-bit counters: a period beyond this launch's iterations is
+    // cut to steps + 1, which the countdown cannot reach before the launch ends.
+    const int period = H > 0 ? (int)(H < (long long)steps + 1 ? H : (long long)steps + 1) : steps + 1;
+    int until = steps + 1;
+    if (H > 0) until = phase0 == 0 ? 0 : (int)(H - phase0 < (long long)steps + 1 ? H - phase0 : (long long)steps + 1);
     int hop_log2 = hop0;        // k mod log2(n)
     float4* ycur = tile_smem;
     float4* ynext = tile_smem + cells;
     float4* gsum = tile_smem + 2 * cells;   // [n / 4 + 2][tile_groups]: the fp32 addends of the column mean
     float4* gmean = gsum + (n / 4 + 2) * tile_groups;   // [tile_groups]: the column means
+    // ring: the cells above and below this one in the tile
+    const int up_cell = (i == 0 ? n - 1 : i - 1) * tile_groups + g, dn_cell = (i == n - 1 ? 0 : i + 1) * tile_groups + g;
     for (int t = 0; t < steps; ++t) {
         const uint32_t k = p.k + (uint32_t)t;
-        const bool global = H > 0 && phase == 0;            // Algorithm 1's test mod(k + 1, H) = 0
+        const bool global = until == 0;                     // Algorithm 1's test mod(k + 1, H) = 0
         const int mix = topology;
-        if (own) ycur[c] = tile_finish<MODE>(p, x, b, i, q, k);
+        float4 y = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (own) {
+            y = tile_finish<MODE>(p, x, b, i, q, k);
+            ycur[c] = y;
+        }
         __syncthreads();
         if (global) {
             // The column mean, formed once per column group instead of once per cell: the first
@@ -314,12 +327,18 @@ __global__ void __launch_bounds__(kTileBlock) run_cell_kernel(const StepParams p
             __syncthreads();
             if (own) x = gmean[g];
         } else if (own) {
-            x = tile_mix(ycur, i, g, n, tile_groups, mix, hop_log2, p.grid_cols, log2n, sw);
+            if (TOPO == GPGA_TOPO_RING) {          // (up + self) + down, as tile_mix forms it
+                x = scale4(add4(add4(ycur[up_cell], y), ycur[dn_cell]), 0.333333343f);
+            } else if (TOPO == GPGA_TOPO_EXP) {
+                x = scale4(add4(y, ycur[((i + (1 << hop_log2)) & (n - 1)) * tile_groups + g]), 0.5f);
+            } else {
+                x = tile_mix(ycur, i, g, n, tile_groups, mix, hop_log2, p.grid_cols, log2n, sw);
+            }
         }
         float4* const swap = ycur;
         ycur = ynext;
         ynext = swap;
-        if (++phase >= H) phase = 0;
+        until = global ? period - 1 : until - 1;
         if (++hop_log2 >= log2n) hop_log2 = 0;
     }
     if (own) store4<VEC>(p.out + (long long)i * p.ld, q * 4, p.d, x);
@@ -414,8 +433,15 @@ cudaError_t launch_run_tile(const StepParams& p, int mode, bool vec, int topolog
         const long long cells = p.n * tile_groups;
         const int blk = (int)((cells + 31) / 32 * 32);
         const size_t smem = (size_t)cells * 32 + (size_t)(p.n / 4 + 3) * tile_groups * 16;
-#define GPGA_RUN_CELL(M, V) \
-    run_cell_kernel<M, V><<<grd, blk, smem, s>>>(p, topology, H, phase0, hop0, steps, tile_groups, log2n, sw)
+#define GPGA_RUN_CELL(M, V)                                                                                         \
+    do {                                                                                                            \
+        if (topology == GPGA_TOPO_RING)                                                                             \
+            run_cell_kernel<M, V, GPGA_TOPO_RING><<<grd, blk, smem, s>>>(p, topology, H, phase0, hop0, steps, tile_groups, log2n, sw); \
+        else if (topology == GPGA_TOPO_EXP)                                                                         \
+            run_cell_kernel<M, V, GPGA_TOPO_EXP><<<grd, blk, smem, s>>>(p, topology, H, phase0, hop0, steps, tile_groups, log2n, sw);  \
+        else                                                                                                        \
+            run_cell_kernel<M, V, -1><<<grd, blk, smem, s>>>(p, topology, H, phase0, hop0, steps, tile_groups, log2n, sw);             \
+    } while (0)
         if (vec) {
             if (mode == GRAD_QUAD) GPGA_RUN_CELL(GRAD_QUAD, true);
             else GPGA_RUN_CELL(GRAD_QUAD_NOISE, true);
