@@ -276,6 +276,7 @@ __global__ void __launch_bounds__(kTileBlock) run_cell_kernel(const StepParams p
     float4* gmean = gsum + (n / 4 + 2) * tile_groups;   // [tile_groups]: the column means
     // ring: the cells above and below this one in the tile
     const int up_cell = (i == 0 ? n - 1 : i - 1) * tile_groups + g, dn_cell = (i == n - 1 ? 0 : i + 1) * tile_groups + g;
+#pragma unroll 2
     for (int t = 0; t < steps; ++t) {
         const uint32_t k = p.k + (uint32_t)t;
         const bool global = until == 0;                     // Algorithm 1's test mod(k + 1, H) = 0
