@@ -223,17 +223,16 @@ int32_t do_step(gpga_ctx* c, int64_t k, bool global, cudaStream_t s, bool after_
 // through many iterations on chip (launch_run_tile) with HBM touched once per launch; the time per
 // iteration is then set by the noise arithmetic, not by memory.  That path is taken
 //  - for a state small enough to sit in L2 (one launch per iteration would be launch-bound), and
-//  - for n <= kFusedWideNodes and runs of at least kFusedMinSteps iterations at any size: there the
-//    arithmetic bound (6.0-6.9e11 updates/s measured for n = 8 ... 64, 5.3e11 at n = 128) is above
-//    what the row-streaming kernels reach from HBM (at most 5.5e11, 4.9-5.3e11 at 0.8 GB of
-//    state), and the one extra pass over the state is amortised.  At n = 256 the two are equal,
-//    and wider n would go through the several-cells-per-thread kernel, which is far slower.  A
-//    global-average iteration costs a little more on chip (the fp64 column mean: 3.15 against
-//    3.02 ms at n = 64, d = 25,557,032), so H = 1 keeps to single steps (H = 2: 2.66 against 3.04).
+//  - for n <= kFusedWideNodes (one cell per thread) and runs of at least kFusedMinSteps iterations at any
+//    size: there the arithmetic bound (7.6-7.8e11 updates/s measured at n = 16 and 64, 6.5e11 at
+//    n = 256) is above what the row-streaming kernels reach from HBM (at most 5.6e11), also when
+//    every iteration is a global average (H = 1: 2.90 against 3.05-3.16 ms at n = 64, d = 25,557,032;
+//    8.55 against 10.18 ms at n = 16, d = 335,141,888), and the one extra pass over the state is
+//    amortised.  Wider n would go through the several-cells-per-thread kernel, which is far slower.
 // A launch is kept to about half a second of work.
 constexpr int64_t kFusedStateBytes = 64ll << 20;
 constexpr int64_t kFusedSteps = 1024;
-constexpr int64_t kFusedWideNodes = 128, kFusedMinSteps = 32;
+constexpr int64_t kFusedWideNodes = 256, kFusedMinSteps = 32;
 constexpr double kFusedUpdatesPerLaunch = 2.75e11;
 
 // Logistic objective, narrow state: many iterations per launch with x_i resident on chip (a pair of
@@ -293,7 +292,7 @@ int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)
         return fail(c, GPGA_ERR_NOT_READY, "topology SPARSE needs gpga_set_weight_matrix");
     const bool fused = c->objective == GPGA_OBJ_QUADRATIC && K >= 2 && run_tile_supports(c->n) &&
                        (12 * c->n * c->ld <= kFusedStateBytes ||
-                        (c->n <= kFusedWideNodes && K >= kFusedMinSteps && c->H != 1));
+                        (c->n <= kFusedWideNodes && K >= kFusedMinSteps));
     int64_t per_launch = (int64_t)(kFusedUpdatesPerLaunch / ((double)c->n * (double)c->d));
     if (per_launch > kFusedSteps) per_launch = kFusedSteps;
     if (per_launch < 16) per_launch = 16;

@@ -266,13 +266,15 @@ def test_partly_overlapping_state_buffers_are_rejected():
 
 @pytest.mark.parametrize("topo,n,d,H,fused", [("exp", 16, 1_500_004, 8, True), ("ring", 32, 600_000, 5, True),
                                               ("ring", 64, 300_000, 4, True), ("ring", 100, 200_000, 3, True),
-                                              ("ring", 200, 100_000, 4, False), ("ring", 16, 1_200_000, 2, True), ("ring", 16, 1_200_000, 1, False)])
+                                              ("ring", 200, 100_000, 4, True), ("exp", 256, 80_000, 0, True),
+                                              ("ring", 300, 70_000, 4, False), ("ring", 16, 1_200_000, 2, True),
+                                              ("ring", 16, 1_200_000, 1, True)])
 def test_long_runs_with_few_nodes_take_the_multi_iteration_launch_at_any_size(topo, n, d, H, fused):
-    """Above 64 MB of state gpga_run still advances many iterations per launch when n <= 128 and the
-    run has at least 32 iterations (the on-chip arithmetic is then faster than streaming the state
-    from HBM every iteration); wider n keeps one launch per iteration, and so does H = 1 (a
-    global-average iteration costs a little more on chip than from HBM).  Either way the result is
-    bit-identical to stepping, and within tolerance of the oracle on a slice of columns."""
+    """Above 64 MB of state gpga_run still advances many iterations per launch when n <= 256 (one cell
+    per thread) and the run has at least 32 iterations (the on-chip arithmetic is then faster than
+    streaming the state from HBM every iteration, also with a global average every iteration); wider
+    n keeps one launch per iteration.  Either way the result is bit-identical to stepping, and within
+    tolerance of the oracle on a slice of columns."""
     X0, B = quadratic_inputs(n, d, 5 + n, x0="shared", x0_std=0.5)
     assert 12 * n * d > 64 << 20
     K = 40
