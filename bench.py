@@ -573,7 +573,7 @@ def run_ours(args):
                  "launches": g.launch_count() - launches_c}
 
     # one gpga_run call over the configuration's own run length (at least 32 iterations): for
-    # n <= 128 and runs that long it advances many iterations per launch with the cells on chip, so
+    # n <= 256 and runs that long it advances many iterations per launch with the cells on chip, so
     # its rate is not tied to 12 bytes per update
     run_info = None
     if not resident:
