@@ -8,15 +8,16 @@
 //    copies, the copies of the next iteration's rows (their indices depend only on the seed,
 //    the node and the iteration) already in flight while this iteration is reduced and mixed,
 //    and the rows that no buffer is free for asked into L2 an iteration before they are copied;
-//  - the per-warp gradient sums are added in shared memory; the chunk sums go to the block that
-//    finishes the column group by asynchronous stores into its shared memory, which count
-//    themselves off on an mbarrier there (no cluster-wide barrier in the loop); each block
-//    finishes one half of the columns: gradient, local update y_i = x_i - gamma g_i;
+//  - the per-warp gradient sums are added in shared memory; the chunk sums go to BOTH blocks of the
+//    pair by asynchronous stores into their shared memory, which count themselves off on an
+//    mbarrier there (no cluster-wide barrier in the loop); each block then finishes all columns
+//    for itself (gradient, local update y_i = x_i - gamma g_i), so x_i^(k+1) never has to cross
+//    from one block to the other, and publishes one half of them;
 //  - y_i is published to global memory as 64-bit words (value, iteration tag), each written and
-//    read whole, so a reader needs no flag and no fence: it reads the rows of its neighbours (ring,
-//    one-peer exponential graph) or of all nodes (global average) until the tags are this
-//    iteration's, forms its half of x_i^(k+1) and sends it to both blocks of the pair, again by
-//    counted asynchronous stores.
+//    read whole, so a reader needs no flag and no fence: both blocks read the rows of the node's
+//    neighbours (ring, one-peer exponential graph) or the column means (global average) until
+//    the tags are this iteration's and form x_i^(k+1), which goes to the block's warps through
+//    shared memory.
 // Every sum is formed in the order the one-iteration kernels use (rows of a warp in order,
 // eight warps of a chunk in order, chunks in order; ring (up + self) + down; global mean by
 // groups of four rows in fp32, groups in fp64), so a run is bit-identical to the same number of
@@ -187,7 +188,7 @@ __device__ __forceinline__ void add4_to(float4& s, const float4 v)
 }
 
 // Shared-memory plan for row width d: row buffers [16 warps][slots][d], the (group, row) items of
-// a column mean [512], the chunk sums of this block's half [4][h0] and x_i [d].  The per-warp
+// a column mean [512], the chunk sums [4][d / 4] and x_i [d].  The per-warp
 // gradient sums have no area of their own: a warp parks them in the buffer of the row it consumed
 // last, which is refilled only after the chunk sums have been formed.
 struct RunSmem {
@@ -196,9 +197,9 @@ struct RunSmem {
 };
 __host__ __device__ inline RunSmem run_smem_plan(int d)
 {
-    const int d4 = d >> 2, h0 = (d4 + 1) >> 1;
+    const int d4 = d >> 2;
     RunSmem s;
-    const size_t fixed = ((size_t)kRunThreads + (size_t)kRunMaxChunks * h0 + (size_t)d4) * sizeof(float4);
+    const size_t fixed = ((size_t)kRunThreads + (size_t)kRunMaxChunks * d4 + (size_t)d4) * sizeof(float4);
     const size_t per_slot = (size_t)kRunWarps * d * sizeof(float);
     long long slots = ((long long)kRunSmemLimit - (long long)fixed) / (long long)per_slot;
     if (slots > kRunMaxSlots) slots = kRunMaxSlots;
@@ -213,14 +214,14 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t bars[kRunWarps * kRunMaxSlots];
-    __shared__ __align__(8) uint64_t sums_bar, x_bar;   // chunk sums of this block's half; x_i^(k+1)
+    __shared__ __align__(8) uint64_t sums_bar;          // the chunk sums of both blocks have arrived
     __shared__ int stage_at[kRunWarps];                 // where each warp parked its gradient sums (float4 index)
     cg::cluster_group cluster = cg::this_cluster();
-    const int r = (int)cluster.block_rank();   // which half of the columns this block finishes
+    const int r = (int)cluster.block_rank();   // which half of the columns this block publishes
     const int i = (int)(blockIdx.x >> 1);      // node
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = p.n, d = p.d, d4 = d >> 2;
-    const int h0 = (d4 + 1) >> 1;              // block 0 finishes groups [0, h0), block 1 [h0, d4)
+    const int h0 = (d4 + 1) >> 1;              // block 0 publishes groups [0, h0), block 1 [h0, d4)
     const int g_lo = r ? h0 : 0;
     const int owned = r ? d4 - h0 : h0;
     const int chunks = (p.batch + kRunChunkRows - 1) / kRunChunkRows;
@@ -230,13 +231,11 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
 
     float* slot_base = reinterpret_cast<float*>(smem_raw);
     float4* items = reinterpret_cast<float4*>(slot_base + (size_t)kRunWarps * slots * d);   // [kRunThreads]
-    float4* pbuf = items + kRunThreads;             // [chunk][h0]: chunk sums of this block's groups
-    float4* xnew = pbuf + kRunMaxChunks * h0;       // [d4]: x_i^(k+1), both halves
+    float4* pbuf = items + kRunThreads;             // [chunk][d4]: the four chunk sums of every group
+    float4* xnew = pbuf + kRunMaxChunks * d4;       // [d4]: x_i^(k+1)
     // the same locations in both blocks of the pair, as cluster addresses
     const uint32_t pbuf_at[2] = {cluster_addr(pbuf, 0), cluster_addr(pbuf, 1)};
-    const uint32_t xnew_at[2] = {cluster_addr(xnew, 0), cluster_addr(xnew, 1)};
     const uint32_t sums_bar_at[2] = {cluster_addr(&sums_bar, 0), cluster_addr(&sums_bar, 1)};
-    const uint32_t x_bar_at[2] = {cluster_addr(&x_bar, 0), cluster_addr(&x_bar, 1)};
     const int* stop = p.stop;
 
     // ---- this warp's rows: warp (chunk c, w) of the one-iteration kernel ----------------------
@@ -266,10 +265,7 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
     }
     if (lane == 0) {
         for (int s = 0; s < slots; ++s) mbar_init(&bar[s], 1);
-        if (warp == 0) {
-            mbar_init(&sums_bar, 1);
-            mbar_init(&x_bar, 1);
-        }
+        if (warp == 0) mbar_init(&sums_bar, 1);
         mbar_init_fence();
     }
     __syncwarp();
@@ -307,9 +303,10 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
             xr[j] = (FULL || g < d4) ? x4[g] : zero2;
         }
     }
-    const bool finisher = tid < owned;   // finishes group g_lo + tid
+    const bool finisher = tid < d4;      // finishes group tid (in both blocks alike)
+    const bool publishes = finisher && tid >= g_lo && tid < g_lo + owned;   // and publishes it
     float4 xo = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (finisher) xo = reinterpret_cast<const float4*>(p.x_in + (long long)i * p.ldx)[g_lo + tid];
+    if (finisher) xo = reinterpret_cast<const float4*>(p.x_in + (long long)i * p.ldx)[tid];
     cluster.sync();   // the partner's barriers are set up before anything is sent to them
 
     bool failed = false;
@@ -318,10 +315,7 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
         const long long k = (long long)p.k0 + it;
         const uint32_t tag = (uint32_t)it + 1u;
         const uint32_t phase = (uint32_t)it & 1u;
-        if (tid == 0) {   // what this iteration will send to this block
-            mbar_arrive_expect_tx(&sums_bar, (uint32_t)(chunks * owned) * 16u);
-            mbar_arrive_expect_tx(&x_bar, (uint32_t)d4 * 16u);
-        }
+        if (tid == 0) mbar_arrive_expect_tx(&sums_bar, (uint32_t)(chunks * d4) * 16u);   // what this iteration will send to this block
         // ---- gradient sums of this warp's rows ----------------------------------------------------
         ulonglong2 acc[kRunGroups];
 #pragma unroll
@@ -393,7 +387,7 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
             if (lane == 0) stage_at[warp] = (warp * slots + stage_slot) * d4;
         }
         __syncthreads();
-        // ---- chunk sums (eight warps in order), sent to the block that finishes the group ---------
+        // ---- chunk sums (eight warps in order), sent to both blocks -------------------------------
         {
             const int cl = tid >> 8, g = tid & 255;
             const int cc = 2 * r + cl;
@@ -402,8 +396,9 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
                 float4 sum = all[stage_at[cl * kRunChunkWarps]];
 #pragma unroll
                 for (int ww = 1; ww < kRunChunkWarps; ++ww) add4_to(sum, all[stage_at[cl * kRunChunkWarps + ww]]);
-                const int to = g >= h0 ? 1 : 0;
-                send4(pbuf_at[to] + (uint32_t)(cc * h0 + (g - (to ? h0 : 0))) * 16u, sums_bar_at[to], sum);
+                const uint32_t off = (uint32_t)(cc * d4 + g) * 16u;
+                send4(pbuf_at[0] + off, sums_bar_at[0], sum);
+                send4(pbuf_at[1] + off, sums_bar_at[1], sum);
             }
         }
         __syncthreads();   // every parked sum has been read: the buffers that carried them can be refilled
@@ -411,9 +406,9 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // this warp's writes before the copy's
             issue(deferred_idx);
         }
-        const bool finisher_warp = warp * 32 < owned;
+        const bool finisher_warp = warp * 32 < d4;
         if (!finisher_warp) roll(it);   // off the path that the next iteration waits for
-        // ---- gradient, local update, publication of this block's half of y_i ----------------------
+        // ---- gradient, local update (all columns), publication of this block's half of y_i --------
         const bool glob = p.H > 0 && ((k + 1) % p.H) == 0;
         const int buf = glob ? gossip_bufs + (int)(((k + 1) / p.H) & 1) : it % gossip_bufs;
         unsigned long long* ybuf = p.ytag + (size_t)buf * buf_words;
@@ -421,12 +416,12 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
         if (finisher) {
             if (!wait_phase(&sums_bar, phase, stop, p.copy_tries)) failed = true;
             float4 gs = pbuf[tid];
-            for (int cc = 1; cc < chunks; ++cc) add4_to(gs, pbuf[cc * h0 + tid]);
+            for (int cc = 1; cc < chunks; ++cc) add4_to(gs, pbuf[cc * d4 + tid]);
             const float4 gr = make_float4(fmaf(gs.x, inv_batch, p.l2 * xo.x), fmaf(gs.y, inv_batch, p.l2 * xo.y),
                                           fmaf(gs.z, inv_batch, p.l2 * xo.z), fmaf(gs.w, inv_batch, p.l2 * xo.w));
             yv = make_float4(fmaf(-p.gamma, gr.x, xo.x), fmaf(-p.gamma, gr.y, xo.y), fmaf(-p.gamma, gr.z, xo.z),
                              fmaf(-p.gamma, gr.w, xo.w));
-            if (!failed) publish4(ybuf + (size_t)i * d + 4 * (g_lo + tid), yv, tag);
+            if (publishes && !failed) publish4(ybuf + (size_t)i * d + 4 * tid, yv, tag);
         }
         // ---- mix ------------------------------------------------------------------------------------
         float4 xp = yv;
@@ -435,7 +430,7 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
             // block (i, r) takes local groups i, i + n, ...; it reads those groups of every node's row,
             // forms their means exactly as the one-iteration kernels do (rows added in fp32 in groups
             // of four, (y0 + y1) + (y2 + y3), the group sums in fp64 in row order) and publishes them;
-            // then every block reads the means of its half.  A block reads n * (groups / n) + groups
+            // then every block reads the means of all groups.  A block reads n * (groups / 2n) + groups
             // words instead of n * groups.
             const int mine_cnt = i < owned ? (owned - i + n - 1) / n : 0;   // groups this block averages
             unsigned long long* means = p.ytag + (size_t)p.nbuf * buf_words + (size_t)(buf - gossip_bufs) * d;
@@ -466,11 +461,11 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
                 asm volatile("st.relaxed.gpu.global.b64 [%0], %1;" ::"l"(means + 4 * (g_lo + i + j * n) + comp), "l"(word)
                              : "memory");
             }
-            if (finisher && !read4(means + 4 * (g_lo + tid), tag, stop, p.poll_tries, &xp)) failed = true;
+            if (finisher && !read4(means + 4 * tid, tag, stop, p.poll_tries, &xp)) failed = true;
         } else if (finisher_warp) {
-            const int seg_last = min(warp * 32 + 31, owned - 1);
-            const unsigned long long* col = ybuf + 4 * (g_lo + min(tid, owned - 1));
-            const unsigned long long* gate = ybuf + 4 * (g_lo + seg_last) + 3;
+            const int seg_last = min(warp * 32 + 31, d4 - 1);
+            const unsigned long long* col = ybuf + 4 * min(tid, d4 - 1);
+            const unsigned long long* gate = ybuf + 4 * seg_last + 3;
             if (p.topology == GPGA_TOPO_RING) {
                 const int up = (i == 0) ? n - 1 : i - 1, dn = (i == n - 1) ? 0 : i + 1;
                 float4 yu = yv, yd = yv;
@@ -493,15 +488,12 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
                                  (yv.w + yp.w) * 0.5f);
             }
         }
-        // ---- x_i^(k+1) to both blocks of the pair ---------------------------------------------------
+        // ---- x_i^(k+1) to the warps of this block ---------------------------------------------------
         if (finisher && !failed) {
-            const uint32_t off = (uint32_t)(g_lo + tid) * 16u;
-            send4(xnew_at[0] + off, x_bar_at[0], xp);
-            send4(xnew_at[1] + off, x_bar_at[1], xp);
-            if (it == p.steps - 1) reinterpret_cast<float4*>(p.x_out + (long long)i * p.ldx)[g_lo + tid] = xp;
+            xnew[tid] = xp;
+            if (publishes && it == p.steps - 1) reinterpret_cast<float4*>(p.x_out + (long long)i * p.ldx)[tid] = xp;
         }
         if (finisher_warp) roll(it);
-        if (!failed && !wait_phase(&x_bar, phase, stop, p.copy_tries)) failed = true;
         if (failed) {   // tell everyone; the partner's and the other nodes' waits end on the stop word
             st_relaxed_gpu(p.stop, 1);
             if (p.error_flag) atomicExch(p.error_flag, 1);
@@ -512,7 +504,7 @@ __global__ void __launch_bounds__(kRunThreads, 1) logreg_run_kernel(const LogRun
             const int g = lane + 32 * j;
             if (FULL || g < d4) xr[j] = reinterpret_cast<const ulonglong2*>(xnew)[g];
         }
-        if (finisher) xo = xnew[g_lo + tid];
+        if (finisher) xo = xp;
     }
     // Copies still in flight target this block's shared memory: give each a bounded chance to land
     // (none is in flight after a run that went through).
