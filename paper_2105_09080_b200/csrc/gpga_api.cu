@@ -296,9 +296,14 @@ int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)
     int64_t per_launch = (int64_t)(kFusedUpdatesPerLaunch / ((double)c->n * (double)c->d));
     if (per_launch > kFusedSteps) per_launch = kFusedSteps;
     if (per_launch < 16) per_launch = 16;
-    // (with a global average every iteration or every other one the two-hop column mean makes the
-    // one-launch kernel no faster than single steps: 11.2 against 10.8 us per iteration at H = 1)
-    if (c->objective == GPGA_OBJ_LOGISTIC && K >= kLogRunMinSteps && (c->H == 0 || c->H >= 3)) {
+    // A global-average iteration costs the one-launch kernel two trips through L2 and a wait for the
+    // slowest node, a gossip iteration costs single steps more the more nodes there are.  Measured
+    // (us per iteration, single steps against one launch, d = 1024, batch 128): H = 1: 7.8 / 8.7 at
+    // n = 8, 8.9 / 9.3 at n = 32, 11.6 / 10.6 at n = 64; H = 2 at n = 64: 10.5 / 9.7; H = 4: 7.6 / 7.9
+    // at n = 8, 8.6 / 8.3 at n = 32, 10.3 / 9.1 at n = 64; no global average: 7.6 / 7.5 at n = 8,
+    // 10.0 / 7.9 at n = 64.
+    const bool run_pays = c->H == 0 || c->H >= 3 || (c->H == 2 && c->n >= 24) || (c->H == 1 && c->n >= 48);
+    if (c->objective == GPGA_OBJ_LOGISTIC && K >= kLogRunMinSteps && run_pays) {
         bool ok = false;
         const cudaError_t e = logreg_run_supported((int)c->n, (int)c->d, (int)c->batch, c->topology, c->H, &ok);
         if (e != cudaSuccess) return cuda_fail(c, e, "occupancy query");

@@ -2,7 +2,7 @@
 on chip, neighbours' half-step rows exchanged through global memory as (value, iteration tag)
 words.  Every sum is formed in the order of the one-iteration kernels, so a run must equal the same
 number of gpga_step calls bit for bit; parity with the oracle is checked on top.  (With H = 1 or 2
-gpga_run keeps to single steps, which are as fast there.)"""
+gpga_run keeps to single steps unless there are many nodes: they are faster there.)"""
 import numpy as np
 import pytest
 
@@ -61,6 +61,28 @@ def test_resident_run_equals_single_steps(topo, H, n, m, d, batch):
     a, b = run.get_x().cpu().numpy(), stepped.get_x().cpu().numpy()
     assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
     assert run.consensus_distance() == stepped.consensus_distance()
+    run.close()
+    stepped.close()
+
+
+@pytest.mark.parametrize("topo,H,n,one_launch", [("ring", 1, 64, True), ("exp", 2, 64, True), ("ring", 2, 32, True),
+                                                 ("ring", 1, 32, False), ("exp", 2, 16, False)])
+def test_short_averaging_periods_take_one_launch_only_with_many_nodes(topo, H, n, one_launch):
+    """With a global average every iteration or every other one the one-launch kernel is taken only
+    where it is faster than single steps (n >= 48 for H = 1, n >= 24 for H = 2); either way the result
+    equals single steps bit for bit."""
+    m, d, batch, K = 64, 1024, 128, 10
+    A, y = logistic_inputs(n, m, d, SEED + n)
+    rng = np.random.default_rng(n + H)
+    X0 = (0.1 * rng.standard_normal((n, d))).astype(np.float32)
+    run, stepped = _pair(n, m, d, batch, topo, H, X0, A, y)
+    launches0 = run.launch_count()
+    run.run(K)
+    assert (run.launch_count() - launches0 == 1) == one_launch
+    for k in range(K):
+        stepped.step(k)
+    a, b = run.get_x().cpu().numpy(), stepped.get_x().cpu().numpy()
+    assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), float(np.abs(a - b).max())
     run.close()
     stepped.close()
 
