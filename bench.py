@@ -720,6 +720,12 @@ def run_node_shard(args):
     xa = torch.randn((n_l, ld), device="cuda") * 0.1
     sh.bind(xa, torch.empty_like(xa), torch.randn((n_l, ld), device="cuda"))
     steps = args.steps or 100
+    if args.fused_send:
+        # stand-ins for the other shards' receive areas, in this device's memory: the export kernel
+        # stores its messages there itself (gpga_shard_export_to), as it would into peer-mapped memory
+        areas = torch.zeros((G, sh.recv.numel()), dtype=torch.uint8, device="cuda")
+        base_of = lambda s: sh.recv.data_ptr() if s == sh.shard else areas[s].data_ptr()
+        sh.export = lambda k: sh.export_to(k, ns.direct_destinations(sh.plan(k), sh.shard, G, base_of))
     for k in range(args.warmup):
         sh.export(k)
         sh.step(k)
@@ -753,7 +759,9 @@ def run_node_shard(args):
                       "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                       "config": {"workload": f"{name}: shard {min(1, G - 1)} of {G} ({n_l} of n={n} nodes x d={d} fp32, "
                                              f"{w['topo']} topology, H={w['H'] or 'inf'}), export + step kernels of the "
-                                             f"node-sharded iteration; the exchange between shards is not timed"},
+                                             f"node-sharded iteration; " + ("the export kernel stores its messages into the receivers' "
+                                             "areas itself (stand-ins in this device's memory)" if args.fused_send
+                                             else "the exchange between shards is not timed")},
                       "per_kind": table, "clocks": clocks, "gpu_launches": sh.g.launch_count()}), flush=True)
     sh.close()
 
@@ -903,6 +911,9 @@ def main(argv=None):
     ap.add_argument("--sustained-seconds", type=float, default=2.0)
     ap.add_argument("--cell-seconds", type=float, default=1.0)
     ap.add_argument("--dry-run", action="store_true", help="multi-rank plumbing only, on CPU with gloo")
+    ap.add_argument("--fused-send", action="store_true",
+                    help="with --node-shards: time gpga_shard_export_to, the export kernel that stores its messages "
+                         "straight into the receivers' areas")
     ap.add_argument("--node-shards", type=int, default=0,
                     help="time the export + step kernels of one shard of a node-sharded run with this many shards")
     args = ap.parse_args(argv)

@@ -311,6 +311,33 @@ int64_t gpga_shard_exchange_bytes(const gpga_t* ctx);
  * exported (a hop of at least n nodes) the step takes the half-step rows from there. */
 int32_t gpga_shard_export(gpga_t* ctx, int64_t k, void* send_dev, void* stream);
 
+/* gpga_shard_export with the send fused into the kernel (Section 3: a gossip step sends the node's
+ * half-step vector to its neighbours; the appendix's implementation details: one copy sent, one
+ * received per one-peer step): the kernel that forms the outgoing rows stores them straight to
+ * where their receivers will read them, so no separate copy or send call follows.
+ * dest_host is a HOST array of ndest device addresses, 16-byte aligned, on this device or on another
+ * one whose memory is mapped for peer access (the kernel only stores there, 16 adjacent bytes per
+ * thread; it never loads from a destination):
+ *   ring (ndest = 2):       dest[m] = where message m of gpga_shard_plan lands, i.e. the receive
+ *                           buffer of shard send_to[m] plus dst_offset[m];
+ *   exponential graph (1):  dest[0] = the receive buffer of shard send_to[0];
+ *   global average (ndest = shards, at most 32): dest[s] = the receive buffer of shard s plus
+ *                           (this shard) * gather_bytes -- the all-gather of the column sums done by
+ *                           the producer's stores; dest[this shard] is the shard's own receive buffer.
+ * keep_dev (may be NULL) is a send-buffer-sized area of this device: when every local row is exported
+ * (a hop of at least n nodes) the rows are stored there too and gpga_shard_step of the same iteration
+ * averages them with the received ones instead of forming the half-step again; otherwise unused.
+ * Ordering is the caller's: (a) a destination must no longer be needed by its owner's step of an
+ * earlier iteration -- alternate between two receive buffers by the parity of k, which suffices when
+ * (b) holds; (b) the receiver launches gpga_shard_step(k) only after the exports of all its senders
+ * have completed (stream order or an event on one device; a barrier across the processes that own
+ * the devices, placed in stream order after the export, otherwise).  No kernel of the library waits
+ * for another one.  Asynchronous on `stream`.
+ * Errors: as gpga_shard_export; INVALID_ARG for a wrong ndest, a NULL or misaligned destination;
+ * UNSUPPORTED for a global average over more than 32 shards. */
+int32_t gpga_shard_export_to(gpga_t* ctx, int64_t k, void* keep_dev, void* const* dest_host, int32_t ndest,
+                             void* stream);
+
 /* Second half: Algorithm 1's update and mix for the local rows, with recv_dev holding the received
  * messages (recv_offset) or all shards' column sums.  Reads the current buffer, writes the other,
  * flips them and sets the counter to k + 1, like gpga_step.  Asynchronous on `stream`. */

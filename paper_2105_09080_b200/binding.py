@@ -60,6 +60,7 @@ SIGNATURES = {
     "gpga_set_node_shard": (_i32, [_P, _i64, _i64]),
     "gpga_shard_exchange_bytes": (_i64, [_P]),
     "gpga_shard_export": (_i32, [_P, _i64, _P, _P]),
+    "gpga_shard_export_to": (_i32, [_P, _i64, _P, _P, _i32, _P]),
     "gpga_shard_step": (_i32, [_P, _i64, _P, _P]),
     "gpga_shard_step_interior": (_i32, [_P, _i64, _P]),
     "gpga_shard_step_boundary": (_i32, [_P, _i64, _P, _P]),

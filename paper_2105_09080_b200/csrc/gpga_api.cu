@@ -919,6 +919,51 @@ int32_t gpga_shard_export(gpga_t* c, int64_t k, void* send_dev, void* stream)
     return GPGA_OK;
 }
 
+int32_t gpga_shard_export_to(gpga_t* c, int64_t k, void* keep_dev, void* const* dest_host, int32_t ndest, void* stream)
+{
+    int32_t st = shard_ready(c, k);
+    if (st) return st;
+    const bool global = is_global_step(k, c->H);
+    const bool ring = c->topology == GPGA_TOPO_RING;
+    const int32_t want = global ? (int32_t)c->shards : (ring ? 2 : 1);
+    if (global && c->shards > kShardMaxDirect)
+        return fail(c, GPGA_ERR_UNSUPPORTED, "the fused all-gather of the column sums serves at most 32 shards");
+    if (!dest_host || ndest != want)
+        return fail(c, GPGA_ERR_INVALID_ARG, "destinations: 2 on the ring, 1 on the exponential graph, one per shard for a global average");
+    for (int32_t m = 0; m < ndest; ++m)
+        if (!dest_host[m] || !aligned16(dest_host[m]))
+            return fail(c, GPGA_ERR_INVALID_ARG, "every destination must be a 16-byte aligned device address");
+    if (keep_dev && !aligned16(keep_dev)) return fail(c, GPGA_ERR_INVALID_ARG, "keep buffer must be 16-byte aligned");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = shard_gradient(c, k, s);
+    if (st) return st;
+    const ShardParams p = shard_params(c, k);
+    const bool vec = vec_ok(c);
+    cudaError_t e;
+    bool kept = false;
+    if (global) {
+        ShardSumDests dl{};
+        dl.count = ndest;
+        for (int32_t m = 0; m < ndest; ++m) dl.dst[m] = static_cast<double*>(dest_host[m]);
+        e = launch_shard_export_sums_to(p, vec, dl, s);
+    } else if (ring) {
+        e = launch_shard_export_rows_to(p, vec, nullptr, static_cast<float*>(dest_host[0]), static_cast<float*>(dest_host[1]),
+                                        1, 0, (int)(c->n - 1), 2, s);
+    } else {
+        const int tau = log2_floor(p.n_total);
+        const int64_t hop = tau > 0 ? (int64_t(1) << (k % tau)) : 1;
+        const int rows = (int)(hop < c->n ? hop : c->n);
+        kept = hop >= c->n && keep_dev != nullptr;   // the step will average these rows with the received ones
+        e = launch_shard_export_rows_to(p, vec, kept ? static_cast<float*>(keep_dev) : nullptr,
+                                        static_cast<float*>(dest_host[0]), nullptr, rows, 0, 1, rows, s);
+    }
+    c->launches += 1;
+    if (e != cudaSuccess) return cuda_fail(c, e, "shard export launch");
+    c->exported = kept ? keep_dev : nullptr;
+    c->exported_k = kept ? k : -1;
+    return GPGA_OK;
+}
+
 namespace {
 
 // Second half of a shard's iteration, whole or in two parts (see ShardPart).

@@ -154,6 +154,75 @@ __global__ void __launch_bounds__(kShardBlock) shard_export_sums_kernel(const Sh
     o[0] = s0; o[1] = s1; o[2] = s2; o[3] = s3;
 }
 
+// ---- export with the send fused in ---------------------------------------------------------------
+// The same rows, stored straight to where their receivers will read them instead of (or besides) a
+// send buffer: row t goes to dst0 row t when t < split, else to dst1 row t - split (ring: split = 1,
+// the first row to the shard above, the last one to the shard below; exponential graph: all rows to
+// the one partner shard).  dst0 / dst1 may be another device's memory mapped for peer access: the
+// kernel only stores there, 16 bytes per thread and row, adjacent threads adjacent addresses.
+// `keep` (may be null) also gets every row, for a step that averages the exported rows themselves.
+template <int NOISE, bool VEC>
+__global__ void __launch_bounds__(kShardBlock) shard_export_rows_to_kernel(const ShardParams p, float* __restrict__ keep,
+                                                                            float* __restrict__ dst0,
+                                                                            float* __restrict__ dst1, int split,
+                                                                            int first, int stride, int rows)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.Q) return;
+    const Group g = group_of(p, q);
+    auto put = [&](int t, float4 y) {
+        if (t < split) store_dense(dst0, t, p, g, y);
+        else store_dense(dst1, t - split, p, g, y);
+        if (keep) store_dense(keep, t, p, g, y);
+    };
+    int t = 0;
+    for (; t + kRowsInFlight <= rows; t += kRowsInFlight) {
+        RowIn r[kRowsInFlight];
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) r[u] = load_row<VEC>(p, g, first + (t + u) * stride);
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) put(t + u, finish_row<NOISE>(p, g, r[u], first + (t + u) * stride));
+    }
+    for (; t < rows; ++t) put(t, half_step_row<NOISE, VEC>(p, g, first + t * stride));
+}
+
+// The shard's column sums, stored into every shard's gather area (its own included): an all-gather
+// done by the producer's stores.  Same sums, formed in the same order, as shard_export_sums_kernel.
+template <int NOISE, bool VEC>
+__global__ void __launch_bounds__(kShardBlock) shard_export_sums_to_kernel(const ShardParams p, const ShardSumDests dl)
+{
+    const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= p.Q) return;
+    const Group g = group_of(p, q);
+    double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+    const int n = (int)p.n;
+    int i = 0;
+    for (; i + 4 <= n; i += 4) {
+        RowIn r[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) r[u] = load_row<VEC>(p, g, i + u);
+        const float4 y0 = finish_row<NOISE>(p, g, r[0], i), y1 = finish_row<NOISE>(p, g, r[1], i + 1);
+        const float4 y2 = finish_row<NOISE>(p, g, r[2], i + 2), y3 = finish_row<NOISE>(p, g, r[3], i + 3);
+        const float4 t = add4(add4(y0, y1), add4(y2, y3));
+        s0 += (double)t.x; s1 += (double)t.y; s2 += (double)t.z; s3 += (double)t.w;
+    }
+    const int rest = n - i;
+    if (rest >= 1) {
+        float4 a = half_step_row<NOISE, VEC>(p, g, i);
+        if (rest >= 2) a = add4(a, half_step_row<NOISE, VEC>(p, g, i + 1));
+        s0 += (double)a.x; s1 += (double)a.y; s2 += (double)a.z; s3 += (double)a.w;
+    }
+    if (rest == 3) {
+        const float4 b = half_step_row<NOISE, VEC>(p, g, i + 2);
+        s0 += (double)b.x; s1 += (double)b.y; s2 += (double)b.z; s3 += (double)b.w;
+    }
+    for (int t = 0; t < dl.count; ++t) {
+        double2* o = reinterpret_cast<double2*>(dl.dst[t] + 4 * q);
+        o[0] = make_double2(s0, s1);
+        o[1] = make_double2(s2, s3);
+    }
+}
+
 // ---- step --------------------------------------------------------------------------------------
 // Ring: recv[0] = half-step of the node above local row 0, recv[1] = of the node below the last.
 // A three-row window slides down the local rows, four rows' loads in flight.
@@ -361,6 +430,21 @@ cudaError_t launch_shard_export_sums(const ShardParams& p, bool vec, double* sum
 {
     const int noise = p.grad;
     GPGA_SHARD_LAUNCH(shard_export_sums_kernel, noise, vec, p, sums);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_shard_export_rows_to(const ShardParams& p, bool vec, float* keep, float* dst0, float* dst1, int split,
+                                        int first, int stride, int rows, cudaStream_t s)
+{
+    const int noise = p.grad;
+    GPGA_SHARD_LAUNCH(shard_export_rows_to_kernel, noise, vec, p, keep, dst0, dst1, split, first, stride, rows);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_shard_export_sums_to(const ShardParams& p, bool vec, const ShardSumDests& dl, cudaStream_t s)
+{
+    const int noise = p.grad;
+    GPGA_SHARD_LAUNCH(shard_export_sums_to_kernel, noise, vec, p, dl);
     return cudaGetLastError();
 }
 

@@ -32,6 +32,17 @@ cudaError_t launch_shard_export_rows(const ShardParams& p, bool vec, float* send
                                      cudaStream_t s);
 // export: the shard's column sums of the half-step (4 Q doubles)
 cudaError_t launch_shard_export_sums(const ShardParams& p, bool vec, double* sums, cudaStream_t s);
+// export with the send fused in: row t to dst0 row t (t < split) or dst1 row t - split, and to
+// `keep` when it is not null; dst0 / dst1 may be peer-mapped memory of another device
+cudaError_t launch_shard_export_rows_to(const ShardParams& p, bool vec, float* keep, float* dst0, float* dst1, int split,
+                                        int first, int stride, int rows, cudaStream_t s);
+// export: the column sums into `count` gather areas (every shard's, possibly peer-mapped)
+constexpr int kShardMaxDirect = 32;   // shards that one kernel can store its column sums to
+struct ShardSumDests {
+    double* dst[kShardMaxDirect];
+    int count;
+};
+cudaError_t launch_shard_export_sums_to(const ShardParams& p, bool vec, const ShardSumDests& dl, cudaStream_t s);
 // Which rows a gossip step kernel writes: all of them, only those whose neighbours are all local
 // (so that they can be formed while the messages are still travelling), or only the others.
 enum ShardPart { SHARD_ALL = 0, SHARD_INTERIOR = 1, SHARD_BOUNDARY = 2 };

@@ -7,6 +7,12 @@ schedule of who sends what to whom is the library's too (`gpga_shard_plan`).  Th
 moves the messages: between shards that live in one process (`exchange_local`: one copy per
 message) or between ranks of a `torch.distributed` group (`exchange_dist`: isend / irecv for the
 gossip messages, an all-gather of the column sums for the global average; NCCL on GPUs, gloo on CPU).
+
+With the send fused into the export kernel (`gpga_shard_export_to`) nothing is moved here at all:
+the kernel stores every outgoing row, or the shard's column sums, straight into the receivers'
+buffers, and this module only works out the destination addresses (`direct_destinations`) and
+orders export and step (`run_local_direct` on one device, `run_dist_direct` over peer-mapped
+symmetric memory between the ranks of a group).
 """
 from __future__ import annotations
 
@@ -70,6 +76,17 @@ class NodeShard:
 
     def step(self, k, stream=None):
         self.g._check(B.lib().gpga_shard_step(self.g._h, k, self.recv.data_ptr(), self.g._sp(stream)))
+
+    def export_to(self, k, dests, stream=None, keep=True):
+        """First half of iteration k with the send fused in: `dests` are the device addresses
+        (`direct_destinations`) the kernel stores the outgoing messages to."""
+        arr = (C.c_void_p * len(dests))(*[int(a) for a in dests])
+        keep_ptr = self.send.data_ptr() if keep else None
+        self.g._check(B.lib().gpga_shard_export_to(self.g._h, k, keep_ptr, arr, len(dests), self.g._sp(stream)))
+
+    def step_from(self, k, recv_ptr, stream=None):
+        """Second half of iteration k from the receive area at device address `recv_ptr`."""
+        self.g._check(B.lib().gpga_shard_step(self.g._h, k, int(recv_ptr), self.g._sp(stream)))
 
     def step_interior(self, k, stream=None):
         """The rows of X^(k+1) that need nothing received (can run while the messages travel)."""
@@ -165,3 +182,58 @@ def run_dist_overlapped(shard, K, k0=0, group=None):
         shard.step_interior(k)
         main.wait_event(delivered)
         shard.step_boundary(k)
+
+
+def direct_destinations(plan, shard, shards, base_of):
+    """Where the export kernel of `shard` stores iteration k's messages (`plan` = its plan for k):
+    `base_of(s)` is the device address of shard s's receive area for this iteration.  Gossip:
+    message m lands in the area of shard send_to[m] at dst_offset[m]; global average: this shard's
+    column sums land in EVERY shard's area, in this shard's slot of the all-gather."""
+    if plan.kind == GPGA_SHARD_GLOBAL:
+        return [base_of(s) + shard * plan.gather_bytes for s in range(shards)]
+    return [base_of(plan.send_to[m]) + plan.dst_offset[m] for m in range(plan.messages)]
+
+
+def run_local_direct(shards, K, k0=0):
+    """K iterations of all shards of one process on one device and stream, no copies between them:
+    every shard's export kernel writes into the other shards' receive areas.  Two receive areas per
+    shard, used alternately by the parity of k (iteration k + 1's exports may run while another
+    shard's step of iteration k still reads its area).  Stream order puts every export of iteration
+    k before every step of iteration k."""
+    import torch
+    if not hasattr(shards[0], "recv_pair"):
+        for sh in shards:
+            sh.recv_pair = (sh.recv, torch.zeros_like(sh.recv))
+    for k in range(k0, k0 + K):
+        par = k & 1
+        for sh in shards:
+            dests = direct_destinations(sh.plan(k), sh.shard, sh.shards, lambda s: shards[s].recv_pair[par].data_ptr())
+            sh.export_to(k, dests)
+        for sh in shards:
+            sh.step_from(k, sh.recv_pair[par].data_ptr())
+
+
+def run_dist_direct(shard, K, k0=0, group=None):
+    """The same between the ranks of a torch.distributed group on several GPUs of one node: the two
+    receive areas of every rank live in symmetric memory (mapped into every peer), the export kernel
+    stores through the peers' addresses, and a barrier of the symmetric-memory group, in stream order
+    between export and step, tells every rank that its senders' kernels have completed.  No library
+    call moves data; nothing loads from a peer's memory."""
+    import torch.distributed as dist
+    import torch.distributed._symmetric_memory as symm
+    import torch
+    group = group or dist.group.WORLD
+    nbytes = shard.recv.numel()
+    area = (nbytes + 255) // 256 * 256
+    buf = symm.empty(2 * area, dtype=torch.uint8, device=shard.recv.device)
+    hdl = symm.rendezvous(buf, group.group_name)
+    bases = [int(a) for a in hdl.buffer_ptrs]
+    me = dist.get_rank(group)
+    for k in range(k0, k0 + K):
+        off = (k & 1) * area
+        dests = direct_destinations(shard.plan(k), me, shard.shards, lambda s: bases[s] + off)
+        shard.export_to(k, dests)
+        hdl.barrier()
+        shard.step_from(k, bases[me] + off)
+    hdl.barrier()   # nobody frees its area while a peer's last export may still be storing to it
+    torch.cuda.synchronize()

@@ -28,7 +28,14 @@ def _sharded_run(n, d, topo, H, gamma, sigma, X0, B, shards, K, col0=0, check_fi
         xa = torch.from_numpy(np.ascontiguousarray(X0[rows])).cuda()
         sh.bind(xa, torch.empty_like(xa), torch.from_numpy(np.ascontiguousarray(B[rows])).cuda())
         parts.append(sh)
-    for k in range(K):
+    if mode == "direct":   # the send fused into the export kernel: no copy between the shards at all
+        if check_first is not None:
+            ns.run_local_direct(parts, 1)
+            check_first(np.concatenate([sh.get_x().cpu().numpy() for sh in parts]))
+            ns.run_local_direct(parts, K - 1, k0=1)
+        else:
+            ns.run_local_direct(parts, K)
+    for k in range(K if mode != "direct" else 0):
         for sh in parts:
             sh.export(k)
         if mode == "whole":
@@ -103,6 +110,60 @@ def test_two_part_step_equals_the_whole_step(topo, H, n, shards, d, mode):
     got = _sharded_run(n, d, topo, H, gamma, sigma, X0, B, shards, K, mode=mode)
     assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), float(np.abs(got - want).max())
     g.close()
+
+
+@pytest.mark.parametrize("d", [4104, 19456, 1031])
+@pytest.mark.parametrize("topo,H,n,shards", [("ring", 4, 16, 2), ("ring", 0, 16, 4), ("ring", 3, 8, 1), ("ring", 5, 24, 3),
+                                             ("exp", 3, 16, 2), ("exp", 0, 16, 4), ("exp", 5, 32, 4), ("exp", 4, 8, 1),
+                                             ("exp", 0, 8, 2)])
+def test_export_with_the_send_fused_in_is_bit_identical_to_the_unsharded_run(topo, H, n, shards, d):
+    """gpga_shard_export_to: the export kernel stores every outgoing row, and the column sums of a
+    global average, straight into the other shards' receive areas (two per shard, alternating with
+    the parity of k); no copy is made between the shards.  Against the unsharded run bit for bit and
+    against the oracle within tolerance, first iteration and whole run."""
+    gamma, sigma, K = 0.1, 0.3, 13
+    X0, B = quadratic_inputs(n, d, SEED + n + d + 2, x0="per_node")
+    g, p = make_quadratic(n, d, topo, H, gamma, SEED, sigma, X0, B)
+    first = {}
+    got = _sharded_run(n, d, topo, H, gamma, sigma, X0, B, shards, K, check_first=lambda x: first.update(x=x),
+                       mode="direct")
+    g.step(0)
+    assert np.array_equal(first["x"].view(np.uint32), g.get_x().cpu().numpy().view(np.uint32))
+    ok, worst = close(first["x"], o.step(p, X0, 0), TOL_STEP)
+    assert ok, worst
+    for k in range(1, K):
+        g.step(k)
+    want = g.get_x().cpu().numpy()
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), float(np.abs(got - want).max())
+    ok, worst = close(got, o.run(p, X0, 0, K), TOL_RUN)
+    assert ok, worst
+    g.close()
+
+
+def test_fused_export_argument_checks():
+    import ctypes as C
+    import torch
+    L = pkg.lib()
+    n, d, shards = 8, 64, 2
+    sh = ns.NodeShard(n, d, TOPO["ring"][0], 4, 0.1, SEED, shards, 0)
+    X0, B = quadratic_inputs(n // shards, d, 3, x0="per_node")
+    xa = torch.from_numpy(X0).cuda()
+    sh.bind(xa, torch.empty_like(xa), torch.from_numpy(B).cuda())
+    good = sh.recv.data_ptr()
+    two = (C.c_void_p * 2)(good, good + 512)
+    one = (C.c_void_p * 1)(good)
+    odd = (C.c_void_p * 2)(good, good + 4)
+    null = (C.c_void_p * 2)(good, None)
+    h = sh.g._h
+    assert L.gpga_shard_export_to(h, 0, None, one, 1, None) == pkg.GPGA_ERR_INVALID_ARG      # the ring sends two messages
+    assert L.gpga_shard_export_to(h, 0, None, odd, 2, None) == pkg.GPGA_ERR_INVALID_ARG      # misaligned destination
+    assert L.gpga_shard_export_to(h, 0, None, null, 2, None) == pkg.GPGA_ERR_INVALID_ARG     # NULL destination
+    assert L.gpga_shard_export_to(h, 0, None, None, 2, None) == pkg.GPGA_ERR_INVALID_ARG
+    assert L.gpga_shard_export_to(h, 3, None, one, 1, None) == pkg.GPGA_ERR_INVALID_ARG      # k = 3, H = 4: one slot per shard
+    assert L.gpga_shard_export_to(h, 0, None, two, 2, None) == pkg.GPGA_OK
+    assert L.gpga_shard_export_to(h, 3, None, two, 2, None) == pkg.GPGA_OK
+    torch.cuda.synchronize()
+    sh.close()
 
 
 def test_sharded_run_with_a_column_offset_and_no_noise():
@@ -201,6 +262,12 @@ def test_logistic_objective_sharded_by_nodes(topo, H, n, shards, m, d, batch):
                   labels=y.astype(np.float64), l2=l2, batch=batch)
     ok, worst = close(got, o.run(p, X0, 0, K), TOL_RUN)
     assert ok, worst
+    # K more iterations with the send fused into the export kernel, against K more single steps
+    ns.run_local_direct(parts, K, k0=K)
+    for k in range(K, 2 * K):
+        g.step(k)
+    got, want = np.concatenate([sh.get_x().cpu().numpy() for sh in parts]), g.get_x().cpu().numpy()
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), float(np.abs(got - want).max())
     for sh in parts:
         sh.close()
     g.close()

@@ -197,3 +197,39 @@ def test_plan_is_consistent_for_every_shape():
                 assert ((g + 1) * n_l) % n == ((g + 1) % shards) * n_l
             glob = ns.shard_plan(pkg.GPGA_TOPO_RING, 4, n, shards, 0, d, 3)
             assert glob.kind == ns.GPGA_SHARD_GLOBAL and glob.gather_bytes == (d + 3) // 4 * 4 * 8
+
+
+def test_direct_destinations_land_where_the_copies_land():
+    """Host logic of the fused export (the kernel stores its messages straight into the receivers'
+    areas): in a flat fake address space, writing every shard's send buffer to the addresses
+    direct_destinations gives must leave every receive area exactly as exchange_local's copies do --
+    ring, every hop of the exponential graph, the all-gather of a global average."""
+    import torch
+    d = 10
+    for topo, H, n, shards in (("ring", 4, 16, 4), ("ring", 0, 8, 2), ("ring", 3, 4, 1), ("exp", 3, 16, 2), ("exp", 0, 32, 8),
+                               ("exp", 5, 16, 4), ("exp", 2, 4, 1)):
+        rng = np.random.default_rng(n + shards)
+        X0, B = quadratic_inputs(n, d, 3, x0="per_node")
+        parts = [OracleShard(n, d, topo, H, 0.2, 0.1, 5, shards, s, X0, B) for s in range(shards)]
+        area = parts[0].recv.numel()
+        for k in range(12):
+            for sh in parts:   # messages with contents that identify (shard, k, byte)
+                sh.send[:] = torch.from_numpy(rng.integers(0, 256, area, dtype=np.uint8))
+                sh.recv[:] = 0
+            ns.exchange_local(parts, k)
+            memory = np.zeros(shards * area, dtype=np.uint8)
+            for sh in parts:
+                plan = sh.plan(k)
+                dests = ns.direct_destinations(plan, sh.shard, shards, lambda s: s * area)
+                if plan.kind == ns.GPGA_SHARD_GLOBAL:
+                    assert len(dests) == shards
+                    for a in dests:
+                        memory[a:a + plan.gather_bytes] = sh.send.numpy()[:plan.gather_bytes]
+                else:
+                    assert len(dests) == plan.messages
+                    for m, a in enumerate(dests):
+                        lo, nb = plan.send_offset[m], plan.bytes[m]
+                        assert a % 16 == 0 and a // area == plan.send_to[m] and a % area + nb <= area
+                        memory[a:a + nb] = sh.send.numpy()[lo:lo + nb]
+            for s, sh in enumerate(parts):
+                assert np.array_equal(memory[s * area:(s + 1) * area], sh.recv.numpy()), (topo, H, n, shards, k, s)
