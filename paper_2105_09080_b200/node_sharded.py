@@ -194,12 +194,13 @@ def direct_destinations(plan, shard, shards, base_of):
     return [base_of(plan.send_to[m]) + plan.dst_offset[m] for m in range(plan.messages)]
 
 
-def run_local_direct(shards, K, k0=0):
+def run_local_direct(shards, K, k0=0, keep=True):
     """K iterations of all shards of one process on one device and stream, no copies between them:
     every shard's export kernel writes into the other shards' receive areas.  Two receive areas per
     shard, used alternately by the parity of k (iteration k + 1's exports may run while another
     shard's step of iteration k still reads its area).  Stream order puts every export of iteration
-    k before every step of iteration k."""
+    k before every step of iteration k.  keep=False: no copy of the exported rows is kept for the
+    shard's own step (it then forms its half-step again when every row was exported)."""
     import torch
     if not hasattr(shards[0], "recv_pair"):
         for sh in shards:
@@ -208,7 +209,7 @@ def run_local_direct(shards, K, k0=0):
         par = k & 1
         for sh in shards:
             dests = direct_destinations(sh.plan(k), sh.shard, sh.shards, lambda s: shards[s].recv_pair[par].data_ptr())
-            sh.export_to(k, dests)
+            sh.export_to(k, dests, keep=keep)
         for sh in shards:
             sh.step_from(k, sh.recv_pair[par].data_ptr())
 

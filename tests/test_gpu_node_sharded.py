@@ -140,6 +140,31 @@ def test_export_with_the_send_fused_in_is_bit_identical_to_the_unsharded_run(top
     g.close()
 
 
+@pytest.mark.parametrize("n,shards,d", [(16, 4, 4104), (32, 2, 1031), (8, 2, 19456)])
+def test_fused_export_without_a_kept_copy(n, shards, d):
+    """With no keep buffer the step of a hop that exported every local row forms the half-step again
+    instead of reading the exported rows: same result, bit for bit."""
+    import torch
+    gamma, sigma, K, H = 0.1, 0.3, 9, 0
+    X0, B = quadratic_inputs(n, d, SEED + n + d + 3, x0="per_node")
+    g, _ = make_quadratic(n, d, "exp", H, gamma, SEED, sigma, X0, B)
+    for k in range(K):
+        g.step(k)
+    want = g.get_x().cpu().numpy()
+    n_l, parts = n // shards, []
+    for s in range(shards):
+        sh = ns.NodeShard(n, d, TOPO["exp"][0], H, gamma, SEED, shards, s, sigma=sigma)
+        xa = torch.from_numpy(np.ascontiguousarray(X0[s * n_l:(s + 1) * n_l])).cuda()
+        sh.bind(xa, torch.empty_like(xa), torch.from_numpy(np.ascontiguousarray(B[s * n_l:(s + 1) * n_l])).cuda())
+        parts.append(sh)
+    ns.run_local_direct(parts, K, keep=False)
+    got = np.concatenate([sh.get_x().cpu().numpy() for sh in parts])
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), float(np.abs(got - want).max())
+    for sh in parts:
+        sh.close()
+    g.close()
+
+
 def test_fused_export_argument_checks():
     import ctypes as C
     import torch
