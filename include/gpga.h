@@ -253,6 +253,17 @@ int32_t gpga_run_adaptive(gpga_t* ctx, int64_t K, int64_t H_init, int64_t warmup
                           int64_t* num_periods_host);
 
 /*
+ * Algorithm 2's period rule by itself (host arithmetic only), for a caller that drives the
+ * iterations itself -- the node-sharded deployment, where the mean loss F is the all-reduced mean of
+ * the shards' gpga_mean_loss values.  Called at a global-average iteration k with that iteration's
+ * F: while k < warmup_iters, F_init <- (F_init + F) / 2 and the period stays; afterwards
+ * H <- ceil(F_init / F * H_init), at least 1 (left as it is when F <= 0 or the ratio is not finite).
+ * Errors: INVALID_ARG for NULL pointers, k < 0, warmup_iters < 0 or H_init < 1.
+ */
+int32_t gpga_aga_update(int64_t k, int64_t warmup_iters, int64_t H_init, double F, double* F_init_inout,
+                        int64_t* H_inout);
+
+/*
  * Node sharding: the deployment of Section 3, where the n nodes live on several devices, a gossip
  * step exchanges the half-step vectors x^(k+1/2) of neighbouring nodes and the global average is
  * an All-Reduce ("All-Reduce v.s. multiple Gossips"); the appendix's implementation details: on

@@ -70,6 +70,7 @@ SIGNATURES = {
     "gpga_set_k": (_i32, [_P, _i64]),
     "gpga_set_gamma": (_i32, [_P, _f32]),
     "gpga_set_period": (_i32, [_P, _i64]),
+    "gpga_aga_update": (_i32, [_i64, _i64, _i64, C.c_double, C.POINTER(C.c_double), C.POINTER(_i64)]),
     "gpga_launch_count": (_i64, [_P]),
     "gpga_last_error": (C.c_char_p, [_P]),
     "gpga_destroy": (_i32, [_P]),

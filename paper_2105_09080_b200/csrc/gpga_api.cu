@@ -1033,6 +1033,19 @@ int32_t gpga_shard_step_boundary(gpga_t* c, int64_t k, const void* recv_dev, voi
     return shard_step_part(c, k, recv_dev, SHARD_BOUNDARY, static_cast<cudaStream_t>(stream));
 }
 
+int32_t gpga_aga_update(int64_t k, int64_t warmup_iters, int64_t H_init, double F, double* F_init_inout, int64_t* H_inout)
+{
+    if (!F_init_inout || !H_inout) return fail(nullptr, GPGA_ERR_INVALID_ARG, "F_init_inout and H_inout must not be NULL");
+    if (k < 0 || warmup_iters < 0 || H_init < 1) return fail(nullptr, GPGA_ERR_INVALID_ARG, "need k >= 0, warmup_iters >= 0, H_init >= 1");
+    if (k < warmup_iters) {
+        *F_init_inout = 0.5 * (*F_init_inout + F);
+    } else if (F > 0.0 && std::isfinite(*F_init_inout / F)) {
+        const double h = std::ceil(*F_init_inout / F * (double)H_init);
+        *H_inout = h < 1.0 ? 1 : (h > 9.0e15 ? (int64_t)9.0e15 : (int64_t)h);
+    }
+    return GPGA_OK;
+}
+
 int32_t gpga_run_adaptive(gpga_t* c, int64_t K, int64_t H_init, int64_t warmup_iters, void* stream,
                           int64_t* periods_host, int64_t max_periods, int64_t* num_periods_host)
 {
@@ -1061,12 +1074,7 @@ int32_t gpga_run_adaptive(gpga_t* c, int64_t K, int64_t H_init, int64_t warmup_i
             if (periods_host && periods < max_periods) periods_host[periods] = H;
             ++periods;
             C = 0;
-            if (k < warmup_iters) {
-                F_init = 0.5 * (F_init + F);
-            } else if (F > 0.0 && std::isfinite(F_init / F)) {
-                const double h = std::ceil(F_init / F * (double)H_init);
-                H = h < 1.0 ? 1 : (h > 9.0e15 ? (int64_t)9.0e15 : (int64_t)h);
-            }
+            gpga_aga_update(k, warmup_iters, H_init, F, &F_init, &H);
         }
     }
     if (num_periods_host) *num_periods_host = periods;

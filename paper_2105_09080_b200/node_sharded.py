@@ -96,6 +96,15 @@ class NodeShard:
         """The remaining rows, from the receive buffer; completes iteration k."""
         self.g._check(B.lib().gpga_shard_step_boundary(self.g._h, k, self.recv.data_ptr(), self.g._sp(stream)))
 
+    def set_period(self, H):
+        """Averaging period of the schedule from now on (Gossip-AGA drives it iteration by iteration)."""
+        self.H = H
+        self.g.set_period(H)
+
+    def mean_loss(self):
+        """Mean over this shard's nodes of the local loss at their own iterates."""
+        return self.g.mean_loss()
+
     def get_x(self):
         return self.g.get_x()
 
@@ -238,3 +247,58 @@ def run_dist_direct(shard, K, k0=0, group=None):
         shard.step_from(k, bases[me] + off)
     hdl.barrier()   # nobody frees its area while a peer's last export may still be storing to it
     torch.cuda.synchronize()
+
+
+def aga_update(k, warmup_iters, H_init, F, F_init, H):
+    """Algorithm 2's period rule (the library's host arithmetic): returns (F_init, H) after a
+    global-average iteration k whose mean loss was F."""
+    fi, h = C.c_double(F_init), C.c_int64(H)
+    st = B.lib().gpga_aga_update(int(k), int(warmup_iters), int(H_init), float(F), C.byref(fi), C.byref(h))
+    if st != B.GPGA_OK:
+        raise B.GpgaError(st, B.lib().gpga_last_error(None).decode())
+    return fi.value, h.value
+
+
+def run_adaptive(shards, K, H_init, warmup_iters, exchange, mean_of_losses, k0=0):
+    """Gossip-AGA (Algorithm 2) on node shards: a counter C counts iterations since the last global
+    average; when it reaches the period H the iteration is a global average, the mean loss F over
+    ALL nodes is taken at that iteration's state (`mean_of_losses(local mean losses)`: the
+    all-reduce of Algorithm 2), and the period is updated by `aga_update`.  `shards`: the shards this
+    process drives; `exchange(k)` delivers iteration k's messages.  Returns the period lengths."""
+    H, count, F_init, periods = H_init, 0, 0.0, []
+    for k in range(k0, k0 + K):
+        count += 1
+        glob = count == H
+        F = mean_of_losses([sh.mean_loss() for sh in shards]) if glob else 0.0
+        for sh in shards:
+            sh.set_period(1 if glob else 0)     # this iteration: a global average, or a gossip step
+        for sh in shards:
+            sh.export(k)
+        exchange(k)
+        for sh in shards:
+            sh.step(k)
+        if glob:
+            periods.append(H)
+            count = 0
+            F_init, H = aga_update(k, warmup_iters, H_init, F, F_init, H)
+    return periods
+
+
+def run_local_adaptive(shards, K, H_init, warmup_iters, k0=0):
+    """Gossip-AGA over all shards of one process (equal shard sizes: the mean of the shard means)."""
+    return run_adaptive(shards, K, H_init, warmup_iters, lambda k: exchange_local(shards, k),
+                        lambda losses: sum(losses) / len(losses), k0)
+
+
+def run_dist_adaptive(shard, K, H_init, warmup_iters, k0=0, group=None):
+    """Gossip-AGA with one shard per rank: the mean loss is all-reduced over the group (the one scalar
+    all-reduce of Algorithm 2), so every rank takes the same period sequence."""
+    import torch
+    import torch.distributed as dist
+
+    def mean_of_losses(losses):
+        t = torch.tensor([losses[0]], dtype=torch.float64, device=shard.recv.device)
+        dist.all_reduce(t, group=group)
+        return float(t.item()) / dist.get_world_size(group)
+
+    return run_adaptive([shard], K, H_init, warmup_iters, lambda k: exchange_dist(shard, k, group), mean_of_losses, k0)

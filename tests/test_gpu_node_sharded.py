@@ -165,6 +165,47 @@ def test_fused_export_without_a_kept_copy(n, shards, d):
     g.close()
 
 
+@pytest.mark.parametrize("topo,n,shards,d", [("ring", 8, 2, 4096), ("exp", 16, 4, 1031), ("ring", 16, 4, 19456)])
+def test_adaptive_period_on_shards_equals_the_unsharded_adaptive_run(topo, n, shards, d):
+    """Gossip-AGA (Algorithm 2) on node shards -- the mean loss is the mean of the shards' mean
+    losses, the period rule is the library's gpga_aga_update -- takes the period sequence of the
+    unsharded gpga_run_adaptive and of the loop driven by the oracle, and ends in the same state."""
+    import torch
+    gamma, sigma, K, H_init, warm = 0.1, 0.05, 60, 2, 6
+    X0, B = quadratic_inputs(n, d, SEED + 5, x0="shared", x0_std=3.0)
+    g, p = make_quadratic(n, d, topo, 0, gamma, SEED, sigma, X0, B)
+    want_periods = g.run_adaptive(K, H_init, warm)
+    want = g.get_x().cpu().numpy()
+    n_l, parts = n // shards, []
+    for s in range(shards):
+        sh = ns.NodeShard(n, d, TOPO[topo][0], 0, gamma, SEED, shards, s, sigma=sigma)
+        xa = torch.from_numpy(np.ascontiguousarray(X0[s * n_l:(s + 1) * n_l])).cuda()
+        sh.bind(xa, torch.empty_like(xa), torch.from_numpy(np.ascontiguousarray(B[s * n_l:(s + 1) * n_l])).cuda())
+        parts.append(sh)
+    periods = ns.run_local_adaptive(parts, K, H_init, warm)
+    assert periods == want_periods and len(set(periods)) > 1
+    got = np.concatenate([sh.get_x().cpu().numpy() for sh in parts])
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), float(np.abs(got - want).max())
+    # the oracle's loop
+    X, H, count, F_init, oracle_periods = X0, H_init, 0, 0.0, []
+    for k in range(K):
+        count += 1
+        glob = count == H
+        F = o.quadratic_mean_loss(X, B) if glob else 0.0
+        p.H = 1 if glob else 0
+        X = o.step(p, X, k)
+        if glob:
+            oracle_periods.append(H)
+            count = 0
+            F_init, H = o.aga_update(k, warm, H_init, F, F_init, H)
+    assert periods == oracle_periods
+    ok, worst = close(got, X, TOL_RUN)
+    assert ok, worst
+    for sh in parts:
+        sh.close()
+    g.close()
+
+
 def test_fused_export_argument_checks():
     import ctypes as C
     import torch

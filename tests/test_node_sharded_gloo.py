@@ -38,6 +38,12 @@ class OracleShard:
     def plan(self, k):
         return ns.shard_plan(self.topology, self.H, self.n_total, self.shards, self.shard, self.d, k)
 
+    def set_period(self, H):
+        self.H = H
+
+    def mean_loss(self):
+        return o.quadratic_mean_loss(self.X, self.B)
+
     def _half_step(self, k):
         """fp64 half-step of the local rows: the rows sit at their global positions of a full-height
         matrix so that the oracle keys the noise by the global node index."""
@@ -94,6 +100,41 @@ def _free_port():
     port = s.getsockname()[1]
     s.close()
     return port
+
+
+def _oracle_adaptive(topo, n, d, K, H_init, warm, gamma, sigma, seed, X0, B):
+    """Algorithm 2 driven by the oracle on the unsharded problem: (periods, X^(K))."""
+    p = o.Problem(TOPOLOGY[topo][1], 0, gamma, seed, sigma=sigma, data=B)
+    X, H, count, F_init, periods = X0, H_init, 0, 0.0, []
+    for k in range(K):
+        count += 1
+        glob = count == H
+        F = o.quadratic_mean_loss(X, B) if glob else 0.0
+        p.H = 1 if glob else 0
+        X = o.step(p, X, k)
+        if glob:
+            periods.append(H)
+            count = 0
+            F_init, H = o.aga_update(k, warm, H_init, F, F_init, H)
+    return periods, X
+
+
+def _adaptive_worker(rank, world, port, topo, n, d, K, H_init, warm, out_dir):
+    import torch.distributed as dist
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    X0, B = quadratic_inputs(n, d, 7, x0="shared", x0_std=3.0)
+    shard = OracleShard(n, d, topo, 0, 0.1, 0.05, 11, world, rank, X0, B)
+    periods = ns.run_dist_adaptive(shard, K, H_init, warm)
+    gathered = [None] * world
+    dist.all_gather_object(gathered, (rank, shard.X, periods))
+    if rank == 0:
+        assert all(g[2] == periods for g in gathered)       # every rank took the same periods
+        np.save(os.path.join(out_dir, "full.npy"), np.concatenate([x for _, x, _ in sorted(gathered, key=lambda t: t[0])]))
+        np.save(os.path.join(out_dir, "periods.npy"), np.array(periods, dtype=np.int64))
+    dist.barrier()
+    dist.destroy_process_group()
 
 
 def _worker(rank, world, port, topo, H, n, d, K, out_dir, tags=True):
@@ -233,3 +274,45 @@ def test_direct_destinations_land_where_the_copies_land():
                         memory[a:a + nb] = sh.send.numpy()[lo:lo + nb]
             for s, sh in enumerate(parts):
                 assert np.array_equal(memory[s * area:(s + 1) * area], sh.recv.numpy()), (topo, H, n, shards, k, s)
+
+
+def test_library_period_rule_equals_the_oracles():
+    """gpga_aga_update (host arithmetic of the library) against the oracle's Algorithm 2 rule wherever
+    the rule is defined (F > 0, F_init > 0); the library's guards for the degenerate cases apart."""
+    rng = np.random.default_rng(4)
+    for _ in range(2000):
+        k, warm, H_init = int(rng.integers(0, 50)), int(rng.integers(0, 30)), int(rng.integers(1, 9))
+        F = float(rng.choice([1e-9, rng.uniform(1e-3, 10.0)]))
+        F_init, H = float(rng.uniform(1e-3, 10.0)), int(rng.integers(1, 40))
+        assert ns.aga_update(k, warm, H_init, F, F_init, H) == o.aga_update(k, warm, H_init, F, F_init, H)
+    assert ns.aga_update(9, 5, 4, 0.0, 2.0, 7) == (2.0, 7)         # F = 0: the ratio is undefined, the period stays
+    assert ns.aga_update(9, 5, 4, 1.0, 0.0, 7) == (0.0, 1)         # ceil(0) = 0: a period is at least 1
+    assert ns.aga_update(9, 5, 4, 1e-9, 1e10, 7)[1] == int(9.0e15)       # beyond int64: clamped
+    assert ns.aga_update(9, 5, 4, 1e-300, 1e300, 7)[1] == 7            # an infinite ratio: the period stays
+    assert pkg.lib().gpga_aga_update(0, 0, 0, 1.0, None, None) == pkg.GPGA_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("topo,n,shards", [("ring", 16, 4), ("exp", 16, 2), ("ring", 8, 1)])
+def test_adaptive_period_on_shards_of_one_process(topo, n, shards):
+    """Gossip-AGA on node shards (the mean loss is the mean of the shards' mean losses): the period
+    sequence and the final state equal those of Algorithm 2 driven by the oracle on the whole problem."""
+    d, K, H_init, warm = 12, 60, 2, 6
+    X0, B = quadratic_inputs(n, d, 7, x0="shared", x0_std=3.0)
+    parts = [OracleShard(n, d, topo, 0, 0.1, 0.05, 11, shards, s, X0, B) for s in range(shards)]
+    periods = ns.run_local_adaptive(parts, K, H_init, warm)
+    want_periods, want = _oracle_adaptive(topo, n, d, K, H_init, warm, 0.1, 0.05, 11, X0, B)
+    assert periods == want_periods and len(set(periods)) > 1 and periods[-1] > periods[0]
+    got = np.concatenate([sh.X for sh in parts])
+    assert np.abs(got - want).max() <= 2e-6 * (1 + np.abs(want).max())
+
+
+def test_adaptive_period_across_ranks(tmp_path):
+    """The same with one shard per gloo rank: the loss is all-reduced, every rank takes the same periods."""
+    import torch.multiprocessing as mp
+    topo, n, d, K, H_init, warm, world = "ring", 8, 12, 40, 2, 6, 2
+    mp.spawn(_adaptive_worker, args=(world, _free_port(), topo, n, d, K, H_init, warm, str(tmp_path)), nprocs=world, join=True)
+    X0, B = quadratic_inputs(n, d, 7, x0="shared", x0_std=3.0)
+    want_periods, want = _oracle_adaptive(topo, n, d, K, H_init, warm, 0.1, 0.05, 11, X0, B)
+    assert np.load(tmp_path / "periods.npy").tolist() == want_periods
+    got = np.load(tmp_path / "full.npy")
+    assert np.abs(got - want).max() <= 2e-6 * (1 + np.abs(want).max())
