@@ -572,12 +572,12 @@ def run_ours(args):
                  "note": "includes the result read-back and stream synchronisation",
                  "launches": g.launch_count() - launches_c}
 
-    # one gpga_run call over the configuration's own run length (at least 32 iterations): for
-    # n <= 256 and runs that long it advances many iterations per launch with the cells on chip, so
-    # its rate is not tied to 12 bytes per update
+    # one gpga_run call over the configuration's own run length: for n <= 256 and runs of 8 or more
+    # iterations it advances many iterations per launch with the cells on chip, so its rate is not
+    # tied to 12 bytes per update
     run_info = None
     if not resident:
-        K_run = max(w["K"], 32)
+        K_run = max(w["K"], 8)
         barrier()
         r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         launches_r = g.launch_count()

@@ -227,12 +227,19 @@ int32_t do_step(gpga_ctx* c, int64_t k, bool global, cudaStream_t s, bool after_
 //    size: there the arithmetic bound (7.6-7.8e11 updates/s measured at n = 16 and 64, 6.5e11 at
 //    n = 256) is above what the row-streaming kernels reach from HBM (at most 5.6e11), also when
 //    every iteration is a global average (H = 1: 2.90 against 3.05-3.16 ms at n = 64, d = 25,557,032;
-//    8.55 against 10.18 ms at n = 16, d = 335,141,888), and the one extra pass over the state is
-//    amortised.  Wider n would go through the several-cells-per-thread kernel, which is far slower.
-// A launch is kept to about half a second of work.
+//    8.55 against 10.18 ms at n = 16, d = 335,141,888), and the launch's fixed cost is amortised: it
+//    loads and stores the state once and dispatches one small block per strip (10.5 M blocks, about
+//    25 ms, at n = 16, d = 335,141,888).  Whole calls measured, single steps against one launch:
+//    n = 16, d = 335,141,888: K = 4: 39.0 / 38.8 ms, 8: 79.6 / 64.9, 20: 198.8 / 145.2; n = 64,
+//    d = 25,557,032: K = 4: 12.0 / 13.7, 6: 18.3 / 15.9, 20: 62.2 / 44.5; n = 128, d = 2^20: K = 6:
+//    1.65 / 2.04, 8: 2.17 / 2.11, 20: 5.48 / 3.94; n = 256, d = 786,432: K = 6: 2.36 / 2.41, 8: 3.17 /
+//    3.09, 20: 7.93 / 6.64 -- one launch wins from 8 iterations on at every n.
+//    Wider n would go through the several-cells-per-thread kernel, which is far slower.
+// A launch is kept to about half a second of work; a longer run is cut into launches of equal length
+// (a short last launch would pay the fixed cost for a few iterations).
 constexpr int64_t kFusedStateBytes = 64ll << 20;
 constexpr int64_t kFusedSteps = 1024;
-constexpr int64_t kFusedWideNodes = 256, kFusedMinSteps = 32;
+constexpr int64_t kFusedWideNodes = 256, kFusedMinSteps = 8;
 constexpr double kFusedUpdatesPerLaunch = 2.75e11;
 
 // Logistic objective, narrow state: many iterations per launch with x_i resident on chip (a pair of
@@ -317,8 +324,10 @@ int32_t run_steps(gpga_ctx* c, int64_t K, cudaStream_t s)
         }
         return GPGA_OK;
     }
+    int64_t launches_left = (K + per_launch - 1) / per_launch;
     while (c->k < k_end) {
-        const int64_t steps = (k_end - c->k < per_launch) ? k_end - c->k : per_launch;
+        const int64_t steps = (k_end - c->k + launches_left - 1) / launches_left;
+        --launches_left;
         StepParams p;
         p.x = c->x[c->cur];
         p.out = c->x[c->cur ^ 1];

@@ -271,7 +271,7 @@ def test_partly_overlapping_state_buffers_are_rejected():
                                               ("ring", 16, 1_200_000, 1, True)])
 def test_long_runs_with_few_nodes_take_the_multi_iteration_launch_at_any_size(topo, n, d, H, fused):
     """Above 64 MB of state gpga_run still advances many iterations per launch when n <= 256 (one cell
-    per thread) and the run has at least 32 iterations (the on-chip arithmetic is then faster than
+    per thread) and the run has at least 8 iterations (the on-chip arithmetic is then faster than
     streaming the state from HBM every iteration, also with a global average every iteration); wider
     n keeps one launch per iteration.  Either way the result is bit-identical to stepping, and within
     tolerance of the oracle on a slice of columns."""
@@ -287,8 +287,10 @@ def test_long_runs_with_few_nodes_take_the_multi_iteration_launch_at_any_size(to
         g2.step(k)
     assert np.array_equal(got, g2.get_x().cpu().numpy())
     g3, _ = make_quadratic(n, d, topo, H, 0.05, 29, 0.1, X0, B)
-    g3.run(K - 1)                      # fewer than 32 left after the first call: falls back to stepping
-    g3.run(1)
+    g3.run(K - 7)                      # fewer than 8 left after the first call: falls back to stepping
+    l0 = g3.launch_count()
+    g3.run(7)
+    assert g3.launch_count() - l0 == (7 if 12 * n * d > 64 << 20 else 1)
     assert np.array_equal(got, g3.get_x().cpu().numpy())
     c0, w = (d // 2) // 4 * 4, 2048
     p = o.Problem(TOPO[topo][1], H, 0.05, 29, sigma=0.1, data=np.ascontiguousarray(B[:, c0:c0 + w]), col0=c0)

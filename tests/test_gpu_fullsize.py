@@ -54,7 +54,7 @@ def _oracle_xi_of_device_state(x, d, chunk=1 << 20):
 
 
 def _run_case(bufs, n, d, topo, H, gamma, sigma, K, x0_kind, x0_std, b_shift, offs, one_step_ks, ld=None,
-              check_xi=False):
+              check_xi=False, stepped=False):
     xa, xb, b, scratch = bufs
     ld = ld or d
     xa, xb, b = (t.view(-1)[:n * ld].view(n, ld) for t in (xa, xb, b))
@@ -80,8 +80,16 @@ def _run_case(bufs, n, d, topo, H, gamma, sigma, K, x0_kind, x0_std, b_shift, of
             ok, worst = close(_gpu_block(x, c0, width(c0)), o.step(p, X0, k), TOL_STEP)
             assert ok, (topo, H, "k", k, "col0", c0, worst)
     # the K-iteration run
+    # (stepped: one launch of the row-streaming kernels per iteration, the loop the benchmark times;
+    # otherwise gpga_run, which takes a run of 8 or more iterations through the multi-iteration launch)
     g.init_from_seed(x0_kind, x0_std, b_shift)
-    g.run(K)
+    launches0 = g.launch_count()
+    if stepped:
+        for k in range(K):
+            g.step(k)
+        assert g.launch_count() - launches0 == K
+    else:
+        g.run(K)
     x = g.get_x()
     for c0 in offs:
         X0, p = ora[c0]
@@ -118,9 +126,11 @@ def test_config_3_resnet50_sized():
             if H == 4:
                 ks = [0, 3] if topo == "ring" else [0, 1, 2, 3, 4, 5]   # hops 1..32; k=3 is global
             # K = 50 ends between global averages for H = 16 and for pure gossip
+            # (H = 4: one launch of the row-streaming kernels per iteration, the loop the benchmark times;
+            # the other periods through gpga_run's multi-iteration launch)
             _run_case((xa, xb, b, scratch), n, d, topo, H, gamma, sigma, K,
                       pkg.GPGA_X0_SHARED_NORMAL, 0.1, 0.5, offs, ks, ld=ld,
-                      check_xi=(topo, H) in (("ring", 16), ("exp", 0)))
+                      check_xi=(topo, H) in (("ring", 16), ("exp", 0)), stepped=(H == 4))
     # the dense layout (row stride d, rows not 128-byte aligned) once as well
     _run_case((xa, xb, b, scratch), n, d, "ring", 4, gamma, sigma, 8, pkg.GPGA_X0_SHARED_NORMAL, 0.1, 0.5,
               offs, [0], ld=d)
@@ -190,14 +200,16 @@ def test_config_4_bert_large_sized():
     b = torch.empty_like(xa)
     scratch = torch.empty(4 << 20, dtype=torch.uint8, device="cuda")   # >= gpga_scratch_bytes at these sizes
     offs = _blocks(d, 48, np.random.default_rng(4))
+    # the configuration's K = 20 iterations with one launch of the row-streaming kernels each (the loop the
+    # benchmark times)
     _run_case((xa, xb, b, scratch), n, d, "exp", H, gamma, sigma, K, pkg.GPGA_X0_ZERO, 1.0, 0.0,
-              offs, [0, 1, 2, 3])
+              offs, [0, 1, 2, 3], stepped=True)
     # K = 18 ends two gossip steps after a global average: a non-zero consensus distance over
     # n d > 2^32 elements, recomputed by the oracle from the downloaded state
     _run_case((xa, xb, b, scratch), n, d, "exp", H, gamma, sigma, 18, pkg.GPGA_X0_ZERO, 1.0, 0.0,
-              offs[::6], [], check_xi=True)
-    # a run of 32 iterations goes through the multi-iteration launch: 10.5 M strips of 8 column groups
-    _run_case((xa, xb, b, scratch), n, d, "exp", H, gamma, sigma, 32, pkg.GPGA_X0_ZERO, 1.0, 0.0,
+              offs[::6], [], check_xi=True, stepped=True)
+    # gpga_run takes 8 or more iterations through the multi-iteration launch: 10.5 M strips of 8 column groups
+    _run_case((xa, xb, b, scratch), n, d, "exp", H, gamma, sigma, K, pkg.GPGA_X0_ZERO, 1.0, 0.0,
               offs[::2], [])
     del xa, xb, b
     torch.cuda.empty_cache()
