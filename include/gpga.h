@@ -245,7 +245,8 @@ int32_t gpga_global_loss(gpga_t* ctx, void* stream, double* out_host);
  * global average; when C == H the step is a global average, the mean loss F of that
  * iteration's state is taken, and H is updated: F_init <- (F_init + F)/2 while
  * k < warmup_iters, afterwards H <- ceil(F_init / F * H_init).  Synchronises at each
- * global-average iteration.  periods_host (may be NULL) receives up to max_periods period
+ * global-average iteration; the gossip iterations between two of them are advanced like a gpga_run
+ * call of that length (in one launch where that is faster), with the same results as single steps.  periods_host (may be NULL) receives up to max_periods period
  * lengths in order; *num_periods_host their count.
  */
 int32_t gpga_run_adaptive(gpga_t* ctx, int64_t K, int64_t H_init, int64_t warmup_iters,

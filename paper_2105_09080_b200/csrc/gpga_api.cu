@@ -1065,26 +1065,37 @@ int32_t gpga_run_adaptive(gpga_t* c, int64_t K, int64_t H_init, int64_t warmup_i
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int64_t H = H_init, C = 0, periods = 0;
     double F_init = 0.0;
-    const int64_t k0 = c->k;
-    for (int64_t k = k0; k < k0 + K; ++k) {
-        ++C;
-        const bool global = (C == H);
+    int64_t k = c->k;
+    const int64_t k_end = k + K;
+    while (k < k_end) {
+        // the gossip iterations before the counter reaches the period, as one run (which takes the
+        // multi-iteration launches where they pay): the handle's own period is out of play meanwhile
+        int64_t gossip = H - 1 - C;
+        if (gossip > k_end - k) gossip = k_end - k;
+        if (gossip > 0) {
+            const int64_t H_handle = c->H;
+            c->H = 0;
+            st = run_steps(c, gossip, s);
+            c->H = H_handle;
+            if (st) return st;
+            C += gossip;
+            k += gossip;
+            continue;
+        }
+        // C + 1 == H: a global average; the loss of this iteration is taken at x^(k) as Algorithm 2 does
         double F = 0.0;
-        if (global) {   // loss of this iteration, taken at x^(k) as Algorithm 2 does
-            double* result = nullptr;
-            st = mean_loss_async(c, s, &result);
-            if (st) return st;
-            st = read_double(c, result, s, &F);
-            if (st) return st;
-        }
-        st = do_step(c, k, global, s);
+        double* result = nullptr;
+        st = mean_loss_async(c, s, &result);
         if (st) return st;
-        if (global) {
-            if (periods_host && periods < max_periods) periods_host[periods] = H;
-            ++periods;
-            C = 0;
-            gpga_aga_update(k, warmup_iters, H_init, F, &F_init, &H);
-        }
+        st = read_double(c, result, s, &F);
+        if (st) return st;
+        st = do_step(c, k, true, s);
+        if (st) return st;
+        if (periods_host && periods < max_periods) periods_host[periods] = H;
+        ++periods;
+        C = 0;
+        gpga_aga_update(k, warmup_iters, H_init, F, &F_init, &H);
+        ++k;
     }
     if (num_periods_host) *num_periods_host = periods;
     return GPGA_OK;

@@ -248,6 +248,36 @@ def test_config_5_logistic_sweep_full_length(c5_data, topo, H):
 
 
 # ------------------------------------------------------------------ Gossip-AGA
+def test_adaptive_run_takes_gossip_stretches_in_one_launch_and_equals_single_steps():
+    """Between two global averages Gossip-AGA's iterations are plain gossip steps; a stretch of 8 or
+    more goes through the multi-iteration launch.  Periods and state must equal those of single steps
+    driven from the host with the same rule."""
+    n, d, K, H_init, warm = 16, 1_200_000, 90, 4, 8
+    X0, B = quadratic_inputs(n, d, SEED + 6, x0="shared", x0_std=3.0)
+    g, _ = make_quadratic(n, d, "exp", 0, 0.1, SEED, 0.05, X0, B)
+    l0 = g.launch_count()
+    periods = g.run_adaptive(K, H_init, warm)
+    launches = g.launch_count() - l0
+    assert max(periods) >= 9                                   # some stretch is long enough for one launch
+    assert launches < K + 2 * len(periods)                     # fewer than one launch per iteration + the losses
+    g2, _ = make_quadratic(n, d, "exp", 0, 0.1, SEED, 0.05, X0, B)
+    H, count, F_init, want_periods = H_init, 0, 0.0, []
+    for k in range(K):
+        count += 1
+        glob = count == H
+        F = g2.mean_loss() if glob else 0.0
+        g2.set_period(1 if glob else 0)
+        g2.step(k)
+        if glob:
+            want_periods.append(H)
+            count = 0
+            F_init, H = o.aga_update(k, warm, H_init, F, F_init, H)
+    assert periods == want_periods
+    assert np.array_equal(g.get_x().cpu().numpy().view(np.uint32), g2.get_x().cpu().numpy().view(np.uint32))
+    g.close()
+    g2.close()
+
+
 def test_adaptive_period_sequence_matches_oracle_driven_loop():
     n, d, K, H_init, warm = 8, 4096, 60, 2, 6
     X0, B = quadratic_inputs(n, d, SEED + 5, x0="shared", x0_std=3.0)
