@@ -178,7 +178,7 @@ int32_t gpga_step(gpga_t* ctx, int64_t k, void* stream);
  * evolve independently, so under the quadratic objective a strip of columns can be advanced many
  * iterations per launch with its cells held on chip (HBM touched once per launch, the time per
  * iteration set by the noise arithmetic).  gpga_run does so for a state of at most 64 MB (X, X+ and b
- * together), and at any size for n <= 256 and K >= 32, where that is faster than
+ * together), and at any size for n <= 256 and K >= 8, where that is faster than
  * streaming the state from HBM every iteration; otherwise it takes one launch per iteration.  Results are bit-identical
  * to K calls of gpga_step either way.
  * Logistic objective: within one call the launches of consecutive iterations overlap (the rows of A and
