@@ -185,7 +185,8 @@ int32_t gpga_step(gpga_t* ctx, int64_t k, void* stream);
  * the labels of iteration k+1 are fetched while iteration k finishes); A and the labels are inputs that
  * no kernel of the library writes, and the caller must not write them while the call's work is in
  * flight on the stream.  For a narrow state (d <= 1024, batch <= 128, ring or one-peer exponential
- * graph, H = 0 or H >= 3, and as many nodes as the device holds pairs of blocks at once: 74 on a B200)
+ * graph, H = 0 or H >= 3, H = 2 with at least 24 nodes, H = 1 with at least 48 (below that single steps
+ * are faster), and as many nodes as the device holds pairs of blocks at once: 74 on a B200)
  * and K >= 2 the whole call is one launch per 16384 iterations: a pair of thread blocks per node keeps
  * x_i on chip and exchanges the half-step rows with its neighbours' pairs through the scratch area.
  * That launch expects the device to itself: its blocks wait for one another, every wait is bounded,
