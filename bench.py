@@ -390,37 +390,43 @@ def run_cell(torch, pkg, bufs, spec, sampler, seconds, peak):
             "ms_x_mhz": med * clocks["sm_mhz"] if clocks["sm_mhz"] else None}
 
 
-def run_logistic_cell(torch, pkg, sampler, peak, iterations=4000):
-    """The convex workload's cell: n = 64 nodes, 4096 samples of 1024 features each, batch 128, ring, H = 4;
-    one gpga_run call (the whole run in one launch), microseconds per iteration."""
+def run_logistic_cells(torch, pkg, sampler, peak, names=("c5_ring_h4", "c5_ring_hinf", "c5_exp_hinf"), iterations=4000):
+    """The convex workload's cells: n = 64 nodes, 4096 samples of 1024 features each, batch 128; ring with
+    H = 4, and ring / one-peer exponential graph without global averaging.  One gpga_run call each (the
+    whole run in one launch), microseconds per iteration; all share one data set."""
     from paper_2105_09080_b200.inputs import logistic_inputs_device
-    w = WORKLOADS["c5_ring_h4"]
-    n, d, m, batch = w["n"], w["d"], w["m"], w["batch"]
-    A, y = logistic_inputs_device(n, m, d, SEED)
-    g = pkg.Gpga(n, d, pkg.GPGA_TOPO_RING, w["H"], w["gamma"], SEED)
-    g.set_objective(pkg.GPGA_OBJ_LOGISTIC, l2=w["l2"], m=m, batch=batch)
-    xa = torch.zeros((n, d), device="cuda")
-    g.bind(xa, torch.empty_like(xa), A, y)
-    g.run(200)
-    torch.cuda.synchronize()
-    launches0 = g.launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler.begin()
-    e0.record()
-    g.run(iterations)
-    e1.record()
-    torch.cuda.synchronize()
-    clocks = sampler.end()
-    us = e0.elapsed_time(e1) / iterations * 1e3
-    algo = n * batch * d * 4 + 4 * n * d * 4        # the batch rows of A once; X read, G written and read, X+ written
-    gbs = algo / (us * 1e-6) / 1e9
-    out = {"kernel": "logreg_run_kernel" if g.launch_count() - launches0 < iterations else "logreg_partial + step_tile",
-           "n": n, "d": d, "m": m, "batch": batch, "iterations": iterations, "launches": g.launch_count() - launches0,
-           "us_per_iteration": us, "GB/s": gbs, "frac": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_PEAK_GBS,
-           "bound": "the chain of hand-overs inside an iteration, not bandwidth",
-           "sm_mhz": clocks["sm_mhz"], "reasons": clocks["reasons"], "global_loss_after": g.global_loss()}
-    g.close()
-    return out
+    first = WORKLOADS[names[0]]
+    A, y = logistic_inputs_device(first["n"], first["m"], first["d"], SEED)
+    cells = {}
+    for name in names:
+        w = WORKLOADS[name]
+        n, d, m, batch = w["n"], w["d"], w["m"], w["batch"]
+        topo = {"ring": pkg.GPGA_TOPO_RING, "exp": pkg.GPGA_TOPO_EXP}[w["topo"]]
+        g = pkg.Gpga(n, d, topo, w["H"], w["gamma"], SEED)
+        g.set_objective(pkg.GPGA_OBJ_LOGISTIC, l2=w["l2"], m=m, batch=batch)
+        xa = torch.zeros((n, d), device="cuda")
+        g.bind(xa, torch.empty_like(xa), A, y)
+        g.run(200)
+        torch.cuda.synchronize()
+        launches0 = g.launch_count()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sampler.begin()
+        e0.record()
+        g.run(iterations)
+        e1.record()
+        torch.cuda.synchronize()
+        clocks = sampler.end()
+        us = e0.elapsed_time(e1) / iterations * 1e3
+        algo = n * batch * d * 4 + 4 * n * d * 4        # the batch rows of A once; X read, G written and read, X+ written
+        gbs = algo / (us * 1e-6) / 1e9
+        cells[name] = {"kernel": "logreg_run_kernel" if g.launch_count() - launches0 < iterations else "logreg_partial + step_tile",
+                       "n": n, "d": d, "m": m, "batch": batch, "topology": w["topo"], "H": w["H"] or "inf",
+                       "iterations": iterations, "launches": g.launch_count() - launches0,
+                       "us_per_iteration": us, "GB/s": gbs, "frac": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_PEAK_GBS,
+                       "bound": "the chain of hand-overs inside an iteration, not bandwidth",
+                       "sm_mhz": clocks["sm_mhz"], "reasons": clocks["reasons"], "global_loss_after": g.global_loss()}
+        g.close()
+    return cells
 
 
 # ---------------------------------------------------------------------------------
@@ -552,9 +558,10 @@ def run_ours(args):
                     roofline[f"cell_{spec[0]}_GBs"] = c["GB/s"]
                     roofline[f"cell_{spec[0]}_frac_of_nominal_8TBs"] = c["frac_of_nominal_8TBs"]
                     roofline[f"cell_{spec[0]}_sm_mhz"] = c["sm_mhz"]
-            cells["c5_ring_h4"] = run_logistic_cell(torch, pkg, sampler, peak)
-            roofline["cell_c5_ring_h4_us_per_iteration"] = cells["c5_ring_h4"]["us_per_iteration"]
-            roofline["cell_c5_ring_h4_frac"] = cells["c5_ring_h4"]["frac"]
+            for cname, cell in run_logistic_cells(torch, pkg, sampler, peak).items():
+                cells[cname] = cell
+                roofline[f"cell_{cname}_us_per_iteration"] = cell["us_per_iteration"]
+                roofline[f"cell_{cname}_frac"] = cell["frac"]
             g.init_from_seed(kind, w["x0_std"], w["b_shift"])     # the cells used the same buffers
             for _ in range(3):
                 g.step(g.get_k())
