@@ -161,6 +161,8 @@ int32_t gpga_bind(gpga_t* ctx, void* x_a, void* x_b, void* data, const void* lab
  *  NODE_SHIFT for node i;  X^(0) per x0_kind with standard deviation x0_std
  *  (Algorithm 1 requires equal initial rows: kinds ZERO and SHARED_NORMAL).
  * Also resets the iteration counter to 0 and makes x_a the current buffer.
+ * On a node shard (gpga_set_node_shard) local row i is filled as node shard * n + i of the whole
+ * problem, so the shards together hold exactly what the unsharded handle would.
  */
 int32_t gpga_init_from_seed(gpga_t* ctx, int32_t x0_kind, float x0_std, float b_shift,
                             void* stream);

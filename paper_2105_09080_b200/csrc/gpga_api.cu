@@ -531,9 +531,10 @@ int32_t gpga_init_from_seed(gpga_t* c, int32_t x0_kind, float x0_std, float b_sh
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool vec = vec_ok(c);
     const uint32_t q_base = (uint32_t)(c->col0 >> 2);
-    cudaError_t e = launch_init_b(c->data, c->n, c->d, c->ld, q_base, b_shift, vec, c->keys, s);
+    const uint32_t row0 = (uint32_t)(c->shard * c->n);   // a node shard fills its own rows of the whole problem
+    cudaError_t e = launch_init_b(c->data, c->n, c->d, c->ld, q_base, row0, b_shift, vec, c->keys, s);
     if (e != cudaSuccess) return cuda_fail(c, e, "init b launch");
-    e = launch_init_x0(c->x[0], c->n, c->d, c->ld, q_base, x0_kind, x0_std, vec, c->keys, s);
+    e = launch_init_x0(c->x[0], c->n, c->d, c->ld, q_base, row0, x0_kind, x0_std, vec, c->keys, s);
     if (e != cudaSuccess) return cuda_fail(c, e, "init x0 launch");
     c->launches += 2;
     c->cur = 0;

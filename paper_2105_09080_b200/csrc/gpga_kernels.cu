@@ -556,14 +556,14 @@ cudaError_t launch_quadratic_loss(const float* x, const float* b, long long n, l
 template <bool VEC>
 __global__ void __launch_bounds__(kBlock) init_b_kernel(float* __restrict__ b, long long n,
                                                         long long d, long long ld, long long Q, uint32_t q_base,
-                                                        float shift, const PhiloxKeys keys)
+                                                        uint32_t row0, float shift, const PhiloxKeys keys)
 {
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (q >= Q) return;
-    for (long long i = 0; i < n; ++i) {
-        float4 z = normal4(q_base + (uint32_t)q, (uint32_t)i, 0u, 1u, keys);
+    for (long long i = 0; i < n; ++i) {   // local row i is node row0 + i of the whole problem
+        float4 z = normal4(q_base + (uint32_t)q, row0 + (uint32_t)i, 0u, 1u, keys);
         if (shift != 0.0f) {
-            const float s = normal4(0u, (uint32_t)i, 0u, 3u, keys).x;
+            const float s = normal4(0u, row0 + (uint32_t)i, 0u, 3u, keys).x;
             z.x = fmaf(shift, s, z.x);
             z.y = fmaf(shift, s, z.y);
             z.z = fmaf(shift, s, z.z);
@@ -576,37 +576,37 @@ __global__ void __launch_bounds__(kBlock) init_b_kernel(float* __restrict__ b, l
 template <bool VEC>
 __global__ void __launch_bounds__(kBlock) init_x0_kernel(float* __restrict__ x, long long n,
                                                          long long d, long long ld, long long Q, uint32_t q_base,
-                                                         int kind, float std, const PhiloxKeys keys)
+                                                         uint32_t row0, int kind, float std, const PhiloxKeys keys)
 {
     const long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (q >= Q) return;
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
     if (kind == 1) v = scale4(normal4(q_base + (uint32_t)q, 0u, 0u, 2u, keys), std);
     for (long long i = 0; i < n; ++i) {
-        if (kind == 2) v = scale4(normal4(q_base + (uint32_t)q, (uint32_t)i, 0u, 2u, keys), std);
+        if (kind == 2) v = scale4(normal4(q_base + (uint32_t)q, row0 + (uint32_t)i, 0u, 2u, keys), std);
         store4<VEC>(x + i * ld, q * 4, d, v);
     }
 }
 
-cudaError_t launch_init_b(float* b, long long n, long long d, long long ld, uint32_t q_base, float shift, bool vec,
-                          const PhiloxKeys& keys, cudaStream_t s)
+cudaError_t launch_init_b(float* b, long long n, long long d, long long ld, uint32_t q_base, uint32_t row0, float shift,
+                          bool vec, const PhiloxKeys& keys, cudaStream_t s)
 {
     const long long Q = (d + 3) / 4;
     if (vec)
-        init_b_kernel<true><<<grid_for(Q, kBlock), kBlock, 0, s>>>(b, n, d, ld, Q, q_base, shift, keys);
+        init_b_kernel<true><<<grid_for(Q, kBlock), kBlock, 0, s>>>(b, n, d, ld, Q, q_base, row0, shift, keys);
     else
-        init_b_kernel<false><<<grid_for(Q, kBlock), kBlock, 0, s>>>(b, n, d, ld, Q, q_base, shift, keys);
+        init_b_kernel<false><<<grid_for(Q, kBlock), kBlock, 0, s>>>(b, n, d, ld, Q, q_base, row0, shift, keys);
     return cudaGetLastError();
 }
 
-cudaError_t launch_init_x0(float* x, long long n, long long d, long long ld, uint32_t q_base, int kind, float std,
-                           bool vec, const PhiloxKeys& keys, cudaStream_t s)
+cudaError_t launch_init_x0(float* x, long long n, long long d, long long ld, uint32_t q_base, uint32_t row0, int kind,
+                           float std, bool vec, const PhiloxKeys& keys, cudaStream_t s)
 {
     const long long Q = (d + 3) / 4;
     if (vec)
-        init_x0_kernel<true><<<grid_for(Q, kBlock), kBlock, 0, s>>>(x, n, d, ld, Q, q_base, kind, std, keys);
+        init_x0_kernel<true><<<grid_for(Q, kBlock), kBlock, 0, s>>>(x, n, d, ld, Q, q_base, row0, kind, std, keys);
     else
-        init_x0_kernel<false><<<grid_for(Q, kBlock), kBlock, 0, s>>>(x, n, d, ld, Q, q_base, kind, std, keys);
+        init_x0_kernel<false><<<grid_for(Q, kBlock), kBlock, 0, s>>>(x, n, d, ld, Q, q_base, row0, kind, std, keys);
     return cudaGetLastError();
 }
 

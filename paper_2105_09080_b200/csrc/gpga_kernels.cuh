@@ -58,11 +58,11 @@ cudaError_t launch_consensus(const float* x, long long n, long long d, long long
 cudaError_t launch_quadratic_loss(const float* x, const float* b, long long n, long long d, long long ld,
                                   bool vec, double* partials, double* result, cudaStream_t s);
 
-// Seeded fills (quadratic objective).
-cudaError_t launch_init_b(float* b, long long n, long long d, long long ld, uint32_t q_base, float shift, bool vec,
-                          const PhiloxKeys& keys, cudaStream_t s);
-cudaError_t launch_init_x0(float* x, long long n, long long d, long long ld, uint32_t q_base, int kind, float std,
-                           bool vec, const PhiloxKeys& keys, cudaStream_t s);
+// Seeded fills (quadratic objective); row0 = global index of local row 0 (node sharding).
+cudaError_t launch_init_b(float* b, long long n, long long d, long long ld, uint32_t q_base, uint32_t row0, float shift,
+                          bool vec, const PhiloxKeys& keys, cudaStream_t s);
+cudaError_t launch_init_x0(float* x, long long n, long long d, long long ld, uint32_t q_base, uint32_t row0, int kind,
+                           float std, bool vec, const PhiloxKeys& keys, cudaStream_t s);
 
 // Generator surface.
 cudaError_t launch_philox_words(const uint32_t* ctr, PhiloxKeys keys, long long count, uint32_t* out,

@@ -68,6 +68,10 @@ class NodeShard:
         """data: the local nodes' b (quadratic) or A (logistic, with their labels)."""
         self.g.bind(x_a, x_b, data, labels)
 
+    def init_from_seed(self, x0_kind, x0_std=1.0, b_shift=0.0):
+        """Fill this shard's rows of b and X^(0) on the device, keyed by the global node index."""
+        self.g.init_from_seed(x0_kind, x0_std, b_shift)
+
     def plan(self, k) -> ShardPlan:
         return shard_plan(self.topology, self.H, self.n_total, self.shards, self.shard, self.d, k)
 

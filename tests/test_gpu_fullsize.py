@@ -213,3 +213,49 @@ def test_config_4_bert_large_sized():
               offs[::2], [])
     del xa, xb, b
     torch.cuda.empty_cache()
+
+
+def test_config_4_sharded_by_nodes_on_one_device():
+    """The BERT-Large-sized problem as two node shards of eight nodes each on one device (a shard's
+    state has 2.7e9 elements: 64-bit offsets in the shard kernels), filled from the seed by each shard
+    for its own nodes, five iterations -- hops 1, 2, 4 inside a shard or across, hop 8 where every row
+    crosses, then a global average -- with one copy per message between the shards; sampled column
+    blocks against the oracle's run of all sixteen nodes."""
+    torch = _torch()
+    from paper_2105_09080_b200 import node_sharded as ns
+    n, d, gamma, sigma, K, H, shards = 16, 335_141_888, 0.01, 0.01, 5, 5, 2
+    n_l = n // shards
+    if _free_gib() < shards * 5 * n_l * d * 4 / 2**30 + 4:
+        pytest.skip("not enough free device memory")
+    parts = []
+    for s in range(shards):
+        sh = ns.NodeShard(n, d, pkg.GPGA_TOPO_EXP, H, gamma, SEED, shards, s, sigma=sigma)
+        xa = torch.empty((n_l, d), dtype=torch.float32, device="cuda")
+        sh.bind(xa, torch.empty_like(xa), torch.empty_like(xa))
+        sh.init_from_seed(pkg.GPGA_X0_PER_NODE_NORMAL, 0.1, 0.5)
+        parts.append(sh)
+    offs = _blocks(d, 12, np.random.default_rng(6))
+    # the shards' fills are the whole problem's rows (keyed by the global node index)
+    for c0 in offs[:4]:
+        want = o.init_x0(n, BLOCK, SEED, o.X0_PER_NODE_NORMAL, 0.1, c0)
+        got = np.concatenate([_gpu_block(sh.get_x(), c0, BLOCK) for sh in parts])
+        assert np.abs(got - want).max() <= 1e-5
+    for k in range(K):
+        for sh in parts:
+            sh.export(k)
+        ns.exchange_local(parts, k)
+        for sh in parts:
+            sh.step(k)
+    for c0 in offs:
+        w = min(BLOCK, d - c0)
+        B = o.init_b(n, w, SEED, 0.5, c0).astype(np.float32)
+        X0 = o.init_x0(n, w, SEED, o.X0_PER_NODE_NORMAL, 0.1, c0).astype(np.float32)
+        p = o.Problem(o.TOPO_EXP, H, gamma, SEED, sigma=sigma, data=B, col0=c0)
+        got = np.concatenate([_gpu_block(sh.get_x(), c0, w) for sh in parts])
+        ok, worst = close(got, o.run(p, X0, 0, K), TOL_RUN)
+        assert ok, ("col0", c0, worst)
+        assert np.all(got == got[0])        # K = H = 5: the run ends on a global average
+    for sh in parts:
+        sh.close()
+    del parts, sh, xa
+    torch.cuda.empty_cache()

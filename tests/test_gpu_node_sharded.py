@@ -206,6 +206,45 @@ def test_adaptive_period_on_shards_equals_the_unsharded_adaptive_run(topo, n, sh
     g.close()
 
 
+@pytest.mark.parametrize("kind", ["shared", "per_node"])
+def test_seeded_fill_of_the_shards_is_the_whole_problems(kind):
+    """gpga_init_from_seed on a shard handle fills local row i as node shard * n + i: the shards
+    together hold bit for bit what the unsharded handle's fill holds, and a run from there agrees."""
+    import torch
+    n, d, shards, K = 16, 4104, 4, 6
+    x0_kind = pkg.GPGA_X0_SHARED_NORMAL if kind == "shared" else pkg.GPGA_X0_PER_NODE_NORMAL
+    g = pkg.Gpga(n, d, TOPO["ring"][0], 3, 0.1, SEED)
+    g.set_objective(pkg.GPGA_OBJ_QUADRATIC, sigma=0.2)
+    xa = torch.empty((n, d), device="cuda")
+    b = torch.empty_like(xa)
+    g.bind(xa, torch.empty_like(xa), b)
+    g.init_from_seed(x0_kind, 0.3, 0.5)
+    x0_full, b_full = g.get_x().cpu().numpy().copy(), b.cpu().numpy().copy()
+    n_l, parts, bs = n // shards, [], []
+    for s in range(shards):
+        sh = ns.NodeShard(n, d, TOPO["ring"][0], 3, 0.1, SEED, shards, s, sigma=0.2)
+        x = torch.empty((n_l, d), device="cuda")
+        bb = torch.empty_like(x)
+        sh.bind(x, torch.empty_like(x), bb)
+        sh.init_from_seed(x0_kind, 0.3, 0.5)
+        parts.append(sh)
+        bs.append(bb)
+    assert np.array_equal(np.concatenate([sh.get_x().cpu().numpy() for sh in parts]), x0_full)
+    assert np.array_equal(np.concatenate([t.cpu().numpy() for t in bs]), b_full)
+    assert len(np.unique(b_full[:, 0])) == n                          # every node has its own b
+    for k in range(K):
+        g.step(k)
+        for sh in parts:
+            sh.export(k)
+        ns.exchange_local(parts, k)
+        for sh in parts:
+            sh.step(k)
+    assert np.array_equal(np.concatenate([sh.get_x().cpu().numpy() for sh in parts]), g.get_x().cpu().numpy())
+    for sh in parts:
+        sh.close()
+    g.close()
+
+
 def test_fused_export_argument_checks():
     import ctypes as C
     import torch
