@@ -281,7 +281,9 @@ int32_t gpga_aga_update(int64_t k, int64_t warmup_iters, int64_t H_init, double 
  *        all-gather of a communication library) --
  *     gpga_shard_step(k, recv)     local update + mix of the local rows with what was received
  * Results equal the unsharded iteration's (same operations in the same order; the column mean adds
- * the shards' fp64 sums in shard order).  Send and receive buffers are caller-owned device memory,
+ * the shards' fp64 sums in shard order).  The diagnostics of a shard handle (gpga_consensus_distance,
+ * gpga_mean_loss, gpga_global_loss) are over the shard's own nodes; gpga_mean_loss values of equal shards
+ * average to the whole problem's.  Send and receive buffers are caller-owned device memory,
  * 16-byte aligned, gpga_shard_exchange_bytes() each; an exchanged row is ceil(d/4)*4 floats.
  * The library reads remote rows only from the receive buffer in this device's own memory.
  */
