@@ -257,6 +257,27 @@ int32_t gpga_run_adaptive(gpga_t* ctx, int64_t K, int64_t H_init, int64_t warmup
                           int64_t* num_periods_host);
 
 /*
+ * Diagnostics of the WHOLE problem on node shards: the consensus distance sum_i ||x_i - xbar||^2
+ * (Section 4) and the global loss f(xbar) = (1/n) sum_i f_i(xbar) of problem (1) need the mean over
+ * all nodes.  gpga_shard_state_sums writes the fp64 column sums of this shard's current rows
+ * (ceil(d/4)*4 doubles, the size and place of a shard's column sums in a global-average exchange:
+ * gpga_shard_plan's gather_bytes) to sums_dev; the caller all-gathers them in shard order, like the
+ * column sums of a global average; gpga_shard_diagnostics then forms xbar = (sum of the gathered
+ * vectors) / (n * shards) and returns this shard's parts,
+ *     *consensus_part_host = sum over the local nodes of ||x_i - xbar||^2,
+ *     *loss_part_host      = (1 / (n * shards)) sum over the local nodes of f_i(xbar),
+ * whose sums over the shards are the whole problem's consensus distance and global loss (f_i as for
+ * gpga_global_loss).  Either host pointer may be NULL.  Synchronises the stream.  On a logistic shard
+ * the call borrows the gradient buffer: a gradient formed by gpga_shard_export for an iteration not yet
+ * stepped is formed again by the step.
+ * Errors: NOT_READY before gpga_bind; INVALID_ARG for NULL or misaligned device buffers or when both
+ * host pointers are NULL; TIMEOUT / CUDA as for the other synchronising calls.
+ */
+int32_t gpga_shard_state_sums(gpga_t* ctx, void* sums_dev, void* stream);
+int32_t gpga_shard_diagnostics(gpga_t* ctx, const void* gathered_dev, void* stream, double* consensus_part_host,
+                               double* loss_part_host);
+
+/*
  * Algorithm 2's period rule by itself (host arithmetic only), for a caller that drives the
  * iterations itself -- the node-sharded deployment, where the mean loss F is the all-reduced mean of
  * the shards' gpga_mean_loss values.  Called at a global-average iteration k with that iteration's

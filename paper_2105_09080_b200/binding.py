@@ -62,6 +62,8 @@ SIGNATURES = {
     "gpga_shard_export": (_i32, [_P, _i64, _P, _P]),
     "gpga_shard_export_to": (_i32, [_P, _i64, _P, _P, _i32, _P]),
     "gpga_shard_step": (_i32, [_P, _i64, _P, _P]),
+    "gpga_shard_state_sums": (_i32, [_P, _P, _P]),
+    "gpga_shard_diagnostics": (_i32, [_P, _P, _P, C.POINTER(C.c_double), C.POINTER(C.c_double)]),
     "gpga_shard_step_interior": (_i32, [_P, _i64, _P]),
     "gpga_shard_step_boundary": (_i32, [_P, _i64, _P, _P]),
     "gpga_run_adaptive": (_i32, [_P, _i64, _i64, _i64, _P, C.POINTER(_i64), _i64, C.POINTER(_i64)]),

@@ -1043,6 +1043,60 @@ int32_t gpga_shard_step_boundary(gpga_t* c, int64_t k, const void* recv_dev, voi
     return shard_step_part(c, k, recv_dev, SHARD_BOUNDARY, static_cast<cudaStream_t>(stream));
 }
 
+int32_t gpga_shard_state_sums(gpga_t* c, void* sums_dev, void* stream)
+{
+    int32_t st = check_ready(c);
+    if (st) return st;
+    if (!sums_dev || !aligned16(sums_dev)) return fail(c, GPGA_ERR_INVALID_ARG, "sums buffer must be a 16-byte aligned device pointer");
+    const cudaError_t e = launch_shard_state_sums(c->x[c->cur], c->n, c->d, c->ld, vec_ok(c), static_cast<double*>(sums_dev),
+                                                  static_cast<cudaStream_t>(stream));
+    c->launches += 1;
+    if (e != cudaSuccess) return cuda_fail(c, e, "state sums launch");
+    return GPGA_OK;
+}
+
+int32_t gpga_shard_diagnostics(gpga_t* c, const void* gathered_dev, void* stream, double* consensus_part_host,
+                               double* loss_part_host)
+{
+    int32_t st = check_ready(c);
+    if (st) return st;
+    if (!gathered_dev || !aligned16(gathered_dev)) return fail(c, GPGA_ERR_INVALID_ARG, "gathered sums must be a 16-byte aligned device pointer");
+    if (!consensus_part_host && !loss_part_host) return fail(c, GPGA_ERR_INVALID_ARG, "nothing asked for");
+    if (c->shards >= (int64_t(1) << 31)) return fail(c, GPGA_ERR_INVALID_ARG, "too many shards");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const ScratchLayout& L = c->L;
+    double* partials = reinterpret_cast<double*>(c->scratch + L.partials_off);
+    double* result = reinterpret_cast<double*>(c->scratch + L.result_off);
+    const double* gathered = static_cast<const double*>(gathered_dev);
+    const long long n_total = c->n * c->shards;
+    cudaError_t e;
+    if (consensus_part_host) {
+        e = launch_shard_consensus_part(c->x[c->cur], c->n, c->d, c->ld, vec_ok(c), gathered, (int)c->shards, n_total,
+                                        partials, result, s);
+        c->launches += 2;
+        if (e != cudaSuccess) return cuda_fail(c, e, "shard consensus launch");
+        st = read_double(c, result, s, consensus_part_host);
+        if (st) return st;
+    }
+    if (loss_part_host) {
+        if (c->objective == GPGA_OBJ_LOGISTIC) {
+            float* xbar = reinterpret_cast<float*>(c->scratch + L.G_off);   // dead between iterations
+            e = launch_shard_logistic_loss_part(c->data, c->labels, c->n, c->d, c->m, c->l2, gathered, (int)c->shards,
+                                                n_total, xbar, partials, L.slots, result, s);
+            c->shard_grad_k = -1;   // the gradient matrix of the coming iteration, if any, has been overwritten
+            c->launches += 3;
+        } else {
+            e = launch_shard_quadratic_loss_part(c->data, c->n, c->d, c->ld, vec_ok(c), gathered, (int)c->shards, n_total,
+                                                 partials, result, s);
+            c->launches += 2;
+        }
+        if (e != cudaSuccess) return cuda_fail(c, e, "shard loss launch");
+        st = read_double(c, result, s, loss_part_host);
+        if (st) return st;
+    }
+    return GPGA_OK;
+}
+
 int32_t gpga_aga_update(int64_t k, int64_t warmup_iters, int64_t H_init, double F, double* F_init_inout, int64_t* H_inout)
 {
     if (!F_init_inout || !H_inout) return fail(nullptr, GPGA_ERR_INVALID_ARG, "F_init_inout and H_inout must not be NULL");

@@ -15,4 +15,20 @@ cudaError_t launch_logistic_global_loss(const float* A, const float* y, const fl
                                         long long d, long long m, float l2, float* xbar, double* partials,
                                         long long slots, double* result, cudaStream_t s);
 
+// Node shards: the whole problem's diagnostics from the shards' parts.  sums: 4 ceil(d/4) doubles, the
+// fp64 column sums of the shard's rows; gathered: `parts` such vectors in shard order.
+cudaError_t launch_shard_state_sums(const float* x, long long n, long long d, long long ld, bool vec, double* sums,
+                                    cudaStream_t s);
+// sum over the local rows of ||x_i - xbar||^2, xbar = (sum of the parts) / n_total
+cudaError_t launch_shard_consensus_part(const float* x, long long n, long long d, long long ld, bool vec,
+                                        const double* gathered, int parts, long long n_total, double* partials,
+                                        double* result, cudaStream_t s);
+// (1 / n_total) sum over the local rows of f_i(xbar)
+cudaError_t launch_shard_quadratic_loss_part(const float* b, long long n, long long d, long long ld, bool vec,
+                                             const double* gathered, int parts, long long n_total, double* partials,
+                                             double* result, cudaStream_t s);
+cudaError_t launch_shard_logistic_loss_part(const float* A, const float* y, long long n, long long d, long long m, float l2,
+                                            const double* gathered, int parts, long long n_total, float* xbar,
+                                            double* partials, long long slots, double* result, cudaStream_t s);
+
 }  // namespace gpga

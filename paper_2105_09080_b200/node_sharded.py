@@ -109,6 +109,21 @@ class NodeShard:
         """Mean over this shard's nodes of the local loss at their own iterates."""
         return self.g.mean_loss()
 
+    def state_sums(self, out=None, stream=None):
+        """The fp64 column sums of this shard's current rows into `out` (a uint8 tensor; default: the
+        start of the send buffer, which is free between two iterations only)."""
+        out = self.send if out is None else out
+        self.g._check(B.lib().gpga_shard_state_sums(self.g._h, out.data_ptr(), self.g._sp(stream)))
+
+    def diagnostics(self, gathered=None, stream=None):
+        """This shard's parts (consensus distance, global loss) of the whole problem's diagnostics, from
+        all shards' column sums in `gathered` (default: the receive buffer, free between two iterations only)."""
+        gathered = self.recv if gathered is None else gathered
+        xi, loss = C.c_double(), C.c_double()
+        self.g._check(B.lib().gpga_shard_diagnostics(self.g._h, gathered.data_ptr(), self.g._sp(stream),
+                                                     C.byref(xi), C.byref(loss)))
+        return xi.value, loss.value
+
     def get_x(self):
         return self.g.get_x()
 
@@ -306,3 +321,49 @@ def run_dist_adaptive(shard, K, H_init, warmup_iters, k0=0, group=None):
         return float(t.item()) / dist.get_world_size(group)
 
     return run_adaptive([shard], K, H_init, warmup_iters, lambda k: exchange_dist(shard, k, group), mean_of_losses, k0)
+
+
+def _gather_bytes(shard):
+    return (shard.d + 3) // 4 * 4 * 8
+
+
+def _diag_buffers(shard, own):
+    """Where the column sums go: the exchange buffers (free between two iterations), or buffers of
+    their own (for a call in the middle of an iteration, while the messages are in the exchange buffers)."""
+    if not own:
+        return shard.send, shard.recv
+    if not hasattr(shard, "_diag"):
+        import torch
+        nb = _gather_bytes(shard)
+        shard._diag = (torch.zeros(nb, dtype=torch.uint8, device=shard.recv.device),
+                       torch.zeros(nb * shard.shards, dtype=torch.uint8, device=shard.recv.device))
+    return shard._diag
+
+
+def diagnostics_local(shards, own_buffers=False):
+    """Consensus distance and global loss f(xbar) of the whole problem from shards of one process:
+    every shard's column sums are copied into every shard's gather area in shard order, the parts
+    are added.  Uses the exchange buffers, so call it between two iterations -- or with
+    own_buffers=True at any point."""
+    nb = _gather_bytes(shards[0])
+    bufs = [_diag_buffers(sh, own_buffers) for sh in shards]
+    for sh, (out, _) in zip(shards, bufs):
+        sh.state_sums(out)
+    for src, (out, _) in zip(shards, bufs):
+        for _, gathered in bufs:
+            gathered[src.shard * nb:(src.shard + 1) * nb].copy_(out[:nb], non_blocking=True)
+    parts = [sh.diagnostics(gathered) for sh, (_, gathered) in zip(shards, bufs)]
+    return sum(p[0] for p in parts), sum(p[1] for p in parts)
+
+
+def diagnostics_dist(shard, group=None, own_buffers=False):
+    """The same with one shard per rank: an all-gather of the column sums, an all-reduce of the two parts."""
+    import torch
+    import torch.distributed as dist
+    nb, world = _gather_bytes(shard), dist.get_world_size(group)
+    out, gathered = _diag_buffers(shard, own_buffers)
+    shard.state_sums(out)
+    dist.all_gather([gathered[r * nb:(r + 1) * nb] for r in range(world)], out[:nb], group=group)
+    t = torch.tensor(shard.diagnostics(gathered), dtype=torch.float64, device=shard.recv.device)
+    dist.all_reduce(t, group=group)
+    return float(t[0].item()), float(t[1].item())

@@ -245,6 +245,86 @@ def test_seeded_fill_of_the_shards_is_the_whole_problems(kind):
     g.close()
 
 
+@pytest.mark.parametrize("topo,H,n,shards,d", [("ring", 0, 16, 4, 4104), ("exp", 5, 16, 2, 1031), ("ring", 3, 8, 1, 19456)])
+def test_whole_problem_diagnostics_from_the_shards_parts(topo, H, n, shards, d):
+    """Consensus distance and global loss of the whole problem, each the sum of the shards' parts
+    (column sums all-gathered, mean over all nodes formed on every shard), against the oracle's values
+    of the same state and against the unsharded handle's diagnostics."""
+    import torch
+    gamma, sigma, K = 0.1, 0.3, 7
+    X0, B = quadratic_inputs(n, d, SEED + n + d + 4, x0="per_node")
+    g, _ = make_quadratic(n, d, topo, H, gamma, SEED, sigma, X0, B)
+    n_l, parts = n // shards, []
+    for s in range(shards):
+        sh = ns.NodeShard(n, d, TOPO[topo][0], H, gamma, SEED, shards, s, sigma=sigma)
+        xa = torch.from_numpy(np.ascontiguousarray(X0[s * n_l:(s + 1) * n_l])).cuda()
+        sh.bind(xa, torch.empty_like(xa), torch.from_numpy(np.ascontiguousarray(B[s * n_l:(s + 1) * n_l])).cuda())
+        parts.append(sh)
+    for k in range(K):
+        g.step(k)
+        for sh in parts:
+            sh.export(k)
+        ns.exchange_local(parts, k)
+        for sh in parts:
+            sh.step(k)
+        if k in (0, 3, K - 1):
+            X = np.concatenate([sh.get_x().cpu().numpy() for sh in parts])
+            xi, loss = ns.diagnostics_local(parts)
+            xi_want = o.consensus_distance(X)
+            xbar = np.repeat(X.astype(np.float64).mean(0, keepdims=True), n, axis=0)
+            loss_want = o.quadratic_mean_loss(xbar, B)                 # (1/n) sum_i 1/2 ||xbar - b_i||^2
+            assert xi_want > 0 and abs(xi - xi_want) <= 1e-5 * xi_want, (k, xi, xi_want)
+            assert abs(loss - loss_want) <= 1e-5 * loss_want, (k, loss, loss_want)
+            assert abs(xi - g.consensus_distance()) <= 1e-5 * xi_want
+            assert abs(loss - g.global_loss()) <= 1e-9 * loss_want
+    for sh in parts:
+        sh.close()
+    g.close()
+
+
+def test_whole_problem_diagnostics_of_logistic_shards():
+    import torch
+    from paper_2105_09080_b200.inputs import logistic_inputs
+    topo, H, n, shards, m, d, batch, gamma, l2, K = "ring", 4, 8, 2, 64, 256, 40, 0.1, 1e-3, 6
+    A, y = logistic_inputs(n, m, d, SEED + n)
+    X0 = (0.1 * np.random.default_rng(n + d).standard_normal((n, d))).astype(np.float32)
+    g = pkg.Gpga(n, d, TOPO[topo][0], H, gamma, SEED)
+    g.set_objective(pkg.GPGA_OBJ_LOGISTIC, l2=l2, m=m, batch=batch)
+    xa = torch.from_numpy(X0).cuda()
+    g.bind(xa, torch.empty_like(xa), torch.from_numpy(A).cuda(), torch.from_numpy(y).cuda())
+    n_l, parts = n // shards, []
+    for s in range(shards):
+        rows = slice(s * n_l, (s + 1) * n_l)
+        sh = ns.NodeShard(n, d, TOPO[topo][0], H, gamma, SEED, shards, s, logistic=dict(l2=l2, m=m, batch=batch))
+        x = torch.from_numpy(np.ascontiguousarray(X0[rows])).cuda()
+        sh.bind(x, torch.empty_like(x), torch.from_numpy(np.ascontiguousarray(A[rows])).cuda(),
+                torch.from_numpy(np.ascontiguousarray(y[rows])).cuda())
+        parts.append(sh)
+    for k in range(K):
+        g.step(k)
+        for sh in parts:
+            sh.export(k)
+        if k == 2:      # between export and step: the step forms the gradient again, the result must not change
+            ns.diagnostics_local(parts, own_buffers=True)
+        ns.exchange_local(parts, k)
+        for sh in parts:
+            sh.step(k)
+        X = np.concatenate([sh.get_x().cpu().numpy() for sh in parts])
+        assert np.array_equal(X.view(np.uint32), g.get_x().cpu().numpy().view(np.uint32))
+        xi, loss = ns.diagnostics_local(parts)
+        xi_want = o.consensus_distance(X)
+        loss_want = o.global_logistic_loss(A.astype(np.float64), y.astype(np.float64), X.astype(np.float64).mean(0), l2)
+        if (k + 1) % H:
+            assert xi_want > 0 and abs(xi - xi_want) <= 1e-5 * xi_want, (k, xi, xi_want)
+        else:
+            assert xi <= 1e-12
+        assert abs(loss - loss_want) <= 1e-5 * loss_want, (k, loss, loss_want)
+        assert abs(loss - g.global_loss()) <= 1e-6 * loss_want
+    for sh in parts:
+        sh.close()
+    g.close()
+
+
 def test_fused_export_argument_checks():
     import ctypes as C
     import torch

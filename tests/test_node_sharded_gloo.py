@@ -41,6 +41,18 @@ class OracleShard:
     def set_period(self, H):
         self.H = H
 
+    def state_sums(self, out=None):
+        sums = np.zeros(self.q4)
+        sums[:self.d] = self.X.astype(np.float64).sum(0)
+        (self.send if out is None else out)[:self.q4 * 8] = _bytes(sums)
+
+    def diagnostics(self, gathered=None):
+        buf = (self.recv if gathered is None else gathered).numpy()[:self.shards * self.q4 * 8]
+        total = np.frombuffer(buf.tobytes(), dtype=np.float64).reshape(self.shards, self.q4).sum(0)[:self.d]
+        xbar = total / self.n_total
+        X = self.X.astype(np.float64)
+        return float(((X - xbar) ** 2).sum()), float(0.5 * ((xbar - self.B) ** 2).sum() / self.n_total)
+
     def mean_loss(self):
         return o.quadratic_mean_loss(self.X, self.B)
 
@@ -133,6 +145,25 @@ def _adaptive_worker(rank, world, port, topo, n, d, K, H_init, warm, out_dir):
         assert all(g[2] == periods for g in gathered)       # every rank took the same periods
         np.save(os.path.join(out_dir, "full.npy"), np.concatenate([x for _, x, _ in sorted(gathered, key=lambda t: t[0])]))
         np.save(os.path.join(out_dir, "periods.npy"), np.array(periods, dtype=np.int64))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def _diag_worker(rank, world, port, n, d, K, out_dir):
+    import torch.distributed as dist
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    X0, B = quadratic_inputs(n, d, 7, x0="per_node")
+    shard = OracleShard(n, d, "ring", 0, 0.1, 0.4, 11, world, rank, X0, B)
+    ns.run_dist(shard, K)
+    xi, loss = ns.diagnostics_dist(shard)
+    gathered = [None] * world
+    dist.all_gather_object(gathered, (rank, shard.X, xi, loss))
+    if rank == 0:
+        assert all(g[2] == xi and g[3] == loss for g in gathered)     # every rank holds the same totals
+        np.save(os.path.join(out_dir, "full.npy"), np.concatenate([x for _, x, _, _ in sorted(gathered, key=lambda t: t[0])]))
+        np.save(os.path.join(out_dir, "diag.npy"), np.array([xi, loss]))
     dist.barrier()
     dist.destroy_process_group()
 
@@ -316,3 +347,18 @@ def test_adaptive_period_across_ranks(tmp_path):
     assert np.load(tmp_path / "periods.npy").tolist() == want_periods
     got = np.load(tmp_path / "full.npy")
     assert np.abs(got - want).max() <= 2e-6 * (1 + np.abs(want).max())
+
+
+def test_whole_problem_diagnostics_across_ranks(tmp_path):
+    """diagnostics_dist: column sums all-gathered in rank order, the two parts all-reduced; against the
+    oracle's consensus distance and global loss of the assembled state."""
+    import torch.multiprocessing as mp
+    n, d, K, world = 12, 10, 5, 3
+    mp.spawn(_diag_worker, args=(world, _free_port(), n, d, K, str(tmp_path)), nprocs=world, join=True)
+    X = np.load(tmp_path / "full.npy")
+    xi, loss = np.load(tmp_path / "diag.npy")
+    _, B = quadratic_inputs(n, d, 7, x0="per_node")
+    xi_want = o.consensus_distance(X)
+    xbar = np.repeat(X.astype(np.float64).mean(0, keepdims=True), n, axis=0)
+    assert xi_want > 0 and abs(xi - xi_want) <= 1e-9 * xi_want
+    assert abs(loss - o.quadratic_mean_loss(xbar, B)) <= 1e-9 * loss
