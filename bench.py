@@ -7,6 +7,7 @@ every H-th iteration.  Prints one JSON line (rank 0).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4_exp_h4] [--impl reference]
     python bench.py --workload c3_ring_h4 --node-shards 4      # one shard's kernels of the node-sharded mode
+    python bench.py --workload c3_ring_h4 --node-shards 4 --fused-send   # ... with the export kernel storing the messages itself
 
 Default workload: the BERT-Large-sized configuration (n = 16, d = 335,141,888, one-peer
 exponential graph, H = 4; 64.35 GB per step), or the ResNet-50-sized ring configuration when
